@@ -1,0 +1,203 @@
+/*
+ * flexspec.h -- C ABI of the B200 (sm_100a) cloud-side verification step of
+ * edge-cloud speculative decoding.
+ *
+ * One verification step (Algorithm 2, "Step 2: cloud-side parallel
+ * verification"; Section III-A system model; Section IV-C KV session): for a
+ * batch of user sequences the cloud receives a block of k_b draft tokens per
+ * sequence, scores the k_b+1 positions in parallel against the user's cached KV
+ * session, decides how many draft tokens to accept (tau) and emits one further
+ * token, so that the verified output is draft[0:tau] followed by that token.
+ *
+ * Three GPU stages, each a hand-written CUDA kernel:
+ *   attention : paged-KV grouped-query attention of the k_b+1 query rows,
+ *               causal inside the draft window (split over the KV range).
+ *   lm_head   : logits[M][V] = attn_out[M][d] . W[V][d]^T on tcgen05 / TMEM.
+ *   sample    : softmax of target and draft logits, acceptance test
+ *               u * q(x) < p(x) with counter-based uniforms, first rejection,
+ *               residual / bonus draw -- or the greedy arg-max rule that
+ *               Algorithm 2 prints.
+ *
+ * Symbols: p = TARGET distribution, q = DRAFT distribution.  (Algorithm 2
+ * writes the target's output as q; that letter is not used here.)
+ *
+ * Conventions
+ *   - Every function returns 0 (FLEXSPEC_OK) or a negative FLEXSPEC_ERR_* code;
+ *     nothing throws, aborts or exits.  Argument errors are detected on the
+ *     host before any launch.
+ *   - "DEVICE" pointers are CUDA global-memory addresses on the handle's
+ *     device, "HOST" pointers ordinary host memory.  The caller owns every
+ *     input and output buffer; the handle owns only its workspace and borrows
+ *     the LM-head weight pointer for its lifetime.
+ *   - Calls that take a stream are asynchronous on it; outputs are valid once
+ *     the stream has been synchronised.  A handle is not thread-safe and must
+ *     be used on one stream at a time.
+ *   - Row layout.  Sequence b owns k_b+1 consecutive query rows, starting at
+ *     row sum_{b'<b}(k_b'+1): row 0 is the position of the last committed
+ *     token, row j>=1 the position of draft token x_{j-1}.  The distribution
+ *     read from row j judges draft token x_j; row k_b is the bonus row.  Draft
+ *     rows (tokens, draft logits) are packed the same way with k_b per sequence.
+ *   - M = sum_b (k_b+1) query rows, S = sum_b k_b draft positions.
+ *   - The library never writes to the KV pages.  KV rollback after a rejection
+ *     (Section IV-C) is the caller's: the next call passes a kv_len truncated
+ *     according to accepted_len.
+ */
+#ifndef FLEXSPEC_H
+#define FLEXSPEC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FLEXSPEC_OK                0
+#define FLEXSPEC_ERR_INVALID_ARG  -1   /* NULL pointer, size out of range, inconsistent lengths */
+#define FLEXSPEC_ERR_UNSUPPORTED  -2   /* shape outside what the kernels are built for          */
+#define FLEXSPEC_ERR_OOM          -3   /* workspace allocation failed                           */
+#define FLEXSPEC_ERR_CUDA         -4   /* a CUDA runtime / driver call failed                   */
+#define FLEXSPEC_ERR_TIMEOUT      -5   /* a bounded device-side wait gave up (status word)      */
+#define FLEXSPEC_ERR_BAD_PAGE     -6   /* page table entry outside [0, num_pages)               */
+#define FLEXSPEC_ERR_BAD_TOKEN    -7   /* draft token outside [0, vocab)                        */
+#define FLEXSPEC_ERR_NO_DEVICE    -8   /* no usable CUDA device / driver                        */
+
+#define FLEXSPEC_MODE_SAMPLE 0   /* speculative sampling: accept w.p. min(1, p/q), residual / bonus draw */
+#define FLEXSPEC_MODE_GREEDY 1   /* Algorithm 2 as printed: accept while x_j == argmax of the target row */
+
+#define FLEXSPEC_FLAG_DEBUG 1u   /* keep p(x_j), q(x_j), u_j per draft position (see flexspec_get_debug) */
+
+typedef struct flexspec_handle flexspec_handle;   /* opaque */
+
+typedef struct {
+    int32_t  n_q_heads;     /* H; d_model = H * head_dim, must be a multiple of 64           */
+    int32_t  n_kv_heads;    /* Hkv, divides H                                                 */
+    int32_t  head_dim;      /* 64 or 128                                                      */
+    int32_t  vocab;         /* V >= 1                                                         */
+    int32_t  page_size;     /* tokens per KV page: must be 16                                 */
+    int32_t  max_batch;     /* 1..1024 sequences per call                                     */
+    int32_t  k_max;         /* largest draft length k_b, 0..63                                */
+    int32_t  max_kv_len;    /* largest kv_len[b] (context + k_b + 1)                          */
+    int32_t  mode;          /* FLEXSPEC_MODE_*                                                */
+    int32_t  device;        /* CUDA device ordinal                                            */
+    uint32_t flags;         /* FLEXSPEC_FLAG_*                                                */
+} flexspec_config;
+
+/* The per-user KV sessions (Section IV-C), as one paged pool. */
+typedef struct {
+    const void*    kv_pages;          /* DEVICE bf16 [num_pages][2][n_kv_heads][page_size][head_dim];
+                                         index 0 of the second axis is K, 1 is V; 16-byte aligned   */
+    int32_t        num_pages;
+    const int32_t* page_table;        /* DEVICE int32 [batch][max_pages_per_seq]: token t of sequence b
+                                         lives in page page_table[b][t/16], slot t%16; entries past
+                                         ceil(kv_len[b]/16) are never read                          */
+    int32_t        max_pages_per_seq;
+    const int32_t* kv_len;            /* DEVICE int32 [batch] = committed context + k_b + 1: the K/V
+                                         of the k_b+1 window positions are already in the pages     */
+    const int32_t* kv_len_host;       /* HOST copy of kv_len (launch geometry only)                 */
+} flexspec_kv;
+
+typedef struct {            /* DEVICE pointers into the handle's workspace, valid until destroy */
+    const void*    attn_out;   /* bf16 [M][d_model], last verify / attention call                 */
+    const float*   logits;     /* fp32 [M][vocab], last verify / lm_head call into the workspace  */
+    const double*  p_tok;      /* fp64 [S]  p_j(x_j)   (FLEXSPEC_FLAG_DEBUG, SAMPLE mode)          */
+    const double*  q_tok;      /* fp64 [S]  q_j(x_j)                                              */
+    const float*   u_acc;      /* fp32 [S]  u_j                                                   */
+    const int32_t* status;     /* int32 [4] device status word: [0] first error code, [1] detail  */
+} flexspec_debug;
+
+/* Create a handle: validates the shape, allocates the workspace on cfg->device
+ * (logits [max_batch*(k_max+1)][vocab] fp32, attention partials, small tables)
+ * and builds the TMA descriptor of the LM-head weights.
+ *   lm_head_w : DEVICE bf16 [vocab][d_model] (row v is the output embedding of
+ *               token v), 16-byte aligned, borrowed until flexspec_destroy.
+ * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA, NO_DEVICE. */
+int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_handle** out);
+
+/* The whole verification step (Algorithm 2, Step 2) on `stream`:
+ * attention -> LM head -> acceptance + emitted token.
+ *   hidden        DEVICE bf16 [M][d_model]; row r viewed as [H][head_dim] is the query of
+ *                 every head (the attention output feeds the LM head directly)
+ *   draft_tokens  DEVICE int32 [S]
+ *   draft_logits  DEVICE fp32 [S][vocab]; may be NULL in GREEDY mode
+ *   draft_len     DEVICE int32 [batch], draft_len_host its HOST copy (launch geometry)
+ *   seeds         DEVICE uint64 [batch]; uniforms are Philox4x32-10 with key =
+ *                 (lo32, hi32) of the seed, counter = (j, stream, 0, 0), word 0,
+ *                 u = (word >> 8) * 2^-24; stream 0 = acceptance test of draft j,
+ *                 stream 1 = draw of the emitted token after j accepted drafts.
+ *                 May be NULL in GREEDY mode.
+ *   temperature   both logit sets are divided by it; 0 selects the greedy rule
+ *   vocab_mask    DEVICE uint32 [batch][ceil(vocab/32)] or NULL: a 0 bit forbids
+ *                 that token for the target (p = 0 exactly)
+ *   accepted_len  DEVICE int32 [batch] out: tau_b in [0, k_b]
+ *   next_token    DEVICE int32 [batch] out: the token emitted after the accepted prefix
+ * Errors: INVALID_ARG (NULLs, batch > max_batch, k_b > k_max, kv_len out of range or
+ * smaller than k_b+1, too few pages per sequence), CUDA. Device-side problems
+ * (bad page id, bad token id, a wait that gave up) are recorded in the status
+ * word, see flexspec_status. */
+int flexspec_verify(flexspec_handle* h, const flexspec_kv* kv, const void* hidden,
+                    const int32_t* draft_tokens, const float* draft_logits,
+                    const int32_t* draft_len, const int32_t* draft_len_host,
+                    const uint64_t* seeds, int32_t batch, float temperature,
+                    const uint32_t* vocab_mask,
+                    int32_t* accepted_len, int32_t* next_token, void* stream);
+
+/* The same step for callers whose per-step inputs live in HOST memory: copies
+ * hidden, draft tokens, draft logits, lengths and seeds to the device, runs
+ * flexspec_verify, copies accepted_len / next_token back and synchronises.
+ * The KV pool and page table stay on the device (they are the persistent
+ * session state); kv->kv_len may be NULL here (taken from kv->kv_len_host).
+ * Every other pointer argument is a HOST pointer. */
+int flexspec_verify_host(flexspec_handle* h, const flexspec_kv* kv, const void* hidden,
+                         const int32_t* draft_tokens, const float* draft_logits,
+                         const int32_t* draft_len, const uint64_t* seeds, int32_t batch,
+                         float temperature, int32_t* accepted_len, int32_t* next_token,
+                         void* stream);
+
+/* Stage 1 alone (Section IV-C; Algorithm 2 "restore KV cache" + target forward over the block):
+ * attn_out DEVICE bf16 [M][d_model] out, or NULL to write the handle's workspace. */
+int flexspec_attention(flexspec_handle* h, const flexspec_kv* kv, const void* hidden,
+                       const int32_t* draft_len, const int32_t* draft_len_host, int32_t batch,
+                       void* attn_out, void* stream);
+
+/* Stage 2 alone: logits[m_rows][vocab] = x[m_rows][d_model] . W^T (the frozen LM head of
+ * the target, Section IV-A).  x DEVICE bf16 (NULL = workspace attn_out), logits DEVICE fp32
+ * (NULL = workspace).  m_rows <= max_batch*(k_max+1). */
+int flexspec_lm_head(flexspec_handle* h, const void* x, int32_t m_rows, float* logits, void* stream);
+
+/* Stage 3 alone (Algorithm 2 acceptance loop and correction token; the stochastic rule of
+ * the speculative-sampling papers it cites).  logits DEVICE fp32 [M][vocab] (NULL = workspace);
+ * other arguments as in flexspec_verify. */
+int flexspec_sample(flexspec_handle* h, const float* logits,
+                    const int32_t* draft_tokens, const float* draft_logits,
+                    const int32_t* draft_len, const int32_t* draft_len_host,
+                    const uint64_t* seeds, int32_t batch, float temperature,
+                    const uint32_t* vocab_mask,
+                    int32_t* accepted_len, int32_t* next_token, void* stream);
+
+/* Workspace pointers for stage-wise comparison. */
+int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);
+
+/* Synchronises the device, copies the status word to status_host[4] (may be NULL), clears it
+ * and returns its first entry (0 or a FLEXSPEC_ERR_* code recorded by a kernel). */
+int flexspec_status(flexspec_handle* h, int32_t* status_host);
+
+/* Per-kernel timing.  With profiling on, verify brackets each kernel with CUDA events on the
+ * caller's stream; flexspec_get_stage_ms synchronises those events and writes the last call's
+ * durations in milliseconds: [0] plan, [1] attention, [2] attention combine, [3] LM head,
+ * [4] sample statistics + decision, [5] sample draw.  Unused stages read 0. */
+int flexspec_set_profiling(flexspec_handle* h, int32_t on);
+int flexspec_get_stage_ms(flexspec_handle* h, float ms[6]);
+
+/* Number of kernels the last verify / stage call launched. */
+int flexspec_last_launches(flexspec_handle* h);
+
+/* Releases the workspace.  NULL is accepted. */
+int flexspec_destroy(flexspec_handle* h);
+
+const char* flexspec_strerror(int code);
+const char* flexspec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,574 @@
+// Host layer of the C ABI declared in include/flexspec.h: argument validation, workspace,
+// TMA descriptors, launch sequencing.  No step of the verification runs on the host.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "internal.h"
+
+using namespace fs;
+
+struct flexspec_handle {
+    Handle h;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is looked up at run time so that the library loads (and its symbols
+// can be inspected) on a machine without a GPU driver.
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major tensor [rows][cols], box [box_rows][64 cols], 128-byte swizzle, zero fill.
+int make_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return FLEXSPEC_ERR_NO_DEVICE;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t elem[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? FLEXSPEC_OK : FLEXSPEC_ERR_CUDA;
+}
+
+template <typename T>
+int dev_alloc(T** p, size_t count)
+{
+    *p = nullptr;
+    if (count == 0) count = 1;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+    if (e != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_OOM; }
+    return FLEXSPEC_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); prev = -1; }
+        ok = (cudaSetDevice(dev) == cudaSuccess);
+        if (!ok) cudaGetLastError();
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+void free_workspace(Handle& h)
+{
+    cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml);
+    cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq);
+    cudaFree(h.stats); cudaFree(h.arg_idx); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.chunk_mass);
+    cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
+    cudaFree(h.stage_dev); cudaFree(h.out_dev);
+    for (int i = 0; i < kNumStageEvents; ++i)
+        if (h.ev[i]) cudaEventDestroy(h.ev[i]);
+}
+
+// geometry of one call, derived from the host copies of the lengths
+struct Geometry {
+    int32_t m_rows = 0, s_rows = 0, k_batch_max = 0, kv_max = 0;
+    int64_t kv_total = 0;
+};
+
+int check_lengths(const Handle& h, const int32_t* draft_len_host, const int32_t* kv_len_host, int32_t batch,
+                  int32_t max_pages_per_seq, Geometry* g)
+{
+    if (batch < 1 || batch > h.cfg.max_batch || draft_len_host == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b) {
+        const int k = draft_len_host[b];
+        if (k < 0 || k > h.cfg.k_max) return FLEXSPEC_ERR_INVALID_ARG;
+        g->m_rows += k + 1;
+        g->s_rows += k;
+        if (k > g->k_batch_max) g->k_batch_max = k;
+        if (kv_len_host != nullptr) {
+            const int l = kv_len_host[b];
+            if (l < k + 1 || l > h.cfg.max_kv_len) return FLEXSPEC_ERR_INVALID_ARG;
+            if ((l + h.cfg.page_size - 1) / h.cfg.page_size > max_pages_per_seq) return FLEXSPEC_ERR_INVALID_ARG;
+            if (l > g->kv_max) g->kv_max = l;
+            g->kv_total += l;
+        }
+    }
+    return FLEXSPEC_OK;
+}
+
+void mark(Handle& h, int idx, cudaStream_t s)
+{
+    if (h.profiling) { cudaEventRecord(h.ev[idx], s); h.ev_used[idx] = 1; }
+}
+
+int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, cudaStream_t s)
+{
+    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, h.plan, h.status, s) != cudaSuccess)
+        return FLEXSPEC_ERR_CUDA;
+    h.launches++;
+    return FLEXSPEC_OK;
+}
+
+int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const int32_t* draft_len,
+                  const Geometry& g, int32_t batch, void* attn_out, cudaStream_t s)
+{
+    const flexspec_config& c = h.cfg;
+    const int group = c.n_q_heads / c.n_kv_heads;
+    // one tensor map over the whole pool: rows of head_dim bf16
+    CUtensorMap kv_map;
+    const uint64_t pool_rows = static_cast<uint64_t>(kv->num_pages) * 2 * c.n_kv_heads * c.page_size;
+    int rc = make_map_2d(&kv_map, kv->kv_pages, pool_rows, static_cast<uint64_t>(c.head_dim), 16);
+    if (rc != FLEXSPEC_OK) return rc;
+
+    // split the KV range so that about three CTAs' worth of work exists per SM
+    const int max_tile_rows = group * (g.k_batch_max + 1);
+    const int row_blocks = (max_tile_rows + 127) / 128;
+    const int64_t units = g.kv_total * c.n_kv_heads * row_blocks;
+    int64_t split_len = (units + 3LL * h.sm_count - 1) / (3LL * h.sm_count);
+    split_len = (split_len + kAttSplitQuantum - 1) / kAttSplitQuantum * kAttSplitQuantum;
+    if (split_len < 2 * kAttSplitQuantum) split_len = 2 * kAttSplitQuantum;
+    int64_t min_len = (static_cast<int64_t>(g.kv_max) + kAttMaxSplits - 1) / kAttMaxSplits;
+    min_len = (min_len + kAttSplitQuantum - 1) / kAttSplitQuantum * kAttSplitQuantum;
+    if (split_len < min_len) split_len = min_len;
+    const int max_splits = static_cast<int>((g.kv_max + split_len - 1) / split_len);
+
+    AttnParams p;
+    p.hidden = static_cast<const __nv_bfloat16*>(hidden);
+    p.page_table = kv->page_table;
+    p.kv_len = kv->kv_len;
+    p.draft_len = draft_len;
+    p.cu_q = h.plan.cu_q;
+    p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = group;
+    p.max_pages_per_seq = kv->max_pages_per_seq; p.num_pages = kv->num_pages;
+    p.split_len = static_cast<int32_t>(split_len);
+    p.row_blocks = row_blocks;
+    p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(c.head_dim)));
+    p.part_o = h.part_o; p.part_ml = h.part_ml;
+    p.part_stride = static_cast<int64_t>(h.max_m) * c.n_q_heads;
+    p.attn_out = static_cast<__nv_bfloat16*>(attn_out);
+    p.status = h.status;
+    if (launch_attention(h, kv_map, p, batch, g.k_batch_max + 1, max_splits, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
+    mark(h, 2, s);
+    if (max_splits > 1) {
+        CombineParams cp;
+        cp.part_o = h.part_o; cp.part_ml = h.part_ml; cp.part_stride = p.part_stride;
+        cp.kv_len = kv->kv_len; cp.draft_len = draft_len; cp.cu_q = h.plan.cu_q;
+        cp.split_len = p.split_len; cp.rows_per_seq_max = g.k_batch_max + 1;
+        cp.n_q_heads = c.n_q_heads; cp.head_dim = c.head_dim;
+        cp.attn_out = p.attn_out;
+        if (launch_attention_combine(cp, batch, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        h.launches++;
+    }
+    return FLEXSPEC_OK;
+}
+
+int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, cudaStream_t s)
+{
+    const flexspec_config& c = h.cfg;
+    LmHeadParams p;
+    p.logits = logits;
+    p.m_rows = m_rows; p.vocab = c.vocab; p.d_model = h.d_model;
+    const int m16 = (m_rows + 15) / 16 * 16;
+    if (m16 <= 256) { p.n_tile = m16; p.n_blocks = 1; }
+    else { p.n_tile = 256; p.n_blocks = 2; }
+    const int rows_per_pass = p.n_tile * p.n_blocks;
+    p.n_pass = (m_rows + rows_per_pass - 1) / rows_per_pass;
+    p.n_vtiles = (c.vocab + 127) / 128;
+    p.num_stages = lm_head_pick_stages(p.n_tile, p.n_blocks);
+    p.acc_stages = (2 * rows_per_pass <= 512) ? 2 : 1;
+    p.status = h.status;
+    CUtensorMap x_map;
+    int rc = make_map_2d(&x_map, x, static_cast<uint64_t>(m_rows), static_cast<uint64_t>(h.d_model),
+                         static_cast<uint32_t>(p.n_tile));
+    if (rc != FLEXSPEC_OK) return rc;
+    if (launch_lm_head(h, x_map, p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
+    return FLEXSPEC_OK;
+}
+
+int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, const float* draft_logits,
+               const int32_t* draft_len, const uint64_t* seeds, const Geometry& g, int32_t batch,
+               float temperature, const uint32_t* vocab_mask, int32_t* accepted_len, int32_t* next_token,
+               cudaStream_t s)
+{
+    const flexspec_config& c = h.cfg;
+    SampleParams p;
+    memset(&p, 0, sizeof(p));
+    p.greedy = (c.mode == FLEXSPEC_MODE_GREEDY || temperature == 0.f) ? 1 : 0;
+    p.logits = logits; p.draft_logits = draft_logits; p.draft_tokens = draft_tokens;
+    p.draft_len = draft_len; p.seeds = seeds; p.vocab_mask = vocab_mask;
+    p.cu_q = h.plan.cu_q; p.cu_d = h.plan.cu_d; p.row_seq = h.plan.row_seq;
+    p.batch = batch; p.vocab = c.vocab; p.m_rows = g.m_rows; p.s_rows = g.s_rows;
+    p.n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
+    p.mask_words = (c.vocab + 31) / 32;
+    p.inv_temp_log2 = p.greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    p.stats = h.stats; p.arg_idx = h.arg_idx; p.counters = h.counters;
+    p.row_info = h.row_info; p.chunk_mass = h.chunk_mass;
+    p.accepted_len = accepted_len; p.next_token = next_token;
+    if (c.flags & FLEXSPEC_FLAG_DEBUG) { p.dbg_p = h.dbg_p; p.dbg_q = h.dbg_q; p.dbg_u = h.dbg_u; }
+    p.status = h.status;
+    if (launch_sample_stats(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
+    mark(h, 5, s);
+    if (!p.greedy) {
+        if (launch_sample_draw(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        h.launches++;
+    }
+    return FLEXSPEC_OK;
+}
+
+bool sample_args_ok(const Handle& h, const int32_t* draft_tokens, const float* draft_logits,
+                    const uint64_t* seeds, float temperature, const Geometry& g)
+{
+    const bool greedy = (h.cfg.mode == FLEXSPEC_MODE_GREEDY || temperature == 0.f);
+    if (!(temperature >= 0.f) || isinf(temperature)) return false;
+    if (g.s_rows > 0 && draft_tokens == nullptr) return false;
+    if (!greedy && (seeds == nullptr || (g.s_rows > 0 && draft_logits == nullptr))) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_handle** out)
+{
+    if (out == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg == nullptr || lm_head_w == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    const flexspec_config& c = *cfg;
+    if (c.n_q_heads < 1 || c.n_kv_heads < 1 || c.vocab < 1 || c.max_batch < 1 || c.k_max < 0 ||
+        c.max_kv_len < 1 || c.device < 0)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    if (c.mode != FLEXSPEC_MODE_SAMPLE && c.mode != FLEXSPEC_MODE_GREEDY) return FLEXSPEC_ERR_INVALID_ARG;
+    if (c.n_q_heads % c.n_kv_heads != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    if (c.max_kv_len < c.k_max + 1) return FLEXSPEC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(lm_head_w) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    if (c.head_dim != 64 && c.head_dim != 128) return FLEXSPEC_ERR_UNSUPPORTED;
+    if (c.page_size != 16) return FLEXSPEC_ERR_UNSUPPORTED;
+    if (c.max_batch > kMaxBatch || c.k_max > kMaxK) return FLEXSPEC_ERR_UNSUPPORTED;
+    const int64_t d_model = static_cast<int64_t>(c.n_q_heads) * c.head_dim;
+    if (d_model % 64 != 0 || d_model > 65536) return FLEXSPEC_ERR_UNSUPPORTED;
+    const int64_t max_m = static_cast<int64_t>(c.max_batch) * (c.k_max + 1);
+    if (max_m * c.vocab > (1LL << 40)) return FLEXSPEC_ERR_UNSUPPORTED;
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || c.device >= n_dev) { cudaGetLastError(); return FLEXSPEC_ERR_NO_DEVICE; }
+    DeviceGuard guard(c.device);
+    if (!guard.ok) return FLEXSPEC_ERR_NO_DEVICE;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (prop.major != 10) return FLEXSPEC_ERR_UNSUPPORTED;       // kernels are built for sm_100a only
+
+    flexspec_handle* fh = new (std::nothrow) flexspec_handle();
+    if (fh == nullptr) return FLEXSPEC_ERR_OOM;
+    Handle& h = fh->h;
+    memset(&h, 0, sizeof(h));
+    h.cfg = c;
+    h.d_model = static_cast<int32_t>(d_model);
+    h.max_m = static_cast<int32_t>(max_m);
+    h.max_s = c.max_batch * c.k_max;
+    h.sm_count = prop.multiProcessorCount;
+    h.w = static_cast<const __nv_bfloat16*>(lm_head_w);
+
+    const int n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
+    int rc = FLEXSPEC_OK;
+    auto A = [&](int r) { if (rc == FLEXSPEC_OK) rc = r; };
+    A(dev_alloc(&h.attn_out, static_cast<size_t>(max_m) * d_model));
+    A(dev_alloc(&h.logits, static_cast<size_t>(max_m) * c.vocab));
+    A(dev_alloc(&h.part_o, static_cast<size_t>(kAttMaxSplits) * max_m * d_model));
+    A(dev_alloc(&h.part_ml, static_cast<size_t>(kAttMaxSplits) * max_m * c.n_q_heads * 2));
+    A(dev_alloc(&h.plan.cu_q, static_cast<size_t>(c.max_batch) + 1));
+    A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
+    A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
+    A(dev_alloc(&h.stats, static_cast<size_t>(max_m + h.max_s) * n_chunks));
+    A(dev_alloc(&h.arg_idx, static_cast<size_t>(max_m) * n_chunks));
+    A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
+    A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 4));
+    A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * n_chunks * 2));
+    A(dev_alloc(&h.dbg_p, static_cast<size_t>(h.max_s)));
+    A(dev_alloc(&h.dbg_q, static_cast<size_t>(h.max_s)));
+    A(dev_alloc(&h.dbg_u, static_cast<size_t>(h.max_s)));
+    A(dev_alloc(&h.status, 4));
+    A(dev_alloc(&h.out_dev, static_cast<size_t>(2) * c.max_batch));
+    if (rc == FLEXSPEC_OK) {
+        // staging for flexspec_verify_host: hidden | draft logits | tokens | lengths (2) | seeds
+        h.stage_bytes = static_cast<size_t>(max_m) * d_model * 2 + static_cast<size_t>(h.max_s) * c.vocab * 4 +
+                        static_cast<size_t>(h.max_s) * 4 + static_cast<size_t>(c.max_batch) * (4 + 4 + 8) + 4096;
+        if (cudaMalloc(&h.stage_dev, h.stage_bytes) != cudaSuccess) { cudaGetLastError(); rc = FLEXSPEC_ERR_OOM; }
+    }
+    if (rc == FLEXSPEC_OK) {
+        if (cudaMemset(h.counters, 0, sizeof(int32_t) * 2 * kMaxBatch) != cudaSuccess ||
+            cudaMemset(h.status, 0, sizeof(int32_t) * 4) != cudaSuccess)
+            rc = FLEXSPEC_ERR_CUDA;
+    }
+    for (int i = 0; i < kNumStageEvents && rc == FLEXSPEC_OK; ++i)
+        if (cudaEventCreate(&h.ev[i]) != cudaSuccess) rc = FLEXSPEC_ERR_CUDA;
+    if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map, lm_head_w, static_cast<uint64_t>(c.vocab),
+                                            static_cast<uint64_t>(d_model), 128);
+    if (rc == FLEXSPEC_OK && (attention_init(c.head_dim) != cudaSuccess || lm_head_init() != cudaSuccess))
+        rc = FLEXSPEC_ERR_CUDA;
+    if (rc != FLEXSPEC_OK) {
+        cudaGetLastError();
+        free_workspace(h);
+        delete fh;
+        return rc;
+    }
+    *out = fh;
+    return FLEXSPEC_OK;
+}
+
+int flexspec_destroy(flexspec_handle* fh)
+{
+    if (fh == nullptr) return FLEXSPEC_OK;
+    DeviceGuard guard(fh->h.cfg.device);
+    cudaDeviceSynchronize();
+    free_workspace(fh->h);
+    delete fh;
+    return FLEXSPEC_OK;
+}
+
+static int kv_args_ok(const Handle& h, const flexspec_kv* kv, bool need_dev_len)
+{
+    if (kv == nullptr || kv->kv_pages == nullptr || kv->page_table == nullptr || kv->kv_len_host == nullptr)
+        return 0;
+    if (need_dev_len && kv->kv_len == nullptr) return 0;
+    if (kv->num_pages < 1 || kv->max_pages_per_seq < 1) return 0;
+    if ((reinterpret_cast<uintptr_t>(kv->kv_pages) & 15u) != 0) return 0;
+    if (static_cast<int64_t>(kv->num_pages) * 2 * h.cfg.n_kv_heads * h.cfg.page_size > 0x7fffffffLL) return 0;
+    return 1;
+}
+
+int flexspec_attention(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
+                       const int32_t* draft_len, const int32_t* draft_len_host, int32_t batch,
+                       void* attn_out, void* stream)
+{
+    if (fh == nullptr || hidden == nullptr || draft_len == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (!kv_args_ok(h, kv, true)) return FLEXSPEC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    Geometry g;
+    int rc = check_lengths(h, draft_len_host, kv->kv_len_host, batch, kv->max_pages_per_seq, &g);
+    if (rc != FLEXSPEC_OK) return rc;
+    DeviceGuard guard(h.cfg.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    h.launches = 0;
+    rc = run_plan(h, draft_len, nullptr, batch, s);
+    if (rc != FLEXSPEC_OK) return rc;
+    return run_attention(h, kv, hidden, draft_len, g, batch, attn_out ? attn_out : h.attn_out, s);
+}
+
+int flexspec_lm_head(flexspec_handle* fh, const void* x, int32_t m_rows, float* logits, void* stream)
+{
+    if (fh == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (m_rows < 1 || m_rows > h.max_m) return FLEXSPEC_ERR_INVALID_ARG;
+    if (x != nullptr && (reinterpret_cast<uintptr_t>(x) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    h.launches = 0;
+    return run_lm_head(h, x ? x : h.attn_out, m_rows, logits ? logits : h.logits, static_cast<cudaStream_t>(stream));
+}
+
+int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* draft_tokens,
+                    const float* draft_logits, const int32_t* draft_len, const int32_t* draft_len_host,
+                    const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
+                    int32_t* accepted_len, int32_t* next_token, void* stream)
+{
+    if (fh == nullptr || draft_len == nullptr || accepted_len == nullptr || next_token == nullptr)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    Geometry g;
+    int rc = check_lengths(h, draft_len_host, nullptr, batch, 0, &g);
+    if (rc != FLEXSPEC_OK) return rc;
+    if (!sample_args_ok(h, draft_tokens, draft_logits, seeds, temperature, g)) return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    h.launches = 0;
+    rc = run_plan(h, draft_len, draft_tokens, batch, s);
+    if (rc != FLEXSPEC_OK) return rc;
+    return run_sample(h, logits ? logits : h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch,
+                      temperature, vocab_mask, accepted_len, next_token, s);
+}
+
+int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
+                    const int32_t* draft_tokens, const float* draft_logits,
+                    const int32_t* draft_len, const int32_t* draft_len_host,
+                    const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
+                    int32_t* accepted_len, int32_t* next_token, void* stream)
+{
+    if (fh == nullptr || hidden == nullptr || draft_len == nullptr || accepted_len == nullptr ||
+        next_token == nullptr)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (!kv_args_ok(h, kv, true)) return FLEXSPEC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    Geometry g;
+    int rc = check_lengths(h, draft_len_host, kv->kv_len_host, batch, kv->max_pages_per_seq, &g);
+    if (rc != FLEXSPEC_OK) return rc;
+    if (!sample_args_ok(h, draft_tokens, draft_logits, seeds, temperature, g)) return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    h.launches = 0;
+    memset(h.ev_used, 0, sizeof(h.ev_used));
+    mark(h, 0, s);
+    rc = run_plan(h, draft_len, draft_tokens, batch, s);
+    if (rc != FLEXSPEC_OK) return rc;
+    mark(h, 1, s);
+    rc = run_attention(h, kv, hidden, draft_len, g, batch, h.attn_out, s);   // marks event 2 after the split kernel
+    if (rc != FLEXSPEC_OK) return rc;
+    mark(h, 3, s);
+    rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, s);
+    if (rc != FLEXSPEC_OK) return rc;
+    mark(h, 4, s);
+    rc = run_sample(h, h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch, temperature,
+                    vocab_mask, accepted_len, next_token, s);                // marks event 5 after the stats kernel
+    if (rc != FLEXSPEC_OK) return rc;
+    mark(h, 6, s);
+    return FLEXSPEC_OK;
+}
+
+int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
+                         const int32_t* draft_tokens, const float* draft_logits, const int32_t* draft_len,
+                         const uint64_t* seeds, int32_t batch, float temperature,
+                         int32_t* accepted_len, int32_t* next_token, void* stream)
+{
+    if (fh == nullptr || hidden == nullptr || draft_len == nullptr || accepted_len == nullptr ||
+        next_token == nullptr)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (!kv_args_ok(h, kv, false)) return FLEXSPEC_ERR_INVALID_ARG;
+    Geometry g;
+    int rc = check_lengths(h, draft_len, kv->kv_len_host, batch, kv->max_pages_per_seq, &g);
+    if (rc != FLEXSPEC_OK) return rc;
+    if (!sample_args_ok(h, draft_tokens, draft_logits, seeds, temperature, g)) return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    // carve the staging buffer (256-byte aligned pieces)
+    uint8_t* base = static_cast<uint8_t*>(h.stage_dev);
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { uint8_t* p = base + off; off = (off + bytes + 255) & ~size_t(255); return p; };
+    void* d_hidden = carve(static_cast<size_t>(g.m_rows) * h.d_model * 2);
+    float* d_dlog = reinterpret_cast<float*>(carve(static_cast<size_t>(g.s_rows) * h.cfg.vocab * 4));
+    int32_t* d_tok = reinterpret_cast<int32_t*>(carve(static_cast<size_t>(g.s_rows) * 4));
+    int32_t* d_len = reinterpret_cast<int32_t*>(carve(static_cast<size_t>(batch) * 4));
+    int32_t* d_kvl = reinterpret_cast<int32_t*>(carve(static_cast<size_t>(batch) * 4));
+    uint64_t* d_seed = reinterpret_cast<uint64_t*>(carve(static_cast<size_t>(batch) * 8));
+    if (off > h.stage_bytes) return FLEXSPEC_ERR_INVALID_ARG;
+
+    bool ok = true;
+    auto H2D = [&](void* dst, const void* src, size_t bytes) {
+        if (bytes > 0 && src != nullptr) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    };
+    H2D(d_hidden, hidden, static_cast<size_t>(g.m_rows) * h.d_model * 2);
+    H2D(d_dlog, draft_logits, static_cast<size_t>(g.s_rows) * h.cfg.vocab * 4);
+    H2D(d_tok, draft_tokens, static_cast<size_t>(g.s_rows) * 4);
+    H2D(d_len, draft_len, static_cast<size_t>(batch) * 4);
+    H2D(d_kvl, kv->kv_len_host, static_cast<size_t>(batch) * 4);
+    H2D(d_seed, seeds, static_cast<size_t>(batch) * 8);
+    if (!ok) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+
+    flexspec_kv kv_dev = *kv;
+    kv_dev.kv_len = d_kvl;
+    rc = flexspec_verify(fh, &kv_dev, d_hidden, d_tok, draft_logits ? d_dlog : nullptr, d_len, draft_len,
+                         seeds ? d_seed : nullptr, batch, temperature, nullptr, h.out_dev, h.out_dev + batch, s);
+    if (rc != FLEXSPEC_OK) return rc;
+    ok = cudaMemcpyAsync(accepted_len, h.out_dev, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(next_token, h.out_dev + batch, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+    return FLEXSPEC_OK;
+}
+
+int flexspec_get_debug(flexspec_handle* fh, flexspec_debug* out)
+{
+    if (fh == nullptr || out == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    const Handle& h = fh->h;
+    out->attn_out = h.attn_out;
+    out->logits = h.logits;
+    out->p_tok = h.dbg_p;
+    out->q_tok = h.dbg_q;
+    out->u_acc = h.dbg_u;
+    out->status = h.status;
+    return FLEXSPEC_OK;
+}
+
+int flexspec_status(flexspec_handle* fh, int32_t* status_host)
+{
+    if (fh == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    DeviceGuard guard(h.cfg.device);
+    int32_t st[4] = {0, 0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+    if (cudaMemcpy(st, h.status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (st[0] != 0 && cudaMemset(h.status, 0, sizeof(st)) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (status_host != nullptr) memcpy(status_host, st, sizeof(st));
+    return st[0];
+}
+
+int flexspec_set_profiling(flexspec_handle* fh, int32_t on)
+{
+    if (fh == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    fh->h.profiling = on ? 1 : 0;
+    memset(fh->h.ev_used, 0, sizeof(fh->h.ev_used));
+    return FLEXSPEC_OK;
+}
+
+int flexspec_get_stage_ms(flexspec_handle* fh, float ms[6])
+{
+    if (fh == nullptr || ms == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    for (int i = 0; i < 6; ++i) ms[i] = 0.f;
+    if (!h.profiling || !h.ev_used[0] || !h.ev_used[6]) return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    if (cudaEventSynchronize(h.ev[6]) != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+    // events: 0 start, 1 after plan, 2 after attention split kernel, 3 after combine, 4 after LM head,
+    // 5 after sample statistics, 6 end
+    for (int i = 0; i < 6; ++i) {
+        if (!h.ev_used[i] || !h.ev_used[i + 1]) continue;
+        if (cudaEventElapsedTime(&ms[i], h.ev[i], h.ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+    }
+    return FLEXSPEC_OK;
+}
+
+int flexspec_last_launches(flexspec_handle* fh)
+{
+    if (fh == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
+    return fh->h.launches;
+}
+
+const char* flexspec_strerror(int code)
+{
+    switch (code) {
+        case FLEXSPEC_OK: return "ok";
+        case FLEXSPEC_ERR_INVALID_ARG: return "invalid argument";
+        case FLEXSPEC_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case FLEXSPEC_ERR_OOM: return "out of device memory";
+        case FLEXSPEC_ERR_CUDA: return "CUDA call failed";
+        case FLEXSPEC_ERR_TIMEOUT: return "device-side wait timed out";
+        case FLEXSPEC_ERR_BAD_PAGE: return "page table entry out of range";
+        case FLEXSPEC_ERR_BAD_TOKEN: return "draft token out of range";
+        case FLEXSPEC_ERR_NO_DEVICE: return "no usable CUDA device";
+        default: return "unknown error";
+    }
+}
+
+const char* flexspec_version(void) { return "flexspec-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,129 @@
+// Host-side internals shared by the .cu files of the library: the handle, launch wrappers.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/flexspec.h"
+
+namespace fs {
+
+constexpr int kMaxBatch = 1024;
+constexpr int kMaxK = 63;
+constexpr int kSampleChunk = 8192;        // vocabulary elements per CTA in the sampling kernels
+constexpr int kAttSplitQuantum = 128;     // tokens per attention pipeline stage
+constexpr int kAttMaxSplits = 32;
+constexpr int kNumStageEvents = 7;
+
+struct Plan {                 // device tables written by the plan kernel, read by all stages
+    int32_t* cu_q;            // [max_batch+1] first query row of each sequence
+    int32_t* cu_d;            // [max_batch+1] first draft row of each sequence
+    int32_t* row_seq;         // [max_m] sequence of each query row
+};
+
+struct AttnParams {
+    const __nv_bfloat16* hidden;
+    const int32_t* page_table;
+    const int32_t* kv_len;
+    const int32_t* draft_len;
+    const int32_t* cu_q;
+    int32_t n_q_heads, n_kv_heads, group;
+    int32_t max_pages_per_seq, num_pages;
+    int32_t split_len;        // tokens per split, multiple of kAttSplitQuantum
+    int32_t row_blocks;       // CTAs along the query rows of one (sequence, kv head)
+    float scale_log2;         // log2(e) / sqrt(head_dim)
+    float* part_o;            // [split][row][H][Dh] unnormalised partial outputs
+    float* part_ml;           // [split][row][H][2]  (running max in log2 units, sum)
+    int64_t part_stride;      // rows * H (elements of part_ml / 2 per split; x Dh for part_o)
+    __nv_bfloat16* attn_out;  // [M][H*Dh]
+    int32_t* status;
+};
+
+struct CombineParams {
+    const float* part_o;
+    const float* part_ml;
+    int64_t part_stride;
+    const int32_t* kv_len;
+    const int32_t* draft_len;
+    const int32_t* cu_q;
+    int32_t split_len, rows_per_seq_max, n_q_heads, head_dim;
+    __nv_bfloat16* attn_out;
+};
+
+struct LmHeadParams {
+    float* logits;            // [m_rows][vocab]
+    int32_t m_rows, vocab, d_model;
+    int32_t n_tile;           // token columns per accumulator block (multiple of 16, <= 256)
+    int32_t n_blocks;         // accumulator blocks per pass (1 or 2)
+    int32_t n_pass;           // passes over W when m_rows > n_tile * n_blocks
+    int32_t n_vtiles;         // ceil(vocab / 128)
+    int32_t num_stages;       // shared-memory pipeline depth
+    int32_t acc_stages;       // TMEM accumulator buffers (1 or 2)
+    int32_t* status;
+};
+
+struct SampleParams {
+    const float* logits;          // [M][V] target
+    const float* draft_logits;    // [S][V]
+    const int32_t* draft_tokens;  // [S]
+    const int32_t* draft_len;     // [B]
+    const uint64_t* seeds;        // [B]
+    const uint32_t* vocab_mask;   // [B][mask_words] or null
+    const int32_t* cu_q;
+    const int32_t* cu_d;
+    const int32_t* row_seq;
+    int32_t batch, vocab, m_rows, s_rows, n_chunks, mask_words;
+    float inv_temp_log2;          // log2(e) / T
+    int32_t greedy;
+    float2* stats;                // [(M+S)][n_chunks] (chunk max in logit units, sum exp)
+    int32_t* arg_idx;             // [M][n_chunks] lowest index of the chunk max (greedy)
+    int32_t* counters;            // [2][max_batch] self-resetting tickets
+    double* row_info;             // [B][4]: max_p, sum_p, max_q, sum_q of row n (log2-scaled max)
+    double* chunk_mass;           // [B][n_chunks][2]: residual mass, p mass
+    int32_t* accepted_len;
+    int32_t* next_token;
+    double* dbg_p; double* dbg_q; float* dbg_u;   // [S] or null
+    int32_t* status;
+};
+
+struct Handle {
+    flexspec_config cfg;
+    int32_t d_model, max_m, max_s;
+    int32_t sm_count;
+    const __nv_bfloat16* w;
+    CUtensorMap w_map;
+    // workspace
+    __nv_bfloat16* attn_out;
+    float* logits;
+    float* part_o; float* part_ml;
+    Plan plan;
+    float2* stats; int32_t* arg_idx; int32_t* counters; double* row_info; double* chunk_mass;
+    double* dbg_p; double* dbg_q; float* dbg_u;
+    int32_t* status;
+    // host staging for flexspec_verify_host
+    void* stage_dev; size_t stage_bytes;
+    int32_t* out_dev;
+    // profiling
+    int32_t profiling, launches;
+    cudaEvent_t ev[kNumStageEvents];
+    int32_t ev_used[kNumStageEvents];
+};
+
+// launch wrappers (each returns a cudaError_t from the launch)
+cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
+                        Plan plan, int32_t* status, cudaStream_t stream);
+cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t batch,
+                             int32_t max_rows_per_seq, int32_t max_splits, cudaStream_t stream);
+cudaError_t launch_attention_combine(const CombineParams& p, int32_t batch, cudaStream_t stream);
+cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
+cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream);
+cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);
+
+cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
+cudaError_t lm_head_init();
+size_t lm_head_smem_bytes(int n_tile, int n_blocks, int num_stages);
+int lm_head_pick_stages(int n_tile, int n_blocks);
+
+}  // namespace fs

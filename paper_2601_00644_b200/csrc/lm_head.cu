@@ -1,0 +1,200 @@
+// Stage 2: LM-head projection logits[M][V] = X[M][d] . W[V][d]^T (the frozen head of the target,
+// Section IV-A; the scores of Algorithm 2, Step 2) on the 5th-generation tensor cores.
+//
+// The vocabulary is the large dimension and M (a few to a few hundred token rows) the small one,
+// so the operands are swapped: a 128-row tile of W is the MMA's A operand (M = 128) and the token
+// rows are its B operand (N = n_tile <= 256), both K-major bf16 staged by TMA with the 128-byte
+// swizzle.  The fp32 accumulator D[128 vocab rows][token columns] lives in TMEM; with lanes =
+// vocabulary rows, a warp's store of one token column is 32 consecutive floats of a logits row.
+//
+// Persistent CTAs (one per SM) walk over the vocabulary tiles.  Warp 0 is the TMA producer, warp 1
+// issues tcgen05.mma from one thread and owns the TMEM allocation, warps 2..5 drain the
+// accumulators.  Shared-memory stages and the (double-buffered, when it fits) accumulators are
+// handed over through mbarriers; every wait is bounded.
+//
+// W is streamed from HBM exactly once per pass; X (M x d bf16, L2 resident) is re-read per tile.
+#include "common.cuh"
+#include "internal.h"
+
+namespace fs {
+
+constexpr int kLmBlockV = 128;          // vocabulary rows per tile (MMA M)
+constexpr int kLmBlockK = 64;           // bf16 elements per 128-byte swizzle row
+constexpr int kLmUmmaK = 16;
+constexpr int kLmThreads = 192;
+constexpr int kLmMaxStages = 12;
+constexpr int kLmATileBytes = kLmBlockV * kLmBlockK * 2;     // 16 KB
+constexpr int kLmTmemCols = 512;
+constexpr int kLmSmemLimit = 232448;    // 227 KB opt-in maximum per CTA
+constexpr int kLmBarBytes = 512;
+
+static inline int lm_stage_bytes(int n_tile, int n_blocks) { return kLmATileBytes + n_blocks * n_tile * 128; }
+
+int lm_head_pick_stages(int n_tile, int n_blocks)
+{
+    int s = (kLmSmemLimit - 1024 - kLmBarBytes) / lm_stage_bytes(n_tile, n_blocks);
+    if (s > kLmMaxStages) s = kLmMaxStages;
+    return s;
+}
+size_t lm_head_smem_bytes(int n_tile, int n_blocks, int num_stages)
+{
+    return static_cast<size_t>(num_stages) * lm_stage_bytes(n_tile, n_blocks) + 1024 + kLmBarBytes;
+}
+
+__global__ void __launch_bounds__(kLmThreads, 1)
+lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
+               const LmHeadParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int b_bytes = p.n_blocks * p.n_tile * 128;
+    const int stage_bytes = kLmATileBytes + b_bytes;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + p.num_stages * stage_bytes);
+    uint64_t* empty_bar = full_bar + kLmMaxStages;
+    uint64_t* tmem_full = empty_bar + kLmMaxStages;
+    uint64_t* tmem_empty = tmem_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+        fence_barrier_init();
+        tma_prefetch_desc(&w_map);
+        tma_prefetch_desc(&x_map);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kLmTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int num_kb = p.d_model / kLmBlockK;
+    const int total_tiles = p.n_vtiles * p.n_pass;
+    const int acc_cols = p.n_blocks * p.n_tile;        // TMEM columns of one accumulator buffer
+    const int rows_per_pass = acc_cols;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t pol_w = l2_policy_evict_first();
+            const uint64_t pol_x = l2_policy_evict_last();
+            int s = 0;
+            uint32_t ph = 0;
+            int last_s = -1;
+            uint32_t last_ph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int vt = tile / p.n_pass, pass = tile % p.n_pass;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, p.status, 2)) { ok = false; break; }
+                    uint8_t* st = smem + s * stage_bytes;
+                    mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(stage_bytes));
+                    tma_load_2d(st, &w_map, &full_bar[s], kb * kLmBlockK, vt * kLmBlockV, pol_w);
+                    for (int nb = 0; nb < p.n_blocks; ++nb)
+                        tma_load_2d(st + kLmATileBytes + nb * p.n_tile * 128, &x_map, &full_bar[s], kb * kLmBlockK,
+                                    pass * rows_per_pass + nb * p.n_tile, pol_x);
+                    last_s = s; last_ph = ph;
+                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                }
+            }
+            // do not leave while a copy of ours may still be landing in shared memory
+            if (last_s >= 0) mbar_wait(&full_bar[last_s], last_ph, p.status, 3);
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(kLmBlockV, static_cast<uint32_t>(p.n_tile));
+            int s = 0;
+            uint32_t ph = 0;
+            int a = 0;
+            uint32_t aph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(&tmem_empty[a], aph ^ 1u, p.status, 4)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem_base + static_cast<uint32_t>(a * acc_cols);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[s], ph, p.status, 5)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+                    const uint32_t b_addr = a_addr + kLmATileBytes;
+                    for (int nb = 0; nb < p.n_blocks; ++nb) {
+#pragma unroll
+                        for (int k = 0; k < kLmBlockK / kLmUmmaK; ++k) {
+                            const uint64_t da = umma_desc_k_sw128(a_addr + k * kLmUmmaK * 2);
+                            const uint64_t db = umma_desc_k_sw128(b_addr + nb * p.n_tile * 128 + k * kLmUmmaK * 2);
+                            umma_bf16(acc + static_cast<uint32_t>(nb * p.n_tile), da, db, idesc,
+                                      (kb > 0 || k > 0) ? 1u : 0u);
+                        }
+                    }
+                    umma_commit(&empty_bar[s]);          // stage is free once these MMAs have read it
+                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                }
+                if (ok) umma_commit(&tmem_full[a]);      // accumulator complete
+                if (++a == p.acc_stages) { a = 0; aph ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (4 warps)
+        const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31
+        int a = 0;
+        uint32_t aph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int vt = tile / p.n_pass, pass = tile % p.n_pass;
+            if (!mbar_wait(&tmem_full[a], aph, p.status, 6)) { ok = false; break; }
+            tc_fence_after();
+            const int v = vt * kLmBlockV + quarter * 32 + lane;
+            const int row_base = pass * rows_per_pass;
+            const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                    static_cast<uint32_t>(a * acc_cols);
+            for (int c0 = 0; c0 < acc_cols; c0 += 16) {
+                if (row_base + c0 >= p.m_rows) break;    // warp-uniform
+                uint32_t r[16];
+                tmem_ld_x16(taddr0 + static_cast<uint32_t>(c0), r);
+                tmem_ld_wait();
+                if (v < p.vocab) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int row = row_base + c0 + i;
+                        if (row < p.m_rows)
+                            p.logits[static_cast<int64_t>(row) * p.vocab + v] = __uint_as_float(r[i]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty[a]);
+            if (++a == p.acc_stages) { a = 0; aph ^= 1u; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kLmTmemCols);
+    }
+}
+
+cudaError_t lm_head_init()
+{
+    return cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmemLimit);
+}
+
+cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream)
+{
+    const int total_tiles = p.n_vtiles * p.n_pass;
+    const int grid = total_tiles < h.sm_count ? total_tiles : h.sm_count;
+    const size_t smem = lm_head_smem_bytes(p.n_tile, p.n_blocks, p.num_stages);
+    lm_head_kernel<<<grid, kLmThreads, smem, stream>>>(h.w_map, x_map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace fs

@@ -1,0 +1,212 @@
+"""GPU parity of each stage in isolation, through the C ABI, against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2601_00644_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2601_00644_b200 import binding
+    return binding
+
+
+def _rand_bf16(gen, shape, std):
+    return (torch.randn(shape, generator=gen, device="cuda") * std).to(torch.bfloat16)
+
+
+# ------------------------------------------------------------------ LM head
+
+@pytest.mark.parametrize("m,d,v", [
+    (5, 512, 4096),          # the tiny config's shape
+    (1, 64, 128),            # smallest legal problem
+    (96, 1024, 5000),        # ragged last vocabulary tile (5000 = 39*128 + 8)
+    (100, 256, 777),         # vocab not a multiple of 4, rows not a multiple of 16
+    (300, 512, 1300),        # two accumulator blocks (single TMEM buffer)
+    (600, 256, 1000),        # two passes over W
+])
+def test_lm_head_matches_oracle(m, d, v):
+    B = _binding()
+    gen = torch.Generator(device="cuda").manual_seed(1000 + m)
+    x = _rand_bf16(gen, (m, d), 1.0)
+    w = _rand_bf16(gen, (v, d), 1.0)
+    hd = 64
+    ver = B.Verifier(w, d // hd, d // hd, hd, max_batch=max(m, 1), k_max=0, max_kv_len=16)
+    logits = torch.full((m, v), float("nan"), device="cuda")
+    ver.lm_head(x, logits)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    ref = oracle.lm_head(wl.bits_u16(x), wl.bits_u16(w))
+    got = logits.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    # fp32 accumulation of exact bf16 products: error ~ d * 2^-24 relative to sum |x||w|
+    bound = d * 2.0 ** -23 * (np.abs(oracle.bf16_to_f64(wl.bits_u16(x))) @ np.abs(oracle.bf16_to_f64(wl.bits_u16(w))).T)
+    assert np.all(np.abs(got - ref) <= bound + 1e-30)
+    assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
+    # run-to-run determinism
+    logits2 = torch.empty_like(logits)
+    ver.lm_head(x, logits2)
+    torch.cuda.synchronize()
+    assert torch.equal(logits, logits2)
+    ver.close()
+
+
+# ------------------------------------------------------------------ attention
+
+def _attn_parity(shape, tol=2e-2):
+    import tests.harness as H
+    case = H.Case(shape)
+    ver = H.make_verifier(case)
+    inp = case.inp
+    out = ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, inp.kv_len.cpu(), inp.hidden,
+                        inp.draft_len, inp.draft_len.cpu())
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    s = shape
+    a64, _ = oracle.attention(case.h_hidden, case.h_kv, case.h_pt, case.kv_len, case.k,
+                              s.n_q_heads, s.n_kv_heads, s.head_dim)
+    got = out.float().cpu().numpy()
+    row_err, ok = H.rel_close(got, a64, tol)
+    assert ok and row_err < tol, (row_err, ok)
+    out2 = ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, inp.kv_len.cpu(), inp.hidden,
+                         inp.draft_len, inp.draft_len.cpu())
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    ver.close()
+    return row_err
+
+
+def _shape(name, idx, **kw):
+    base = dict(batch=1, n_q_heads=8, n_kv_heads=2, head_dim=64, vocab=256, k_min=4, k_max=4,
+                ctx_min=128, ctx_max=128, sigma_min=0.5, sigma_max=0.5)
+    base.update(kw)
+    return wl.VerifyShape(name=name, index=idx, **base)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),                                                              # tiny config: one split
+    dict(input_std=1.0),                                                 # peaked scores
+    dict(batch=5, k_min=0, k_max=12, ctx_min=1, ctx_max=700),            # ragged, several splits, k=0
+    dict(batch=3, n_q_heads=32, n_kv_heads=8, head_dim=128, k_min=5, k_max=5, ctx_min=2048,
+         ctx_max=2048, input_std=1.0),                                   # 8B heads
+    dict(batch=2, n_q_heads=64, n_kv_heads=8, head_dim=128, k_min=8, k_max=8, ctx_min=1000,
+         ctx_max=1300, input_std=1.0),                                   # 70B heads: 72 rows per kv head
+    dict(batch=2, n_q_heads=32, n_kv_heads=8, head_dim=128, k_min=16, k_max=16, ctx_min=5000,
+         ctx_max=6000, input_std=1.0),                                   # 68 rows, long context
+    dict(batch=2, n_q_heads=16, n_kv_heads=1, head_dim=64, k_min=9, k_max=10, ctx_min=0,
+         ctx_max=40, input_std=1.0),                                     # 176 rows per kv head: two row blocks
+    dict(batch=4, n_q_heads=4, n_kv_heads=4, head_dim=128, k_min=1, k_max=3, ctx_min=0, ctx_max=3,
+         input_std=1.0),                                                 # plain MHA, almost no context
+])
+def test_attention_matches_oracle(kw):
+    _attn_parity(_shape("attn_case", 100 + len(kw), **kw))
+
+
+# ------------------------------------------------------------------ decision stage
+
+def _sample_case(seed, batch, vocab, k_lo, k_hi, mode, temperature, logit_std=3.0, holes=False, mask=False):
+    rng = np.random.RandomState(seed)
+    k = rng.randint(k_lo, k_hi + 1, batch).astype(np.int32)
+    m, s = int(k.sum()) + batch, int(k.sum())
+    zt = (rng.standard_normal((m, vocab)) * logit_std).astype(np.float32)
+    zd = (rng.standard_normal((s, vocab)) * logit_std).astype(np.float32)
+    # make the draft resemble the target so that acceptances and rejections both occur
+    r0 = np.concatenate([[0], np.cumsum(k + 1)]); t0 = np.concatenate([[0], np.cumsum(k)])
+    for b in range(batch):
+        zd[t0[b]:t0[b + 1]] = zt[r0[b]:r0[b] + k[b]] + 0.7 * zd[t0[b]:t0[b + 1]] / logit_std
+    if holes:
+        zd[rng.rand(s, vocab) < 0.1] = -np.inf
+        zt[rng.rand(m, vocab) < 0.05] = -np.inf
+        zt[:, 0] = 1e4 * (rng.rand(m) < 0.1)                # a few rows with one huge logit
+    q = torch.softmax(torch.from_numpy(zd).double() / max(temperature, 1e-3), -1).numpy() if s else np.zeros((0, vocab))
+    toks = np.array([rng.choice(vocab, p=q[i] / q[i].sum()) for i in range(s)], np.int32)
+    if mode == 1:      # greedy: make most drafts the arg-max so that prefixes get accepted
+        am = np.concatenate([zt[r0[b]:r0[b] + k[b]].argmax(-1) for b in range(batch)]) if s else toks
+        toks = np.where(rng.rand(s) < 0.7, am, toks).astype(np.int32)
+    seeds = rng.randint(0, 2 ** 62, batch).astype(np.uint64)
+    vmask = None
+    if mask:
+        vmask = rng.randint(0, 2 ** 32, (batch, (vocab + 31) // 32), dtype=np.uint64).astype(np.uint32)
+        vmask[:, 0] |= 1
+    return k, zt, zd, toks, seeds, vmask
+
+
+@pytest.mark.parametrize("mode,temperature", [(0, 1.0), (0, 0.7), (1, 1.0), (0, 0.0)])
+@pytest.mark.parametrize("vocab,batch,k_hi,holes,mask", [
+    (4096, 3, 4, False, False),
+    (777, 9, 7, True, False),            # vocab % 4 != 0, -inf entries, huge logits
+    (20000, 16, 12, False, True),        # several chunks with a ragged last one, vocabulary mask
+    (8192 * 2 + 1, 5, 33, False, False), # k > 32: two ballot rounds
+])
+def test_sample_stage_matches_oracle(mode, temperature, vocab, batch, k_hi, holes, mask):
+    B = _binding()
+    k, zt, zd, toks, seeds, vmask = _sample_case(vocab + batch, batch, vocab, 0, k_hi, mode, temperature,
+                                                 holes=holes, mask=mask)
+    greedy = (mode == 1 or temperature == 0.0)
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=max(k_hi, 1), max_kv_len=64, mode=mode, debug=True)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).cuda()
+    zt_d, zd_d = dev(zt, torch.float32), dev(zd, torch.float32)
+    toks_d = dev(toks, torch.int32)
+    k_d = dev(k, torch.int32)
+    seeds_d = dev(seeds.view(np.int64), torch.int64)
+    vm_d = None if vmask is None else dev(vmask.view(np.int32), torch.int32)
+    outs = []
+    for _ in range(2):                   # twice: the self-resetting tickets must be reusable
+        acc, nxt = ver.sample(zt_d, toks_d, zd_d, k_d, k_d.cpu(), seeds_d, temperature=temperature, vocab_mask=vm_d)
+        torch.cuda.synchronize()
+        assert ver.status()[0] == 0
+        outs.append((acc.cpu().numpy(), nxt.cpu().numpy()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    acc, nxt = outs[0]
+    ref = oracle.accept(1 if greedy else 0, zt.astype(np.float64), zd, toks, k, seeds,
+                        temperature if not greedy else 1.0, vmask)
+    t0 = np.concatenate([[0], np.cumsum(k)])
+    n_ties = 0
+    for b in range(batch):
+        if acc[b] != ref["accepted_len"][b]:
+            assert not greedy
+            j = min(acc[b], ref["accepted_len"][b])
+            assert ref["acc_margin"][t0[b] + j] < 1e-5
+            n_ties += 1
+            continue
+        if nxt[b] != ref["next_token"][b]:
+            assert not greedy and ref["cdf_margin"][b] < 1e-9, (b, nxt[b], ref["next_token"][b], ref["cdf_margin"][b])
+    assert n_ties <= 1
+    if not greedy and k.sum() > 0:
+        dbg = ver.debug(int(k.sum()) + batch, int(k.sum()))
+        assert np.abs(dbg["p_tok"].cpu().numpy() - ref["p_tok"]).max() < 1e-5
+        assert np.abs(dbg["q_tok"].cpu().numpy() - ref["q_tok"]).max() < 1e-5
+        assert np.array_equal(dbg["u"].cpu().numpy().astype(np.float64), ref["u"])
+    ver.close()
+
+
+def test_sample_invariants_on_gpu():
+    """p == q accepts every draft; a draft outside the target's support is rejected at 0."""
+    B = _binding()
+    vocab, batch, kk = 5000, 6, 5
+    rng = np.random.RandomState(5)
+    k = np.full(batch, kk, np.int32)
+    zt = (rng.standard_normal((batch * (kk + 1), vocab)) * 2).astype(np.float32)
+    zd = zt.reshape(batch, kk + 1, vocab)[:, :kk].reshape(-1, vocab).copy()
+    toks = rng.randint(0, vocab, batch * kk).astype(np.int32)
+    seeds = rng.randint(0, 2 ** 62, batch).astype(np.int64)
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=kk, max_kv_len=64)
+    t = lambda a, dt: torch.from_numpy(a).to(dt).cuda()
+    acc, nxt = ver.sample(t(zt, torch.float32), t(toks, torch.int32), t(zd, torch.float32), t(k, torch.int32),
+                          torch.from_numpy(k), t(seeds, torch.int64), temperature=0.7)
+    assert np.all(acc.cpu().numpy() == kk)
+    # disjoint support through the vocabulary mask: drafts live on masked tokens only
+    toks2 = (rng.randint(0, vocab // 2, batch * kk) * 2 + 1).astype(np.int32)          # odd ids
+    words = (vocab + 31) // 32
+    mask = np.full((batch, words), 0x55555555, np.uint32)                               # even ids allowed
+    acc, nxt = ver.sample(t(zt, torch.float32), t(toks2, torch.int32), t(zd, torch.float32), t(k, torch.int32),
+                          torch.from_numpy(k), t(seeds, torch.int64), temperature=0.7,
+                          vocab_mask=t(mask.view(np.int32), torch.int32))
+    assert np.all(acc.cpu().numpy() == 0)
+    assert np.all(nxt.cpu().numpy() % 2 == 0)
+    ver.close()

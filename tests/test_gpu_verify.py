@@ -1,0 +1,192 @@
+"""GPU parity of the whole verification step (flexspec_verify through the C ABI) against the
+oracle: reduced cases compared on every sequence, the full-size configs on a subset of whole
+sequences (sequences are independent) plus properties that hold for all of them."""
+import math
+
+import numpy as np
+import pytest
+import scipy.stats
+import torch
+
+from paper_2601_00644_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _H():
+    import tests.harness as H
+    return H
+
+
+def _run(shape, check=None, mode=0, e2e_cdf_tol=1e-6):
+    H = _H()
+    case = H.Case(shape, check_seqs=check, mode=mode)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    rep = H.full_parity(case, ver, e2e_cdf_tol=e2e_cdf_tol)
+    # same call again: identical outputs (tickets reset, no stale state)
+    acc2, nxt2 = H.run_gpu_verify(case, ver)
+    assert np.array_equal(acc2, rep["accepted_len"]) and np.array_equal(nxt2, rep["next_token"])
+    ver.close()
+    return case, rep
+
+
+def test_tiny_config_every_mode():
+    shape = wl.CONFIGS["tiny"]
+    case, rep = _run(shape)
+    assert rep["e2e_ties"] == 0
+    _run(shape, mode=1)
+    _run(wl.peaked(shape))
+
+
+def test_reduced_8b_shape_flat_and_peaked():
+    base = wl.scaled(wl.CONFIGS["llama3_8b"], batch=3, vocab=20000, ctx_min=700, ctx_max=700, index=11)
+    case, rep = _run(base)
+    assert rep["e2e_ties"] + rep["e2e_cdf_ties"] <= 1
+    # peaked logits: the bf16 rounding of the attention output moves the logits by ~1e-2, so
+    # end-to-end decisions may legitimately differ; the isolated comparison stays exact
+    H = _H()
+    pk = wl.peaked(base)
+    case = H.Case(pk)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    acc, nxt = H.run_gpu_verify(case, ver)
+    dbg = ver.debug(case.inp.m_rows, case.inp.s_rows)
+    a64, a16, logits_o = case.oracle_front()
+    err, ok = H.rel_close(dbg["logits"].cpu().numpy(), logits_o)
+    assert ok and err < H.REL_TOL
+    ref_iso = case.oracle_accept(dbg["logits"].cpu().numpy().astype(np.float64))
+    H.compare_decisions(case, acc, nxt, ref_iso, H.CDF_TIE_TOL, "isolated/peaked")
+    assert np.abs(dbg["p_tok"].cpu().numpy() - ref_iso["p_tok"]).max() < H.PROB_TOL
+    ver.close()
+
+
+def test_ragged_batch_with_k0_and_greedy():
+    shape = wl.scaled(wl.CONFIGS["adaptive_k"], batch=7, vocab=9000, k_min=0, k_max=12, ctx_min=30,
+                      ctx_max=900, index=12)
+    _run(shape)
+    _run(shape, mode=1)
+
+
+def test_degenerate_cases_p_equals_q_and_disjoint_support():
+    """Long-context config's sub-cases on a reduced shape: a sequence whose draft logits are the
+    target's own (every draft accepted) and one whose drafts lie outside the target's support
+    (rejected at position 0, emitted token from p)."""
+    H = _H()
+    shape = wl.scaled(wl.CONFIGS["long_ctx"], batch=3, vocab=12000, ctx_min=3000, ctx_max=3000,
+                      k_min=6, k_max=6, index=13)
+    case = H.Case(shape)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    inp = case.inp
+    # phase 1: the GPU's own target logits
+    ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, inp.kv_len.cpu(), inp.hidden,
+                  inp.draft_len, inp.draft_len.cpu(), attn_out=None)
+    attn = ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, inp.kv_len.cpu(), inp.hidden,
+                         inp.draft_len, inp.draft_len.cpu())
+    logits = ver.lm_head(attn)
+    kk = 6
+    # sequence 0: q == p bit for bit
+    case.draft_logits[case.tok0[0]:case.tok0[0] + kk] = logits[case.row0[0]:case.row0[0] + kk]
+    # sequence 1: drafts on odd ids, the target restricted to even ids
+    case.draft_tokens[case.tok0[1]:case.tok0[1] + kk] = torch.tensor([1, 3, 5, 7, 9, 11], dtype=torch.int32, device="cuda")
+    words = (shape.vocab + 31) // 32
+    mask = np.full((3, words), 0xFFFFFFFF, np.uint32)
+    mask[1] = 0x55555555
+    mask_dev = torch.from_numpy(mask.view(np.int32)).cuda()
+    acc, nxt = H.run_gpu_verify(case, ver, vocab_mask_dev=mask_dev)
+    assert acc[0] == kk
+    assert acc[1] == 0 and nxt[1] % 2 == 0
+    # oracle on the same inputs (its own logits; masks applied identically)
+    case.vocab_mask = mask
+    _, _, logits_o = case.oracle_front()
+    ref = case.oracle_accept(logits_o)
+    assert ref["accepted_len"][1] == 0 and ref["next_token"][1] % 2 == 0
+    ref_iso = case.oracle_accept(logits.cpu().numpy().astype(np.float64))
+    assert ref_iso["accepted_len"][0] == kk
+    H.compare_decisions(case, acc, nxt, ref_iso, H.CDF_TIE_TOL, "degenerate")
+    ver.close()
+
+
+def test_bad_inputs_are_reported_not_faulted():
+    H = _H()
+    from paper_2601_00644_b200 import binding as B
+    shape = wl.scaled(wl.CONFIGS["tiny"], index=14)
+    case = H.Case(shape)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    inp = case.inp
+    args = dict(kv_pages=inp.kv_pages, page_table=inp.page_table, kv_len=inp.kv_len, kv_len_host=inp.kv_len.cpu(),
+                hidden=inp.hidden, draft_tokens=case.draft_tokens, draft_logits=case.draft_logits,
+                draft_len=inp.draft_len, draft_len_host=inp.draft_len.cpu(), seeds=inp.seeds)
+    # host-side rejections
+    with pytest.raises(B.FlexSpecError) as e:
+        ver.verify(**{**args, "draft_len_host": torch.tensor([9], dtype=torch.int32)})
+    assert e.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.FlexSpecError):
+        ver.verify(**{**args, "kv_len_host": torch.tensor([2], dtype=torch.int32)})
+    with pytest.raises(B.FlexSpecError):
+        ver.verify(**{**args, "draft_logits": None})
+    with pytest.raises(B.FlexSpecError):
+        ver.verify(**{**args, "temperature": -1.0})
+    # device-side: a page id outside the pool is reported through the status word, no fault
+    bad_pt = inp.page_table.clone()
+    bad_pt[0, 1] = inp.kv_pages.shape[0] + 5
+    ver.verify(**{**args, "page_table": bad_pt})
+    torch.cuda.synchronize()
+    code, st = ver.status()
+    assert code == B.ERR_BAD_PAGE and st[1] == inp.kv_pages.shape[0] + 5
+    # a token id outside the vocabulary
+    bad_tok = case.draft_tokens.clone()
+    bad_tok[2] = shape.vocab + 3
+    ver.verify(**{**args, "draft_tokens": bad_tok})
+    torch.cuda.synchronize()
+    code, st = ver.status()
+    assert code == B.ERR_BAD_TOKEN
+    # the handle is still usable
+    acc, nxt = H.run_gpu_verify(case, ver)
+    assert 0 <= acc[0] <= 4
+    ver.close()
+
+
+def test_verify_host_entry_matches_device_entry():
+    H = _H()
+    shape = wl.scaled(wl.CONFIGS["llama3_8b"], batch=4, vocab=6000, ctx_min=300, ctx_max=400, index=15)
+    case = H.Case(shape)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    acc, nxt = H.run_gpu_verify(case, ver)
+    inp = case.inp
+    pin = lambda t: t.cpu().pin_memory()
+    acc_h = torch.empty(case.batch, dtype=torch.int32).pin_memory()
+    nxt_h = torch.empty(case.batch, dtype=torch.int32).pin_memory()
+    ver.verify_host(inp.kv_pages, inp.page_table, inp.kv_len.cpu(), pin(inp.hidden), pin(case.draft_tokens),
+                    pin(case.draft_logits), pin(inp.draft_len), pin(inp.seeds), acc_h, nxt_h,
+                    temperature=shape.temperature)
+    assert np.array_equal(acc_h.numpy(), acc) and np.array_equal(nxt_h.numpy(), nxt)
+    ver.close()
+
+
+# ------------------------------------------------------------------ full-size configs
+
+@pytest.mark.parametrize("name,check", [
+    ("llama3_8b", [0, 7, 15]),
+    ("adaptive_k", [1, 20, 41, 63]),
+    ("llama3_70b", [3, 30]),
+    ("long_ctx", [2, 6]),
+])
+def test_full_config_subset_parity_and_properties(name, check):
+    shape = wl.CONFIGS[name]
+    case, rep = _run(shape, check=check)
+    acc = rep["accepted_len"]
+    k = case.k
+    assert np.all((acc >= 0) & (acc <= k))
+    assert np.all((rep["next_token"] >= 0) & (rep["next_token"] < shape.vocab))
+    # per-position acceptance follows the flat-target closed form 2*Phi(-sigma/(2T)):
+    # position j is reached iff all earlier ones were accepted, so count tests actually taken
+    sig = case.inp.sigma.cpu().numpy()
+    taken = np.minimum(acc + 1, k).sum()
+    accepted = acc.sum()
+    want = float(np.sum(np.minimum(acc + 1, k) * 2 * scipy.stats.norm.cdf(-sig / (2 * shape.temperature))) / max(taken, 1))
+    assert abs(accepted / max(taken, 1) - want) < 5 * math.sqrt(0.25 / max(taken, 1)) + 0.02
+    assert rep["e2e_ties"] + rep["e2e_cdf_ties"] <= 1
