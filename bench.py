@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the cloud-side verification step (Algorithm 2, Step 2) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+A step is one flexspec_verify call (plan + attention [+ split merge] + LM head + acceptance /
+emitted token) over one batch of seeded synthetic input.  The default workload is the
+Llama-3-8B-shaped config (B=16, k=5, context 2048, V=128256).  Prints ONE JSON line.
+
+N > 1 (torchrun, one rank per GPU): sequences are independent, so every rank verifies its own
+batch against its own replica of the LM head; there is no data-path collective (weak scaling).
+`--impl reference` times the fp64 CPU oracle on the host cores over a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch at the default
+# workload, from the ncu capture summarised in profiles/ (None until captured)
+LM_HEAD_TRAFFIC_BYTES = None
+FALLBACK_HBM_GBS = 6650.0
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+# ------------------------------------------------------------------------------ reference arm
+def run_reference(args):
+    """The oracle as it stands, on the host cores: each step verifies `sample` whole sequences
+    of the workload (attention -> bf16 -> LM head -> acceptance), fp64."""
+    rank, _, world = _dist_env()
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2601_00644_b200 import workloads as wl
+    shape = wl.CONFIGS[args.config]
+    n_seq = 1
+    small = wl.scaled(shape, batch=n_seq)            # same shape, a sample of whole sequences
+    inp = wl.make_inputs(small, device="cpu")
+    k = inp.draft_len.numpy()
+    hid, kvp, w = wl.bits_u16(inp.hidden), wl.bits_u16(inp.kv_pages), wl.bits_u16(inp.lm_head_w)
+    pt, kvl, seeds = inp.page_table.numpy(), inp.kv_len.numpy(), wl.seeds_u64(inp.seeds)
+    noise = inp.noise.numpy()
+    toks = wl.draw_draft_tokens(inp.noise, shape.temperature, inp.token_uniforms).numpy()
+
+    def step():
+        return oracle.verify(oracle.SAMPLE, hid, kvp, pt, kvl, k, w, toks, noise, seeds,
+                             shape.n_q_heads, shape.n_kv_heads, shape.head_dim, 16, shape.temperature)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    verified = 0
+    for _ in range(args.steps):
+        res = step()
+        verified += int(res["accepted_len"].sum()) + n_seq
+    dt = time.perf_counter() - t0
+    value = verified / dt
+    cores = oracle.num_threads()
+    sample = f"{n_seq} of {shape.batch} sequences of '{shape.name}' per step (whole sequences, k={int(k[0])})"
+    line = {
+        "impl": "reference", "metric": "verified_tokens_per_s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ our arm
+def cpu_baseline(shape, seconds_target=12.0):
+    """Oracle timed on the host cores over a bounded sample of whole sequences."""
+    import numpy as np
+    import oracle
+    from paper_2601_00644_b200 import workloads as wl
+    small = wl.scaled(shape, batch=1)
+    inp = wl.make_inputs(small, device="cpu")
+    k = inp.draft_len.numpy()
+    toks = wl.draw_draft_tokens(inp.noise, shape.temperature, inp.token_uniforms).numpy()
+    args = (wl.bits_u16(inp.hidden), wl.bits_u16(inp.kv_pages), inp.page_table.numpy(), inp.kv_len.numpy(), k,
+            wl.bits_u16(inp.lm_head_w), toks, inp.noise.numpy(), wl.seeds_u64(inp.seeds),
+            shape.n_q_heads, shape.n_kv_heads, shape.head_dim, 16, shape.temperature)
+    t0 = time.perf_counter()
+    reps, verified = 0, 0
+    while True:
+        res = oracle.verify(oracle.SAMPLE, *args)
+        verified += int(res["accepted_len"].sum()) + 1
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt > seconds_target or reps >= 8:
+            break
+    return {"value": verified / dt, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{reps} x 1 of {shape.batch} sequences of '{shape.name}' (whole sequences), {dt:.1f} s"}
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2601_00644_b200 import binding, workloads as wl
+
+    rank, local_rank, world = _dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    shape = wl.CONFIGS[args.config]
+    if world > 1:
+        shape = wl.scaled(shape, index=shape.index + 100 * rank)        # every rank its own batch
+    inp = wl.make_inputs(shape, device=str(dev))
+    k_host, kv_host = inp.draft_len.cpu(), inp.kv_len.cpu()
+    batch, m_rows, s_rows = inp.batch, inp.m_rows, inp.s_rows
+    ver = binding.Verifier(inp.lm_head_w, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                           max_batch=batch, k_max=int(k_host.max()), max_kv_len=int(kv_host.max()))
+
+    # draft logits = target logits (from this library's attention + LM head) + sigma * noise
+    attn = ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, kv_host, inp.hidden, inp.draft_len, k_host)
+    tgt = ver.lm_head(attn)
+    row0, tok0 = inp.row_offsets(), inp.tok_offsets()
+    draft_logits = inp.noise
+    for b in range(batch):
+        kb = int(k_host[b])
+        draft_logits[tok0[b]:tok0[b] + kb] += tgt[row0[b]:row0[b] + kb]
+    del tgt, attn
+    draft_tokens = wl.draw_draft_tokens(draft_logits, shape.temperature, inp.token_uniforms)
+    acc = torch.empty(batch, dtype=torch.int32, device=dev)
+    nxt = torch.empty(batch, dtype=torch.int32, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)       # 4x the 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    def step():
+        ver.verify(inp.kv_pages, inp.page_table, inp.kv_len, kv_host, inp.hidden, draft_tokens, draft_logits,
+                   inp.draft_len, k_host, inp.seeds, temperature=shape.temperature,
+                   accepted_len=acc, next_token=nxt, stream=stream)
+
+    def flush_l2():
+        flush.view(torch.int64).sum()                                   # read-only sweep: leaves clean lines
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush_l2(); step()
+    barrier()
+    code, st = ver.status()
+    if code != 0:
+        raise RuntimeError(f"device status {code} {st}")
+    launches_per_step = ver.last_launches()
+
+    # ---- timed region: K steps, each bracketed by CUDA events on the launching stream; the L2
+    # sweep between steps is outside the event pairs
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush_l2()
+        starts[i].record(stream)
+        step()
+        ends[i].record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    total_ms = sum(step_ms)
+    verified = int(acc.sum().item()) + batch                              # tau + 1 tokens per sequence
+    accept_rate = float(acc.sum().item()) / max(1, s_rows)
+
+    # ---- per-kernel durations (second loop, events between the kernels inside the library)
+    ver.set_profiling(True)
+    stage_acc = np.zeros(6)
+    n_prof = min(args.steps, 20)
+    for _ in range(n_prof):
+        flush_l2(); step()
+        stage_acc += np.array(ver.stage_ms())
+    ver.set_profiling(False)
+    stage_ms = (stage_acc / n_prof).tolist()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host-buffer entry point (H2D of the step's inputs, D2H of results)
+    pin = lambda t: t.cpu().pin_memory()
+    h_hidden, h_tok, h_dlog = pin(inp.hidden), pin(draft_tokens), pin(draft_logits)
+    h_len, h_seeds = pin(inp.draft_len), pin(inp.seeds)
+    h_acc = torch.empty(batch, dtype=torch.int32).pin_memory()
+    h_nxt = torch.empty(batch, dtype=torch.int32).pin_memory()
+
+    def step_host():
+        ver.verify_host(inp.kv_pages, inp.page_table, kv_host, h_hidden, h_tok, h_dlog, h_len, h_seeds,
+                        h_acc, h_nxt, temperature=shape.temperature, stream=stream)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        step_host()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        step_host()
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    h2d = h_hidden.numel() * 2 + h_tok.numel() * 4 + h_dlog.numel() * 4 + h_len.numel() * 4 * 2 + h_seeds.numel() * 8
+    d2h = 2 * batch * 4
+    assert torch.equal(h_acc.to(dev), acc) and torch.equal(h_nxt.to(dev), nxt)
+
+    # ---- reduce over ranks: max time, summed tokens
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_s = float(t[0]), float(t[1])
+        v = torch.tensor([verified], dtype=torch.float64, device=dev)
+        dist.all_reduce(v, op=dist.ReduceOp.SUM)
+        verified_all = float(v[0])
+    else:
+        verified_all = float(verified)
+    ms_per_step = total_ms / args.steps
+
+    if rank == 0:
+        peak, peak_kind = _peaks()
+        d, v = shape.d_model, shape.vocab
+        kv_bytes = int(kv_host.sum()) * shape.n_kv_heads * shape.head_dim * 2 * 2
+        alg_bytes = v * d * 2 + kv_bytes + 3 * m_rows * d * 2 + s_rows * v * 4
+        lm_bytes = v * d * 2                                             # 2*d bytes per vocabulary row
+        lm_ms = stage_ms[3]
+        achieved = lm_bytes / (lm_ms * 1e-3) / 1e9 if lm_ms > 0 else 0.0
+        line = {
+            "metric": "verified_tokens_per_s", "value": verified_all / (ms_per_step * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": shape.name, "batch_per_gpu": batch, "k": [int(k_host.min()), int(k_host.max())],
+                       "context": [shape.ctx_min, shape.ctx_max], "vocab": v, "d_model": d,
+                       "heads": [shape.n_q_heads, shape.n_kv_heads, shape.head_dim],
+                       "temperature": shape.temperature, "mode": "sample",
+                       "l2": "read sweep of a 512 MiB buffer between steps, outside the event pairs"},
+            "step_us": ms_per_step * 1e3,
+            "step_us_median": statistics.median(step_ms) * 1e3,
+            "scored_positions_per_s": world * m_rows / (ms_per_step * 1e-3),
+            "mean_acceptance": accept_rate,
+            "algorithmic_bytes_per_step": alg_bytes,
+            "hbm_roofline_frac_of_8TBs": alg_bytes / (ms_per_step * 1e-3) / 8e12,
+            "hbm_roofline_frac_of_measured": alg_bytes / (ms_per_step * 1e-3) / (peak * 1e9),
+            "stage_us": {"plan": stage_ms[0] * 1e3, "attention": stage_ms[1] * 1e3,
+                         "attention_combine": stage_ms[2] * 1e3, "lm_head": stage_ms[3] * 1e3,
+                         "sample_stats": stage_ms[4] * 1e3, "sample_draw": stage_ms[5] * 1e3},
+            "roofline": {"kernel": "lm_head_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                         "traffic": LM_HEAD_TRAFFIC_BYTES, "algorithmic_bytes": lm_bytes},
+            "e2e": {"value": verified_all / e2e_s, "unit": "tokens/s", "ms_per_step": e2e_s * 1e3,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "note": "flexspec_verify_host: per-step inputs from pinned host memory; KV pool and W resident"},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+            "wall_s_timed_region": t_wall,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl.CONFIGS[args.config])
+        print(json.dumps(line))
+    ver.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default="llama3_8b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
