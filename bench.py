@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch at the default
 # workload, from the ncu capture summarised in profiles/ (None until captured)
-LM_HEAD_TRAFFIC_BYTES = None
+LM_HEAD_TRAFFIC_BYTES = 1051598000 + 7260672
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -317,7 +317,7 @@ def run_ours(args):
             "step_us": ms_per_step * 1e3,
             "step_us_median": statistics.median(step_ms) * 1e3,
             "scored_positions_per_s": world * m_rows / (ms_per_step * 1e-3),
-            "mean_acceptance": accept_rate,
+            "mean_tau_over_k": accept_rate,
             "algorithmic_bytes_per_step": alg_bytes,
             "hbm_roofline_frac_of_8TBs": alg_bytes / (ms_per_step * 1e-3) / 8e12,
             "hbm_roofline_frac_of_measured": alg_bytes / (ms_per_step * 1e-3) / (peak * 1e9),
@@ -345,7 +345,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="llama3_8b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
