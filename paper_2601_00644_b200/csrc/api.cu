@@ -77,6 +77,7 @@ void free_workspace(Handle& h)
 {
     cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml);
     cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq);
+    cudaFree(h.plan.seq_blk0); cudaFree(h.plan.seq_pair0); cudaFree(h.plan.cta_start);
     cudaFree(h.stats); cudaFree(h.arg_idx); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.chunk_mass);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
@@ -87,7 +88,8 @@ void free_workspace(Handle& h)
 // geometry of one call, derived from the host copies of the lengths
 struct Geometry {
     int32_t m_rows = 0, s_rows = 0, k_batch_max = 0, kv_max = 0;
-    int64_t kv_total = 0;
+    int64_t att_blocks = 0;      // attention work blocks (128 tokens of one pair), as the plan kernel counts them
+    int32_t att_ctas = 0;
 };
 
 int check_lengths(const Handle& h, const int32_t* draft_len_host, const int32_t* kv_len_host, int32_t batch,
@@ -105,9 +107,14 @@ int check_lengths(const Handle& h, const int32_t* draft_len_host, const int32_t*
             if (l < k + 1 || l > h.cfg.max_kv_len) return FLEXSPEC_ERR_INVALID_ARG;
             if ((l + h.cfg.page_size - 1) / h.cfg.page_size > max_pages_per_seq) return FLEXSPEC_ERR_INVALID_ARG;
             if (l > g->kv_max) g->kv_max = l;
-            g->kv_total += l;
+            const int group = h.cfg.n_q_heads / h.cfg.n_kv_heads;
+            const int64_t pairs = static_cast<int64_t>(h.cfg.n_kv_heads) *
+                                  ((group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
+            g->att_blocks += pairs * ((l + kAttBlockTokens - 1) / kAttBlockTokens);
         }
     }
+    if (g->att_blocks > 0x7fffffffLL) return FLEXSPEC_ERR_UNSUPPORTED;
+    g->att_ctas = static_cast<int32_t>(g->att_blocks < h.sm_count ? g->att_blocks : h.sm_count);
     return FLEXSPEC_OK;
 }
 
@@ -116,9 +123,11 @@ void mark(Handle& h, int idx, cudaStream_t s)
     if (h.profiling) { cudaEventRecord(h.ev[idx], s); h.ev_used[idx] = 1; }
 }
 
-int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, cudaStream_t s)
+int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, const int32_t* kv_len,
+             const Geometry& g, int32_t batch, cudaStream_t s)
 {
-    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, h.plan, h.status, s) != cudaSuccess)
+    if (launch_plan(draft_len, draft_tokens, kv_len, batch, h.cfg.vocab, h.cfg.n_kv_heads,
+                    h.cfg.n_q_heads / h.cfg.n_kv_heads, g.att_ctas, h.plan, h.status, s) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
     h.launches++;
     return FLEXSPEC_OK;
@@ -135,17 +144,8 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     int rc = make_map_2d(&kv_map, kv->kv_pages, pool_rows, static_cast<uint64_t>(c.head_dim), 16);
     if (rc != FLEXSPEC_OK) return rc;
 
-    // split the KV range so that about three CTAs' worth of work exists per SM
     const int max_tile_rows = group * (g.k_batch_max + 1);
-    const int row_blocks = (max_tile_rows + 127) / 128;
-    const int64_t units = g.kv_total * c.n_kv_heads * row_blocks;
-    int64_t split_len = (units + 3LL * h.sm_count - 1) / (3LL * h.sm_count);
-    split_len = (split_len + kAttSplitQuantum - 1) / kAttSplitQuantum * kAttSplitQuantum;
-    if (split_len < 2 * kAttSplitQuantum) split_len = 2 * kAttSplitQuantum;
-    int64_t min_len = (static_cast<int64_t>(g.kv_max) + kAttMaxSplits - 1) / kAttMaxSplits;
-    min_len = (min_len + kAttSplitQuantum - 1) / kAttSplitQuantum * kAttSplitQuantum;
-    if (split_len < min_len) split_len = min_len;
-    const int max_splits = static_cast<int>((g.kv_max + split_len - 1) / split_len);
+    const int n_cw = attention_consumer_warps(max_tile_rows);
 
     AttnParams p;
     p.hidden = static_cast<const __nv_bfloat16*>(hidden);
@@ -153,28 +153,27 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     p.kv_len = kv->kv_len;
     p.draft_len = draft_len;
     p.cu_q = h.plan.cu_q;
+    p.seq_blk0 = h.plan.seq_blk0; p.seq_pair0 = h.plan.seq_pair0; p.cta_start = h.plan.cta_start;
+    p.batch = batch;
     p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = group;
     p.max_pages_per_seq = kv->max_pages_per_seq; p.num_pages = kv->num_pages;
-    p.split_len = static_cast<int32_t>(split_len);
-    p.row_blocks = row_blocks;
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(c.head_dim)));
     p.part_o = h.part_o; p.part_ml = h.part_ml;
-    p.part_stride = static_cast<int64_t>(h.max_m) * c.n_q_heads;
-    p.attn_out = static_cast<__nv_bfloat16*>(attn_out);
     p.status = h.status;
-    if (launch_attention(h, kv_map, p, batch, g.k_batch_max + 1, max_splits, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_attention(h, kv_map, p, g.att_ctas, n_cw, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 2, s);
-    if (max_splits > 1) {
-        CombineParams cp;
-        cp.part_o = h.part_o; cp.part_ml = h.part_ml; cp.part_stride = p.part_stride;
-        cp.kv_len = kv->kv_len; cp.draft_len = draft_len; cp.cu_q = h.plan.cu_q;
-        cp.split_len = p.split_len; cp.rows_per_seq_max = g.k_batch_max + 1;
-        cp.n_q_heads = c.n_q_heads; cp.head_dim = c.head_dim;
-        cp.attn_out = p.attn_out;
-        if (launch_attention_combine(cp, batch, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-        h.launches++;
-    }
+    CombineParams cp;
+    cp.part_o = h.part_o; cp.part_ml = h.part_ml;
+    cp.kv_len = kv->kv_len; cp.draft_len = draft_len; cp.cu_q = h.plan.cu_q;
+    cp.seq_blk0 = h.plan.seq_blk0; cp.seq_pair0 = h.plan.seq_pair0;
+    cp.batch = batch; cp.n_q_heads = c.n_q_heads; cp.n_kv_heads = c.n_kv_heads; cp.group = group;
+    cp.head_dim = c.head_dim;
+    cp.n_ctas = g.att_ctas; cp.n_cw = n_cw;
+    cp.pairs_per_seq_max = c.n_kv_heads * ((max_tile_rows + kAttRowsPerPair - 1) / kAttRowsPerPair);
+    cp.attn_out = static_cast<__nv_bfloat16*>(attn_out);
+    if (launch_attention_combine(cp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
     return FLEXSPEC_OK;
 }
 
@@ -216,6 +215,7 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
     p.cu_q = h.plan.cu_q; p.cu_d = h.plan.cu_d; p.row_seq = h.plan.row_seq;
     p.batch = batch; p.vocab = c.vocab; p.m_rows = g.m_rows; p.s_rows = g.s_rows;
     p.n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
+    p.n_dchunks = (c.vocab + kDrawChunk - 1) / kDrawChunk;
     p.mask_words = (c.vocab + 31) / 32;
     p.inv_temp_log2 = p.greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     p.stats = h.stats; p.arg_idx = h.arg_idx; p.counters = h.counters;
@@ -292,8 +292,15 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     auto A = [&](int r) { if (rc == FLEXSPEC_OK) rc = r; };
     A(dev_alloc(&h.attn_out, static_cast<size_t>(max_m) * d_model));
     A(dev_alloc(&h.logits, static_cast<size_t>(max_m) * c.vocab));
-    A(dev_alloc(&h.part_o, static_cast<size_t>(kAttMaxSplits) * max_m * d_model));
-    A(dev_alloc(&h.part_ml, static_cast<size_t>(kAttMaxSplits) * max_m * c.n_q_heads * 2));
+    // attention partial slots: one per (pair, CTA) segment, index pair + CTA
+    const int group = c.n_q_heads / c.n_kv_heads;
+    const size_t att_slots = static_cast<size_t>(c.max_batch) * c.n_kv_heads *
+                                 ((group * (c.k_max + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair) + h.sm_count;
+    A(dev_alloc(&h.part_o, att_slots * kAttMaxConsumerWarps * 16 * c.head_dim));
+    A(dev_alloc(&h.part_ml, att_slots * kAttMaxConsumerWarps * 16 * 2));
+    A(dev_alloc(&h.plan.seq_blk0, static_cast<size_t>(c.max_batch) + 1));
+    A(dev_alloc(&h.plan.seq_pair0, static_cast<size_t>(c.max_batch) + 1));
+    A(dev_alloc(&h.plan.cta_start, static_cast<size_t>(h.sm_count)));
     A(dev_alloc(&h.plan.cu_q, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
@@ -301,7 +308,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.arg_idx, static_cast<size_t>(max_m) * n_chunks));
     A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
     A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 4));
-    A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * n_chunks * 2));
+    A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * ((c.vocab + kDrawChunk - 1) / kDrawChunk) * 2));
     A(dev_alloc(&h.dbg_p, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.dbg_q, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.dbg_u, static_cast<size_t>(h.max_s)));
@@ -369,7 +376,7 @@ int flexspec_attention(flexspec_handle* fh, const flexspec_kv* kv, const void* h
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    rc = run_plan(h, draft_len, nullptr, batch, s);
+    rc = run_plan(h, draft_len, nullptr, kv->kv_len, g, batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     return run_attention(h, kv, hidden, draft_len, g, batch, attn_out ? attn_out : h.attn_out, s);
 }
@@ -400,7 +407,7 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    rc = run_plan(h, draft_len, draft_tokens, batch, s);
+    rc = run_plan(h, draft_len, draft_tokens, nullptr, g, batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     return run_sample(h, logits ? logits : h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch,
                       temperature, vocab_mask, accepted_len, next_token, s);
@@ -427,7 +434,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     h.launches = 0;
     memset(h.ev_used, 0, sizeof(h.ev_used));
     mark(h, 0, s);
-    rc = run_plan(h, draft_len, draft_tokens, batch, s);
+    rc = run_plan(h, draft_len, draft_tokens, kv->kv_len, g, batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 1, s);
     rc = run_attention(h, kv, hidden, draft_len, g, batch, h.attn_out, s);   // marks event 2 after the split kernel

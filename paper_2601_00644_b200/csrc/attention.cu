@@ -2,24 +2,30 @@
 // inside the draft window (Section IV-C: the cloud keeps each user's KV session and scores only
 // the newly received block; Algorithm 2, Step 2).
 //
-// One CTA handles (sequence b, kv head, KV split).  The query rows of all `group` heads that
-// share the kv head form one tile of group*(k_b+1) rows, so every K/V page is read from HBM once
-// per kv head.  K/V pages (16 tokens) are brought in by TMA with the 128-byte swizzle, 8 pages
-// per pipeline stage; QK^T and PV run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with an
-// fp32 online softmax in registers (row max / sum over the 4 lanes of a quad by shuffles).
-// Each warp owns one 16-row tile and a subset of the pages of every stage; warps that share a
-// row tile are merged through shared memory at the end.  With more than one split the CTA writes
-// an unnormalised partial (running max, sum, output); a second kernel merges splits.
+// Work decomposition.  A "pair" is (sequence b, kv head, block of up to 128 query rows): the
+// query rows of all `group` heads that share the kv head, group*(k_b+1) of them, so every K/V
+// page is read from HBM once per kv head.  A pair's KV range is cut into blocks of 128 tokens
+// (8 pages of 16).  All blocks of the batch, numbered sequence by sequence and pair by pair, are
+// divided into equal contiguous ranges, one per CTA, with one CTA per SM: a single balanced wave
+// whatever the mix of context lengths and draft lengths.  A CTA therefore works on a few
+// "segments" (runs of blocks of one pair).
+//
+// Inside a CTA: warp 0 is the TMA producer (one 4 KB K and V page per lane, 128-byte swizzle,
+// 3 stages of 128 tokens, full/empty mbarriers, every wait bounded); the other warps consume.
+// Each consumer warp owns one 16-row tile of the pair and a subset of the pages of every stage:
+// QK^T and PV on mma.sync m16n8k16 (bf16 in, fp32 accumulate), fp32 online softmax in registers
+// with the row max / sum reduced over the 4 lanes of a quad by shuffles.  At the end of a segment
+// every consumer warp writes its unnormalised partial (running max, sum, output tile); a second
+// small kernel merges the partials of a pair by log-sum-exp and rounds to bf16.
 #include "common.cuh"
 #include "internal.h"
 
 namespace fs {
 
-constexpr int kAttPagesPerStage = 8;     // 8 pages = 128 tokens = kAttSplitQuantum
+constexpr int kAttPagesPerStage = 8;     // 8 pages = 128 tokens = kAttBlockTokens
 constexpr int kAttStages = 3;
-constexpr int kAttMaxWarps = 10;
-constexpr int kAttRowsPerCta = 128;
 constexpr int kPageTokens = 16;
+constexpr int kAttMaxThreads = (kAttMaxConsumerWarps + 1) * 32;
 
 template <int DH>
 struct AttCfg {
@@ -27,11 +33,8 @@ struct AttCfg {
     static constexpr int kSlabBytes = kPageTokens * 128;       // 16 tokens x 64 bf16
     static constexpr int kPageBytes = kHalves * kSlabBytes;    // K (or V) of one page, one kv head
     static constexpr int kStageBytes = kAttPagesPerStage * 2 * kPageBytes;
-    static constexpr int kQSlabBytes = kAttRowsPerCta * 128;
-    static constexpr int kQBytes = kHalves * kQSlabBytes;
-    static constexpr int kBarOffset = kAttStages * kStageBytes + kQBytes;
-    static constexpr int kSmemBytes = kBarOffset + 64 + 1024;  // + barriers/misc + alignment slack
-    static constexpr int kMergeRowFloats = DH + 4;             // padded row of the merge buffer
+    static constexpr int kBarOffset = kAttStages * kStageBytes;
+    static constexpr int kSmemBytes = kBarOffset + 128 + 1024;  // + barriers + alignment slack
 };
 
 // byte offset of 16-byte chunk `c` of row `r` inside a 128-byte-swizzled slab
@@ -40,141 +43,166 @@ __device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t c)
     return r * 128u + ((c ^ (r & 7u)) << 4);
 }
 
+// Position in the batch-wide block list; producer and consumers walk it in lock step.
+struct AttCursor {
+    int b, pair, blk;             // sequence, pair inside it, block inside the pair
+    int k, kvl, nb, rbc, pairs;   // of sequence b: draft length, kv length, blocks per pair,
+                                  // row blocks per kv head, pairs
+    __device__ __forceinline__ void load_seq(const AttnParams& p)
+    {
+        k = p.draft_len[b];
+        kvl = p.kv_len[b];
+        nb = (kvl + kAttBlockTokens - 1) / kAttBlockTokens;
+        rbc = (p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair;
+        pairs = p.n_kv_heads * rbc;
+    }
+    __device__ __forceinline__ void start(const AttnParams& p, int2 where)
+    {
+        b = where.x;
+        load_seq(p);
+        pair = where.y / nb;
+        blk = where.y % nb;
+    }
+    // returns true when the step left the current pair
+    __device__ __forceinline__ bool advance(const AttnParams& p, bool more)
+    {
+        if (++blk < nb) return false;
+        blk = 0;
+        if (++pair == pairs) {
+            pair = 0;
+            ++b;
+            if (more && b < p.batch) load_seq(p);
+        }
+        return true;
+    }
+};
+
 template <int DH>
-__global__ void __launch_bounds__(kAttMaxWarps * 32, 1)
-attention_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
+__global__ void __launch_bounds__(kAttMaxThreads, 1)
+attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
     using Cfg = AttCfg<DH>;
-    const int split = blockIdx.x;
-    const int kvh = blockIdx.y / p.row_blocks;
-    const int rb = blockIdx.y % p.row_blocks;
-    const int b = blockIdx.z;
-
-    const int k_b = p.draft_len[b];
-    const int kvl = p.kv_len[b];
-    const int ctx = kvl - (k_b + 1);
-    const int n_rows = p.group * (k_b + 1);           // query rows of this (sequence, kv head)
-    const int row_lo = rb * kAttRowsPerCta;
-    if (row_lo >= n_rows) return;
-    const int n_split = (kvl + p.split_len - 1) / p.split_len;
-    if (split >= n_split) return;
-    const int rows_here = min(kAttRowsPerCta, n_rows - row_lo);
-    const int n_rt = (rows_here + 15) >> 4;           // 16-row tiles in this CTA
-    const int t_begin = split * p.split_len;
-    const int t_end = min(kvl, t_begin + p.split_len);
-    const int n_pages = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
-    const int n_iter = (n_pages + kAttPagesPerStage - 1) / kAttPagesPerStage;
-    const int q_row0 = p.cu_q[b];
+    const int64_t total_blocks = p.seq_blk0[p.batch];
+    const int cta = blockIdx.x;
+    const int blk_begin = static_cast<int>(cta * total_blocks / gridDim.x);
+    const int blk_end = static_cast<int>((cta + 1) * total_blocks / gridDim.x);
+    const int n_my = blk_end - blk_begin;
+    if (n_my <= 0) return;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* q_smem = smem + kAttStages * Cfg::kStageBytes;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOffset);
+    uint64_t* empty_bar = full_bar + kAttStages;
 
-    const int tid = threadIdx.x;
-    const int warp = tid >> 5;
-    const int lane = tid & 31;
-    const int n_warps = blockDim.x >> 5;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int n_cw = (blockDim.x >> 5) - 1;             // consumer warps
 
-    if (tid == 0) {
-        for (int s = 0; s < kAttStages; ++s) mbar_init(&full_bar[s], 1);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kAttStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], n_cw); }
         fence_barrier_init();
         tma_prefetch_desc(&kv_map);
     }
     __syncthreads();
 
-    // ---- producer: lanes 0..7 of warp 0 each fetch one page (K and V) of the stage
-    const uint64_t pol = l2_policy_evict_first();
-    auto issue_stage = [&](int it) {
-        const int s = it % kAttStages;
-        const int pg0 = it * kAttPagesPerStage;
-        const int npg = min(kAttPagesPerStage, n_pages - pg0);
-        if (lane == 0) mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(npg * 2 * Cfg::kPageBytes));
-        __syncwarp();
-        if (lane < npg) {
-            const int page_idx = t_begin / kPageTokens + pg0 + lane;
-            int phys = p.page_table[static_cast<int64_t>(b) * p.max_pages_per_seq + page_idx];
-            if (phys < 0 || phys >= p.num_pages) {
-                report_error(p.status, kErrBadPage, phys, 1);
-                phys = 0;                                   // stay inside the pool
-            }
-            uint8_t* dst = smem + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes;
-            const int row_k = ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens;
-            const int row_v = ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens;
-#pragma unroll
-            for (int hf = 0; hf < Cfg::kHalves; ++hf) {
-                tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &full_bar[s], hf * 64, row_k, pol);
-                tma_load_2d(dst + Cfg::kPageBytes + hf * Cfg::kSlabBytes, &kv_map, &full_bar[s], hf * 64, row_v, pol);
-            }
-        }
-        __syncwarp();
-    };
+    AttCursor cur;
+    cur.start(p, p.cta_start[cta]);
+
     if (warp == 0) {
-        for (int it = 0; it < min(kAttStages, n_iter); ++it) issue_stage(it);
-    }
-
-    // ---- query tile -> shared memory (swizzled like the K/V slabs), then per-warp fragments
-    {
-        const int chunks_per_row = DH / 8;
-        const int total = n_rt * 16 * chunks_per_row;
-        for (int idx = tid; idx < total; idx += blockDim.x) {
-            const int r = idx / chunks_per_row;
-            const int ch = idx % chunks_per_row;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            const int rho = row_lo + r;
-            if (rho < n_rows) {
-                const int j = rho / p.group, hh = rho % p.group;
-                const __nv_bfloat16* src = p.hidden +
-                    (static_cast<int64_t>(q_row0 + j) * p.n_q_heads + kvh * p.group + hh) * DH + ch * 8;
-                v = *reinterpret_cast<const uint4*>(src);
+        // ------------------------------------------------------------------ TMA producer
+        const uint64_t pol = l2_policy_evict_first();
+        for (int q = 0; q < n_my; ++q) {
+            const int s = q % kAttStages;
+            const int use = q / kAttStages;
+            if (use > 0) mbar_wait(&empty_bar[s], (use - 1) & 1, p.status, 1);
+            const int kvh = cur.pair / cur.rbc;
+            const int t_begin = cur.blk * kAttBlockTokens;
+            const int t_end = min(cur.kvl, t_begin + kAttBlockTokens);
+            const int npg = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
+            if (lane == 0) mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(npg * 2 * Cfg::kPageBytes));
+            __syncwarp();
+            if (lane < npg) {
+                const int page_idx = cur.blk * kAttPagesPerStage + lane;
+                int phys = p.page_table[static_cast<int64_t>(cur.b) * p.max_pages_per_seq + page_idx];
+                if (phys < 0 || phys >= p.num_pages) {
+                    report_error(p.status, kErrBadPage, phys, 1);
+                    phys = 0;                               // stay inside the pool
+                }
+                uint8_t* dst = smem + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes;
+                const int row_k = ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens;
+                const int row_v = ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens;
+#pragma unroll
+                for (int hf = 0; hf < Cfg::kHalves; ++hf) {
+                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &full_bar[s], hf * 64, row_k, pol);
+                    tma_load_2d(dst + Cfg::kPageBytes + hf * Cfg::kSlabBytes, &kv_map, &full_bar[s], hf * 64, row_v, pol);
+                }
             }
-            *reinterpret_cast<uint4*>(q_smem + (ch >> 3) * Cfg::kQSlabBytes + swz(r, ch & 7)) = v;
+            __syncwarp();
+            cur.advance(p, q + 1 < n_my);
         }
+        return;     // consumers wait on every full barrier, so no copy is in flight when the CTA ends
     }
-    __syncthreads();
 
-    // warp -> (row tile, slice of the pages of each stage)
-    const int rt = warp % n_rt;
-    const int slice = warp / n_rt;
-    const int n_slices = (n_warps - rt + n_rt - 1) / n_rt;       // warps sharing this row tile
+    // ---------------------------------------------------------------------- consumers
+    const int cw = warp - 1;
+    const int g = lane >> 2, tq = lane & 3;
 
     uint32_t qa[DH / 16][4];
-    {
-        const int mi = lane >> 3;
-        const int r = rt * 16 + (mi & 1) * 8 + (lane & 7);
-#pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-            const int ch = 2 * kk + (mi >> 1);
-            ldmatrix_x4(qa[kk], smem_u32(q_smem + (ch >> 3) * Cfg::kQSlabBytes + swz(r, ch & 7)));
-        }
-    }
-
-    // rows of this thread inside the tile: g and g+8; their causal limits
-    const int g = lane >> 2, tq = lane & 3;
-    int limit[2];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int rho = row_lo + rt * 16 + g + i * 8;
-        limit[i] = (rho < n_rows) ? ctx + rho / p.group + 1 : kvl;    // padded rows see everything
-    }
-
     float o[DH / 8][4];
-#pragma unroll
-    for (int nt = 0; nt < DH / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
-    float m_run[2] = {-INFINITY, -INFINITY};
-    float l_run[2] = {0.f, 0.f};
+    float m_run[2], l_run[2];
+    int limit[2];
+    int rt = 0, slice = 0, n_slices = 1, n_rt = 1, ctx = 0;
+    bool new_segment = true;
 
-    for (int it = 0; it < n_iter; ++it) {
-        const int s = it % kAttStages;
-        mbar_wait(&full_bar[s], (it / kAttStages) & 1, p.status, 1);
-        const int pg0 = it * kAttPagesPerStage;
-        const int npg = min(kAttPagesPerStage, n_pages - pg0);
+    for (int q = 0; q < n_my; ++q) {
+        if (new_segment) {
+            // ---- set up the pair: row tile of this warp, query fragments, causal limits
+            const int kvh = cur.pair / cur.rbc;
+            const int row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
+            const int n_rows = p.group * (cur.k + 1);
+            const int rows_here = min(kAttRowsPerPair, n_rows - row_lo);
+            n_rt = (rows_here + 15) >> 4;
+            rt = cw % n_rt;
+            slice = cw / n_rt;
+            n_slices = (n_cw - rt + n_rt - 1) / n_rt;
+            ctx = cur.kvl - (cur.k + 1);
+            const int q_row0 = p.cu_q[cur.b];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int rho = row_lo + rt * 16 + g + i * 8;
+                const bool real = rho < n_rows;
+                limit[i] = real ? ctx + rho / p.group + 1 : cur.kvl;     // padded rows see everything
+                const uint32_t* src = nullptr;
+                if (real) {
+                    const int j = rho / p.group, hh = rho % p.group;
+                    src = reinterpret_cast<const uint32_t*>(
+                        p.hidden + (static_cast<int64_t>(q_row0 + j) * p.n_q_heads + kvh * p.group + hh) * DH);
+                }
+#pragma unroll
+                for (int kk = 0; kk < DH / 16; ++kk) {
+                    // A fragment of m16n8k16: regs 0/1 = rows g / g+8, cols 2tq..; regs 2/3 = cols 8+2tq..
+                    qa[kk][i] = real ? __ldg(src + kk * 8 + tq) : 0u;
+                    qa[kk][i + 2] = real ? __ldg(src + kk * 8 + 4 + tq) : 0u;
+                }
+            }
+#pragma unroll
+            for (int nt = 0; nt < DH / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+            m_run[0] = m_run[1] = -INFINITY;
+            l_run[0] = l_run[1] = 0.f;
+            new_segment = false;
+        }
+
+        const int s = q % kAttStages;
+        mbar_wait(&full_bar[s], (q / kAttStages) & 1, p.status, 2);
+        const int t_begin = cur.blk * kAttBlockTokens;
+        const int t_end = min(cur.kvl, t_begin + kAttBlockTokens);
+        const int npg = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
         const uint8_t* stage = smem + s * Cfg::kStageBytes;
 
         for (int pi = slice; pi < npg; pi += n_slices) {
             const uint8_t* kp = stage + pi * 2 * Cfg::kPageBytes;
             const uint8_t* vp = kp + Cfg::kPageBytes;
-            const int tok0 = t_begin + (pg0 + pi) * kPageTokens;
+            const int tok0 = t_begin + pi * kPageTokens;
 
             // S = Q K^T for 16 rows x 16 tokens
             float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -238,159 +266,149 @@ attention_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnPar
                     uint32_t vb[4];
                     ldmatrix_x4_trans(vb, smem_u32(vp + (ch >> 3) * Cfg::kSlabBytes + swz(tok, ch & 7)));
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        float (&acc)[4] = o[2 * dp + q];
+                    for (int h2 = 0; h2 < 2; ++h2) {
+                        float (&acc)[4] = o[2 * dp + h2];
                         acc[0] *= alpha[0]; acc[1] *= alpha[0];
                         acc[2] *= alpha[1]; acc[3] *= alpha[1];
-                        mma_bf16_16816(acc, pa, vb[2 * q], vb[2 * q + 1]);
+                        mma_bf16_16816(acc, pa, vb[2 * h2], vb[2 * h2 + 1]);
                     }
                 }
             }
         }
-        __syncthreads();                               // every warp is done with stage s
-        if (warp == 0 && it + kAttStages < n_iter) issue_stage(it + kAttStages);
-    }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);           // this warp is done with stage s
 
-    // ---- merge the warps that share a row tile, then write the result / the split partial
+        const int pair_global = p.seq_pair0[cur.b] + cur.pair;
+        const bool left_pair = cur.advance(p, q + 1 < n_my);
+        if (left_pair || q + 1 == n_my) {
+            // ---- end of the segment: this warp's partial -> slot (pair + CTA), unique per segment
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
-        l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
-    }
-    float* mo = reinterpret_cast<float*>(smem);                                   // [warp][16][DH+4]
-    float* mml = mo + kAttMaxWarps * 16 * Cfg::kMergeRowFloats;                   // [warp][16][2]
-    {
-        float* my = mo + warp * 16 * Cfg::kMergeRowFloats;
-#pragma unroll
-        for (int nt = 0; nt < DH / 8; ++nt) {
-            *reinterpret_cast<float2*>(my + g * Cfg::kMergeRowFloats + nt * 8 + tq * 2) = make_float2(o[nt][0], o[nt][1]);
-            *reinterpret_cast<float2*>(my + (g + 8) * Cfg::kMergeRowFloats + nt * 8 + tq * 2) = make_float2(o[nt][2], o[nt][3]);
-        }
-        if (tq == 0) {
-            mml[(warp * 16 + g) * 2 + 0] = m_run[0];
-            mml[(warp * 16 + g) * 2 + 1] = l_run[0];
-            mml[(warp * 16 + g + 8) * 2 + 0] = m_run[1];
-            mml[(warp * 16 + g + 8) * 2 + 1] = l_run[1];
-        }
-    }
-    __syncthreads();
-
-    const int cols4 = DH / 4;
-    for (int idx = tid; idx < rows_here * cols4; idx += blockDim.x) {
-        const int r = idx / cols4;
-        const int c4 = (idx % cols4) * 4;
-        const int tile = r >> 4, rr = r & 15;
-        const int slices = (n_warps - tile + n_rt - 1) / n_rt;
-        float m_all = -INFINITY;
-        for (int sl = 0; sl < slices; ++sl) m_all = fmaxf(m_all, mml[((tile + sl * n_rt) * 16 + rr) * 2]);
-        const float m_safe = (m_all == -INFINITY) ? 0.f : m_all;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float l_all = 0.f;
-        for (int sl = 0; sl < slices; ++sl) {
-            const int w = tile + sl * n_rt;
-            const float wgt = fast_exp2(mml[(w * 16 + rr) * 2] - m_safe);
-            l_all += wgt * mml[(w * 16 + rr) * 2 + 1];
-            const float4 v = *reinterpret_cast<const float4*>(mo + (w * 16 + rr) * Cfg::kMergeRowFloats + c4);
-            acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-        }
-        const int rho = row_lo + r;
-        const int j = rho / p.group, hh = rho % p.group;
-        const int64_t out_row = static_cast<int64_t>(q_row0 + j) * p.n_q_heads + kvh * p.group + hh;
-        if (n_split == 1) {
-            const float inv = 1.f / l_all;
-            __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-            __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-            uint2 pk;
-            pk.x = *reinterpret_cast<uint32_t*>(&lo);
-            pk.y = *reinterpret_cast<uint32_t*>(&hi);
-            *reinterpret_cast<uint2*>(p.attn_out + out_row * DH + c4) = pk;
-        } else {
-            const int64_t prow = static_cast<int64_t>(split) * p.part_stride + out_row;
-            *reinterpret_cast<float4*>(p.part_o + prow * DH + c4) = acc;
-            if (c4 == 0) {
-                p.part_ml[prow * 2 + 0] = m_all;
-                p.part_ml[prow * 2 + 1] = l_all;
+            for (int i = 0; i < 2; ++i) {
+                l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
+                l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
             }
+            const int64_t slot = static_cast<int64_t>(pair_global + cta) * kAttMaxConsumerWarps + cw;
+            float* po = p.part_o + slot * 16 * DH;
+            float* pml = p.part_ml + slot * 16 * 2;
+            const bool has = (m_run[0] != -INFINITY) || (m_run[1] != -INFINITY);
+            if (has) {
+#pragma unroll
+                for (int nt = 0; nt < DH / 8; ++nt) {
+                    *reinterpret_cast<float2*>(po + g * DH + nt * 8 + tq * 2) = make_float2(o[nt][0], o[nt][1]);
+                    *reinterpret_cast<float2*>(po + (g + 8) * DH + nt * 8 + tq * 2) = make_float2(o[nt][2], o[nt][3]);
+                }
+            }
+            if (tq == 0) {
+                *reinterpret_cast<float2*>(pml + g * 2) = make_float2(m_run[0], l_run[0]);
+                *reinterpret_cast<float2*>(pml + (g + 8) * 2) = make_float2(m_run[1], l_run[1]);
+            }
+            new_segment = true;
         }
     }
 }
 
-// Merge of the KV splits: out = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s, rounded to bf16.
+// Merge of a pair's partials: out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i, rounded to bf16.
+// The partials of pair P were written by the CTAs whose block ranges intersect the pair's blocks,
+// by every consumer warp that shares the row tile.
 __global__ void __launch_bounds__(256)
 attention_combine_kernel(const CombineParams p)
 {
     const int b = blockIdx.y;
-    const int j = blockIdx.x;
     const int k_b = p.draft_len[b];
-    if (j > k_b) return;
     const int kvl = p.kv_len[b];
-    const int n_split = (kvl + p.split_len - 1) / p.split_len;
-    if (n_split <= 1) return;                       // the attention kernel wrote the result itself
-    const int64_t row = p.cu_q[b] + j;
-    const int dh4 = p.head_dim / 4;
-    const int total = p.n_q_heads * dh4;
-    for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
-        const int h = idx / dh4;
-        const int c4 = (idx % dh4) * 4;
-        const int64_t rh = row * p.n_q_heads + h;
+    const int nb = (kvl + kAttBlockTokens - 1) / kAttBlockTokens;
+    const int n_rows = p.group * (k_b + 1);
+    const int rbc = (n_rows + kAttRowsPerPair - 1) / kAttRowsPerPair;
+    const int pair = blockIdx.x;
+    if (pair >= p.n_kv_heads * rbc) return;
+    const int kvh = pair / rbc;
+    const int row_lo = (pair % rbc) * kAttRowsPerPair;
+    const int rows_here = min(kAttRowsPerPair, n_rows - row_lo);
+    const int n_rt = (rows_here + 15) >> 4;
+
+    const int64_t total_blocks = p.seq_blk0[p.batch];
+    const int64_t blk_first = p.seq_blk0[b] + static_cast<int64_t>(pair) * nb;
+    const int64_t blk_last = blk_first + nb - 1;
+    // CTA c owns blocks [c*T/G, (c+1)*T/G): the owner of block x is ceil((x+1)*G/T) - 1
+    const int c0 = static_cast<int>(((blk_first + 1) * p.n_ctas - 1) / total_blocks);
+    const int c1 = static_cast<int>(((blk_last + 1) * p.n_ctas - 1) / total_blocks);
+    const int pair_global = p.seq_pair0[b] + pair;
+    const int q_row0 = p.cu_q[b];
+    const int dh = p.head_dim;
+    const int cols4 = dh / 4;
+
+    for (int idx = threadIdx.x; idx < rows_here * cols4; idx += blockDim.x) {
+        const int r = idx / cols4;
+        const int c4 = (idx % cols4) * 4;
+        const int tile = r >> 4, rr = r & 15;
+        const int slices = (p.n_cw - tile + n_rt - 1) / n_rt;
         float m_all = -INFINITY;
-        for (int s = 0; s < n_split; ++s) m_all = fmaxf(m_all, p.part_ml[(s * p.part_stride + rh) * 2]);
+        for (int c = c0; c <= c1; ++c)
+            for (int sl = 0; sl < slices; ++sl) {
+                const int64_t slot = static_cast<int64_t>(pair_global + c) * kAttMaxConsumerWarps + tile + sl * n_rt;
+                m_all = fmaxf(m_all, p.part_ml[(slot * 16 + rr) * 2]);
+            }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float l_all = 0.f;
-        for (int s = 0; s < n_split; ++s) {
-            const int64_t pr = s * p.part_stride + rh;
-            const float wgt = fast_exp2(p.part_ml[pr * 2] - m_all);
-            l_all += wgt * p.part_ml[pr * 2 + 1];
-            const float4 v = *reinterpret_cast<const float4*>(p.part_o + pr * p.head_dim + c4);
-            acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-        }
+        for (int c = c0; c <= c1; ++c)
+            for (int sl = 0; sl < slices; ++sl) {
+                const int64_t slot = static_cast<int64_t>(pair_global + c) * kAttMaxConsumerWarps + tile + sl * n_rt;
+                const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (slot * 16 + rr) * 2);
+                if (ml.x == -INFINITY) continue;             // that warp saw no visible token
+                const float wgt = fast_exp2(ml.x - m_all);
+                l_all += wgt * ml.y;
+                const float4 v = *reinterpret_cast<const float4*>(p.part_o + (slot * 16 + rr) * dh + c4);
+                acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
+            }
+        const int rho = row_lo + r;
+        const int j = rho / p.group, hh = rho % p.group;
+        const int64_t out_row = static_cast<int64_t>(q_row0 + j) * p.n_q_heads + kvh * p.group + hh;
         const float inv = 1.f / l_all;
         __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
         __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
         uint2 pk;
         pk.x = *reinterpret_cast<uint32_t*>(&lo);
         pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(p.attn_out + rh * p.head_dim + c4) = pk;
+        *reinterpret_cast<uint2*>(p.attn_out + out_row * dh + c4) = pk;
     }
 }
 
 cudaError_t attention_init(int head_dim)
 {
     if (head_dim == 128)
-        return cudaFuncSetAttribute(attention_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        return cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     AttCfg<128>::kSmemBytes);
-    return cudaFuncSetAttribute(attention_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 AttCfg<64>::kSmemBytes);
 }
 
-// warps per CTA for a batch whose largest (sequence, kv head) tile has `max_rows` query rows
-static int attention_warps(int max_rows)
+// consumer warps per CTA for a batch whose largest pair has `max_tile_rows` query rows
+int attention_consumer_warps(int max_tile_rows)
 {
-    const int rows = max_rows > kAttRowsPerCta ? kAttRowsPerCta : max_rows;
+    const int rows = max_tile_rows > kAttRowsPerPair ? kAttRowsPerPair : max_tile_rows;
     const int rt = rows > 0 ? (rows + 15) / 16 : 1;
     int slices = (8 + rt / 2) / rt;                  // round(8 / rt) ...
     if (slices < 1) slices = 1;                      // ... at least 1
     int w = rt * slices;
-    if (w > kAttMaxWarps) w = rt;
+    if (w > kAttMaxConsumerWarps) w = rt;
     return w;
 }
 
-cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t batch,
-                             int32_t max_rows_per_seq, int32_t max_splits, cudaStream_t stream)
+cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
+                             int32_t n_cw, cudaStream_t stream)
 {
-    const int max_tile_rows = p.group * max_rows_per_seq;
-    dim3 grid(max_splits, p.n_kv_heads * p.row_blocks, batch);
-    dim3 block(attention_warps(max_tile_rows) * 32);
+    dim3 grid(n_ctas);
+    dim3 block((n_cw + 1) * 32);
     if (h.cfg.head_dim == 128)
-        attention_split_kernel<128><<<grid, block, AttCfg<128>::kSmemBytes, stream>>>(kv_map, p);
+        attention_kernel<128><<<grid, block, AttCfg<128>::kSmemBytes, stream>>>(kv_map, p);
     else
-        attention_split_kernel<64><<<grid, block, AttCfg<64>::kSmemBytes, stream>>>(kv_map, p);
+        attention_kernel<64><<<grid, block, AttCfg<64>::kSmemBytes, stream>>>(kv_map, p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_attention_combine(const CombineParams& p, int32_t batch, cudaStream_t stream)
+cudaError_t launch_attention_combine(const CombineParams& p, cudaStream_t stream)
 {
-    dim3 grid(p.rows_per_seq_max, batch);
+    dim3 grid(p.pairs_per_seq_max, p.batch);
     attention_combine_kernel<<<grid, 256, 0, stream>>>(p);
     return cudaGetLastError();
 }

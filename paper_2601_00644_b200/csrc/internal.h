@@ -12,16 +12,25 @@ namespace fs {
 
 constexpr int kMaxBatch = 1024;
 constexpr int kMaxK = 63;
-constexpr int kSampleChunk = 8192;        // vocabulary elements per CTA in the sampling kernels
-constexpr int kAttSplitQuantum = 128;     // tokens per attention pipeline stage
-constexpr int kAttMaxSplits = 32;
+constexpr int kSampleChunk = 8192;        // vocabulary entries per CTA of the statistics kernel
+constexpr int kDrawChunk = 2048;          // vocabulary entries per CTA of the draw kernel
+constexpr int kAttBlockTokens = 128;      // KV tokens per attention work block / pipeline stage
+constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block
 constexpr int kNumStageEvents = 7;
 
 struct Plan {                 // device tables written by the plan kernel, read by all stages
     int32_t* cu_q;            // [max_batch+1] first query row of each sequence
     int32_t* cu_d;            // [max_batch+1] first draft row of each sequence
     int32_t* row_seq;         // [max_m] sequence of each query row
+    // attention work list: a "block" is 128 KV tokens of one (sequence, kv head, 128-row block)
+    // pair; blocks are numbered sequence by sequence, pair by pair, and cut into equal
+    // contiguous ranges, one per CTA
+    int32_t* seq_blk0;        // [max_batch+1] first block of each sequence; [batch] = total
+    int32_t* seq_pair0;       // [max_batch+1] first pair of each sequence
+    int2* cta_start;          // [sm_count] (sequence, block index inside it) where CTA c starts
 };
+
+constexpr int kAttMaxConsumerWarps = 10;
 
 struct AttnParams {
     const __nv_bfloat16* hidden;
@@ -29,26 +38,29 @@ struct AttnParams {
     const int32_t* kv_len;
     const int32_t* draft_len;
     const int32_t* cu_q;
-    int32_t n_q_heads, n_kv_heads, group;
+    const int32_t* seq_blk0;
+    const int32_t* seq_pair0;
+    const int2* cta_start;
+    int32_t batch, n_q_heads, n_kv_heads, group;
     int32_t max_pages_per_seq, num_pages;
-    int32_t split_len;        // tokens per split, multiple of kAttSplitQuantum
-    int32_t row_blocks;       // CTAs along the query rows of one (sequence, kv head)
     float scale_log2;         // log2(e) / sqrt(head_dim)
-    float* part_o;            // [split][row][H][Dh] unnormalised partial outputs
-    float* part_ml;           // [split][row][H][2]  (running max in log2 units, sum)
-    int64_t part_stride;      // rows * H (elements of part_ml / 2 per split; x Dh for part_o)
-    __nv_bfloat16* attn_out;  // [M][H*Dh]
+    float* part_o;            // [slot][consumer warp][16][Dh] unnormalised partial outputs
+    float* part_ml;           // [slot][consumer warp][16][2]  (running max in log2 units, sum)
     int32_t* status;
 };
 
 struct CombineParams {
     const float* part_o;
     const float* part_ml;
-    int64_t part_stride;
     const int32_t* kv_len;
     const int32_t* draft_len;
     const int32_t* cu_q;
-    int32_t split_len, rows_per_seq_max, n_q_heads, head_dim;
+    const int32_t* seq_blk0;
+    const int32_t* seq_pair0;
+    int32_t batch, n_q_heads, n_kv_heads, group, head_dim;
+    int32_t n_ctas;           // grid of the attention kernel
+    int32_t n_cw;             // its consumer warps
+    int32_t pairs_per_seq_max;
     __nv_bfloat16* attn_out;
 };
 
@@ -74,14 +86,14 @@ struct SampleParams {
     const int32_t* cu_q;
     const int32_t* cu_d;
     const int32_t* row_seq;
-    int32_t batch, vocab, m_rows, s_rows, n_chunks, mask_words;
+    int32_t batch, vocab, m_rows, s_rows, n_chunks, n_dchunks, mask_words;
     float inv_temp_log2;          // log2(e) / T
     int32_t greedy;
     float2* stats;                // [(M+S)][n_chunks] (chunk max in logit units, sum exp)
     int32_t* arg_idx;             // [M][n_chunks] lowest index of the chunk max (greedy)
     int32_t* counters;            // [2][max_batch] self-resetting tickets
-    double* row_info;             // [B][4]: max_p, sum_p, max_q, sum_q of row n (log2-scaled max)
-    double* chunk_mass;           // [B][n_chunks][2]: residual mass, p mass
+    double* row_info;             // [B][4]: max_p, 1/sum_p, max_q, 1/sum_q of row n
+    double* chunk_mass;           // [B][n_dchunks][2]: residual mass, p mass
     int32_t* accepted_len;
     int32_t* next_token;
     double* dbg_p; double* dbg_q; float* dbg_u;   // [S] or null
@@ -112,11 +124,13 @@ struct Handle {
 };
 
 // launch wrappers (each returns a cudaError_t from the launch)
-cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
+cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, const int32_t* kv_len,
+                        int32_t batch, int32_t vocab, int32_t n_kv_heads, int32_t group, int32_t n_ctas,
                         Plan plan, int32_t* status, cudaStream_t stream);
-cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t batch,
-                             int32_t max_rows_per_seq, int32_t max_splits, cudaStream_t stream);
-cudaError_t launch_attention_combine(const CombineParams& p, int32_t batch, cudaStream_t stream);
+int attention_consumer_warps(int max_tile_rows);
+cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
+                             int32_t n_cw, cudaStream_t stream);
+cudaError_t launch_attention_combine(const CombineParams& p, cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream);
 cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);

@@ -8,110 +8,41 @@
 // as Algorithm 2 prints it: accept while x_j equals the arg-max of the target row, emit the
 // arg-max of the first row that disagrees (or of the bonus row).
 //
-//   plan   : prefix sums of the draft lengths, row -> sequence table, token range check.
-//   stats  : grid (vocabulary chunk, row) over all M target rows and S draft rows: chunk max
-//            and sum of exp in fp32 (one streaming read of both logit sets).  The last CTA to
-//            finish for a sequence (atomic ticket, no waiting) merges the chunk statistics in
-//            fp64, evaluates the acceptance tests with Philox uniforms, finds the first
-//            rejection by warp vote and stores accepted_len.
-//   draw   : grid (chunk, sequence): probability mass of the residual (or of p) per chunk in
-//            fp64; the last CTA of a sequence picks the chunk that holds u' * Z and scans it in
-//            vocabulary order (inverse CDF).
+//   stats  : grid (vocabulary chunk of 8192, row) over all M target rows and S draft rows: one
+//            streaming read of both logit sets; per chunk the max and the sum of 2^((z-max)*c),
+//            c = log2(e)/T, in fp32 (online per thread, merged by shuffles, one block barrier).
+//            The last CTA to finish for a sequence (atomic ticket, nobody waits) merges the chunk
+//            statistics in fp64, evaluates the acceptance tests with Philox uniforms, finds the
+//            first rejection by warp vote and stores accepted_len.
+//   draw   : grid (chunk of 2048, sequence) over row n of each sequence only: probability mass of
+//            the residual (and of p) per chunk, fp32 exponentials accumulated in fp64; the last
+//            CTA of a sequence picks the chunk that holds u' * Z and scans it in vocabulary order
+//            (inverse CDF).
 #include "common.cuh"
 #include "internal.h"
 
 namespace fs {
 
 constexpr int kSampleThreads = 256;
+constexpr int kSampleWarps = kSampleThreads / 32;
 constexpr int kElemsPerThread = kSampleChunk / kSampleThreads;   // 32
+constexpr int kDrawElems = kDrawChunk / kSampleThreads;          // 8
 
-// ------------------------------------------------------------------------------------ plan
-__global__ void __launch_bounds__(kMaxBatch)
-plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ draft_tokens, int32_t batch,
-            int32_t vocab, Plan plan, int32_t* status)
-{
-    __shared__ int32_t scan_q[kMaxBatch];
-    __shared__ int32_t scan_d[kMaxBatch];
-    const int t = threadIdx.x;
-    const int k = (t < batch) ? draft_len[t] : 0;
-    scan_q[t] = (t < batch) ? k + 1 : 0;
-    scan_d[t] = k;
-    __syncthreads();
-    for (int off = 1; off < kMaxBatch; off <<= 1) {          // inclusive Hillis-Steele scan
-        const int aq = (t >= off) ? scan_q[t - off] : 0;
-        const int ad = (t >= off) ? scan_d[t - off] : 0;
-        __syncthreads();
-        scan_q[t] += aq;
-        scan_d[t] += ad;
-        __syncthreads();
-    }
-    if (t < batch) {
-        const int q0 = scan_q[t] - (k + 1);
-        const int d0 = scan_d[t] - k;
-        plan.cu_q[t] = q0;
-        plan.cu_d[t] = d0;
-        for (int j = 0; j <= k; ++j) plan.row_seq[q0 + j] = t;
-        if (draft_tokens != nullptr)
-            for (int j = 0; j < k; ++j) {
-                const int x = draft_tokens[d0 + j];
-                if (x < 0 || x >= vocab) report_error(status, kErrBadToken, x, 7);
-            }
-        if (t == batch - 1) {
-            plan.cu_q[batch] = scan_q[t];
-            plan.cu_d[batch] = scan_d[t];
-        }
-    }
-}
-
-cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
-                        Plan plan, int32_t* status, cudaStream_t stream)
-{
-    plan_kernel<<<1, kMaxBatch, 0, stream>>>(draft_len, draft_tokens, batch, vocab, plan, status);
-    return cudaGetLastError();
-}
-
-// ------------------------------------------------------------------------------------ helpers
 __device__ __forceinline__ bool mask_allows(const uint32_t* mask_row, int v)
 {
     return mask_row == nullptr || ((mask_row[v >> 5] >> (v & 31)) & 1u);
 }
 
-// block-wide reductions over kSampleThreads threads (8 warps)
-__device__ __forceinline__ float block_max(float v, float* red)
+// (max, sum of 2^((z - max) * c)) pairs: merge of two partial softmax statistics
+__device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2, float c)
 {
-    v = warp_max(v);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    float r = red[0];
-#pragma unroll
-    for (int w = 1; w < kSampleThreads / 32; ++w) r = fmaxf(r, red[w]);
-    __syncthreads();
-    return r;
-}
-__device__ __forceinline__ float block_sum(float v, float* red)
-{
-    v = warp_sum(v);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    float r = 0.f;
-#pragma unroll
-    for (int w = 0; w < kSampleThreads / 32; ++w) r += red[w];      // fixed order: deterministic
-    __syncthreads();
-    return r;
-}
-__device__ __forceinline__ double block_sum(double v, double* red)
-{
-    v = warp_sum(v);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    double r = 0.0;
-#pragma unroll
-    for (int w = 0; w < kSampleThreads / 32; ++w) r += red[w];
-    __syncthreads();
-    return r;
+    const float mm = fmaxf(m, m2);
+    const float base = (mm == -INFINITY) ? 0.f : mm;
+    s = s * fast_exp2((m - base) * c) + s2 * fast_exp2((m2 - base) * c);
+    m = mm;
 }
 
-// Merge of per-chunk (max, sum exp2((z - max) * scale)) in chunk order, fp64.
+// Merge of per-chunk statistics in chunk order, fp64.
 __device__ __forceinline__ void merge_row_stats(const float2* st, int n_chunks, double scale, double& mx, double& sum)
 {
     double m = -INFINITY;
@@ -130,12 +61,14 @@ __device__ __forceinline__ void merge_row_stats(const float2* st, int n_chunks, 
 __global__ void __launch_bounds__(kSampleThreads)
 sample_stats_kernel(const SampleParams p)
 {
-    __shared__ float red[kSampleThreads / 32];
-    __shared__ int red_idx[kSampleThreads / 32];
-    __shared__ int s_is_last;
+    __shared__ float red_m[kSampleWarps];
+    __shared__ float red_s[kSampleWarps];
+    __shared__ int red_i[kSampleWarps];
+    __shared__ int s_argmax[kMaxK + 1];
 
     const int chunk = blockIdx.x;
     const int row = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool is_target = row < p.m_rows;
     int b;
     const float* src;
@@ -146,8 +79,7 @@ sample_stats_kernel(const SampleParams p)
         if (p.vocab_mask != nullptr) mask_row = p.vocab_mask + static_cast<int64_t>(b) * p.mask_words;
     } else {
         const int dr = row - p.m_rows;
-        // sequence of a draft row: the target row with the same (b, j) is row dr + b, so search
-        int lo = 0, hi = p.batch - 1;                     // largest b with cu_d[b] <= dr and k_b > 0
+        int lo = 0, hi = p.batch - 1;                     // largest b with cu_d[b] <= dr: owns draft row dr
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
             if (p.cu_d[mid] <= dr) lo = mid; else hi = mid - 1;
@@ -185,65 +117,90 @@ sample_stats_kernel(const SampleParams p)
     float mx = -INFINITY;
 #pragma unroll
     for (int i = 0; i < kElemsPerThread; ++i) mx = fmaxf(mx, z[i]);
+    const float c = p.inv_temp_log2;
 
     if (p.greedy) {
-        if (is_target) {
-            // lowest index holding the chunk maximum
-            int best = 0x7fffffff;
-            const float bm = block_max(mx, red);
+        // (max, lowest index holding it)
+        int best = 0x7fffffff;
 #pragma unroll
-            for (int i = 0; i < kElemsPerThread; ++i) {
-                const int v = v0 + ((i >> 2) * kSampleThreads + threadIdx.x) * 4 + (i & 3);
-                if (z[i] == bm && v < v_end) best = min(best, v);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, o));
-            if ((threadIdx.x & 31) == 0) red_idx[threadIdx.x >> 5] = best;
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                for (int w = 1; w < kSampleThreads / 32; ++w) best = min(best, red_idx[w]);
-                p.stats[static_cast<int64_t>(row) * p.n_chunks + chunk] = make_float2(bm, 0.f);
-                p.arg_idx[static_cast<int64_t>(row) * p.n_chunks + chunk] = best;
-            }
+        for (int i = 0; i < kElemsPerThread; ++i) {
+            const int v = v0 + ((i >> 2) * kSampleThreads + threadIdx.x) * 4 + (i & 3);
+            if (z[i] == mx && v < v_end) best = min(best, v);
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mx, o);
+            const int i2 = __shfl_xor_sync(0xffffffffu, best, o);
+            if (m2 > mx || (m2 == mx && i2 < best)) { mx = m2; best = i2; }
+        }
+        if (lane == 0) { red_m[warp] = mx; red_i[warp] = best; }
     } else {
-        const float bm = block_max(mx, red);
-        const float base = (bm == -INFINITY) ? 0.f : bm;
+        const float base = (mx == -INFINITY) ? 0.f : mx;
         float se = 0.f;
 #pragma unroll
-        for (int i = 0; i < kElemsPerThread; ++i) se += fast_exp2((z[i] - base) * p.inv_temp_log2);
-        const float bs = block_sum(se, red);
-        if (threadIdx.x == 0) p.stats[static_cast<int64_t>(row) * p.n_chunks + chunk] = make_float2(bm, bs);
+        for (int i = 0; i < kElemsPerThread; ++i) se += fast_exp2((z[i] - base) * c);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, mx, o);
+            const float s2 = __shfl_xor_sync(0xffffffffu, se, o);
+            merge_ms(mx, se, m2, s2, c);
+        }
+        if (lane == 0) { red_m[warp] = mx; red_s[warp] = se; }
     }
+    __syncthreads();
+    if (warp != 0) return;
 
-    // ---- ticket: the last CTA of sequence b takes the decision
+    // ---- warp 0: merge the 8 warps, publish, take a ticket
+    {
+        float m = (lane < kSampleWarps) ? red_m[lane] : -INFINITY;
+        if (p.greedy) {
+            int bi = (lane < kSampleWarps) ? red_i[lane] : 0x7fffffff;
+#pragma unroll
+            for (int o = kSampleWarps / 2; o > 0; o >>= 1) {
+                const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+                const int i2 = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (m2 > m || (m2 == m && i2 < bi)) { m = m2; bi = i2; }
+            }
+            if (lane == 0 && is_target) {
+                p.stats[static_cast<int64_t>(row) * p.n_chunks + chunk] = make_float2(m, 0.f);
+                p.arg_idx[static_cast<int64_t>(row) * p.n_chunks + chunk] = bi;
+            }
+        } else {
+            float s = (lane < kSampleWarps) ? red_s[lane] : 0.f;
+#pragma unroll
+            for (int o = kSampleWarps / 2; o > 0; o >>= 1) {
+                const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+                const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
+                merge_ms(m, s, m2, s2, c);
+            }
+            if (lane == 0) p.stats[static_cast<int64_t>(row) * p.n_chunks + chunk] = make_float2(m, s);
+        }
+    }
     const int k_b = p.draft_len[b];
-    const int expected = (p.greedy ? (k_b + 1) : (2 * k_b + 1)) * p.n_chunks;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
+    int is_last = 0;
+    if (lane == 0) {
+        const int expected = (p.greedy ? (k_b + 1) : (2 * k_b + 1)) * p.n_chunks;
+        __threadfence();
         const int t = atomicAdd(&p.counters[b], 1);
-        s_is_last = (t == expected - 1);
-        if (s_is_last) p.counters[b] = 0;                 // ready for the next call
+        is_last = (t == expected - 1);
+        if (is_last) { p.counters[b] = 0; __threadfence(); }      // ready for the next call
     }
-    __syncthreads();
-    if (!s_is_last) return;
+    is_last = __shfl_sync(0xffffffffu, is_last, 0);
+    if (!is_last) return;
     __threadfence();
-    if (threadIdx.x >= 32) return;
 
+    // ---- the last CTA of sequence b takes the decision
     const int q0 = p.cu_q[b], d0 = p.cu_d[b];
-    const int lane = threadIdx.x;
     const double scale = static_cast<double>(p.inv_temp_log2);
     int n = k_b;
     if (p.greedy) {
-        __shared__ int s_argmax[kMaxK + 1];
         for (int j = lane; j <= k_b; j += 32) {
             const float2* st = p.stats + static_cast<int64_t>(q0 + j) * p.n_chunks;
             const int32_t* ai = p.arg_idx + static_cast<int64_t>(q0 + j) * p.n_chunks;
             float bm = -INFINITY;
             int best = 0;
-            for (int c = 0; c < p.n_chunks; ++c)
-                if (c == 0 || st[c].x > bm) { bm = st[c].x; best = ai[c]; }     // strict: lowest index wins
+            for (int cc = 0; cc < p.n_chunks; ++cc)
+                if (cc == 0 || st[cc].x > bm) { bm = st[cc].x; best = ai[cc]; }     // strict: lowest index wins
             s_argmax[j] = best;
         }
         __syncwarp();
@@ -289,12 +246,12 @@ sample_stats_kernel(const SampleParams p)
     }
     if (lane == 0) {
         p.accepted_len[b] = n;
-        double mp, sp, mq = 0.0, sq = 0.0;
+        double mp, sp, mq = 0.0, sq = 1.0;
         merge_row_stats(p.stats + static_cast<int64_t>(q0 + n) * p.n_chunks, p.n_chunks, scale, mp, sp);
         if (n < k_b)
             merge_row_stats(p.stats + static_cast<int64_t>(p.m_rows + d0 + n) * p.n_chunks, p.n_chunks, scale, mq, sq);
         double* ri = p.row_info + static_cast<int64_t>(b) * 4;
-        ri[0] = mp; ri[1] = sp; ri[2] = mq; ri[3] = sq;
+        ri[0] = mp; ri[1] = 1.0 / sp; ri[2] = mq; ri[3] = 1.0 / sq;
     }
 }
 
@@ -307,40 +264,60 @@ cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream)
 }
 
 // ------------------------------------------------------------------------------------ draw
-// Residual (or bonus) probability of vocabulary entry v of sequence b, fp64.
+// Row n of one sequence: p_v and the residual max(0, p_v - q_v).  The exponentials are the same
+// fp32 2^x as in the statistics pass, so numerator and normaliser share their rounding; products
+// and all sums are fp64.
 struct DrawRow {
     const float* zt; const float* zd; const uint32_t* mask;
-    double mp, sp, mq, sq, scale;
+    float mp, mq, c;
+    double inv_sp, inv_sq;
     bool residual;
-    __device__ __forceinline__ double prob_p(int v) const
+    __device__ __forceinline__ double prob_p(float z, int v) const
     {
-        const float z = zt[v];
         if (z == -INFINITY || !mask_allows(mask, v)) return 0.0;
-        return exp2((static_cast<double>(z) - mp) * scale) / sp;
+        return static_cast<double>(fast_exp2((z - mp) * c)) * inv_sp;
     }
-    __device__ __forceinline__ double prob_q(int v) const
+    __device__ __forceinline__ double prob_q(float z) const
     {
-        const float z = zd[v];
         if (z == -INFINITY) return 0.0;
-        return exp2((static_cast<double>(z) - mq) * scale) / sq;
+        return static_cast<double>(fast_exp2((z - mq) * c)) * inv_sq;
     }
-    __device__ __forceinline__ double resid(int v) const
+    // loads the 8 consecutive entries starting at v (v % 8 == 0) of the target / draft row
+    __device__ __forceinline__ void load8(const float* row, int v, int v_end, bool vec_ok, float (&out)[8]) const
     {
-        const double d = prob_p(v) - prob_q(v);
-        return d > 0.0 ? d : 0.0;
+        if (vec_ok && v + 7 < v_end) {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(row + v));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(row + v + 4));
+            out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+            out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) out[i] = (v + i < v_end) ? __ldg(row + v + i) : -INFINITY;
+        }
     }
 };
+
+__device__ __forceinline__ double warp_inclusive_scan(double v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
 
 __global__ void __launch_bounds__(kSampleThreads)
 sample_draw_kernel(const SampleParams p)
 {
-    __shared__ double red[kSampleThreads / 32];
-    __shared__ double scan[kSampleThreads];
-    __shared__ int s_is_last, s_chunk, s_use_p, s_found;
+    __shared__ double red_r[kSampleWarps];
+    __shared__ double red_p[kSampleWarps];
+    __shared__ int s_is_last, s_chunk, s_use_p, s_found, s_last;
     __shared__ double s_before, s_thr;
 
     const int chunk = blockIdx.x;
     const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int k_b = p.draft_len[b];
     const int n = p.accepted_len[b];
     DrawRow row;
@@ -349,103 +326,140 @@ sample_draw_kernel(const SampleParams p)
     row.zd = row.residual ? p.draft_logits + static_cast<int64_t>(p.cu_d[b] + n) * p.vocab : nullptr;
     row.mask = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(b) * p.mask_words : nullptr;
     const double* ri = p.row_info + static_cast<int64_t>(b) * 4;
-    row.mp = ri[0]; row.sp = ri[1]; row.mq = ri[2]; row.sq = ri[3];
-    row.scale = static_cast<double>(p.inv_temp_log2);
+    row.mp = static_cast<float>(ri[0]); row.inv_sp = ri[1];
+    row.mq = static_cast<float>(ri[2]); row.inv_sq = ri[3];
+    row.c = p.inv_temp_log2;
+    const bool vec_ok = ((p.vocab & 3) == 0);
 
-    // thread t owns the contiguous elements [v0 + t*32, v0 + t*32 + 32): vocabulary order is kept
-    const int v0 = chunk * kSampleChunk;
-    const int v_end = min(p.vocab, v0 + kSampleChunk);
-    const int my0 = v0 + threadIdx.x * kElemsPerThread;
-    double mass_r = 0.0, mass_p = 0.0;
-    for (int i = 0; i < kElemsPerThread; ++i) {
-        const int v = my0 + i;
-        if (v < v_end) {
-            const double pv = row.prob_p(v);
-            mass_p += pv;
-            if (row.residual) { const double d = pv - row.prob_q(v); mass_r += d > 0.0 ? d : 0.0; }
+    // thread t owns the contiguous entries [v0 + 8t, v0 + 8t + 8): vocabulary order is kept
+    {
+        const int v0 = chunk * kDrawChunk;
+        const int v_end = min(p.vocab, v0 + kDrawChunk);
+        const int my0 = v0 + threadIdx.x * kDrawElems;
+        double mass_r = 0.0, mass_p = 0.0;
+        if (my0 < v_end) {
+            float zt[8], zd[8];
+            row.load8(row.zt, my0, v_end, vec_ok, zt);
+            if (row.residual) row.load8(row.zd, my0, v_end, vec_ok, zd);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const double pv = row.prob_p(zt[i], my0 + i);
+                mass_p += pv;
+                if (row.residual) { const double d = pv - row.prob_q(zd[i]); mass_r += d > 0.0 ? d : 0.0; }
+            }
         }
+        mass_r = warp_sum(mass_r);
+        mass_p = warp_sum(mass_p);
+        if (lane == 0) { red_r[warp] = mass_r; red_p[warp] = mass_p; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double tr = 0.0, tp = 0.0;
+#pragma unroll
+            for (int w = 0; w < kSampleWarps; ++w) { tr += red_r[w]; tp += red_p[w]; }
+            double* cm = p.chunk_mass + (static_cast<int64_t>(b) * p.n_dchunks + chunk) * 2;
+            cm[0] = tr; cm[1] = tp;
+            __threadfence();
+            const int t = atomicAdd(&p.counters[kMaxBatch + b], 1);
+            s_is_last = (t == p.n_dchunks - 1);
+            if (s_is_last) { p.counters[kMaxBatch + b] = 0; __threadfence(); }
+        }
+        __syncthreads();
+        if (!s_is_last) return;
+        __threadfence();
     }
-    const double tot_r = block_sum(mass_r, red);
-    const double tot_p = block_sum(mass_p, red);
-    double* cm = p.chunk_mass + (static_cast<int64_t>(b) * p.n_chunks) * 2;
-    if (threadIdx.x == 0) { cm[chunk * 2 + 0] = tot_r; cm[chunk * 2 + 1] = tot_p; }
 
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int t = atomicAdd(&p.counters[kMaxBatch + b], 1);
-        s_is_last = (t == p.n_chunks - 1);
-        if (s_is_last) p.counters[kMaxBatch + b] = 0;
-    }
-    __syncthreads();
-    if (!s_is_last) return;
-    __threadfence();
-
-    // ---- the last CTA of the sequence: pick the chunk, then scan it in vocabulary order
-    if (threadIdx.x == 0) {
+    // ---- the last CTA of the sequence: pick the chunk that holds u' * Z ...
+    const double* cm = p.chunk_mass + static_cast<int64_t>(b) * p.n_dchunks * 2;
+    if (warp == 0) {
         double z_r = 0.0, z_p = 0.0;
-        for (int c = 0; c < p.n_chunks; ++c) { z_r += cm[c * 2]; z_p += cm[c * 2 + 1]; }
+        for (int c0 = 0; c0 < p.n_dchunks; c0 += 32) {
+            const int cc = c0 + lane;
+            z_r += (cc < p.n_dchunks) ? cm[cc * 2] : 0.0;
+            z_p += (cc < p.n_dchunks) ? cm[cc * 2 + 1] : 0.0;
+        }
+        z_r = warp_sum(z_r);
+        z_p = warp_sum(z_p);
         const int use_p = !(row.residual && z_r > 0.0);       // bonus row, or a residual lost to rounding
         const double z_mass = use_p ? z_p : z_r;
-        const double u2 = philox_uniform(p.seeds[b], static_cast<uint32_t>(n), 1u);
-        const double thr = u2 * z_mass;
-        double c_run = 0.0, before = 0.0;
+        const double thr = philox_uniform(p.seeds[b], static_cast<uint32_t>(n), 1u) * z_mass;
+        double carry = 0.0, last_before = 0.0;
         int pick = -1, last_pos = 0;
-        double last_before = 0.0;
-        for (int c = 0; c < p.n_chunks; ++c) {
-            const double m = cm[c * 2 + use_p];
-            if (m > 0.0) { last_pos = c; last_before = c_run; }
-            if (c_run + m > thr) { pick = c; before = c_run; break; }
-            c_run += m;
+        double before = 0.0;
+        for (int c0 = 0; c0 < p.n_dchunks && pick < 0; c0 += 32) {
+            const int cc = c0 + lane;
+            const double m = (cc < p.n_dchunks) ? cm[cc * 2 + use_p] : 0.0;
+            const double incl = warp_inclusive_scan(m, lane) + carry;
+            const unsigned hit = __ballot_sync(0xffffffffu, cc < p.n_dchunks && incl > thr);
+            const unsigned pos = __ballot_sync(0xffffffffu, m > 0.0);
+            if (hit != 0u) {
+                const int l = __ffs(hit) - 1;
+                pick = c0 + l;
+                before = __shfl_sync(0xffffffffu, incl - m, l);
+            } else if (pos != 0u) {
+                const int l = 31 - __clz(pos);
+                last_pos = c0 + l;
+                last_before = __shfl_sync(0xffffffffu, incl - m, l);
+            }
+            carry = __shfl_sync(0xffffffffu, incl, 31);
         }
         if (pick < 0) { pick = last_pos; before = last_before; }
-        s_chunk = pick; s_use_p = use_p; s_before = before; s_thr = thr;
-        s_found = 0x7fffffff;
+        if (lane == 0) {
+            s_chunk = pick; s_use_p = use_p; s_before = before; s_thr = thr;
+            s_found = 0x7fffffff; s_last = -1;
+        }
     }
     __syncthreads();
-    const int pc = s_chunk;
+
+    // ... and scan it in vocabulary order
     const bool use_p = s_use_p != 0;
-    const int w0 = pc * kSampleChunk + threadIdx.x * kElemsPerThread;
-    const int w_end = min(p.vocab, (pc + 1) * kSampleChunk);
-    double r[kElemsPerThread];
+    const int w0 = s_chunk * kDrawChunk + threadIdx.x * kDrawElems;
+    const int w_end = min(p.vocab, (s_chunk + 1) * kDrawChunk);
+    double r[8];
     double mine = 0.0;
-    for (int i = 0; i < kElemsPerThread; ++i) {
-        const int v = w0 + i;
-        r[i] = (v < w_end) ? (use_p ? row.prob_p(v) : row.resid(v)) : 0.0;
-        mine += r[i];
+    {
+        float zt[8], zd[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { zt[i] = -INFINITY; zd[i] = -INFINITY; }
+        if (w0 < w_end) {
+            row.load8(row.zt, w0, w_end, vec_ok, zt);
+            if (!use_p) row.load8(row.zd, w0, w_end, vec_ok, zd);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            double v = 0.0;
+            if (w0 + i < w_end) {
+                const double pv = row.prob_p(zt[i], w0 + i);
+                if (use_p) v = pv;
+                else { const double d = pv - row.prob_q(zd[i]); v = d > 0.0 ? d : 0.0; }
+            }
+            r[i] = v;
+            mine += v;
+        }
     }
-    scan[threadIdx.x] = mine;
+    const double incl = warp_inclusive_scan(mine, lane);
+    if (lane == 31) red_r[warp] = incl;
     __syncthreads();
-    if (threadIdx.x == 0) {                                   // exclusive scan, sequential: exact order
-        double run = s_before;
-        for (int t = 0; t < kSampleThreads; ++t) { const double m = scan[t]; scan[t] = run; run += m; }
-    }
-    __syncthreads();
-    double run = scan[threadIdx.x];
+    double run = s_before + (incl - mine);
+    for (int w = 0; w < warp; ++w) run += red_r[w];
     int found = 0x7fffffff, last_pos = -1;
-    for (int i = 0; i < kElemsPerThread; ++i) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
         run += r[i];
         if (r[i] > 0.0) last_pos = w0 + i;
-        if (run > s_thr && found == 0x7fffffff && w0 + i < w_end) found = w0 + i;
+        if (run > s_thr && found == 0x7fffffff && r[i] > 0.0) found = w0 + i;
     }
     if (found != 0x7fffffff) atomicMin(&s_found, found);
+    if (last_pos >= 0) atomicMax(&s_last, last_pos);
     __syncthreads();
-    if (s_found == 0x7fffffff) {
-        // rounding left no entry above the threshold: take the last entry with positive mass
-        __shared__ int s_last;
-        if (threadIdx.x == 0) s_last = -1;
-        __syncthreads();
-        if (last_pos >= 0) atomicMax(&s_last, last_pos);
-        __syncthreads();
-        if (threadIdx.x == 0) p.next_token[b] = s_last >= 0 ? s_last : 0;
-    } else if (threadIdx.x == 0) {
-        p.next_token[b] = s_found;
+    if (threadIdx.x == 0) {
+        // if rounding left no entry above the threshold: the last entry with positive mass
+        p.next_token[b] = (s_found != 0x7fffffff) ? s_found : (s_last >= 0 ? s_last : 0);
     }
 }
 
 cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream)
 {
-    dim3 grid(p.n_chunks, p.batch);
+    dim3 grid(p.n_dchunks, p.batch);
     sample_draw_kernel<<<grid, kSampleThreads, 0, stream>>>(p);
     return cudaGetLastError();
 }

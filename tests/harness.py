@@ -17,7 +17,7 @@ from paper_2601_00644_b200 import workloads as wl
 REL_TOL = 2e-2        # attention outputs and logits: bf16 inputs, fp32 accumulation
 PROB_TOL = 1e-5       # probabilities, absolute
 TIE_TOL = 1e-5        # |u - min(1, p/q)| below this is a near-tie: counted, not required to match
-CDF_TIE_TOL = 1e-9    # same for the inverse-CDF boundary when both sides see identical logits
+CDF_TIE_TOL = 1e-6    # inverse-CDF boundary, same logits on both sides: fp32 exponentials (2^-22 rel.) vs fp64
 
 
 def rel_close(got: np.ndarray, ref: np.ndarray, tol: float = REL_TOL):

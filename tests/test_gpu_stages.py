@@ -174,7 +174,7 @@ def test_sample_stage_matches_oracle(mode, temperature, vocab, batch, k_hi, hole
             n_ties += 1
             continue
         if nxt[b] != ref["next_token"][b]:
-            assert not greedy and ref["cdf_margin"][b] < 1e-9, (b, nxt[b], ref["next_token"][b], ref["cdf_margin"][b])
+            assert not greedy and ref["cdf_margin"][b] < 1e-6, (b, nxt[b], ref["next_token"][b], ref["cdf_margin"][b])
     assert n_ties <= 1
     if not greedy and k.sum() > 0:
         dbg = ver.debug(int(k.sum()) + batch, int(k.sum()))
