@@ -75,9 +75,8 @@ struct DeviceGuard {
 
 void free_workspace(Handle& h)
 {
-    cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml);
+    cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml); cudaFree(h.att_tickets);
     cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq);
-    cudaFree(h.plan.seq_blk0); cudaFree(h.plan.seq_pair0); cudaFree(h.plan.cta_start);
     cudaFree(h.stats); cudaFree(h.arg_idx); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.chunk_mass);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
@@ -123,11 +122,9 @@ void mark(Handle& h, int idx, cudaStream_t s)
     if (h.profiling) { cudaEventRecord(h.ev[idx], s); h.ev_used[idx] = 1; }
 }
 
-int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, const int32_t* kv_len,
-             const Geometry& g, int32_t batch, cudaStream_t s)
+int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, cudaStream_t s)
 {
-    if (launch_plan(draft_len, draft_tokens, kv_len, batch, h.cfg.vocab, h.cfg.n_kv_heads,
-                    h.cfg.n_q_heads / h.cfg.n_kv_heads, g.att_ctas, h.plan, h.status, s) != cudaSuccess)
+    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, h.plan, h.status, s) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
     h.launches++;
     return FLEXSPEC_OK;
@@ -144,35 +141,19 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     int rc = make_map_2d(&kv_map, kv->kv_pages, pool_rows, static_cast<uint64_t>(c.head_dim), 16);
     if (rc != FLEXSPEC_OK) return rc;
 
-    const int max_tile_rows = group * (g.k_batch_max + 1);
-    const int n_cw = attention_consumer_warps(max_tile_rows);
-
     AttnParams p;
     p.hidden = static_cast<const __nv_bfloat16*>(hidden);
     p.page_table = kv->page_table;
     p.kv_len = kv->kv_len;
     p.draft_len = draft_len;
-    p.cu_q = h.plan.cu_q;
-    p.seq_blk0 = h.plan.seq_blk0; p.seq_pair0 = h.plan.seq_pair0; p.cta_start = h.plan.cta_start;
     p.batch = batch;
     p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = group;
     p.max_pages_per_seq = kv->max_pages_per_seq; p.num_pages = kv->num_pages;
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(c.head_dim)));
-    p.part_o = h.part_o; p.part_ml = h.part_ml;
+    p.part_o = h.part_o; p.part_ml = h.part_ml; p.tickets = h.att_tickets;
+    p.attn_out = static_cast<__nv_bfloat16*>(attn_out);
     p.status = h.status;
-    if (launch_attention(h, kv_map, p, g.att_ctas, n_cw, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    h.launches++;
-    mark(h, 2, s);
-    CombineParams cp;
-    cp.part_o = h.part_o; cp.part_ml = h.part_ml;
-    cp.kv_len = kv->kv_len; cp.draft_len = draft_len; cp.cu_q = h.plan.cu_q;
-    cp.seq_blk0 = h.plan.seq_blk0; cp.seq_pair0 = h.plan.seq_pair0;
-    cp.batch = batch; cp.n_q_heads = c.n_q_heads; cp.n_kv_heads = c.n_kv_heads; cp.group = group;
-    cp.head_dim = c.head_dim;
-    cp.n_ctas = g.att_ctas; cp.n_cw = n_cw;
-    cp.pairs_per_seq_max = c.n_kv_heads * ((max_tile_rows + kAttRowsPerPair - 1) / kAttRowsPerPair);
-    cp.attn_out = static_cast<__nv_bfloat16*>(attn_out);
-    if (launch_attention_combine(cp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_attention(h, kv_map, p, g.att_ctas, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     return FLEXSPEC_OK;
 }
@@ -294,13 +275,12 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.logits, static_cast<size_t>(max_m) * c.vocab));
     // attention partial slots: one per (pair, CTA) segment, index pair + CTA
     const int group = c.n_q_heads / c.n_kv_heads;
-    const size_t att_slots = static_cast<size_t>(c.max_batch) * c.n_kv_heads *
-                                 ((group * (c.k_max + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair) + h.sm_count;
-    A(dev_alloc(&h.part_o, att_slots * kAttMaxConsumerWarps * 16 * c.head_dim));
-    A(dev_alloc(&h.part_ml, att_slots * kAttMaxConsumerWarps * 16 * 2));
-    A(dev_alloc(&h.plan.seq_blk0, static_cast<size_t>(c.max_batch) + 1));
-    A(dev_alloc(&h.plan.seq_pair0, static_cast<size_t>(c.max_batch) + 1));
-    A(dev_alloc(&h.plan.cta_start, static_cast<size_t>(h.sm_count)));
+    h.att_pairs_max = c.max_batch * c.n_kv_heads * ((group * (c.k_max + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
+    // split-merge scratch: every CTA parks at most its first and its last segment
+    const size_t att_slots = static_cast<size_t>(2) * h.sm_count;
+    A(dev_alloc(&h.part_o, att_slots * kAttRowsPerPair * c.head_dim));
+    A(dev_alloc(&h.part_ml, att_slots * kAttRowsPerPair * 2));
+    A(dev_alloc(&h.att_tickets, static_cast<size_t>(h.att_pairs_max)));
     A(dev_alloc(&h.plan.cu_q, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
@@ -322,6 +302,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     }
     if (rc == FLEXSPEC_OK) {
         if (cudaMemset(h.counters, 0, sizeof(int32_t) * 2 * kMaxBatch) != cudaSuccess ||
+            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max)) != cudaSuccess ||
             cudaMemset(h.status, 0, sizeof(int32_t) * 4) != cudaSuccess)
             rc = FLEXSPEC_ERR_CUDA;
     }
@@ -370,14 +351,13 @@ int flexspec_attention(flexspec_handle* fh, const flexspec_kv* kv, const void* h
     Handle& h = fh->h;
     if (!kv_args_ok(h, kv, true)) return FLEXSPEC_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(attn_out) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
     Geometry g;
     int rc = check_lengths(h, draft_len_host, kv->kv_len_host, batch, kv->max_pages_per_seq, &g);
     if (rc != FLEXSPEC_OK) return rc;
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    rc = run_plan(h, draft_len, nullptr, kv->kv_len, g, batch, s);
-    if (rc != FLEXSPEC_OK) return rc;
     return run_attention(h, kv, hidden, draft_len, g, batch, attn_out ? attn_out : h.attn_out, s);
 }
 
@@ -407,7 +387,7 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    rc = run_plan(h, draft_len, draft_tokens, nullptr, g, batch, s);
+    rc = run_plan(h, draft_len, draft_tokens, batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     return run_sample(h, logits ? logits : h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch,
                       temperature, vocab_mask, accepted_len, next_token, s);
@@ -434,11 +414,12 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     h.launches = 0;
     memset(h.ev_used, 0, sizeof(h.ev_used));
     mark(h, 0, s);
-    rc = run_plan(h, draft_len, draft_tokens, kv->kv_len, g, batch, s);
+    rc = run_plan(h, draft_len, draft_tokens, batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 1, s);
-    rc = run_attention(h, kv, hidden, draft_len, g, batch, h.attn_out, s);   // marks event 2 after the split kernel
+    rc = run_attention(h, kv, hidden, draft_len, g, batch, h.attn_out, s);
     if (rc != FLEXSPEC_OK) return rc;
+    mark(h, 2, s);
     mark(h, 3, s);
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, s);
     if (rc != FLEXSPEC_OK) return rc;

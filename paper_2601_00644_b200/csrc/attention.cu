@@ -8,46 +8,146 @@
 // (8 pages of 16).  All blocks of the batch, numbered sequence by sequence and pair by pair, are
 // divided into equal contiguous ranges, one per CTA, with one CTA per SM: a single balanced wave
 // whatever the mix of context lengths and draft lengths.  A CTA therefore works on a few
-// "segments" (runs of blocks of one pair).
+// "segments" (runs of blocks of one pair).  Every CTA derives its own range from draft_len[] and
+// kv_len[] (a block-wide prefix sum over the sequences), so no planning kernel runs first.
 //
-// Inside a CTA: warp 0 is the TMA producer (one 4 KB K and V page per lane, 128-byte swizzle,
-// 3 stages of 128 tokens, full/empty mbarriers, every wait bounded); the other warps consume.
-// Each consumer warp owns one 16-row tile of the pair and a subset of the pages of every stage:
-// QK^T and PV on mma.sync m16n8k16 (bf16 in, fp32 accumulate), fp32 online softmax in registers
-// with the row max / sum reduced over the 4 lanes of a quad by shuffles.  At the end of a segment
-// every consumer warp writes its unnormalised partial (running max, sum, output tile); a second
-// small kernel merges the partials of a pair by log-sum-exp and rounds to bf16.
+// Both contractions run on the 5th-generation tensor cores with accumulators in tensor memory
+// (the legacy warp-level MMA path cannot keep up with the KV stream):
+//   S[128 query rows][128 tokens] = Q K^T     A = Q tile, B = K tile, both K-major in shared memory
+//   O[128 query rows][Dh]        += P V       A = P (bf16, written by the softmax threads),
+//                                             B = V tile as TMA delivers it ([token][Dh]: MN-major)
+// The query rows of the pair occupy the first rows of the M = 128 tile; the remaining rows are
+// padding whose results are never read.
+//
+// Warp roles.  Warp 0: TMA producer (one 16-token K and V page per lane, 128-byte swizzle, a ring
+// of 128-token stages).  Warp 1: one thread issues every tcgen05.mma; the warp owns the TMEM
+// allocation.  Warps 2..5: softmax, one thread per TMEM lane (= tile row, so a row's maximum and
+// sum need no shuffles): two passes over the scores of the block with tcgen05.ld -- maximum, then
+// p = 2^(s - m) written to shared memory as bf16 -- with S double buffered so that the next
+// block's QK^T overlaps.  A pair with at most 32 (64) rows is replicated 4 (2) times over the
+// tile rows and each copy takes a quarter (half) of the block's tokens, so all four warps work
+// on small pairs.  The running maximum is only raised when it grew by more than 2^8 (O in TMEM
+// is then rescaled); the final division by the row sum makes the stale maximum cancel.  At the end of a segment the softmax threads read O from TMEM; if the
+// pair spans several CTAs they park (m, l, O) in global scratch and the CTA that completes the
+// pair last (atomic ticket, nobody waits) merges the parts by log-sum-exp in CTA order.
+// Every mbarrier wait is bounded.
 #include "common.cuh"
 #include "internal.h"
 
 namespace fs {
 
-constexpr int kAttPagesPerStage = 8;     // 8 pages = 128 tokens = kAttBlockTokens
-constexpr int kAttStages = 3;
 constexpr int kPageTokens = 16;
-constexpr int kAttMaxThreads = (kAttMaxConsumerWarps + 1) * 32;
+constexpr int kAttPagesPerStage = kAttBlockTokens / kPageTokens;    // 8
+constexpr int kAttSoftmaxThreads = 128;
+constexpr int kAttTmemCols = 512;
+constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column offsets
+constexpr float kRescaleThreshold = 8.f;                             // log2 units
 
 template <int DH>
 struct AttCfg {
-    static constexpr int kHalves = DH / 64;                    // 128-byte column slabs per row
-    static constexpr int kSlabBytes = kPageTokens * 128;       // 16 tokens x 64 bf16
-    static constexpr int kPageBytes = kHalves * kSlabBytes;    // K (or V) of one page, one kv head
-    static constexpr int kStageBytes = kAttPagesPerStage * 2 * kPageBytes;
-    static constexpr int kBarOffset = kAttStages * kStageBytes;
-    static constexpr int kSmemBytes = kBarOffset + 128 + 1024;  // + barriers + alignment slack
+    static constexpr int kSlabs = DH / 64;                     // 128-byte column slabs per row
+    static constexpr int kSlabBytes = 128 * 128;               // 128 rows x 64 bf16
+    static constexpr int kStageBytes = 2 * kSlabs * kSlabBytes;      // K slabs, then V slabs
+    static constexpr int kStages = (DH == 128) ? 2 : 4;
+    static constexpr int kQOffset = kStages * kStageBytes;
+    static constexpr int kQBytes = kSlabs * kSlabBytes;
+    static constexpr int kPOffset = kQOffset + kQBytes;
+    static constexpr int kPBytes = 2 * kSlabBytes;             // 128 rows x 128 tokens bf16
+    static constexpr int kBarOffset = kPOffset + 2 * kPBytes;
+    static constexpr int kSmemBytes = kBarOffset + 256 + 1024; // + barriers + alignment slack
 };
 
-// byte offset of 16-byte chunk `c` of row `r` inside a 128-byte-swizzled slab
-__device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t c)
+struct AttBars {
+    uint64_t kv_full[4], kv_empty[4];
+    uint64_t s_full[2], s_empty[2];
+    uint64_t p_full[2], p_empty[2];
+    uint64_t q_full, o_full, group;
+    uint32_t tmem_slot;
+};
+static_assert(sizeof(AttBars) <= 256, "barrier block");
+
+__device__ __forceinline__ void prefetch_l2(const void* p)
 {
-    return r * 128u + ((c ^ (r & 7u)) << 4);
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
-// Position in the batch-wide block list; producer and consumers walk it in lock step.
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp reads TMEM lane (base lane + i).
+__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr),
+          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait()
+{
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of an MN-major bf16 operand laid out by TMA with the 128-byte
+// swizzle: rows of 64 MN-elements (128 B) indexed by k, groups of 8 k-rows `sbo` bytes apart,
+// the next 64 MN-elements `lbo` bytes away.
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo, uint32_t sbo)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;                       // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                       // 128-byte swizzle
+    return d;
+}
+constexpr uint32_t kIdescBMajorMN = 1u << 16;
+
+// Exclusive prefix sum over the block of one int per thread; returns the block total in `total`.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int& total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_warps = (blockDim.x + 31) >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int before = 0, sum = 0;
+    for (int w = 0; w < n_warps; ++w) {
+        const int t = warp_tot[w];
+        if (w < warp) before += t;
+        sum += t;
+    }
+    __syncthreads();
+    total = sum;
+    return before + incl - v;
+}
+
+// Position in the batch-wide block list; every role walks it in lock step.
 struct AttCursor {
     int b, pair, blk;             // sequence, pair inside it, block inside the pair
     int k, kvl, nb, rbc, pairs;   // of sequence b: draft length, kv length, blocks per pair,
                                   // row blocks per kv head, pairs
+    int q_row0, pair0, blk0;      // first query row / first pair / first block of sequence b
     __device__ __forceinline__ void load_seq(const AttnParams& p)
     {
         k = p.draft_len[b];
@@ -56,13 +156,6 @@ struct AttCursor {
         rbc = (p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair;
         pairs = p.n_kv_heads * rbc;
     }
-    __device__ __forceinline__ void start(const AttnParams& p, int2 where)
-    {
-        b = where.x;
-        load_seq(p);
-        pair = where.y / nb;
-        blk = where.y % nb;
-    }
     // returns true when the step left the current pair
     __device__ __forceinline__ bool advance(const AttnParams& p, bool more)
     {
@@ -70,6 +163,9 @@ struct AttCursor {
         blk = 0;
         if (++pair == pairs) {
             pair = 0;
+            q_row0 += k + 1;
+            pair0 += pairs;
+            blk0 += pairs * nb;
             ++b;
             if (more && b < p.batch) load_seq(p);
         }
@@ -77,49 +173,125 @@ struct AttCursor {
     }
 };
 
+struct AttStart { int b, blk_off, q_row0, pair0, blk0, total; };
+
 template <int DH>
-__global__ void __launch_bounds__(kAttMaxThreads, 1)
+__global__ void __launch_bounds__(kAttThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
     using Cfg = AttCfg<DH>;
-    const int64_t total_blocks = p.seq_blk0[p.batch];
-    const int cta = blockIdx.x;
-    const int blk_begin = static_cast<int>(cta * total_blocks / gridDim.x);
-    const int blk_end = static_cast<int>((cta + 1) * total_blocks / gridDim.x);
-    const int n_my = blk_end - blk_begin;
-    if (n_my <= 0) return;
-
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOffset);
-    uint64_t* empty_bar = full_bar + kAttStages;
+    AttBars* bars = reinterpret_cast<AttBars*>(smem + Cfg::kBarOffset);
+    __shared__ int s_warp_tot[32];
+    __shared__ AttStart s_start;
+    __shared__ int s_flag;
+    __shared__ float s_xch[3][kAttSoftmaxThreads];          // [0..1] row maxima (by block parity), [2] row sums, exchanged between the copies of a row
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int n_cw = (blockDim.x >> 5) - 1;             // consumer warps
+    const int cta = blockIdx.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kAttStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], n_cw); }
+        for (int s = 0; s < 4; ++s) { mbar_init(&bars->kv_full[s], 1); mbar_init(&bars->kv_empty[s], 1); }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], kAttSoftmaxThreads);
+            mbar_init(&bars->p_full[a], kAttSoftmaxThreads); mbar_init(&bars->p_empty[a], 1);
+        }
+        mbar_init(&bars->q_full, kAttSoftmaxThreads);
+        mbar_init(&bars->o_full, 1);
+        mbar_init(&bars->group, kAttSoftmaxThreads);
         fence_barrier_init();
         tma_prefetch_desc(&kv_map);
     }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_slot, kAttTmemCols);
+        tmem_relinquish();
+    }
+
+    // ---- where this CTA starts: prefix sums of blocks / pairs / rows over the sequences
+    int blk_begin, n_my;
+    {
+        const int per = (p.batch + blockDim.x - 1) / blockDim.x;
+        const int b_lo = min(p.batch, static_cast<int>(threadIdx.x) * per);
+        const int b_hi = min(p.batch, b_lo + per);
+        int my_blocks = 0, my_pairs = 0, my_rows = 0;
+        for (int b = b_lo; b < b_hi; ++b) {
+            const int k = p.draft_len[b];
+            const int nb = (p.kv_len[b] + kAttBlockTokens - 1) / kAttBlockTokens;
+            const int pairs = p.n_kv_heads * ((p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
+            my_blocks += pairs * nb;
+            my_pairs += pairs;
+            my_rows += k + 1;
+        }
+        int total, unused;
+        const int ex_blocks = block_exclusive_scan(my_blocks, s_warp_tot, total);
+        const int ex_pairs = block_exclusive_scan(my_pairs, s_warp_tot, unused);
+        const int ex_rows = block_exclusive_scan(my_rows, s_warp_tot, unused);
+        const int64_t t64 = total;
+        blk_begin = static_cast<int>(cta * t64 / gridDim.x);
+        n_my = static_cast<int>((cta + 1) * t64 / gridDim.x) - blk_begin;
+        if (n_my > 0 && blk_begin >= ex_blocks && blk_begin < ex_blocks + my_blocks) {
+            int blk0 = ex_blocks, pair0 = ex_pairs, row0 = ex_rows;
+            for (int b = b_lo; b < b_hi; ++b) {
+                const int k = p.draft_len[b];
+                const int nb = (p.kv_len[b] + kAttBlockTokens - 1) / kAttBlockTokens;
+                const int pairs = p.n_kv_heads * ((p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
+                if (blk_begin < blk0 + pairs * nb) {
+                    s_start.b = b; s_start.blk_off = blk_begin - blk0;
+                    s_start.q_row0 = row0; s_start.pair0 = pair0; s_start.blk0 = blk0;
+                    break;
+                }
+                blk0 += pairs * nb; pair0 += pairs; row0 += k + 1;
+            }
+        }
+        if (threadIdx.x == 0) s_start.total = total;
+    }
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_slot;
+    const int64_t total_blocks = s_start.total;
 
     AttCursor cur;
-    cur.start(p, p.cta_start[cta]);
+    if (n_my > 0) {
+        cur.b = s_start.b;
+        cur.q_row0 = s_start.q_row0; cur.pair0 = s_start.pair0; cur.blk0 = s_start.blk0;
+        cur.load_seq(p);
+        cur.pair = s_start.blk_off / cur.nb;
+        cur.blk = s_start.blk_off % cur.nb;
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         const uint64_t pol = l2_policy_evict_first();
-        for (int q = 0; q < n_my; ++q) {
-            const int s = q % kAttStages;
-            const int use = q / kAttStages;
-            if (use > 0) mbar_wait(&empty_bar[s], (use - 1) & 1, p.status, 1);
+        bool new_pair = true;
+        bool ok = true;
+        int last_st = -1;
+        uint32_t last_ph = 0;
+        for (int q = 0; q < n_my && ok; ++q) {
             const int kvh = cur.pair / cur.rbc;
+            if (new_pair) {
+                // bring the pair's query rows into L2 ahead of the softmax threads that copy them
+                const int row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
+                const int rows_here = min(kAttRowsPerPair, p.group * (cur.k + 1) - row_lo);
+                const int j_lo = row_lo / p.group, j_hi = (row_lo + rows_here - 1) / p.group;
+                const int lines_per_j = (p.group * DH * 2 + 127) / 128;
+                for (int i = lane; i < (j_hi - j_lo + 1) * lines_per_j; i += 32) {
+                    const int j = j_lo + i / lines_per_j;
+                    const uint8_t* base = reinterpret_cast<const uint8_t*>(
+                        p.hidden + (static_cast<int64_t>(cur.q_row0 + j) * p.n_q_heads + kvh * p.group) * DH);
+                    prefetch_l2(base + (i % lines_per_j) * 128);
+                }
+            }
+            const int st = q % Cfg::kStages;
+            const int use = q / Cfg::kStages;
+            if (use > 0 && !mbar_wait(&bars->kv_empty[st], (use - 1) & 1, p.status, 1)) { ok = false; break; }
             const int t_begin = cur.blk * kAttBlockTokens;
             const int t_end = min(cur.kvl, t_begin + kAttBlockTokens);
             const int npg = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
-            if (lane == 0) mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(npg * 2 * Cfg::kPageBytes));
+            if (lane == 0)
+                mbar_arrive_expect_tx(&bars->kv_full[st], static_cast<uint32_t>(npg * 2 * Cfg::kSlabs * kPageTokens * 128));
             __syncwarp();
             if (lane < npg) {
                 const int page_idx = cur.blk * kAttPagesPerStage + lane;
@@ -128,248 +300,389 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
                     report_error(p.status, kErrBadPage, phys, 1);
                     phys = 0;                               // stay inside the pool
                 }
-                uint8_t* dst = smem + s * Cfg::kStageBytes + lane * 2 * Cfg::kPageBytes;
+                uint8_t* dst = smem + st * Cfg::kStageBytes + lane * (kPageTokens * 128);
                 const int row_k = ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens;
                 const int row_v = ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens;
 #pragma unroll
-                for (int hf = 0; hf < Cfg::kHalves; ++hf) {
-                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &full_bar[s], hf * 64, row_k, pol);
-                    tma_load_2d(dst + Cfg::kPageBytes + hf * Cfg::kSlabBytes, &kv_map, &full_bar[s], hf * 64, row_v, pol);
+                for (int hf = 0; hf < Cfg::kSlabs; ++hf) {
+                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &bars->kv_full[st], hf * 64, row_k, pol);
+                    tma_load_2d(dst + (Cfg::kSlabs + hf) * Cfg::kSlabBytes, &kv_map, &bars->kv_full[st], hf * 64, row_v, pol);
                 }
             }
             __syncwarp();
-            cur.advance(p, q + 1 < n_my);
+            last_st = st; last_ph = use & 1;
+            new_pair = cur.advance(p, q + 1 < n_my);
         }
-        return;     // consumers wait on every full barrier, so no copy is in flight when the CTA ends
-    }
+        // do not leave while a copy of ours may still be landing in shared memory
+        if (last_st >= 0) mbar_wait(&bars->kv_full[last_st], last_ph, p.status, 9);
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && n_my > 0) {
+            const uint32_t idesc_s = umma_idesc_bf16(128, 128);
+            const uint32_t idesc_o = umma_idesc_bf16(128, DH) | kIdescBMajorMN;
+            const uint32_t q_addr = smem_u32(smem + Cfg::kQOffset);
+            bool ok = true;
+            int seg = 0;
+            // S[q & 1] = Q K^T of block q (waits: the pair's Q tile, the K/V stage, the S buffer)
+            auto issue_s = [&](int q, bool seg_first, int seg_idx) -> bool {
+                const int st = q % Cfg::kStages, buf = q & 1, u = q >> 1;
+                if (seg_first && !mbar_wait(&bars->q_full, seg_idx & 1, p.status, 2)) return false;
+                if (!mbar_wait(&bars->kv_full[st], (q / Cfg::kStages) & 1, p.status, 3)) return false;
+                if (u > 0 && !mbar_wait(&bars->s_empty[buf], (u - 1) & 1, p.status, 4)) return false;
+                tc_fence_after();
+                const uint32_t k_addr = smem_u32(smem + st * Cfg::kStageBytes);
+                const uint32_t acc = tmem_base + (buf ? kTmemS1 : kTmemS0);
+#pragma unroll
+                for (int kk = 0; kk < DH / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32;
+                    umma_bf16(acc, umma_desc_k_sw128(q_addr + off), umma_desc_k_sw128(k_addr + off), idesc_s, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(&bars->s_full[buf]);
+                return true;
+            };
+            bool seg_first = true;
+            ok = issue_s(0, true, 0);
+            for (int q = 0; q < n_my && ok; ++q) {
+                const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
+                const int st = q % Cfg::kStages, buf = q & 1, u = q >> 1;
+                if (!seg_last && q + 1 < n_my) { if (!issue_s(q + 1, false, seg)) { ok = false; break; } }   // overlap with softmax of q
+                if (!mbar_wait(&bars->p_full[buf], u & 1, p.status, 5)) { ok = false; break; }
+                tc_fence_after();
+                {
+                    const uint32_t p_addr = smem_u32(smem + Cfg::kPOffset + buf * Cfg::kPBytes);
+                    const uint32_t v_addr = smem_u32(smem + st * Cfg::kStageBytes + Cfg::kSlabs * Cfg::kSlabBytes);
+#pragma unroll
+                    for (int ks = 0; ks < kAttBlockTokens / 16; ++ks) {
+                        const uint64_t da = umma_desc_k_sw128(p_addr + (ks >> 2) * Cfg::kSlabBytes + (ks & 3) * 32);
+                        const uint64_t db = umma_desc_mn_sw128(v_addr + ks * 2048, Cfg::kSlabBytes, 1024);
+                        umma_bf16(tmem_base + kTmemO, da, db, idesc_o, (seg_first && ks == 0) ? 0u : 1u);
+                    }
+                }
+                umma_commit(&bars->kv_empty[st]);
+                umma_commit(&bars->p_empty[buf]);
+                umma_commit(&bars->o_full);
+                cur.advance(p, q + 1 < n_my);
+                seg_first = seg_last;
+                if (seg_last) {
+                    ++seg;
+                    if (q + 1 < n_my && !issue_s(q + 1, true, seg)) { ok = false; break; }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax
+        // Thread t owns TMEM lane t.  When the pair has at most 32 (64) query rows the Q tile holds
+        // 4 (2) copies of them, copy c in tile rows [c*span, (c+1)*span), span = 128 / copies, and
+        // the thread of tile row c*span + r handles tokens [c*span, (c+1)*span) of row r in every
+        // block: all four warps share the work of a small pair.  The copies agree on the row
+        // maximum through shared memory and write their part of P into row r of ONE P tile, so O is
+        // complete in tile rows [0, span) and needs no merge.
+        const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
+        const int t = quarter * 32 + lane;                  // tile row
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        uint8_t* q_smem = smem + Cfg::kQOffset;
+        bool ok = true;
+        bool seg_first = true;
+        int seg = 0;
+        uint32_t group_phase = 0;
+        float m_used = -INFINITY, l_run = 0.f;
+        int rows_here = 0, row_lo = 0, limit = 0, ctx = 0;
+        int copies = 1, span = 128, c = 0, r = t;
 
-    // ---------------------------------------------------------------------- consumers
-    const int cw = warp - 1;
-    const int g = lane >> 2, tq = lane & 3;
+        // all softmax threads meet; bounded like every other wait
+        auto group_sync = [&](int where) -> bool {
+            mbar_arrive(&bars->group);
+            const bool done = mbar_wait(&bars->group, group_phase, p.status, where);
+            group_phase ^= 1u;
+            return done;
+        };
 
-    uint32_t qa[DH / 16][4];
-    float o[DH / 8][4];
-    float m_run[2], l_run[2];
-    int limit[2];
-    int rt = 0, slice = 0, n_slices = 1, n_rt = 1, ctx = 0;
-    bool new_segment = true;
-
-    for (int q = 0; q < n_my; ++q) {
-        if (new_segment) {
-            // ---- set up the pair: row tile of this warp, query fragments, causal limits
+        for (int q = 0; q < n_my && ok; ++q) {
             const int kvh = cur.pair / cur.rbc;
-            const int row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
-            const int n_rows = p.group * (cur.k + 1);
-            const int rows_here = min(kAttRowsPerPair, n_rows - row_lo);
-            n_rt = (rows_here + 15) >> 4;
-            rt = cw % n_rt;
-            slice = cw / n_rt;
-            n_slices = (n_cw - rt + n_rt - 1) / n_rt;
-            ctx = cur.kvl - (cur.k + 1);
-            const int q_row0 = p.cu_q[cur.b];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const int rho = row_lo + rt * 16 + g + i * 8;
-                const bool real = rho < n_rows;
-                limit[i] = real ? ctx + rho / p.group + 1 : cur.kvl;     // padded rows see everything
-                const uint32_t* src = nullptr;
-                if (real) {
+            if (seg_first) {
+                // ---- the pair's query rows -> shared memory in the K-major swizzled layout of operand A
+                row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
+                const int n_rows = p.group * (cur.k + 1);
+                rows_here = min(kAttRowsPerPair, n_rows - row_lo);
+                ctx = cur.kvl - (cur.k + 1);
+                copies = rows_here <= 32 ? 4 : (rows_here <= 64 ? 2 : 1);
+                span = kAttRowsPerPair / copies;
+                c = t / span;
+                r = t % span;
+                if (r < rows_here) {
+                    const int rho = row_lo + r;
                     const int j = rho / p.group, hh = rho % p.group;
-                    src = reinterpret_cast<const uint32_t*>(
-                        p.hidden + (static_cast<int64_t>(q_row0 + j) * p.n_q_heads + kvh * p.group + hh) * DH);
-                }
+                    limit = ctx + j + 1;
+                    const uint4* src = reinterpret_cast<const uint4*>(
+                        p.hidden + (static_cast<int64_t>(cur.q_row0 + j) * p.n_q_heads + kvh * p.group + hh) * DH);
+                    uint4 v[DH / 8];
 #pragma unroll
-                for (int kk = 0; kk < DH / 16; ++kk) {
-                    // A fragment of m16n8k16: regs 0/1 = rows g / g+8, cols 2tq..; regs 2/3 = cols 8+2tq..
-                    qa[kk][i] = real ? __ldg(src + kk * 8 + tq) : 0u;
-                    qa[kk][i + 2] = real ? __ldg(src + kk * 8 + 4 + tq) : 0u;
+                    for (int ch = 0; ch < DH / 8; ++ch) v[ch] = __ldg(src + ch);
+#pragma unroll
+                    for (int ch = 0; ch < DH / 8; ++ch)
+                        *reinterpret_cast<uint4*>(q_smem + (ch >> 3) * Cfg::kSlabBytes + t * 128 + (((ch & 7) ^ (t & 7)) << 4)) = v[ch];
                 }
+                m_used = -INFINITY;
+                l_run = 0.f;
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(&bars->q_full);
             }
-#pragma unroll
-            for (int nt = 0; nt < DH / 8; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
-            m_run[0] = m_run[1] = -INFINITY;
-            l_run[0] = l_run[1] = 0.f;
-            new_segment = false;
-        }
+            const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
+            const int st = q % Cfg::kStages, buf = q & 1, u = q >> 1;
+            const int t_begin = cur.blk * kAttBlockTokens;
+            const bool real = r < rows_here;
+            const bool warp_real = (quarter * 32) % span < rows_here;    // warp-uniform: a real row among this warp's lanes
+            const bool o_owner = (quarter * 32 < span) && warp_real;      // warp-uniform: this warp's lanes hold real rows of O
+            const uint32_t t_s = t_lane + (buf ? kTmemS1 : kTmemS0) + static_cast<uint32_t>(c * span);
+            const int lim_local = (real ? limit : 0) - t_begin - c * span;   // my tokens [0, lim_local) are visible
+            const bool need_mask = (t_begin + kAttBlockTokens > ctx + 1);
 
-        const int s = q % kAttStages;
-        mbar_wait(&full_bar[s], (q / kAttStages) & 1, p.status, 2);
-        const int t_begin = cur.blk * kAttBlockTokens;
-        const int t_end = min(cur.kvl, t_begin + kAttBlockTokens);
-        const int npg = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
-        const uint8_t* stage = smem + s * Cfg::kStageBytes;
+            if (!mbar_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
+            tc_fence_after();
 
-        for (int pi = slice; pi < npg; pi += n_slices) {
-            const uint8_t* kp = stage + pi * 2 * Cfg::kPageBytes;
-            const uint8_t* vp = kp + Cfg::kPageBytes;
-            const int tok0 = t_begin + pi * kPageTokens;
-
-            // S = Q K^T for 16 rows x 16 tokens
-            float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            {
-                const int mi = lane >> 3;
-                const uint32_t tok = (mi >> 1) * 8 + (lane & 7);
+            // ---- pass 1: maximum over my tokens of the block, then over the copies of the row
+            float mx = -INFINITY;
+            if (warp_real) {
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                for (int c0 = 0; c0 < span; c0 += 32) {
+                    uint32_t sv[32];
+                    tmem_ld_x32(t_s + c0, sv);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int kk = 0; kk < DH / 16; ++kk) {
-                    const int ch = 2 * kk + (mi & 1);
-                    uint32_t kb[4];
-                    ldmatrix_x4(kb, smem_u32(kp + (ch >> 3) * Cfg::kSlabBytes + swz(tok, ch & 7)));
-                    mma_bf16_16816(sc[0], qa[kk], kb[0], kb[1]);
-                    mma_bf16_16816(sc[1], qa[kk], kb[2], kb[3]);
-                }
-            }
-            // scale to log2 units, causal mask inside the draft window
-            const bool need_mask = (tok0 + kPageTokens > ctx + 1);
-#pragma unroll
-            for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = sc[nt][e] * p.scale_log2;
-                    if (need_mask) {
-                        const int t = tok0 + nt * 8 + tq * 2 + (e & 1);
-                        if (t >= limit[e >> 1]) v = -INFINITY;
-                    }
-                    sc[nt][e] = v;
-                }
-            // online softmax: row max over the quad, rescale, exponentiate
-            float alpha[2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                float mx = fmaxf(fmaxf(sc[0][2 * i], sc[0][2 * i + 1]), fmaxf(sc[1][2 * i], sc[1][2 * i + 1]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run[i], mx);
-                const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-                alpha[i] = fast_exp2(m_run[i] - m_safe);
-                m_run[i] = m_new;
-                float rs = 0.f;
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-                    sc[nt][2 * i] = fast_exp2(sc[nt][2 * i] - m_safe);
-                    sc[nt][2 * i + 1] = fast_exp2(sc[nt][2 * i + 1] - m_safe);
-                    rs += sc[nt][2 * i] + sc[nt][2 * i + 1];
-                }
-                l_run[i] = l_run[i] * alpha[i] + rs;
-            }
-            uint32_t pa[4];
-            pa[0] = pack_bf16(sc[0][0], sc[0][1]);
-            pa[1] = pack_bf16(sc[0][2], sc[0][3]);
-            pa[2] = pack_bf16(sc[1][0], sc[1][1]);
-            pa[3] = pack_bf16(sc[1][2], sc[1][3]);
-            // O = alpha * O + P V
-            {
-                const int mi = lane >> 3;
-                const uint32_t tok = (mi & 1) * 8 + (lane & 7);
-#pragma unroll
-                for (int dp = 0; dp < DH / 16; ++dp) {
-                    const int ch = 2 * dp + (mi >> 1);
-                    uint32_t vb[4];
-                    ldmatrix_x4_trans(vb, smem_u32(vp + (ch >> 3) * Cfg::kSlabBytes + swz(tok, ch & 7)));
-#pragma unroll
-                    for (int h2 = 0; h2 < 2; ++h2) {
-                        float (&acc)[4] = o[2 * dp + h2];
-                        acc[0] *= alpha[0]; acc[1] *= alpha[0];
-                        acc[2] *= alpha[1]; acc[3] *= alpha[1];
-                        mma_bf16_16816(acc, pa, vb[2 * h2], vb[2 * h2 + 1]);
+                    for (int i = 0; i < 32; ++i) {
+                        float v = __uint_as_float(sv[i]);
+                        if (need_mask && c0 + i >= lim_local) v = -INFINITY;
+                        mx4[i & 3] = fmaxf(mx4[i & 3], v);
                     }
                 }
+                mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;   // scale > 0: the maximum commutes
+                if (!real) mx = -INFINITY;                                 // padding rows stay inert
             }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[s]);           // this warp is done with stage s
+            if (copies > 1) {
+                float* xch = s_xch[q & 1];
+                xch[t] = mx;
+                if (!group_sync(13)) { ok = false; break; }
+                mx = xch[r];
+                for (int cc = 1; cc < copies; ++cc) mx = fmaxf(mx, xch[cc * span + r]);
+            }
+            // ---- raise the running maximum only if it grew by more than the threshold
+            float alpha = 1.f;
+            if (seg_first) {
+                m_used = mx;
+            } else if (mx > m_used + kRescaleThreshold) {
+                alpha = fast_exp2(m_used - mx);                            // m_used == -inf gives 0
+                m_used = mx;
+                l_run *= alpha;
+            }
+            if (o_owner && !seg_first && __any_sync(0xffffffffu, alpha != 1.f)) {
+                // O += P V of the previous block must have landed before O is rescaled
+                if (!mbar_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int c0 = 0; c0 < DH; c0 += 32) {
+                    uint32_t o[32];
+                    tmem_ld_x32(t_lane + kTmemO + c0, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st_x32(t_lane + kTmemO + c0, o);
+                }
+                tmem_st_wait();
+            }
+            // the P buffer is free once the P V product of two blocks ago has read it
+            if (u > 0 && !mbar_wait(&bars->p_empty[buf], (u - 1) & 1, p.status, 8)) { ok = false; break; }
+            if (warp_real) {
+                // ---- pass 2: p = 2^(s * scale - m), bf16, into row r of operand A of the P V product
+                const float m_safe = (m_used == -INFINITY) ? 0.f : m_used;
+                uint8_t* p_row = smem + Cfg::kPOffset + buf * Cfg::kPBytes + r * 128;
+                float rs0 = 0.f, rs1 = 0.f;
+                for (int c0 = 0; c0 < span; c0 += 32) {
+                    uint32_t sv[32];
+                    tmem_ld_x32(t_s + c0, sv);
+                    tmem_ld_wait();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float e0 = fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -m_safe));
+                        float e1 = fast_exp2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -m_safe));
+                        if (need_mask) {
+                            if (c0 + i >= lim_local) e0 = 0.f;
+                            if (c0 + i + 1 >= lim_local) e1 = 0.f;
+                        }
+                        rs0 += e0;
+                        rs1 += e1;
+                        pk[i >> 1] = pack_bf16(e0, e1);
+                    }
+                    if (real) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            const int chunk = ((c * span + c0) >> 3) + ch;  // 16-byte chunk (8 tokens) of the row
+                            *reinterpret_cast<uint4*>(p_row + (chunk >> 3) * Cfg::kSlabBytes + (((chunk & 7) ^ (r & 7)) << 4)) =
+                                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+                        }
+                    }
+                }
+                l_run += rs0 + rs1;
+            }
+            // rows of V past the end of the sequence may hold anything (the pool is the caller's, or
+            // the page was never loaded): their weight is exactly 0, but 0 * NaN is NaN, so clear them
+            if (t_begin + kAttBlockTokens > cur.kvl && t >= cur.kvl - t_begin) {
+                uint8_t* v_row = smem + st * Cfg::kStageBytes + Cfg::kSlabs * Cfg::kSlabBytes + t * 128;
+#pragma unroll
+                for (int hf = 0; hf < Cfg::kSlabs; ++hf)
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch)
+                        *reinterpret_cast<uint4*>(v_row + hf * Cfg::kSlabBytes + ch * 16) = make_uint4(0u, 0u, 0u, 0u);
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&bars->p_full[buf]);
+            mbar_arrive(&bars->s_empty[buf]);
 
-        const int pair_global = p.seq_pair0[cur.b] + cur.pair;
-        const bool left_pair = cur.advance(p, q + 1 < n_my);
-        if (left_pair || q + 1 == n_my) {
-            // ---- end of the segment: this warp's partial -> slot (pair + CTA), unique per segment
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
-                l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
+            const int pair_global = cur.pair0 + cur.pair;
+            const int64_t pair_blk_first = static_cast<int64_t>(cur.blk0) + static_cast<int64_t>(cur.pair) * cur.nb;
+            const int pair_nb = cur.nb, pair_q_row0 = cur.q_row0;
+            cur.advance(p, q + 1 < n_my);
+            seg_first = seg_last;
+            if (!seg_last) continue;
+
+            // ------------------------------------------------------------ end of the segment
+            ++seg;
+            if (copies > 1) {
+                // the copies of a row hold the sums over their own tokens (same maximum): add them up
+                float* xch = s_xch[2];
+                xch[t] = l_run;
+                if (!group_sync(14)) { ok = false; break; }
+                l_run = xch[r];
+                for (int cc = 1; cc < copies; ++cc) l_run += xch[cc * span + r];
             }
-            const int64_t slot = static_cast<int64_t>(pair_global + cta) * kAttMaxConsumerWarps + cw;
-            float* po = p.part_o + slot * 16 * DH;
-            float* pml = p.part_ml + slot * 16 * 2;
-            const bool has = (m_run[0] != -INFINITY) || (m_run[1] != -INFINITY);
-            if (has) {
+            if (!mbar_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
+            tc_fence_after();
+            // which CTAs hold blocks of this pair: CTA c owns blocks [c*T/G, (c+1)*T/G), so the owner of
+            // block x is ceil((x+1)*G/T) - 1
+            const int64_t pair_blk_last = pair_blk_first + pair_nb - 1;
+            const int c_first = static_cast<int>(((pair_blk_first + 1) * gridDim.x - 1) / total_blocks);
+            const int c_last = static_cast<int>(((pair_blk_last + 1) * gridDim.x - 1) / total_blocks);
+            const int rho = row_lo + r;
+            const int64_t out_row = static_cast<int64_t>(pair_q_row0 + rho / p.group) * p.n_q_heads + kvh * p.group + rho % p.group;
+            __nv_bfloat16* out = p.attn_out + out_row * DH;
+            const bool writer = o_owner && real;                           // c == 0 and a real row
+
+            if (c_first == c_last) {
+                // the whole pair was ours: normalise and store
+                if (o_owner) {
+                    const float inv = 1.f / l_run;
 #pragma unroll
-                for (int nt = 0; nt < DH / 8; ++nt) {
-                    *reinterpret_cast<float2*>(po + g * DH + nt * 8 + tq * 2) = make_float2(o[nt][0], o[nt][1]);
-                    *reinterpret_cast<float2*>(po + (g + 8) * DH + nt * 8 + tq * 2) = make_float2(o[nt][2], o[nt][3]);
+                    for (int cc = 0; cc < DH; cc += 32) {
+                        uint32_t o[32];
+                        tmem_ld_x32(t_lane + kTmemO + cc, o);
+                        tmem_ld_wait();
+                        if (writer) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 8) {
+                                uint4 w;
+                                w.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+                                w.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                                w.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                                w.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                                *reinterpret_cast<uint4*>(out + cc + i) = w;
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                continue;
+            }
+
+            // ---- the pair spans CTAs c_first..c_last: park (m, l, O); a CTA's parts are its first and its last segment
+            const int my_slot = cta * 2 + ((seg == 1) ? 0 : 1);
+            if (o_owner) {
+                float* po = p.part_o + (static_cast<int64_t>(my_slot) * kAttRowsPerPair + r) * DH;
+#pragma unroll
+                for (int cc = 0; cc < DH; cc += 32) {
+                    uint32_t o[32];
+                    tmem_ld_x32(t_lane + kTmemO + cc, o);
+                    tmem_ld_wait();
+                    if (writer) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            __stcg(reinterpret_cast<float4*>(po + cc + i),
+                                   make_float4(__uint_as_float(o[i]), __uint_as_float(o[i + 1]),
+                                               __uint_as_float(o[i + 2]), __uint_as_float(o[i + 3])));
+                    }
+                }
+                if (writer)
+                    __stcg(reinterpret_cast<float2*>(p.part_ml + (static_cast<int64_t>(my_slot) * kAttRowsPerPair + r) * 2),
+                           make_float2(m_used, l_run));
+            }
+            tc_fence_before();
+            __threadfence();
+            if (!group_sync(11)) { ok = false; break; }                    // every softmax thread has published
+            if (t == 0) {
+                const int tk = atomicAdd(&p.tickets[pair_global], 1);
+                const int last = (tk == c_last - c_first);
+                if (last) p.tickets[pair_global] = 0;                      // ready for the next call
+                s_flag = last;
+            }
+            if (!group_sync(12)) { ok = false; break; }
+            if (s_flag && writer) {
+                // ---- this CTA completed the pair: out = sum_c 2^(m_c - M) O_c / sum_c 2^(m_c - M) l_c,
+                // parts taken in CTA order.  The first CTA holds the head of the pair in its last segment unless
+                // its range starts exactly there; every later CTA holds its part in its first segment.
+                __threadfence();
+                const int blk_begin_c0 = static_cast<int>(static_cast<int64_t>(c_first) * total_blocks / gridDim.x);
+                const int slot_c0 = c_first * 2 + ((blk_begin_c0 == pair_blk_first) ? 0 : 1);
+                float m_all = -INFINITY;
+                for (int cc = c_first; cc <= c_last; ++cc) {
+                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+                    m_all = fmaxf(m_all, __ldcg(p.part_ml + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * 2));
+                }
+                float l_all = 0.f;
+                for (int cc = c_first; cc <= c_last; ++cc) {
+                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * 2));
+                    if (ml.x != -INFINITY) l_all += fast_exp2(ml.x - m_all) * ml.y;
+                }
+                const float inv = 1.f / l_all;
+#pragma unroll 1
+                for (int col = 0; col < DH; col += 32) {
+                    float acc[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+                    for (int cc = c_first; cc <= c_last; ++cc) {
+                        const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+                        const float mc = __ldcg(p.part_ml + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * 2);
+                        if (mc == -INFINITY) continue;                     // that part saw no visible token
+                        const float wgt = fast_exp2(mc - m_all);
+                        const float4* po = reinterpret_cast<const float4*>(
+                            p.part_o + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * DH + col);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 v = __ldcg(po + i);
+                            acc[4 * i] += wgt * v.x; acc[4 * i + 1] += wgt * v.y;
+                            acc[4 * i + 2] += wgt * v.z; acc[4 * i + 3] += wgt * v.w;
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 w;
+                        w.x = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
+                        w.y = pack_bf16(acc[i + 2] * inv, acc[i + 3] * inv);
+                        w.z = pack_bf16(acc[i + 4] * inv, acc[i + 5] * inv);
+                        w.w = pack_bf16(acc[i + 6] * inv, acc[i + 7] * inv);
+                        *reinterpret_cast<uint4*>(out + col + i) = w;
+                    }
                 }
             }
-            if (tq == 0) {
-                *reinterpret_cast<float2*>(pml + g * 2) = make_float2(m_run[0], l_run[0]);
-                *reinterpret_cast<float2*>(pml + (g + 8) * 2) = make_float2(m_run[1], l_run[1]);
-            }
-            new_segment = true;
         }
     }
-}
 
-// Merge of a pair's partials: out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i, rounded to bf16.
-// The partials of pair P were written by the CTAs whose block ranges intersect the pair's blocks,
-// by every consumer warp that shares the row tile.
-__global__ void __launch_bounds__(256)
-attention_combine_kernel(const CombineParams p)
-{
-    const int b = blockIdx.y;
-    const int k_b = p.draft_len[b];
-    const int kvl = p.kv_len[b];
-    const int nb = (kvl + kAttBlockTokens - 1) / kAttBlockTokens;
-    const int n_rows = p.group * (k_b + 1);
-    const int rbc = (n_rows + kAttRowsPerPair - 1) / kAttRowsPerPair;
-    const int pair = blockIdx.x;
-    if (pair >= p.n_kv_heads * rbc) return;
-    const int kvh = pair / rbc;
-    const int row_lo = (pair % rbc) * kAttRowsPerPair;
-    const int rows_here = min(kAttRowsPerPair, n_rows - row_lo);
-    const int n_rt = (rows_here + 15) >> 4;
-
-    const int64_t total_blocks = p.seq_blk0[p.batch];
-    const int64_t blk_first = p.seq_blk0[b] + static_cast<int64_t>(pair) * nb;
-    const int64_t blk_last = blk_first + nb - 1;
-    // CTA c owns blocks [c*T/G, (c+1)*T/G): the owner of block x is ceil((x+1)*G/T) - 1
-    const int c0 = static_cast<int>(((blk_first + 1) * p.n_ctas - 1) / total_blocks);
-    const int c1 = static_cast<int>(((blk_last + 1) * p.n_ctas - 1) / total_blocks);
-    const int pair_global = p.seq_pair0[b] + pair;
-    const int q_row0 = p.cu_q[b];
-    const int dh = p.head_dim;
-    const int cols4 = dh / 4;
-
-    for (int idx = threadIdx.x; idx < rows_here * cols4; idx += blockDim.x) {
-        const int r = idx / cols4;
-        const int c4 = (idx % cols4) * 4;
-        const int tile = r >> 4, rr = r & 15;
-        const int slices = (p.n_cw - tile + n_rt - 1) / n_rt;
-        float m_all = -INFINITY;
-        for (int c = c0; c <= c1; ++c)
-            for (int sl = 0; sl < slices; ++sl) {
-                const int64_t slot = static_cast<int64_t>(pair_global + c) * kAttMaxConsumerWarps + tile + sl * n_rt;
-                m_all = fmaxf(m_all, p.part_ml[(slot * 16 + rr) * 2]);
-            }
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float l_all = 0.f;
-        for (int c = c0; c <= c1; ++c)
-            for (int sl = 0; sl < slices; ++sl) {
-                const int64_t slot = static_cast<int64_t>(pair_global + c) * kAttMaxConsumerWarps + tile + sl * n_rt;
-                const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (slot * 16 + rr) * 2);
-                if (ml.x == -INFINITY) continue;             // that warp saw no visible token
-                const float wgt = fast_exp2(ml.x - m_all);
-                l_all += wgt * ml.y;
-                const float4 v = *reinterpret_cast<const float4*>(p.part_o + (slot * 16 + rr) * dh + c4);
-                acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
-            }
-        const int rho = row_lo + r;
-        const int j = rho / p.group, hh = rho % p.group;
-        const int64_t out_row = static_cast<int64_t>(q_row0 + j) * p.n_q_heads + kvh * p.group + hh;
-        const float inv = 1.f / l_all;
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-        __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(p.attn_out + out_row * dh + c4) = pk;
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kAttTmemCols);
     }
 }
 
@@ -382,34 +695,15 @@ cudaError_t attention_init(int head_dim)
                                 AttCfg<64>::kSmemBytes);
 }
 
-// consumer warps per CTA for a batch whose largest pair has `max_tile_rows` query rows
-int attention_consumer_warps(int max_tile_rows)
-{
-    const int rows = max_tile_rows > kAttRowsPerPair ? kAttRowsPerPair : max_tile_rows;
-    const int rt = rows > 0 ? (rows + 15) / 16 : 1;
-    int slices = (8 + rt / 2) / rt;                  // round(8 / rt) ...
-    if (slices < 1) slices = 1;                      // ... at least 1
-    int w = rt * slices;
-    if (w > kAttMaxConsumerWarps) w = rt;
-    return w;
-}
-
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
-                             int32_t n_cw, cudaStream_t stream)
+                             cudaStream_t stream)
 {
     dim3 grid(n_ctas);
-    dim3 block((n_cw + 1) * 32);
+    dim3 block(kAttThreads);
     if (h.cfg.head_dim == 128)
         attention_kernel<128><<<grid, block, AttCfg<128>::kSmemBytes, stream>>>(kv_map, p);
     else
         attention_kernel<64><<<grid, block, AttCfg<64>::kSmemBytes, stream>>>(kv_map, p);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_attention_combine(const CombineParams& p, cudaStream_t stream)
-{
-    dim3 grid(p.pairs_per_seq_max, p.batch);
-    attention_combine_kernel<<<grid, 256, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

@@ -15,53 +15,29 @@ constexpr int kMaxK = 63;
 constexpr int kSampleChunk = 8192;        // vocabulary entries per CTA of the statistics kernel
 constexpr int kDrawChunk = 2048;          // vocabulary entries per CTA of the draw kernel
 constexpr int kAttBlockTokens = 128;      // KV tokens per attention work block / pipeline stage
-constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block
+constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block (MMA M)
+constexpr int kAttThreads = 192;          // TMA warp + MMA warp + 4 softmax warps
 constexpr int kNumStageEvents = 7;
 
-struct Plan {                 // device tables written by the plan kernel, read by all stages
+struct Plan {                 // device tables written by the plan kernel, read by the sampling stage
     int32_t* cu_q;            // [max_batch+1] first query row of each sequence
     int32_t* cu_d;            // [max_batch+1] first draft row of each sequence
     int32_t* row_seq;         // [max_m] sequence of each query row
-    // attention work list: a "block" is 128 KV tokens of one (sequence, kv head, 128-row block)
-    // pair; blocks are numbered sequence by sequence, pair by pair, and cut into equal
-    // contiguous ranges, one per CTA
-    int32_t* seq_blk0;        // [max_batch+1] first block of each sequence; [batch] = total
-    int32_t* seq_pair0;       // [max_batch+1] first pair of each sequence
-    int2* cta_start;          // [sm_count] (sequence, block index inside it) where CTA c starts
 };
-
-constexpr int kAttMaxConsumerWarps = 10;
 
 struct AttnParams {
     const __nv_bfloat16* hidden;
     const int32_t* page_table;
     const int32_t* kv_len;
     const int32_t* draft_len;
-    const int32_t* cu_q;
-    const int32_t* seq_blk0;
-    const int32_t* seq_pair0;
-    const int2* cta_start;
     int32_t batch, n_q_heads, n_kv_heads, group;
     int32_t max_pages_per_seq, num_pages;
     float scale_log2;         // log2(e) / sqrt(head_dim)
-    float* part_o;            // [slot][consumer warp][16][Dh] unnormalised partial outputs
-    float* part_ml;           // [slot][consumer warp][16][2]  (running max in log2 units, sum)
+    float* part_o;            // [2 * CTAs][128][Dh] unnormalised partial outputs (a CTA's first / last segment)
+    float* part_ml;           // [2 * CTAs][128][2]  (running max in log2 units, sum)
+    int32_t* tickets;         // [pairs] self-resetting arrival counters of the split merge
+    __nv_bfloat16* attn_out;  // [M][d_model]
     int32_t* status;
-};
-
-struct CombineParams {
-    const float* part_o;
-    const float* part_ml;
-    const int32_t* kv_len;
-    const int32_t* draft_len;
-    const int32_t* cu_q;
-    const int32_t* seq_blk0;
-    const int32_t* seq_pair0;
-    int32_t batch, n_q_heads, n_kv_heads, group, head_dim;
-    int32_t n_ctas;           // grid of the attention kernel
-    int32_t n_cw;             // its consumer warps
-    int32_t pairs_per_seq_max;
-    __nv_bfloat16* attn_out;
 };
 
 struct LmHeadParams {
@@ -109,7 +85,7 @@ struct Handle {
     // workspace
     __nv_bfloat16* attn_out;
     float* logits;
-    float* part_o; float* part_ml;
+    float* part_o; float* part_ml; int32_t* att_tickets; int32_t att_pairs_max;
     Plan plan;
     float2* stats; int32_t* arg_idx; int32_t* counters; double* row_info; double* chunk_mass;
     double* dbg_p; double* dbg_q; float* dbg_u;
@@ -124,13 +100,10 @@ struct Handle {
 };
 
 // launch wrappers (each returns a cudaError_t from the launch)
-cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, const int32_t* kv_len,
-                        int32_t batch, int32_t vocab, int32_t n_kv_heads, int32_t group, int32_t n_ctas,
+cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
                         Plan plan, int32_t* status, cudaStream_t stream);
-int attention_consumer_warps(int max_tile_rows);
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
-                             int32_t n_cw, cudaStream_t stream);
-cudaError_t launch_attention_combine(const CombineParams& p, cudaStream_t stream);
+                             cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream);
 cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);

@@ -1,8 +1,7 @@
-// Plan kernel: the small per-call tables every stage reads.  One CTA; thread b handles
+// Plan kernel: the small per-call tables the sampling stage reads.  One CTA; thread b handles
 // sequence b.  Prefix sums of (k_b + 1) and k_b give the packed row offsets of the ragged batch
-// (FlexSpec's channel-aware stride makes k_b differ per sequence, Section IV-B); prefix sums of
-// the attention block and pair counts give the batch-wide work list that the attention kernel
-// cuts into one equal range per CTA.  Draft tokens are range-checked here.
+// (FlexSpec's channel-aware stride makes k_b differ per sequence, Section IV-B).  Draft tokens
+// are range-checked here.
 #include "common.cuh"
 #include "internal.h"
 
@@ -35,34 +34,21 @@ __device__ __forceinline__ int block_inclusive_scan(int v, int* warp_tot)
 }
 
 __global__ void __launch_bounds__(kMaxBatch)
-plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ draft_tokens,
-            const int32_t* __restrict__ kv_len, int32_t batch, int32_t vocab, int32_t n_kv_heads, int32_t group,
-            int32_t n_ctas, Plan plan, int32_t* status)
+plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ draft_tokens, int32_t batch,
+            int32_t vocab, Plan plan, int32_t* status)
 {
     __shared__ int warp_tot[32];
-    __shared__ int s_blk0[kMaxBatch + 1];
     const int t = threadIdx.x;
     const bool live = t < batch;
     const int k = live ? draft_len[t] : 0;
-    int blocks = 0, pairs = 0;
-    if (live && kv_len != nullptr) {
-        const int nb = (kv_len[t] + kAttBlockTokens - 1) / kAttBlockTokens;
-        pairs = n_kv_heads * ((group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
-        blocks = pairs * nb;
-    }
     if (t < 32) warp_tot[t] = 0;
     __syncthreads();
     const int q_end = block_inclusive_scan(live ? k + 1 : 0, warp_tot);
     const int d_end = block_inclusive_scan(k, warp_tot);
-    const int b_end = block_inclusive_scan(blocks, warp_tot);
-    const int p_end = block_inclusive_scan(pairs, warp_tot);
     if (live) {
         const int q0 = q_end - (k + 1), d0 = d_end - k;
         plan.cu_q[t] = q0;
         plan.cu_d[t] = d0;
-        plan.seq_blk0[t] = b_end - blocks;
-        plan.seq_pair0[t] = p_end - pairs;
-        s_blk0[t] = b_end - blocks;
         for (int j = 0; j <= k; ++j) plan.row_seq[q0 + j] = t;
         if (draft_tokens != nullptr)
             for (int j = 0; j < k; ++j) {
@@ -72,36 +58,15 @@ plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ d
         if (t == batch - 1) {
             plan.cu_q[batch] = q_end;
             plan.cu_d[batch] = d_end;
-            plan.seq_blk0[batch] = b_end;
-            plan.seq_pair0[batch] = p_end;
-            s_blk0[batch] = b_end;
-        }
-    }
-    __syncthreads();
-    // where each attention CTA starts: the sequence that holds block floor(c * T / G)
-    if (kv_len != nullptr) {
-        const int64_t total = s_blk0[batch];
-        for (int c = t; c < n_ctas; c += blockDim.x) {
-            const int first = static_cast<int>(c * total / n_ctas);
-            int lo = 0, hi = batch - 1;                    // largest b with s_blk0[b] <= first
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (s_blk0[mid] <= first) lo = mid; else hi = mid - 1;
-            }
-            plan.cta_start[c] = make_int2(lo, first - s_blk0[lo]);
         }
     }
 }
 
-cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, const int32_t* kv_len,
-                        int32_t batch, int32_t vocab, int32_t n_kv_heads, int32_t group, int32_t n_ctas,
+cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
                         Plan plan, int32_t* status, cudaStream_t stream)
 {
-    int threads = (batch + 31) / 32 * 32;
-    if (threads < n_ctas) threads = (n_ctas + 31) / 32 * 32;
-    if (threads > kMaxBatch) threads = kMaxBatch;
-    plan_kernel<<<1, threads, 0, stream>>>(draft_len, draft_tokens, kv_len, batch, vocab, n_kv_heads, group,
-                                           n_ctas, plan, status);
+    const int threads = (batch + 31) / 32 * 32;
+    plan_kernel<<<1, threads, 0, stream>>>(draft_len, draft_tokens, batch, vocab, plan, status);
     return cudaGetLastError();
 }
 
