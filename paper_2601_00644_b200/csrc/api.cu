@@ -149,6 +149,11 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     p.batch = batch;
     p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = group;
     p.max_pages_per_seq = kv->max_pages_per_seq; p.num_pages = kv->num_pages;
+    const int rows_max = group * (g.k_batch_max + 1) < kAttRowsPerPair ? group * (g.k_batch_max + 1) : kAttRowsPerPair;
+    p.n_pad = (rows_max + 15) / 16 * 16;
+    p.p_bufs = attention_p_bufs(p.n_pad);
+    attention_stages(c.head_dim, p.n_pad, &p.k_stages, &p.v_stages);
+    if (p.k_stages < 1 || p.v_stages < 2) return FLEXSPEC_ERR_UNSUPPORTED;
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(c.head_dim)));
     p.part_o = h.part_o; p.part_ml = h.part_ml; p.tickets = h.att_tickets;
     p.attn_out = static_cast<__nv_bfloat16*>(attn_out);
@@ -279,8 +284,8 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     // split-merge scratch: every CTA parks at most its first and its last segment
     const size_t att_slots = static_cast<size_t>(2) * h.sm_count;
     A(dev_alloc(&h.part_o, att_slots * kAttRowsPerPair * c.head_dim));
-    A(dev_alloc(&h.part_ml, att_slots * kAttRowsPerPair * 2));
-    A(dev_alloc(&h.att_tickets, static_cast<size_t>(h.att_pairs_max)));
+    A(dev_alloc(&h.part_ml, att_slots * 4 * kAttRowsPerPair * 2));
+    A(dev_alloc(&h.att_tickets, static_cast<size_t>(h.att_pairs_max) * 4));
     A(dev_alloc(&h.plan.cu_q, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
@@ -302,7 +307,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     }
     if (rc == FLEXSPEC_OK) {
         if (cudaMemset(h.counters, 0, sizeof(int32_t) * 2 * kMaxBatch) != cudaSuccess ||
-            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max)) != cudaSuccess ||
+            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 4) != cudaSuccess ||
             cudaMemset(h.status, 0, sizeof(int32_t) * 4) != cudaSuccess)
             rc = FLEXSPEC_ERR_CUDA;
     }

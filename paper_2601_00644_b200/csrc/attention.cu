@@ -12,25 +12,28 @@
 // kv_len[] (a block-wide prefix sum over the sequences), so no planning kernel runs first.
 //
 // Both contractions run on the 5th-generation tensor cores with accumulators in tensor memory
-// (the legacy warp-level MMA path cannot keep up with the KV stream):
-//   S[128 query rows][128 tokens] = Q K^T     A = Q tile, B = K tile, both K-major in shared memory
-//   O[128 query rows][Dh]        += P V       A = P (bf16, written by the softmax threads),
-//                                             B = V tile as TMA delivers it ([token][Dh]: MN-major)
-// The query rows of the pair occupy the first rows of the M = 128 tile; the remaining rows are
-// padding whose results are never read.
+// (the legacy warp-level MMA path cannot keep up with the KV stream).  A verification step has
+// few query rows per kv head (8..72 in the paper-shaped workloads), so the operands are swapped:
+// the 128 tokens of a block are the MMA's M dimension and the query rows its N dimension
+// (n_pad = rows rounded up to 16), which makes tensor work, the Q tile and the P tile scale with
+// the real row count:
+//   S^T[128 tokens][n_pad] = K Q^T      A = K tile, B = Q tile, both K-major, 128-byte swizzle
+//   O^T[Dh][n_pad]        += V^T P^T    A = V tile as TMA delivers it ([token][Dh]: MN-major),
+//                                       B = P^T written by the softmax threads ([token][row]:
+//                                       MN-major, unswizzled 8x8 core matrices)
 //
-// Warp roles.  Warp 0: TMA producer (one 16-token K and V page per lane, 128-byte swizzle, a ring
-// of 128-token stages).  Warp 1: one thread issues every tcgen05.mma; the warp owns the TMEM
-// allocation.  Warps 2..5: softmax, one thread per TMEM lane (= tile row, so a row's maximum and
-// sum need no shuffles): two passes over the scores of the block with tcgen05.ld -- maximum, then
-// p = 2^(s - m) written to shared memory as bf16 -- with S double buffered so that the next
-// block's QK^T overlaps.  A pair with at most 32 (64) rows is replicated 4 (2) times over the
-// tile rows and each copy takes a quarter (half) of the block's tokens, so all four warps work
-// on small pairs.  The running maximum is only raised when it grew by more than 2^8 (O in TMEM
-// is then rescaled); the final division by the row sum makes the stale maximum cancel.  At the end of a segment the softmax threads read O from TMEM; if the
-// pair spans several CTAs they park (m, l, O) in global scratch and the CTA that completes the
-// pair last (atomic ticket, nobody waits) merges the parts by log-sum-exp in CTA order.
-// Every mbarrier wait is bounded.
+// Warp roles.  Warp 0: TMA producer (one 16-token K and V page per lane, separate rings of
+// 128-token K and V tiles; the page ids of the next block are fetched one block ahead).  Warp 1:
+// one thread issues every tcgen05.mma; the warp owns the TMEM allocation.  Warps 2..5: softmax,
+// thread t = token t of the block (TMEM lane t of S^T).  The maximum of a query row over the
+// block is a column maximum: redux.sync.max over each warp, then over the four warps through
+// shared memory.  The running maximum is only raised when it grew by more than 2^8 (O^T in TMEM
+// is then rescaled); the final division by the row sum makes the stale maximum cancel.  Row sums
+// are kept per thread and added up across lanes once per segment.  At the end of a segment
+// thread t owns row Dh-index t of O^T; if the pair spans several CTAs every warp parks its 32
+// rows of (m, l, O^T) in global scratch and the warp that arrives last for those rows (atomic
+// ticket, nobody waits) merges the parts by log-sum-exp in CTA order.  Every mbarrier wait is
+// bounded.
 #include "common.cuh"
 #include "internal.h"
 
@@ -42,33 +45,64 @@ constexpr int kAttSoftmaxThreads = 128;
 constexpr int kAttTmemCols = 512;
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column offsets
 constexpr float kRescaleThreshold = 8.f;                             // log2 units
-
-template <int DH>
-struct AttCfg {
-    static constexpr int kSlabs = DH / 64;                     // 128-byte column slabs per row
-    static constexpr int kSlabBytes = 128 * 128;               // 128 rows x 64 bf16
-    static constexpr int kStageBytes = 2 * kSlabs * kSlabBytes;      // K slabs, then V slabs
-    static constexpr int kStages = (DH == 128) ? 2 : 4;
-    static constexpr int kQOffset = kStages * kStageBytes;
-    static constexpr int kQBytes = kSlabs * kSlabBytes;
-    static constexpr int kPOffset = kQOffset + kQBytes;
-    static constexpr int kPBytes = 2 * kSlabBytes;             // 128 rows x 128 tokens bf16
-    static constexpr int kBarOffset = kPOffset + 2 * kPBytes;
-    static constexpr int kSmemBytes = kBarOffset + 256 + 1024; // + barriers + alignment slack
-};
+constexpr int kAttSmemLimit = 232448;                                // 227 KB opt-in maximum per CTA
+constexpr int kAttStaticReserve = 512;                               // __shared__ variables of the kernel
 
 struct AttBars {
-    uint64_t kv_full[4], kv_empty[4];
+    uint64_t k_full[kAttMaxStages], k_empty[kAttMaxStages];
+    uint64_t v_full[kAttMaxStages], v_empty[kAttMaxStages];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_full[2], p_empty[2];
     uint64_t q_full, o_full, group;
     uint32_t tmem_slot;
 };
-static_assert(sizeof(AttBars) <= 256, "barrier block");
+static_assert(sizeof(AttBars) <= 512, "barrier block");
+
+// Dynamic shared memory, all offsets from a 1024-byte aligned base:
+//   [k_stages x K slabs] [v_stages x V slabs] [Q: slabs x n_pad x 128 B] [P^T: p_bufs x n_pad x 256 B]
+//   [barriers] [exchange of column maxima / row sums between the warps: 3 x 4 x n_pad floats]
+// K and V travel in separate rings: a K tile is free again after the QK^T product, a V tile only
+// after the softmax and the second product, so V gets the deeper ring.
+template <int DH>
+struct AttCfg {
+    static constexpr int kSlabs = DH / 64;                     // 128-byte column slabs per row
+    static constexpr int kSlabBytes = 128 * 128;               // 128 tokens x 64 bf16
+    static constexpr int kTileBytes = kSlabs * kSlabBytes;     // K (or V) of one 128-token block
+    __host__ __device__ static constexpr int q_bytes(int n_pad) { return kSlabs * n_pad * 128; }
+    __host__ __device__ static constexpr int p_bytes(int n_pad) { return n_pad * 256; }
+    __host__ __device__ static constexpr int col_bytes(int n_pad) { return 3 * 4 * n_pad * 4; }
+    __host__ __device__ static constexpr int fixed_bytes(int n_pad, int p_bufs)
+    {
+        return q_bytes(n_pad) + p_bufs * p_bytes(n_pad) + 512 + col_bytes(n_pad) + 1024;
+    }
+};
+
+// the widest tile leaves room for enough K/V tiles only with a single P^T buffer
+int attention_p_bufs(int n_pad) { return n_pad > 112 ? 1 : 2; }
+
+// ring depths that fit: two K tiles when there is room for at least four tiles, the rest V
+void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages)
+{
+    const int pb = attention_p_bufs(n_pad);
+    const int tile = head_dim == 128 ? AttCfg<128>::kTileBytes : AttCfg<64>::kTileBytes;
+    const int fixed = head_dim == 128 ? AttCfg<128>::fixed_bytes(n_pad, pb) : AttCfg<64>::fixed_bytes(n_pad, pb);
+    const int tiles = (kAttSmemLimit - kAttStaticReserve - fixed) / tile;
+    int ks = tiles >= 4 ? 2 : 1;
+    int vs = tiles - ks;
+    if (vs > kAttMaxStages) vs = kAttMaxStages;
+    *k_stages = ks;
+    *v_stages = vs;
+}
 
 __device__ __forceinline__ void prefetch_l2(const void* p)
 {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+__device__ __forceinline__ float redux_max(float v)
+{
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
 }
 
 // 32 lanes x 32 consecutive fp32 columns: thread i of the warp reads TMEM lane (base lane + i).
@@ -104,18 +138,30 @@ __device__ __forceinline__ void tmem_st_wait()
 }
 
 // Shared-memory matrix descriptor of an MN-major bf16 operand laid out by TMA with the 128-byte
-// swizzle: rows of 64 MN-elements (128 B) indexed by k, groups of 8 k-rows `sbo` bytes apart,
-// the next 64 MN-elements `lbo` bytes away.
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo, uint32_t sbo)
+// swizzle: rows of 64 MN-elements (128 B) indexed by k, groups of 8 k-rows `k_stride` bytes apart,
+// the next 64 MN-elements `mn_stride` bytes away.
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t mn_stride, uint32_t k_stride)
 {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
-    d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
-    d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
-    d |= static_cast<uint64_t>(1) << 46;                       // descriptor version of this architecture
-    d |= static_cast<uint64_t>(2) << 61;                       // 128-byte swizzle
+    d |= static_cast<uint64_t>((mn_stride >> 4) & 0x3FFFu) << 16;   // leading byte offset
+    d |= static_cast<uint64_t>((k_stride >> 4) & 0x3FFFu) << 32;    // stride byte offset
+    d |= static_cast<uint64_t>(1) << 46;                             // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                             // 128-byte swizzle
     return d;
 }
+// MN-major bf16 operand without swizzle: 8 (k) x 8 (mn) core matrices of 128 contiguous bytes
+// (a k-row is 16 B), the next 8 k-rows `k_stride` bytes away, the next 8 MN-elements `mn_stride`.
+__device__ __forceinline__ uint64_t umma_desc_mn_plain(uint32_t smem_addr, uint32_t mn_stride, uint32_t k_stride)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((k_stride >> 4) & 0x3FFFu) << 16;    // leading byte offset
+    d |= static_cast<uint64_t>((mn_stride >> 4) & 0x3FFFu) << 32;   // stride byte offset
+    d |= static_cast<uint64_t>(1) << 46;
+    return d;
+}
+constexpr uint32_t kIdescAMajorMN = 1u << 15;
 constexpr uint32_t kIdescBMajorMN = 1u << 16;
 
 // Exclusive prefix sum over the block of one int per thread; returns the block total in `total`.
@@ -175,6 +221,369 @@ struct AttCursor {
 
 struct AttStart { int b, blk_off, q_row0, pair0, blk0, total; };
 
+struct AttSmem {                  // pointers into dynamic shared memory
+    uint8_t* k_ring;
+    uint8_t* v_ring;
+    uint8_t* q;
+    uint8_t* pt;                  // P^T buffers
+    AttBars* bars;
+    float* xch;                   // [3][4][n_pad]: column maxima (by block parity) and row sums, one row per warp
+};
+
+// ------------------------------------------------------------------------------------ softmax role
+// NCH = chunks of 32 columns (query rows) of S^T: n_pad <= 32 * NCH.  Per-column state (running
+// maximum, row sum, output row) lives in lane i of every warp for column 32*ci + i and is
+// broadcast by shuffles, so the four warps only meet once per block (column maxima) and once
+// per segment (row sums).
+template <int DH, int NCH>
+__device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& sm, uint32_t tmem_base, AttCursor cur,
+                                            int n_my, int64_t total_blocks)
+{
+    using Cfg = AttCfg<DH>;
+    AttBars* bars = sm.bars;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
+    const int t = quarter * 32 + lane;                  // token of the block (S^T), Dh index (O^T)
+    const int cta = blockIdx.x;
+    const int n_pad = p.n_pad;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const int q_slab = n_pad * 128;
+    const bool o_lane = quarter * 32 < DH;              // warp-uniform: this warp's lanes hold rows of O^T
+
+    bool ok = true, seg_first = true;
+    int seg = 0;
+    uint32_t group_phase = 0;
+    auto group_sync = [&](int where) -> bool {
+        mbar_arrive(&bars->group);
+        const bool done = mbar_wait(&bars->group, group_phase, p.status, where);
+        group_phase ^= 1u;
+        return done;
+    };
+
+    float lsum[NCH * 32];                               // my token's share of the row sums, per column
+    float m_used[NCH];                                  // lane i: running maximum of column 32*ci + i (log2 units)
+    int row_c[NCH];                                     // lane i: output row index (row * n_q_heads + head) of that column
+    int rows_here = 0, row_lo = 0, ctx = 0;
+
+    for (int q = 0; q < n_my && ok; ++q) {
+        const int kvh = cur.pair / cur.rbc;
+        if (seg_first) {
+            // ---- the pair's query rows -> shared memory, K-major swizzled rows of operand B
+            row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
+            rows_here = min(kAttRowsPerPair, p.group * (cur.k + 1) - row_lo);
+            ctx = cur.kvl - (cur.k + 1);
+            for (int idx = t; idx < rows_here * (DH / 8); idx += kAttSoftmaxThreads) {
+                const int row = idx / (DH / 8), ch = idx % (DH / 8);
+                const int rho = row_lo + row;
+                const int64_t src_row = static_cast<int64_t>(cur.q_row0 + rho / p.group) * p.n_q_heads + kvh * p.group + rho % p.group;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.hidden + src_row * DH) + ch);
+                *reinterpret_cast<uint4*>(sm.q + (ch >> 3) * q_slab + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = v;
+            }
+#pragma unroll
+            for (int i = 0; i < NCH * 32; ++i) lsum[i] = 0.f;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                m_used[ci] = -INFINITY;
+                const int rho = row_lo + ci * 32 + lane;
+                row_c[ci] = (cur.q_row0 + rho / p.group) * p.n_q_heads + kvh * p.group + rho % p.group;
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&bars->q_full);
+        }
+        const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
+        const int buf = q & 1, u = q >> 1;
+        const int t_begin = cur.blk * kAttBlockTokens;
+        // token t of the block sees query row (column) c iff col_min <= c < rows_here: it is at
+        // distance d = t_abs - ctx into the draft window and row c belongs to window position c / group
+        const int d = t_begin + t - ctx;
+        const int col_min = d > 0 ? d * p.group - row_lo : 0;
+        const uint32_t col_span = static_cast<uint32_t>(max(0, rows_here - col_min));
+        const uint32_t t_s = t_lane + (buf ? kTmemS1 : kTmemS0);
+
+        if (!mbar_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
+        tc_fence_after();
+
+        // ---- pass 1: column maxima over my warp's 32 tokens, then over the four warps
+        uint32_t sv[32];                                 // kept for pass 2 when there is a single chunk
+        float* xch = sm.xch + (q & 1) * 4 * n_pad;
+#pragma unroll
+        for (int ci = 0; ci < NCH; ++ci) {
+            if (ci * 32 < n_pad) {
+                tmem_ld_x32(t_s + ci * 32, sv);
+                tmem_ld_wait();
+                float mine = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;
+                    const float w = redux_max(masked ? -INFINITY : __uint_as_float(sv[i]));
+                    if (lane == i) mine = w;
+                }
+                if (ci * 32 + lane < n_pad) xch[quarter * n_pad + ci * 32 + lane] = mine;
+            }
+        }
+        if (!group_sync(14)) { ok = false; break; }
+        float alpha[NCH];
+        bool rescale = false;
+#pragma unroll
+        for (int ci = 0; ci < NCH; ++ci) {
+            alpha[ci] = 1.f;
+            const int col = ci * 32 + lane;
+            if (col < n_pad) {
+                const float mx = fmaxf(fmaxf(xch[col], xch[n_pad + col]), fmaxf(xch[2 * n_pad + col], xch[3 * n_pad + col])) *
+                                 p.scale_log2;           // scale > 0: the maximum commutes
+                // ---- raise the running maximum only if it grew by more than the threshold
+                if (seg_first) {
+                    m_used[ci] = mx;
+                } else if (mx > m_used[ci] + kRescaleThreshold) {
+                    alpha[ci] = fast_exp2(m_used[ci] - mx);                // m_used == -inf gives 0
+                    m_used[ci] = mx;
+                    rescale = true;
+                }
+            }
+        }
+        if (!seg_first && __any_sync(0xffffffffu, rescale)) {
+            // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
+            if (!mbar_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 < n_pad) {
+                    uint32_t o[32];
+                    if (o_lane) {
+                        tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
+                        tmem_ld_wait();
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float a = __shfl_sync(0xffffffffu, alpha[ci], i);
+                        lsum[ci * 32 + i] *= a;
+                        if (o_lane) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
+                    }
+                    if (o_lane) tmem_st_x32(t_lane + kTmemO + ci * 32, o);
+                }
+            }
+            if (o_lane) tmem_st_wait();
+        }
+        // the P^T buffer is free once the product that last read it has completed
+        const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
+        if (pu > 0 && !mbar_wait(&bars->p_empty[pbuf], (pu - 1) & 1, p.status, 8)) { ok = false; break; }
+        // ---- pass 2: p = 2^(s * scale - m), bf16, into row t of operand B of the second product
+        {
+            uint8_t* p_row = sm.pt + pbuf * Cfg::p_bytes(n_pad) + t * 16;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 < n_pad) {
+                    if (NCH > 1) {
+                        tmem_ld_x32(t_s + ci * 32, sv);
+                        tmem_ld_wait();
+                    }
+                    const float m_safe = (m_used[ci] == -INFINITY) ? 0.f : m_used[ci];
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float m0 = __shfl_sync(0xffffffffu, m_safe, i);
+                        const float m1 = __shfl_sync(0xffffffffu, m_safe, i + 1);
+                        float e0 = fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -m0));
+                        float e1 = fast_exp2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -m1));
+                        if (static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span) e0 = 0.f;
+                        if (static_cast<uint32_t>(ci * 32 + i + 1 - col_min) >= col_span) e1 = 0.f;
+                        lsum[ci * 32 + i] += e0;
+                        lsum[ci * 32 + i + 1] += e1;
+                        pk[i >> 1] = pack_bf16(e0, e1);
+                    }
+#pragma unroll
+                    for (int g8 = 0; g8 < 4; ++g8)
+                        if (ci * 32 + g8 * 8 < n_pad)
+                            *reinterpret_cast<uint4*>(p_row + (ci * 4 + g8) * 2048) =
+                                make_uint4(pk[4 * g8], pk[4 * g8 + 1], pk[4 * g8 + 2], pk[4 * g8 + 3]);
+                }
+            }
+        }
+        // rows of V past the end of the sequence may hold anything (the pool is the caller's, or
+        // the page was never loaded): their weight is exactly 0, but 0 * NaN is NaN, so clear them
+        if (t_begin + kAttBlockTokens > cur.kvl && t >= cur.kvl - t_begin) {
+            uint8_t* v_row = sm.v_ring + (q % p.v_stages) * Cfg::kTileBytes + t * 128;
+#pragma unroll
+            for (int hf = 0; hf < Cfg::kSlabs; ++hf)
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch)
+                    *reinterpret_cast<uint4*>(v_row + hf * Cfg::kSlabBytes + ch * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(&bars->p_full[pbuf]);
+        mbar_arrive(&bars->s_empty[buf]);
+
+        const int pair_global = cur.pair0 + cur.pair;
+        const int64_t pair_blk_first = static_cast<int64_t>(cur.blk0) + static_cast<int64_t>(cur.pair) * cur.nb;
+        const int pair_nb = cur.nb;
+        cur.advance(p, q + 1 < n_my);
+        seg_first = seg_last;
+        if (!seg_last) continue;
+
+        // ---------------------------------------------------------------- end of the segment
+        ++seg;
+        // ---- row sums: add my warp's tokens, then the four warps; lane i ends up with column 32*ci + i
+        float* xl = sm.xch + 2 * 4 * n_pad;
+        float l_c[NCH];
+#pragma unroll
+        for (int ci = 0; ci < NCH; ++ci) {
+            l_c[ci] = 0.f;
+            if (ci * 32 < n_pad) {
+                float mine = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float w = warp_sum(lsum[ci * 32 + i]);
+                    if (lane == i) mine = w;
+                }
+                if (ci * 32 + lane < n_pad) xl[quarter * n_pad + ci * 32 + lane] = mine;
+            }
+        }
+        if (!group_sync(15)) { ok = false; break; }
+#pragma unroll
+        for (int ci = 0; ci < NCH; ++ci) {
+            const int col = ci * 32 + lane;
+            if (col < n_pad) l_c[ci] = (xl[col] + xl[n_pad + col]) + (xl[2 * n_pad + col] + xl[3 * n_pad + col]);
+        }
+        if (!mbar_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
+        tc_fence_after();
+        if (!o_lane) continue;                                         // nothing of O^T in this warp's lanes
+        // which CTAs hold blocks of this pair: CTA c owns blocks [c*T/G, (c+1)*T/G), so the owner of
+        // block x is ceil((x+1)*G/T) - 1
+        const int64_t pair_blk_last = pair_blk_first + pair_nb - 1;
+        const int c_first = static_cast<int>(((pair_blk_first + 1) * gridDim.x - 1) / total_blocks);
+        const int c_last = static_cast<int>(((pair_blk_last + 1) * gridDim.x - 1) / total_blocks);
+
+        if (c_first == c_last) {
+            // the whole pair was ours: normalise and store; thread t holds element t of every row
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 < n_pad) {
+                    uint32_t o[32];
+                    tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (ci * 32 + i < rows_here) {                 // uniform
+                            const float l = __shfl_sync(0xffffffffu, l_c[ci], i);
+                            const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
+                            p.attn_out[static_cast<int64_t>(row) * DH + t] = __float2bfloat16_rn(__uint_as_float(o[i]) / l);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            continue;
+        }
+
+        // ---- the pair spans CTAs c_first..c_last: every warp parks its 32 rows of O^T with its own copy
+        // of (m, l) and takes its own ticket; the warp that arrives last for (pair, warp) merges those
+        // rows.  A CTA's parts are its first and its last segment.
+        const int my_slot = cta * 2 + ((seg == 1) ? 0 : 1);
+        {
+            float* po = p.part_o + (static_cast<int64_t>(my_slot) * DH + t) * kAttRowsPerPair;
+            float* pml = p.part_ml + (static_cast<int64_t>(my_slot) * 4 + quarter) * kAttRowsPerPair * 2;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 < n_pad) {
+                    uint32_t o[32];
+                    tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        if (ci * 32 + i < n_pad)
+                            __stcg(reinterpret_cast<float4*>(po + ci * 32 + i),
+                                   make_float4(__uint_as_float(o[i]), __uint_as_float(o[i + 1]),
+                                               __uint_as_float(o[i + 2]), __uint_as_float(o[i + 3])));
+                    if (ci * 32 + lane < n_pad)
+                        __stcg(reinterpret_cast<float2*>(pml + (ci * 32 + lane) * 2), make_float2(m_used[ci], l_c[ci]));
+                }
+            }
+        }
+        tc_fence_before();
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+            int32_t* tk = p.tickets + static_cast<int64_t>(pair_global) * 4 + quarter;
+            last = (atomicAdd(tk, 1) == c_last - c_first);
+            if (last) *tk = 0;                                         // ready for the next call
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (!last) continue;
+
+        // ---- this warp completed its rows of the pair: out = sum_c 2^(m_c - M) O_c / sum_c 2^(m_c - M) l_c,
+        // parts taken in CTA order.  The first CTA holds the head of the pair in its last segment unless its
+        // range starts exactly there; every later CTA holds its part in its first segment.
+        __threadfence();
+        const int blk_begin_c0 = static_cast<int>(static_cast<int64_t>(c_first) * total_blocks / gridDim.x);
+        const int slot_c0 = c_first * 2 + ((blk_begin_c0 == pair_blk_first) ? 0 : 1);
+        float m_all[NCH], l_all[NCH];
+#pragma unroll
+        for (int ci = 0; ci < NCH; ++ci) {
+            m_all[ci] = -INFINITY;
+            l_all[ci] = 0.f;
+            const int col = ci * 32 + lane;
+            if (col < n_pad) {
+                for (int cc = c_first; cc <= c_last; ++cc) {
+                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+                    m_all[ci] = fmaxf(m_all[ci], __ldcg(p.part_ml + ((static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair + col) * 2));
+                }
+                for (int cc = c_first; cc <= c_last; ++cc) {
+                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(
+                        p.part_ml + ((static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair + col) * 2));
+                    if (ml.x != -INFINITY) l_all[ci] += fast_exp2(ml.x - m_all[ci]) * ml.y;
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < NCH * 32; ++i) lsum[i] = 0.f;              // reused as the accumulator of my O^T row
+        for (int cc = c_first; cc <= c_last; ++cc) {
+            const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+            const float4* po = reinterpret_cast<const float4*>(p.part_o + (static_cast<int64_t>(slot) * DH + t) * kAttRowsPerPair);
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 < n_pad) {
+                    const int col = ci * 32 + lane;
+                    float wgt = 0.f;                                   // weight of this part for my column
+                    if (col < n_pad) {
+                        const float mc = __ldcg(p.part_ml + ((static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair + col) * 2);
+                        wgt = (mc == -INFINITY) ? 0.f : fast_exp2(mc - m_all[ci]);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        if (ci * 32 + i < rows_here) {                 // uniform
+                            const float4 v = __ldcg(po + ci * 8 + (i >> 2));
+                            const float w0 = __shfl_sync(0xffffffffu, wgt, i), w1 = __shfl_sync(0xffffffffu, wgt, i + 1);
+                            const float w2 = __shfl_sync(0xffffffffu, wgt, i + 2), w3 = __shfl_sync(0xffffffffu, wgt, i + 3);
+                            // a part that saw no visible token has weight 0
+                            if (w0 != 0.f) lsum[ci * 32 + i + 0] += w0 * v.x;
+                            if (w1 != 0.f) lsum[ci * 32 + i + 1] += w1 * v.y;
+                            if (w2 != 0.f) lsum[ci * 32 + i + 2] += w2 * v.z;
+                            if (w3 != 0.f) lsum[ci * 32 + i + 3] += w3 * v.w;
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int ci = 0; ci < NCH; ++ci) {
+            if (ci * 32 < n_pad) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    if (ci * 32 + i < rows_here) {                     // uniform
+                        const float l = __shfl_sync(0xffffffffu, l_all[ci], i);
+                        const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
+                        p.attn_out[static_cast<int64_t>(row) * DH + t] = __float2bfloat16_rn(lsum[ci * 32 + i] / l);
+                    }
+                }
+            }
+        }
+    }
+}
+
 template <int DH>
 __global__ void __launch_bounds__(kAttThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
@@ -182,18 +591,25 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
     using Cfg = AttCfg<DH>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    AttBars* bars = reinterpret_cast<AttBars*>(smem + Cfg::kBarOffset);
+    const int n_pad = p.n_pad;
+    AttSmem sm;
+    sm.k_ring = smem;
+    sm.v_ring = smem + p.k_stages * Cfg::kTileBytes;
+    sm.q = sm.v_ring + p.v_stages * Cfg::kTileBytes;
+    sm.pt = sm.q + Cfg::q_bytes(n_pad);
+    sm.bars = reinterpret_cast<AttBars*>(sm.pt + p.p_bufs * Cfg::p_bytes(n_pad));
+    sm.xch = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sm.bars) + 512);
+    AttBars* bars = sm.bars;
     __shared__ int s_warp_tot[32];
     __shared__ AttStart s_start;
-    __shared__ int s_flag;
-    __shared__ float s_xch[3][kAttSoftmaxThreads];          // [0..1] row maxima (by block parity), [2] row sums, exchanged between the copies of a row
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 4; ++s) { mbar_init(&bars->kv_full[s], 1); mbar_init(&bars->kv_empty[s], 1); }
+        for (int s = 0; s < p.k_stages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+        for (int s = 0; s < p.v_stages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], kAttSoftmaxThreads);
             mbar_init(&bars->p_full[a], kAttSoftmaxThreads); mbar_init(&bars->p_empty[a], 1);
@@ -267,8 +683,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         const uint64_t pol = l2_policy_evict_first();
         bool new_pair = true;
         bool ok = true;
-        int last_st = -1;
-        uint32_t last_ph = 0;
+        int phys_next = 0;
+        bool have_next = false;
         for (int q = 0; q < n_my && ok; ++q) {
             const int kvh = cur.pair / cur.rbc;
             if (new_pair) {
@@ -284,82 +700,110 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
                     prefetch_l2(base + (i % lines_per_j) * 128);
                 }
             }
-            const int st = q % Cfg::kStages;
-            const int use = q / Cfg::kStages;
-            if (use > 0 && !mbar_wait(&bars->kv_empty[st], (use - 1) & 1, p.status, 1)) { ok = false; break; }
+            const int ks = q % p.k_stages, k_use = q / p.k_stages;
+            const int vs = q % p.v_stages, v_use = q / p.v_stages;
             const int t_begin = cur.blk * kAttBlockTokens;
             const int t_end = min(cur.kvl, t_begin + kAttBlockTokens);
             const int npg = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
-            if (lane == 0)
-                mbar_arrive_expect_tx(&bars->kv_full[st], static_cast<uint32_t>(npg * 2 * Cfg::kSlabs * kPageTokens * 128));
+            int phys = phys_next;
+            if (!have_next && lane < npg)
+                phys = p.page_table[static_cast<int64_t>(cur.b) * p.max_pages_per_seq + cur.blk * kAttPagesPerStage + lane];
+            if (lane < npg && (phys < 0 || phys >= p.num_pages)) {
+                report_error(p.status, kErrBadPage, phys, 1);
+                phys = 0;                                   // stay inside the pool
+            }
+            const uint32_t tile_tx = static_cast<uint32_t>(npg * Cfg::kSlabs * kPageTokens * 128);
+            // K tile
+            if (k_use > 0 && !mbar_wait(&bars->k_empty[ks], (k_use - 1) & 1, p.status, 1)) { ok = false; break; }
+            if (lane == 0) mbar_arrive_expect_tx(&bars->k_full[ks], tile_tx);
             __syncwarp();
             if (lane < npg) {
-                const int page_idx = cur.blk * kAttPagesPerStage + lane;
-                int phys = p.page_table[static_cast<int64_t>(cur.b) * p.max_pages_per_seq + page_idx];
-                if (phys < 0 || phys >= p.num_pages) {
-                    report_error(p.status, kErrBadPage, phys, 1);
-                    phys = 0;                               // stay inside the pool
-                }
-                uint8_t* dst = smem + st * Cfg::kStageBytes + lane * (kPageTokens * 128);
+                uint8_t* dst = sm.k_ring + ks * Cfg::kTileBytes + lane * (kPageTokens * 128);
                 const int row_k = ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens;
+#pragma unroll
+                for (int hf = 0; hf < Cfg::kSlabs; ++hf)
+                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &bars->k_full[ks], hf * 64, row_k, pol);
+            }
+            // V tile
+            if (v_use > 0 && !mbar_wait(&bars->v_empty[vs], (v_use - 1) & 1, p.status, 20)) { ok = false; break; }
+            if (lane == 0) mbar_arrive_expect_tx(&bars->v_full[vs], tile_tx);
+            __syncwarp();
+            if (lane < npg) {
+                uint8_t* dst = sm.v_ring + vs * Cfg::kTileBytes + lane * (kPageTokens * 128);
                 const int row_v = ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens;
 #pragma unroll
-                for (int hf = 0; hf < Cfg::kSlabs; ++hf) {
-                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &bars->kv_full[st], hf * 64, row_k, pol);
-                    tma_load_2d(dst + (Cfg::kSlabs + hf) * Cfg::kSlabBytes, &kv_map, &bars->kv_full[st], hf * 64, row_v, pol);
-                }
+                for (int hf = 0; hf < Cfg::kSlabs; ++hf)
+                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &bars->v_full[vs], hf * 64, row_v, pol);
             }
             __syncwarp();
-            last_st = st; last_ph = use & 1;
             new_pair = cur.advance(p, q + 1 < n_my);
+            // page ids of the next block, fetched while this block's copies are in flight
+            have_next = false;
+            if (q + 1 < n_my) {
+                const int nt_begin = cur.blk * kAttBlockTokens;
+                const int n_npg = (min(cur.kvl, nt_begin + kAttBlockTokens) - nt_begin + kPageTokens - 1) / kPageTokens;
+                if (lane < n_npg)
+                    phys_next = p.page_table[static_cast<int64_t>(cur.b) * p.max_pages_per_seq + cur.blk * kAttPagesPerStage + lane];
+                have_next = true;
+            }
         }
         // do not leave while a copy of ours may still be landing in shared memory
-        if (last_st >= 0) mbar_wait(&bars->kv_full[last_st], last_ph, p.status, 9);
+        if (ok && n_my > 0) {
+            const int ql = n_my - 1;
+            mbar_wait(&bars->k_full[ql % p.k_stages], (ql / p.k_stages) & 1, p.status, 9);
+            mbar_wait(&bars->v_full[ql % p.v_stages], (ql / p.v_stages) & 1, p.status, 9);
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_my > 0) {
-            const uint32_t idesc_s = umma_idesc_bf16(128, 128);
-            const uint32_t idesc_o = umma_idesc_bf16(128, DH) | kIdescBMajorMN;
-            const uint32_t q_addr = smem_u32(smem + Cfg::kQOffset);
+            const uint32_t idesc_s = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad));
+            const uint32_t idesc_o = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad)) | kIdescAMajorMN | kIdescBMajorMN;
+            const uint32_t q_addr = smem_u32(sm.q);
+            const uint32_t q_slab = static_cast<uint32_t>(n_pad) * 128u;
             bool ok = true;
             int seg = 0;
-            // S[q & 1] = Q K^T of block q (waits: the pair's Q tile, the K/V stage, the S buffer)
+            // S^T[q & 1] = K Q^T of block q (waits: the pair's Q tile, the K tile, the S^T buffer)
             auto issue_s = [&](int q, bool seg_first, int seg_idx) -> bool {
-                const int st = q % Cfg::kStages, buf = q & 1, u = q >> 1;
+                const int ks = q % p.k_stages, buf = q & 1, u = q >> 1;
                 if (seg_first && !mbar_wait(&bars->q_full, seg_idx & 1, p.status, 2)) return false;
-                if (!mbar_wait(&bars->kv_full[st], (q / Cfg::kStages) & 1, p.status, 3)) return false;
+                if (!mbar_wait(&bars->k_full[ks], (q / p.k_stages) & 1, p.status, 3)) return false;
                 if (u > 0 && !mbar_wait(&bars->s_empty[buf], (u - 1) & 1, p.status, 4)) return false;
                 tc_fence_after();
-                const uint32_t k_addr = smem_u32(smem + st * Cfg::kStageBytes);
+                const uint32_t k_addr = smem_u32(sm.k_ring + ks * Cfg::kTileBytes);
                 const uint32_t acc = tmem_base + (buf ? kTmemS1 : kTmemS0);
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32;
-                    umma_bf16(acc, umma_desc_k_sw128(q_addr + off), umma_desc_k_sw128(k_addr + off), idesc_s, kk > 0 ? 1u : 0u);
+                    const uint64_t da = umma_desc_k_sw128(k_addr + (kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32);
+                    const uint64_t db = umma_desc_k_sw128(q_addr + (kk >> 2) * q_slab + (kk & 3) * 32);
+                    umma_bf16(acc, da, db, idesc_s, kk > 0 ? 1u : 0u);
                 }
                 umma_commit(&bars->s_full[buf]);
+                umma_commit(&bars->k_empty[ks]);
                 return true;
             };
             bool seg_first = true;
             ok = issue_s(0, true, 0);
             for (int q = 0; q < n_my && ok; ++q) {
                 const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
-                const int st = q % Cfg::kStages, buf = q & 1, u = q >> 1;
-                if (!seg_last && q + 1 < n_my) { if (!issue_s(q + 1, false, seg)) { ok = false; break; } }   // overlap with softmax of q
-                if (!mbar_wait(&bars->p_full[buf], u & 1, p.status, 5)) { ok = false; break; }
+                const int vs = q % p.v_stages;
+                if (!seg_last && q + 1 < n_my) { if (!issue_s(q + 1, false, seg)) { ok = false; break; } }   // overlaps the softmax of q
+                const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
+                if (!mbar_wait(&bars->v_full[vs], (q / p.v_stages) & 1, p.status, 21)) { ok = false; break; }
+                if (!mbar_wait(&bars->p_full[pbuf], pu & 1, p.status, 5)) { ok = false; break; }
                 tc_fence_after();
                 {
-                    const uint32_t p_addr = smem_u32(smem + Cfg::kPOffset + buf * Cfg::kPBytes);
-                    const uint32_t v_addr = smem_u32(smem + st * Cfg::kStageBytes + Cfg::kSlabs * Cfg::kSlabBytes);
+                    const uint32_t p_addr = smem_u32(sm.pt + pbuf * Cfg::p_bytes(n_pad));
+                    const uint32_t v_addr = smem_u32(sm.v_ring + vs * Cfg::kTileBytes);
 #pragma unroll
                     for (int ks = 0; ks < kAttBlockTokens / 16; ++ks) {
-                        const uint64_t da = umma_desc_k_sw128(p_addr + (ks >> 2) * Cfg::kSlabBytes + (ks & 3) * 32);
-                        const uint64_t db = umma_desc_mn_sw128(v_addr + ks * 2048, Cfg::kSlabBytes, 1024);
+                        // 16 tokens: two groups of 8 k-rows in both operands
+                        const uint64_t da = umma_desc_mn_sw128(v_addr + ks * 2048, Cfg::kSlabBytes, 1024);
+                        const uint64_t db = umma_desc_mn_plain(p_addr + ks * 256, 2048, 128);
                         umma_bf16(tmem_base + kTmemO, da, db, idesc_o, (seg_first && ks == 0) ? 0u : 1u);
                     }
                 }
-                umma_commit(&bars->kv_empty[st]);
-                umma_commit(&bars->p_empty[buf]);
+                umma_commit(&bars->v_empty[vs]);
+                umma_commit(&bars->p_empty[pbuf]);
                 umma_commit(&bars->o_full);
                 cur.advance(p, q + 1 < n_my);
                 seg_first = seg_last;
@@ -369,313 +813,11 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
                 }
             }
         }
-    } else {
-        // ------------------------------------------------------------------ softmax
-        // Thread t owns TMEM lane t.  When the pair has at most 32 (64) query rows the Q tile holds
-        // 4 (2) copies of them, copy c in tile rows [c*span, (c+1)*span), span = 128 / copies, and
-        // the thread of tile row c*span + r handles tokens [c*span, (c+1)*span) of row r in every
-        // block: all four warps share the work of a small pair.  The copies agree on the row
-        // maximum through shared memory and write their part of P into row r of ONE P tile, so O is
-        // complete in tile rows [0, span) and needs no merge.
-        const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
-        const int t = quarter * 32 + lane;                  // tile row
-        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-        uint8_t* q_smem = smem + Cfg::kQOffset;
-        bool ok = true;
-        bool seg_first = true;
-        int seg = 0;
-        uint32_t group_phase = 0;
-        float m_used = -INFINITY, l_run = 0.f;
-        int rows_here = 0, row_lo = 0, limit = 0, ctx = 0;
-        int copies = 1, span = 128, c = 0, r = t;
-
-        // all softmax threads meet; bounded like every other wait
-        auto group_sync = [&](int where) -> bool {
-            mbar_arrive(&bars->group);
-            const bool done = mbar_wait(&bars->group, group_phase, p.status, where);
-            group_phase ^= 1u;
-            return done;
-        };
-
-        for (int q = 0; q < n_my && ok; ++q) {
-            const int kvh = cur.pair / cur.rbc;
-            if (seg_first) {
-                // ---- the pair's query rows -> shared memory in the K-major swizzled layout of operand A
-                row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
-                const int n_rows = p.group * (cur.k + 1);
-                rows_here = min(kAttRowsPerPair, n_rows - row_lo);
-                ctx = cur.kvl - (cur.k + 1);
-                copies = rows_here <= 32 ? 4 : (rows_here <= 64 ? 2 : 1);
-                span = kAttRowsPerPair / copies;
-                c = t / span;
-                r = t % span;
-                if (r < rows_here) {
-                    const int rho = row_lo + r;
-                    const int j = rho / p.group, hh = rho % p.group;
-                    limit = ctx + j + 1;
-                    const uint4* src = reinterpret_cast<const uint4*>(
-                        p.hidden + (static_cast<int64_t>(cur.q_row0 + j) * p.n_q_heads + kvh * p.group + hh) * DH);
-                    uint4 v[DH / 8];
-#pragma unroll
-                    for (int ch = 0; ch < DH / 8; ++ch) v[ch] = __ldg(src + ch);
-#pragma unroll
-                    for (int ch = 0; ch < DH / 8; ++ch)
-                        *reinterpret_cast<uint4*>(q_smem + (ch >> 3) * Cfg::kSlabBytes + t * 128 + (((ch & 7) ^ (t & 7)) << 4)) = v[ch];
-                }
-                m_used = -INFINITY;
-                l_run = 0.f;
-                fence_proxy_async();
-                tc_fence_before();
-                mbar_arrive(&bars->q_full);
-            }
-            const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
-            const int st = q % Cfg::kStages, buf = q & 1, u = q >> 1;
-            const int t_begin = cur.blk * kAttBlockTokens;
-            const bool real = r < rows_here;
-            const bool warp_real = (quarter * 32) % span < rows_here;    // warp-uniform: a real row among this warp's lanes
-            const bool o_owner = (quarter * 32 < span) && warp_real;      // warp-uniform: this warp's lanes hold real rows of O
-            const uint32_t t_s = t_lane + (buf ? kTmemS1 : kTmemS0) + static_cast<uint32_t>(c * span);
-            const int lim_local = (real ? limit : 0) - t_begin - c * span;   // my tokens [0, lim_local) are visible
-            const bool need_mask = (t_begin + kAttBlockTokens > ctx + 1);
-
-            if (!mbar_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
-            tc_fence_after();
-
-            // ---- pass 1: maximum over my tokens of the block, then over the copies of the row
-            float mx = -INFINITY;
-            if (warp_real) {
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                for (int c0 = 0; c0 < span; c0 += 32) {
-                    uint32_t sv[32];
-                    tmem_ld_x32(t_s + c0, sv);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        float v = __uint_as_float(sv[i]);
-                        if (need_mask && c0 + i >= lim_local) v = -INFINITY;
-                        mx4[i & 3] = fmaxf(mx4[i & 3], v);
-                    }
-                }
-                mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;   // scale > 0: the maximum commutes
-                if (!real) mx = -INFINITY;                                 // padding rows stay inert
-            }
-            if (copies > 1) {
-                float* xch = s_xch[q & 1];
-                xch[t] = mx;
-                if (!group_sync(13)) { ok = false; break; }
-                mx = xch[r];
-                for (int cc = 1; cc < copies; ++cc) mx = fmaxf(mx, xch[cc * span + r]);
-            }
-            // ---- raise the running maximum only if it grew by more than the threshold
-            float alpha = 1.f;
-            if (seg_first) {
-                m_used = mx;
-            } else if (mx > m_used + kRescaleThreshold) {
-                alpha = fast_exp2(m_used - mx);                            // m_used == -inf gives 0
-                m_used = mx;
-                l_run *= alpha;
-            }
-            if (o_owner && !seg_first && __any_sync(0xffffffffu, alpha != 1.f)) {
-                // O += P V of the previous block must have landed before O is rescaled
-                if (!mbar_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int c0 = 0; c0 < DH; c0 += 32) {
-                    uint32_t o[32];
-                    tmem_ld_x32(t_lane + kTmemO + c0, o);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st_x32(t_lane + kTmemO + c0, o);
-                }
-                tmem_st_wait();
-            }
-            // the P buffer is free once the P V product of two blocks ago has read it
-            if (u > 0 && !mbar_wait(&bars->p_empty[buf], (u - 1) & 1, p.status, 8)) { ok = false; break; }
-            if (warp_real) {
-                // ---- pass 2: p = 2^(s * scale - m), bf16, into row r of operand A of the P V product
-                const float m_safe = (m_used == -INFINITY) ? 0.f : m_used;
-                uint8_t* p_row = smem + Cfg::kPOffset + buf * Cfg::kPBytes + r * 128;
-                float rs0 = 0.f, rs1 = 0.f;
-                for (int c0 = 0; c0 < span; c0 += 32) {
-                    uint32_t sv[32];
-                    tmem_ld_x32(t_s + c0, sv);
-                    tmem_ld_wait();
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float e0 = fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -m_safe));
-                        float e1 = fast_exp2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -m_safe));
-                        if (need_mask) {
-                            if (c0 + i >= lim_local) e0 = 0.f;
-                            if (c0 + i + 1 >= lim_local) e1 = 0.f;
-                        }
-                        rs0 += e0;
-                        rs1 += e1;
-                        pk[i >> 1] = pack_bf16(e0, e1);
-                    }
-                    if (real) {
-#pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
-                            const int chunk = ((c * span + c0) >> 3) + ch;  // 16-byte chunk (8 tokens) of the row
-                            *reinterpret_cast<uint4*>(p_row + (chunk >> 3) * Cfg::kSlabBytes + (((chunk & 7) ^ (r & 7)) << 4)) =
-                                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-                        }
-                    }
-                }
-                l_run += rs0 + rs1;
-            }
-            // rows of V past the end of the sequence may hold anything (the pool is the caller's, or
-            // the page was never loaded): their weight is exactly 0, but 0 * NaN is NaN, so clear them
-            if (t_begin + kAttBlockTokens > cur.kvl && t >= cur.kvl - t_begin) {
-                uint8_t* v_row = smem + st * Cfg::kStageBytes + Cfg::kSlabs * Cfg::kSlabBytes + t * 128;
-#pragma unroll
-                for (int hf = 0; hf < Cfg::kSlabs; ++hf)
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch)
-                        *reinterpret_cast<uint4*>(v_row + hf * Cfg::kSlabBytes + ch * 16) = make_uint4(0u, 0u, 0u, 0u);
-            }
-            fence_proxy_async();
-            tc_fence_before();
-            mbar_arrive(&bars->p_full[buf]);
-            mbar_arrive(&bars->s_empty[buf]);
-
-            const int pair_global = cur.pair0 + cur.pair;
-            const int64_t pair_blk_first = static_cast<int64_t>(cur.blk0) + static_cast<int64_t>(cur.pair) * cur.nb;
-            const int pair_nb = cur.nb, pair_q_row0 = cur.q_row0;
-            cur.advance(p, q + 1 < n_my);
-            seg_first = seg_last;
-            if (!seg_last) continue;
-
-            // ------------------------------------------------------------ end of the segment
-            ++seg;
-            if (copies > 1) {
-                // the copies of a row hold the sums over their own tokens (same maximum): add them up
-                float* xch = s_xch[2];
-                xch[t] = l_run;
-                if (!group_sync(14)) { ok = false; break; }
-                l_run = xch[r];
-                for (int cc = 1; cc < copies; ++cc) l_run += xch[cc * span + r];
-            }
-            if (!mbar_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
-            tc_fence_after();
-            // which CTAs hold blocks of this pair: CTA c owns blocks [c*T/G, (c+1)*T/G), so the owner of
-            // block x is ceil((x+1)*G/T) - 1
-            const int64_t pair_blk_last = pair_blk_first + pair_nb - 1;
-            const int c_first = static_cast<int>(((pair_blk_first + 1) * gridDim.x - 1) / total_blocks);
-            const int c_last = static_cast<int>(((pair_blk_last + 1) * gridDim.x - 1) / total_blocks);
-            const int rho = row_lo + r;
-            const int64_t out_row = static_cast<int64_t>(pair_q_row0 + rho / p.group) * p.n_q_heads + kvh * p.group + rho % p.group;
-            __nv_bfloat16* out = p.attn_out + out_row * DH;
-            const bool writer = o_owner && real;                           // c == 0 and a real row
-
-            if (c_first == c_last) {
-                // the whole pair was ours: normalise and store
-                if (o_owner) {
-                    const float inv = 1.f / l_run;
-#pragma unroll
-                    for (int cc = 0; cc < DH; cc += 32) {
-                        uint32_t o[32];
-                        tmem_ld_x32(t_lane + kTmemO + cc, o);
-                        tmem_ld_wait();
-                        if (writer) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 8) {
-                                uint4 w;
-                                w.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-                                w.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-                                w.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-                                w.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-                                *reinterpret_cast<uint4*>(out + cc + i) = w;
-                            }
-                        }
-                    }
-                }
-                tc_fence_before();
-                continue;
-            }
-
-            // ---- the pair spans CTAs c_first..c_last: park (m, l, O); a CTA's parts are its first and its last segment
-            const int my_slot = cta * 2 + ((seg == 1) ? 0 : 1);
-            if (o_owner) {
-                float* po = p.part_o + (static_cast<int64_t>(my_slot) * kAttRowsPerPair + r) * DH;
-#pragma unroll
-                for (int cc = 0; cc < DH; cc += 32) {
-                    uint32_t o[32];
-                    tmem_ld_x32(t_lane + kTmemO + cc, o);
-                    tmem_ld_wait();
-                    if (writer) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            __stcg(reinterpret_cast<float4*>(po + cc + i),
-                                   make_float4(__uint_as_float(o[i]), __uint_as_float(o[i + 1]),
-                                               __uint_as_float(o[i + 2]), __uint_as_float(o[i + 3])));
-                    }
-                }
-                if (writer)
-                    __stcg(reinterpret_cast<float2*>(p.part_ml + (static_cast<int64_t>(my_slot) * kAttRowsPerPair + r) * 2),
-                           make_float2(m_used, l_run));
-            }
-            tc_fence_before();
-            __threadfence();
-            if (!group_sync(11)) { ok = false; break; }                    // every softmax thread has published
-            if (t == 0) {
-                const int tk = atomicAdd(&p.tickets[pair_global], 1);
-                const int last = (tk == c_last - c_first);
-                if (last) p.tickets[pair_global] = 0;                      // ready for the next call
-                s_flag = last;
-            }
-            if (!group_sync(12)) { ok = false; break; }
-            if (s_flag && writer) {
-                // ---- this CTA completed the pair: out = sum_c 2^(m_c - M) O_c / sum_c 2^(m_c - M) l_c,
-                // parts taken in CTA order.  The first CTA holds the head of the pair in its last segment unless
-                // its range starts exactly there; every later CTA holds its part in its first segment.
-                __threadfence();
-                const int blk_begin_c0 = static_cast<int>(static_cast<int64_t>(c_first) * total_blocks / gridDim.x);
-                const int slot_c0 = c_first * 2 + ((blk_begin_c0 == pair_blk_first) ? 0 : 1);
-                float m_all = -INFINITY;
-                for (int cc = c_first; cc <= c_last; ++cc) {
-                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
-                    m_all = fmaxf(m_all, __ldcg(p.part_ml + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * 2));
-                }
-                float l_all = 0.f;
-                for (int cc = c_first; cc <= c_last; ++cc) {
-                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
-                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * 2));
-                    if (ml.x != -INFINITY) l_all += fast_exp2(ml.x - m_all) * ml.y;
-                }
-                const float inv = 1.f / l_all;
-#pragma unroll 1
-                for (int col = 0; col < DH; col += 32) {
-                    float acc[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-                    for (int cc = c_first; cc <= c_last; ++cc) {
-                        const int slot = (cc == c_first) ? slot_c0 : cc * 2;
-                        const float mc = __ldcg(p.part_ml + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * 2);
-                        if (mc == -INFINITY) continue;                     // that part saw no visible token
-                        const float wgt = fast_exp2(mc - m_all);
-                        const float4* po = reinterpret_cast<const float4*>(
-                            p.part_o + (static_cast<int64_t>(slot) * kAttRowsPerPair + r) * DH + col);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float4 v = __ldcg(po + i);
-                            acc[4 * i] += wgt * v.x; acc[4 * i + 1] += wgt * v.y;
-                            acc[4 * i + 2] += wgt * v.z; acc[4 * i + 3] += wgt * v.w;
-                        }
-                    }
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 w;
-                        w.x = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
-                        w.y = pack_bf16(acc[i + 2] * inv, acc[i + 3] * inv);
-                        w.z = pack_bf16(acc[i + 4] * inv, acc[i + 5] * inv);
-                        w.w = pack_bf16(acc[i + 6] * inv, acc[i + 7] * inv);
-                        *reinterpret_cast<uint4*>(out + col + i) = w;
-                    }
-                }
-            }
-        }
+    } else if (n_my > 0) {
+        if (n_pad <= 32) att_softmax<DH, 1>(p, sm, tmem_base, cur, n_my, total_blocks);
+        else if (n_pad <= 64) att_softmax<DH, 2>(p, sm, tmem_base, cur, n_my, total_blocks);
+        else if (n_pad <= 96) att_softmax<DH, 3>(p, sm, tmem_base, cur, n_my, total_blocks);
+        else att_softmax<DH, 4>(p, sm, tmem_base, cur, n_my, total_blocks);
     }
 
     tc_fence_before();
@@ -690,9 +832,9 @@ cudaError_t attention_init(int head_dim)
 {
     if (head_dim == 128)
         return cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    AttCfg<128>::kSmemBytes);
+                                    kAttSmemLimit - kAttStaticReserve);
     return cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                AttCfg<64>::kSmemBytes);
+                                kAttSmemLimit - kAttStaticReserve);
 }
 
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
@@ -700,10 +842,15 @@ cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const A
 {
     dim3 grid(n_ctas);
     dim3 block(kAttThreads);
-    if (h.cfg.head_dim == 128)
-        attention_kernel<128><<<grid, block, AttCfg<128>::kSmemBytes, stream>>>(kv_map, p);
-    else
-        attention_kernel<64><<<grid, block, AttCfg<64>::kSmemBytes, stream>>>(kv_map, p);
+    if (h.cfg.head_dim == 128) {
+        const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<128>::kTileBytes +
+                            AttCfg<128>::fixed_bytes(p.n_pad, p.p_bufs);
+        attention_kernel<128><<<grid, block, smem, stream>>>(kv_map, p);
+    } else {
+        const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<64>::kTileBytes +
+                            AttCfg<64>::fixed_bytes(p.n_pad, p.p_bufs);
+        attention_kernel<64><<<grid, block, smem, stream>>>(kv_map, p);
+    }
     return cudaGetLastError();
 }
 

@@ -17,6 +17,7 @@ constexpr int kDrawChunk = 2048;          // vocabulary entries per CTA of the d
 constexpr int kAttBlockTokens = 128;      // KV tokens per attention work block / pipeline stage
 constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block (MMA M)
 constexpr int kAttThreads = 192;          // TMA warp + MMA warp + 4 softmax warps
+constexpr int kAttMaxStages = 8;          // K / V ring depth (what fits in shared memory is used)
 constexpr int kNumStageEvents = 7;
 
 struct Plan {                 // device tables written by the plan kernel, read by the sampling stage
@@ -32,10 +33,14 @@ struct AttnParams {
     const int32_t* draft_len;
     int32_t batch, n_q_heads, n_kv_heads, group;
     int32_t max_pages_per_seq, num_pages;
+    int32_t n_pad;            // MMA N: the largest pair's query rows rounded up to 16 (<= 128)
+    int32_t k_stages;         // depth of the K ring (128-token tiles)
+    int32_t v_stages;         // depth of the V ring
+    int32_t p_bufs;           // P^T buffers (2, or 1 when shared memory is short)
     float scale_log2;         // log2(e) / sqrt(head_dim)
-    float* part_o;            // [2 * CTAs][128][Dh] unnormalised partial outputs (a CTA's first / last segment)
-    float* part_ml;           // [2 * CTAs][128][2]  (running max in log2 units, sum)
-    int32_t* tickets;         // [pairs] self-resetting arrival counters of the split merge
+    float* part_o;            // [2 * CTAs][Dh][128] unnormalised partial outputs (a CTA's first / last segment)
+    float* part_ml;           // [2 * CTAs][4 warps][128][2]  (running max in log2 units, sum)
+    int32_t* tickets;         // [pairs][4 warps] self-resetting arrival counters of the split merge
     __nv_bfloat16* attn_out;  // [M][d_model]
     int32_t* status;
 };
@@ -109,6 +114,8 @@ cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream);
 cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);
 
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
+int attention_p_bufs(int n_pad);
+void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages);
 cudaError_t lm_head_init();
 size_t lm_head_smem_bytes(int n_tile, int n_blocks, int num_stages);
 int lm_head_pick_stages(int n_tile, int n_blocks);
