@@ -62,29 +62,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after a limit of polls, records a timeout in the status word and
+// Bounded wait: gives up after `limit` polls, records a timeout in the status word and
 // returns false; the caller carries on to its normal teardown so nothing is left waiting.
-// The first polls use the non-blocking test (lowest hand-over latency between pipeline roles);
-// after that try_wait, which suspends the thread for a hardware-chosen interval per poll.
-constexpr uint32_t kWaitSpin = 1u << 12;
+// try_wait itself suspends the thread for a hardware-chosen interval, so the loop neither
+// burns issue slots (a non-blocking test_wait spin measurably slowed the other warps of the
+// SM) nor adds the wake-up latency of a sleep.
 constexpr uint32_t kWaitLimit = 1u << 24;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
 {
-    for (uint32_t i = 0; i < kWaitSpin; ++i) {
-        if (mbar_test_wait(bar, parity)) return true;
-    }
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
     }
