@@ -174,6 +174,33 @@ int flexspec_sample(flexspec_handle* h, const float* logits,
                     const uint32_t* vocab_mask,
                     int32_t* accepted_len, int32_t* next_token, void* stream);
 
+/* The acceptance / emitted-token stage (flexspec_sample) without a handle and without any
+ * allocation.  (No counterpart in the paper: it exists for how some hosts have to run.)
+ * Meant for callers that cannot obtain device memory at call time: a serving process whose
+ * memory pool took the whole device at start-up, so that a cudaMalloc inside the library would
+ * fail or eat into the pool's reserve; or a step loop that must never stall on the implicit
+ * device synchronisation of an allocation or a free.  Such callers cannot use flexspec_create,
+ * which allocates the workspace.
+ *   - The working memory is one fixed array inside the loaded library (about 0.5 MB, held on
+ *     every GPU that loads the library until the process exits).  Limits that follow from it:
+ *     batch <= 64, sum_b (k_b + 1) <= 1024, vocab <= 131072; larger calls return
+ *     FLEXSPEC_ERR_UNSUPPORTED and launch nothing.
+ *   - Runs on the CURRENT device of the calling thread.  The first call on a device looks up
+ *     the device address of the array (a cheap runtime query, no allocation); make that first
+ *     call outside any stream capture.
+ *   - All calls on a device share the array, and it keeps the previous call's contents; each
+ *     call clears the part that has to start at zero on `stream` before its kernels.  Two calls
+ *     whose GPU work may overlap (different streams, no ordering) race on the array: serialise
+ *     them.
+ *   - Arguments as flexspec_sample, all DEVICE pointers except draft_len_host; `mode` is a
+ *     FLEXSPEC_MODE_* value.  A draft token outside [0, vocab) is clamped, not reported.
+ * Errors: INVALID_ARG, UNSUPPORTED (limits above), NO_DEVICE, CUDA. */
+int flexspec_sample_static(const float* logits, const int32_t* draft_tokens, const float* draft_logits,
+                           const int32_t* draft_len, const int32_t* draft_len_host, const uint64_t* seeds,
+                           int32_t batch, int32_t vocab, int32_t mode, float temperature,
+                           const uint32_t* vocab_mask, int32_t* accepted_len, int32_t* next_token,
+                           void* stream);
+
 /* Workspace pointers for stage-wise comparison. */
 int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);
 

@@ -24,7 +24,7 @@ ERR_TIMEOUT, ERR_BAD_PAGE, ERR_BAD_TOKEN, ERR_NO_DEVICE = -5, -6, -7, -8
 
 EXPORTS = [
     "flexspec_create", "flexspec_verify", "flexspec_verify_host", "flexspec_attention",
-    "flexspec_lm_head", "flexspec_sample", "flexspec_get_debug", "flexspec_status",
+    "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_get_debug", "flexspec_status",
     "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
     "flexspec_destroy", "flexspec_strerror", "flexspec_version",
 ]
@@ -61,6 +61,7 @@ def _load() -> C.CDLL:
     lib.flexspec_attention.argtypes = [vp, C.POINTER(KV), vp, vp, vp, i32, vp, vp]
     lib.flexspec_lm_head.argtypes = [vp, vp, i32, vp, vp]
     lib.flexspec_sample.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
+    lib.flexspec_sample_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp]
     lib.flexspec_get_debug.argtypes = [vp, C.POINTER(Debug)]
     lib.flexspec_status.argtypes = [vp, vp]
     lib.flexspec_set_profiling.argtypes = [vp, i32]
@@ -111,6 +112,31 @@ def _host_i32(t, name):
     if t.is_cuda or t.dtype != torch.int32 or not t.is_contiguous():
         raise TypeError(f"{name}: expected a contiguous CPU int32 tensor")
     return t
+
+
+def sample_static(logits, draft_tokens, draft_logits, draft_len, draft_len_host, seeds, mode=MODE_SAMPLE,
+                  temperature=1.0, vocab_mask=None, accepted_len=None, next_token=None, stream=None):
+    """flexspec_sample_static: the acceptance / emitted-token stage for hosts that cannot allocate
+    device memory at call time.  No handle; the library's built-in scratch array is used, so calls
+    on one device must not overlap.  Outputs may be passed in (then nothing at all is allocated,
+    not even by torch); otherwise two int32 tensors are created for convenience."""
+    batch = int(draft_len_host.numel())
+    _dev(logits, torch.float32, "logits")
+    vocab = int(logits.shape[-1])
+    dev = logits.device
+    if accepted_len is None:
+        accepted_len = torch.empty(batch, dtype=torch.int32, device=dev)
+    if next_token is None:
+        next_token = torch.empty(batch, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(LIB.flexspec_sample_static(
+            _ptr(logits), _ptr(_dev(draft_tokens, torch.int32, "draft_tokens")),
+            _ptr(_dev(draft_logits, torch.float32, "draft_logits")), _ptr(_dev(draft_len, torch.int32, "draft_len")),
+            _ptr(_host_i32(draft_len_host, "draft_len_host")), _ptr(_dev(seeds, torch.int64, "seeds")),
+            batch, vocab, int(mode), float(temperature), _ptr(_dev(vocab_mask, torch.int32, "vocab_mask")),
+            _ptr(_dev(accepted_len, torch.int32, "accepted_len")), _ptr(_dev(next_token, torch.int32, "next_token")),
+            _stream_ptr(stream)), "flexspec_sample_static")
+    return accepted_len, next_token
 
 
 class Verifier:
