@@ -82,6 +82,9 @@ void free_workspace(Handle& h)
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
     for (int i = 0; i < kNumStageEvents; ++i)
         if (h.ev[i]) cudaEventDestroy(h.ev[i]);
+    if (h.ev_fork) cudaEventDestroy(h.ev_fork);
+    if (h.ev_join) cudaEventDestroy(h.ev_join);
+    if (h.side) cudaStreamDestroy(h.side);
 }
 
 // geometry of one call, derived from the host copies of the lengths
@@ -187,13 +190,12 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, cudaStr
     return FLEXSPEC_OK;
 }
 
-int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, const float* draft_logits,
-               const int32_t* draft_len, const uint64_t* seeds, const Geometry& g, int32_t batch,
-               float temperature, const uint32_t* vocab_mask, int32_t* accepted_len, int32_t* next_token,
-               cudaStream_t s)
+void fill_sample_params(Handle& h, SampleParams& p, const float* logits, const int32_t* draft_tokens,
+                        const float* draft_logits, const int32_t* draft_len, const uint64_t* seeds, const Geometry& g,
+                        int32_t batch, float temperature, const uint32_t* vocab_mask, int32_t* accepted_len,
+                        int32_t* next_token)
 {
     const flexspec_config& c = h.cfg;
-    SampleParams p;
     memset(&p, 0, sizeof(p));
     p.greedy = (c.mode == FLEXSPEC_MODE_GREEDY || temperature == 0.f) ? 1 : 0;
     p.logits = logits; p.draft_logits = draft_logits; p.draft_tokens = draft_tokens;
@@ -209,9 +211,19 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
     p.accepted_len = accepted_len; p.next_token = next_token;
     if (c.flags & FLEXSPEC_FLAG_DEBUG) { p.dbg_p = h.dbg_p; p.dbg_q = h.dbg_q; p.dbg_u = h.dbg_u; }
     p.status = h.status;
-    if (launch_sample_stats(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+}
+
+// the whole stage on one stream: statistics of every row, decision, draw
+int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, const float* draft_logits,
+               const int32_t* draft_len, const uint64_t* seeds, const Geometry& g, int32_t batch,
+               float temperature, const uint32_t* vocab_mask, int32_t* accepted_len, int32_t* next_token,
+               cudaStream_t s)
+{
+    SampleParams p;
+    fill_sample_params(h, p, logits, draft_tokens, draft_logits, draft_len, seeds, g, batch, temperature, vocab_mask,
+                       accepted_len, next_token);
+    if (launch_sample_stats(p, 0, p.greedy ? p.m_rows : p.m_rows + p.s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
-    mark(h, 5, s);
     if (!p.greedy) {
         if (launch_sample_draw(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
@@ -313,6 +325,11 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     }
     for (int i = 0; i < kNumStageEvents && rc == FLEXSPEC_OK; ++i)
         if (cudaEventCreate(&h.ev[i]) != cudaSuccess) rc = FLEXSPEC_ERR_CUDA;
+    if (rc == FLEXSPEC_OK &&
+        (cudaStreamCreateWithFlags(&h.side, cudaStreamNonBlocking) != cudaSuccess ||
+         cudaEventCreateWithFlags(&h.ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&h.ev_join, cudaEventDisableTiming) != cudaSuccess))
+        rc = FLEXSPEC_ERR_CUDA;
     if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map, lm_head_w, static_cast<uint64_t>(c.vocab),
                                             static_cast<uint64_t>(d_model), 128);
     if (rc == FLEXSPEC_OK && (attention_init(c.head_dim) != cudaSuccess || lm_head_init() != cudaSuccess))
@@ -418,9 +435,22 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
     memset(h.ev_used, 0, sizeof(h.ev_used));
+    SampleParams sp;
+    fill_sample_params(h, sp, h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch, temperature, vocab_mask,
+                       accepted_len, next_token);
     mark(h, 0, s);
-    rc = run_plan(h, draft_len, draft_tokens, batch, s);
+    // ---- second stream: row offsets of the ragged batch and the statistics of the draft logits need
+    // nothing from the target model, so they run beside attention and the LM head
+    if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess)
+        return FLEXSPEC_ERR_CUDA;
+    rc = run_plan(h, draft_len, draft_tokens, batch, h.side);
     if (rc != FLEXSPEC_OK) return rc;
+    if (!sp.greedy && sp.s_rows > 0) {
+        if (launch_sample_stats(sp, sp.m_rows, sp.s_rows, h.side) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        h.launches++;
+    }
+    if (cudaEventRecord(h.ev_join, h.side) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    // ---- main stream
     mark(h, 1, s);
     rc = run_attention(h, kv, hidden, draft_len, g, batch, h.attn_out, s);
     if (rc != FLEXSPEC_OK) return rc;
@@ -429,9 +459,14 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);
-    rc = run_sample(h, h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch, temperature,
-                    vocab_mask, accepted_len, next_token, s);                // marks event 5 after the stats kernel
-    if (rc != FLEXSPEC_OK) return rc;
+    if (cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_stats(sp, 0, sp.m_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;   // the last CTA of a sequence decides
+    h.launches++;
+    mark(h, 5, s);
+    if (!sp.greedy) {
+        if (launch_sample_draw(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        h.launches++;
+    }
     mark(h, 6, s);
     return FLEXSPEC_OK;
 }

@@ -68,6 +68,7 @@ struct SampleParams {
     const int32_t* cu_d;
     const int32_t* row_seq;
     int32_t batch, vocab, m_rows, s_rows, n_chunks, n_dchunks, mask_words;
+    int32_t row_begin;            // first row of this launch of the statistics kernel
     float inv_temp_log2;          // log2(e) / T
     int32_t greedy;
     float2* stats;                // [(M+S)][n_chunks] (chunk max in logit units, sum exp)
@@ -98,6 +99,8 @@ struct Handle {
     // host staging for flexspec_verify_host
     void* stage_dev; size_t stage_bytes;
     int32_t* out_dev;
+    // second stream: the plan and the draft-logit statistics run beside attention and the LM head
+    cudaStream_t side; cudaEvent_t ev_fork, ev_join;
     // profiling
     int32_t profiling, launches;
     cudaEvent_t ev[kNumStageEvents];
@@ -110,7 +113,7 @@ cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, i
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
                              cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
-cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream);
+cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
 cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);
 
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes

@@ -8,7 +8,9 @@
 // as Algorithm 2 prints it: accept while x_j equals the arg-max of the target row, emit the
 // arg-max of the first row that disagrees (or of the bonus row).
 //
-//   stats  : grid (vocabulary chunk of 8192, row) over all M target rows and S draft rows: one
+//   stats  : grid (vocabulary chunk of 8192, row) over all M target rows and S draft rows (in one
+//            launch, or the draft rows ahead of time on a second stream and the target rows
+//            after the LM head): one
 //            streaming read of both logit sets; per chunk the max and the sum of 2^((z-max)*c),
 //            c = log2(e)/T, in fp32 (online per thread, merged by shuffles, one block barrier).
 //            The last CTA to finish for a sequence (atomic ticket, nobody waits) merges the chunk
@@ -67,7 +69,7 @@ sample_stats_kernel(const SampleParams p)
     __shared__ int s_argmax[kMaxK + 1];
 
     const int chunk = blockIdx.x;
-    const int row = blockIdx.y;
+    const int row = blockIdx.y + p.row_begin;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool is_target = row < p.m_rows;
     int b;
@@ -255,11 +257,16 @@ sample_stats_kernel(const SampleParams p)
     }
 }
 
-cudaError_t launch_sample_stats(const SampleParams& p, cudaStream_t stream)
+// Rows [row_begin, row_begin + row_count) of the (target rows, then draft rows) list.  The launch may
+// be split (draft rows early on another stream, target rows once the logits exist): whichever CTA
+// arrives last for a sequence takes its decision.
+cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream)
 {
-    const int rows = p.greedy ? p.m_rows : p.m_rows + p.s_rows;
-    dim3 grid(p.n_chunks, rows);
-    sample_stats_kernel<<<grid, kSampleThreads, 0, stream>>>(p);
+    if (row_count <= 0) return cudaSuccess;
+    SampleParams q = p;
+    q.row_begin = row_begin;
+    dim3 grid(p.n_chunks, row_count);
+    sample_stats_kernel<<<grid, kSampleThreads, 0, stream>>>(q);
     return cudaGetLastError();
 }
 
