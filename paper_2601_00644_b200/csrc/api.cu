@@ -77,7 +77,7 @@ void free_workspace(Handle& h)
 {
     cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml); cudaFree(h.att_tickets);
     cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq);
-    cudaFree(h.stats); cudaFree(h.arg_idx); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.chunk_mass);
+    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.row_stats); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.chunk_mass);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
     for (int i = 0; i < kNumStageEvents; ++i)
@@ -166,7 +166,7 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     return FLEXSPEC_OK;
 }
 
-int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, cudaStream_t s)
+int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, const SampleParams* sp, cudaStream_t s)
 {
     const flexspec_config& c = h.cfg;
     LmHeadParams p;
@@ -180,6 +180,12 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, cudaStr
     p.n_vtiles = (c.vocab + 127) / 128;
     p.num_stages = lm_head_pick_stages(p.n_tile, p.n_blocks);
     p.acc_stages = (2 * rows_per_pass <= 512) ? 2 : 1;
+    p.tstats = nullptr; p.n_tparts = 0; p.inv_temp_log2 = 1.f; p.greedy = 0;
+    p.row_seq = nullptr; p.vocab_mask = nullptr; p.mask_words = 0;
+    if (sp != nullptr) {
+        p.tstats = h.tstats; p.n_tparts = 4 * p.n_vtiles; p.inv_temp_log2 = sp->inv_temp_log2; p.greedy = sp->greedy;
+        p.row_seq = sp->row_seq; p.vocab_mask = sp->vocab_mask; p.mask_words = sp->mask_words;
+    }
     p.status = h.status;
     CUtensorMap x_map;
     int rc = make_map_2d(&x_map, x, static_cast<uint64_t>(m_rows), static_cast<uint64_t>(h.d_model),
@@ -206,8 +212,9 @@ void fill_sample_params(Handle& h, SampleParams& p, const float* logits, const i
     p.n_dchunks = (c.vocab + kDrawChunk - 1) / kDrawChunk;
     p.mask_words = (c.vocab + 31) / 32;
     p.inv_temp_log2 = p.greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
-    p.stats = h.stats; p.arg_idx = h.arg_idx; p.counters = h.counters;
-    p.row_info = h.row_info; p.chunk_mass = h.chunk_mass;
+    p.stats = h.stats; p.counters = h.counters;
+    p.tstats = h.stats; p.n_tparts = p.n_chunks;          // target parts from the statistics kernel unless the LM head wrote them
+    p.row_info = h.row_info; p.row_stats = h.row_stats; p.chunk_mass = h.chunk_mass;
     p.accepted_len = accepted_len; p.next_token = next_token;
     if (c.flags & FLEXSPEC_FLAG_DEBUG) { p.dbg_p = h.dbg_p; p.dbg_q = h.dbg_q; p.dbg_u = h.dbg_u; }
     p.status = h.status;
@@ -223,6 +230,8 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
     fill_sample_params(h, p, logits, draft_tokens, draft_logits, draft_len, seeds, g, batch, temperature, vocab_mask,
                        accepted_len, next_token);
     if (launch_sample_stats(p, 0, p.greedy ? p.m_rows : p.m_rows + p.s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
+    if (launch_sample_decide(p, g.k_batch_max, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     if (!p.greedy) {
         if (launch_sample_draw(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
@@ -302,9 +311,10 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
     A(dev_alloc(&h.stats, static_cast<size_t>(max_m + h.max_s) * n_chunks));
-    A(dev_alloc(&h.arg_idx, static_cast<size_t>(max_m) * n_chunks));
+    A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128)));
     A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
     A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 4));
+    A(dev_alloc(&h.row_stats, static_cast<size_t>(c.max_batch) * (kMaxK + 1) * 4));
     A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * ((c.vocab + kDrawChunk - 1) / kDrawChunk) * 2));
     A(dev_alloc(&h.dbg_p, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.dbg_q, static_cast<size_t>(h.max_s)));
@@ -391,7 +401,7 @@ int flexspec_lm_head(flexspec_handle* fh, const void* x, int32_t m_rows, float* 
     if (x != nullptr && (reinterpret_cast<uintptr_t>(x) & 15u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
     DeviceGuard guard(h.cfg.device);
     h.launches = 0;
-    return run_lm_head(h, x ? x : h.attn_out, m_rows, logits ? logits : h.logits, static_cast<cudaStream_t>(stream));
+    return run_lm_head(h, x ? x : h.attn_out, m_rows, logits ? logits : h.logits, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* draft_tokens,
@@ -456,11 +466,14 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 2, s);
     mark(h, 3, s);
-    rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, s);
+    // the vocabulary mask needs the row -> sequence table of the plan kernel
+    if (sp.vocab_mask != nullptr && cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    sp.tstats = h.tstats; sp.n_tparts = 4 * ((h.cfg.vocab + 127) / 128);     // the LM head leaves the target rows' parts
+    rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);
     if (cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (launch_sample_stats(sp, 0, sp.m_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;   // the last CTA of a sequence decides
+    if (launch_sample_decide(sp, g.k_batch_max, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 5, s);
     if (!sp.greedy) {

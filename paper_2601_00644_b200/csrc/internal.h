@@ -54,6 +54,15 @@ struct LmHeadParams {
     int32_t n_vtiles;         // ceil(vocab / 128)
     int32_t num_stages;       // shared-memory pipeline depth
     int32_t acc_stages;       // TMEM accumulator buffers (1 or 2)
+    // optional: softmax statistics of the rows, one part per (row, 32 vocabulary rows), for the
+    // sampling stage (null = not wanted)
+    float2* tstats;           // [m_rows][n_tparts], n_tparts = 4 * n_vtiles
+    int32_t n_tparts;
+    float inv_temp_log2;      // log2(e) / T
+    int32_t greedy;           // parts are (max, arg-max index) instead of (max, sum exp)
+    const int32_t* row_seq;   // [m_rows] sequence of each row (for the vocabulary mask)
+    const uint32_t* vocab_mask;
+    int32_t mask_words;
     int32_t* status;
 };
 
@@ -71,9 +80,12 @@ struct SampleParams {
     int32_t row_begin;            // first row of this launch of the statistics kernel
     float inv_temp_log2;          // log2(e) / T
     int32_t greedy;
-    float2* stats;                // [(M+S)][n_chunks] (chunk max in logit units, sum exp)
-    int32_t* arg_idx;             // [M][n_chunks] lowest index of the chunk max (greedy)
-    int32_t* counters;            // [2][max_batch] self-resetting tickets
+    float2* stats;                // [(M+S)][n_chunks] parts written by the statistics kernel: (chunk max in logit
+                                  // units, sum exp), or (max, arg-max index as int bits) in greedy mode
+    const float2* tstats;         // parts of the target rows: [M][n_tparts] (from the LM head), or = stats
+    int32_t n_tparts;
+    int32_t* counters;            // [2][max_batch] self-resetting tickets (decision, draw)
+    double* row_stats;            // [B][kMaxK+1][4]: (max_p, sum_p, max_q, sum_q) of every row, or the arg-max in [0]
     double* row_info;             // [B][4]: max_p, 1/sum_p, max_q, 1/sum_q of row n
     double* chunk_mass;           // [B][n_dchunks][2]: residual mass, p mass
     int32_t* accepted_len;
@@ -93,7 +105,7 @@ struct Handle {
     float* logits;
     float* part_o; float* part_ml; int32_t* att_tickets; int32_t att_pairs_max;
     Plan plan;
-    float2* stats; int32_t* arg_idx; int32_t* counters; double* row_info; double* chunk_mass;
+    float2* stats; float2* tstats; int32_t* counters; double* row_stats; double* row_info; double* chunk_mass;
     double* dbg_p; double* dbg_q; float* dbg_u;
     int32_t* status;
     // host staging for flexspec_verify_host
@@ -114,6 +126,7 @@ cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const A
                              cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
+cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, cudaStream_t stream);
 cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);
 
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes

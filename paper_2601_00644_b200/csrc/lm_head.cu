@@ -13,6 +13,9 @@
 // handed over through mbarriers; every wait is bounded.
 //
 // W is streamed from HBM exactly once per pass; X (M x d bf16, L2 resident) is re-read per tile.
+// On request the epilogue also leaves the softmax statistics of every row (maximum and sum of
+// exponentials, or maximum and arg-max) per 32 vocabulary rows, so that the sampling stage does
+// not have to read the logits again to normalise them.
 #include "common.cuh"
 #include "internal.h"
 
@@ -166,6 +169,47 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                         if (row < p.m_rows)
                             p.logits[static_cast<int64_t>(row) * p.vocab + v] = __uint_as_float(r[i]);
                     }
+                }
+                if (p.tstats != nullptr) {
+                    // softmax statistics of this warp's 32 vocabulary rows for each of the 16 token
+                    // columns; the 16 reductions are interleaved so that their shuffle chains overlap.
+                    // Columns past m_rows hold zeros (out-of-range rows of X) and are not stored.
+                    float zv[16], mx[16], sc[16];
+                    uint32_t allow = 0xffffu;
+                    if (p.vocab_mask != nullptr && v < p.vocab) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int row = min(row_base + c0 + i, p.m_rows - 1);
+                            const uint32_t w = __ldg(p.vocab_mask + static_cast<int64_t>(__ldg(p.row_seq + row)) * p.mask_words + (v >> 5));
+                            if (((w >> (v & 31)) & 1u) == 0u) allow &= ~(1u << i);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) zv[i] = (v < p.vocab && ((allow >> i) & 1u)) ? __uint_as_float(r[i]) : -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) mx[i] = redux_max(zv[i]);
+                    if (p.greedy) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const unsigned eq = __ballot_sync(0xffffffffu, zv[i] == mx[i]);
+                            sc[i] = __int_as_float(vt * kLmBlockV + quarter * 32 + __ffs(eq) - 1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            sc[i] = fast_exp2((zv[i] - ((mx[i] == -INFINITY) ? 0.f : mx[i])) * p.inv_temp_log2);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) sc[i] += __shfl_xor_sync(0xffffffffu, sc[i], o);
+                    }
+                    float part_m = -INFINITY, part_s = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (lane == i) { part_m = mx[i]; part_s = sc[i]; }
+                    if (lane < 16 && row_base + c0 + lane < p.m_rows)
+                        p.tstats[static_cast<int64_t>(row_base + c0 + lane) * p.n_tparts + vt * 4 + quarter] =
+                            make_float2(part_m, part_s);
                 }
             }
             tc_fence_before();

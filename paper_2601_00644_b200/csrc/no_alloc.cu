@@ -24,9 +24,9 @@ constexpr size_t kOffCuQ = kOffCounters + align256(sizeof(int32_t) * 2 * kMaxBat
 constexpr size_t kOffCuD = kOffCuQ + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));
 constexpr size_t kOffRowSeq = kOffCuD + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));
 constexpr size_t kOffStats = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);
-constexpr size_t kOffArg = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
-constexpr size_t kOffRowInfo = kOffArg + align256(sizeof(int32_t) * kStaticMaxRows * kStaticChunks);
-constexpr size_t kOffMass = kOffRowInfo + align256(sizeof(double) * kStaticMaxBatch * 4);
+constexpr size_t kOffRowInfo = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
+constexpr size_t kOffRowStats = kOffRowInfo + align256(sizeof(double) * kStaticMaxBatch * 4);
+constexpr size_t kOffMass = kOffRowStats + align256(sizeof(double) * kStaticMaxBatch * (kMaxK + 1) * 4);
 constexpr size_t kScratchBytes = kOffMass + align256(sizeof(double) * kStaticMaxBatch * kStaticDrawChunks * 2);
 
 // In host code this name is only a handle for the runtime: the device address comes from
@@ -52,10 +52,11 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     if (batch < 1 || vocab < 1) return FLEXSPEC_ERR_INVALID_ARG;
     // sizes beyond what the fixed array was laid out for
     if (batch > kStaticMaxBatch || vocab > kStaticMaxVocab) return FLEXSPEC_ERR_UNSUPPORTED;
-    int32_t m_rows = 0, s_rows = 0;
+    int32_t m_rows = 0, s_rows = 0, k_batch_max = 0;
     for (int b = 0; b < batch; ++b) {
         const int k = draft_len_host[b];
         if (k < 0 || k > kMaxK) return FLEXSPEC_ERR_INVALID_ARG;
+        if (k > k_batch_max) k_batch_max = k;
         m_rows += k + 1;
         s_rows += k;
     }
@@ -105,13 +106,15 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     p.mask_words = (vocab + 31) / 32;
     p.inv_temp_log2 = greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     p.stats = reinterpret_cast<float2*>(base + kOffStats);
-    p.arg_idx = reinterpret_cast<int32_t*>(base + kOffArg);
+    p.tstats = p.stats; p.n_tparts = p.n_chunks;
     p.counters = reinterpret_cast<int32_t*>(base + kOffCounters);
     p.row_info = reinterpret_cast<double*>(base + kOffRowInfo);
+    p.row_stats = reinterpret_cast<double*>(base + kOffRowStats);
     p.chunk_mass = reinterpret_cast<double*>(base + kOffMass);
     p.accepted_len = accepted_len; p.next_token = next_token;
     p.status = status;
     if (launch_sample_stats(p, 0, greedy ? m_rows : m_rows + s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_decide(p, k_batch_max, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     if (!greedy && launch_sample_draw(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     return FLEXSPEC_OK;
 }

@@ -8,14 +8,13 @@
 // as Algorithm 2 prints it: accept while x_j equals the arg-max of the target row, emit the
 // arg-max of the first row that disagrees (or of the bonus row).
 //
-//   stats  : grid (vocabulary chunk of 8192, row) over all M target rows and S draft rows (in one
-//            launch, or the draft rows ahead of time on a second stream and the target rows
-//            after the LM head): one
-//            streaming read of both logit sets; per chunk the max and the sum of 2^((z-max)*c),
-//            c = log2(e)/T, in fp32 (online per thread, merged by shuffles, one block barrier).
-//            The last CTA to finish for a sequence (atomic ticket, nobody waits) merges the chunk
-//            statistics in fp64, evaluates the acceptance tests with Philox uniforms, finds the
-//            first rejection by warp vote and stores accepted_len.
+//   stats  : grid (vocabulary chunk of 8192, row): one streaming read of the logits; per chunk the
+//            max and the sum of 2^((z-max)*c), c = log2(e)/T, in fp32 (online per thread, merged
+//            by shuffles, one block barrier).  Serves the draft rows (ahead of time, on a second
+//            stream) and, for the stand-alone stage, the target rows; inside flexspec_verify the
+//            LM-head kernel writes the target rows' parts from its epilogue.
+//   decide : one CTA per sequence merges the parts of its rows, evaluates the acceptance tests
+//            with Philox uniforms, finds the first rejection by warp vote, stores accepted_len.
 //   draw   : grid (chunk of 2048, sequence) over row n of each sequence only: probability mass of
 //            the residual (and of p) per chunk, fp32 exponentials accumulated in fp64; the last
 //            CTA of a sequence picks the chunk that holds u' * Z and scans it in vocabulary order
@@ -44,50 +43,29 @@ __device__ __forceinline__ void merge_ms(float& m, float& s, float m2, float s2,
     m = mm;
 }
 
-// Merge of per-chunk statistics in chunk order, fp64.
-__device__ __forceinline__ void merge_row_stats(const float2* st, int n_chunks, double scale, double& mx, double& sum)
-{
-    double m = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) m = fmax(m, static_cast<double>(st[c].x));
-    double s = 0.0;
-    for (int c = 0; c < n_chunks; ++c) {
-        const double mc = static_cast<double>(st[c].x);
-        if (mc != -INFINITY) s += static_cast<double>(st[c].y) * exp2((mc - m) * scale);
-    }
-    mx = m;
-    sum = s;
-}
-
-// ------------------------------------------------------------------------------------ stats + decision
-// Rows [0, M) are target rows, rows [M, M+S) draft rows.
+// ------------------------------------------------------------------------------------ statistics
+// One part per (row, vocabulary chunk): SAMPLE (max, sum of 2^((z - max) * c)); GREEDY (max, lowest
+// index holding it, as int bits).  Rows [0, M) are target rows, rows [M, M+S) draft rows.  The
+// LM-head kernel can write the target rows' parts itself (one part per 32 vocabulary rows); this
+// kernel serves the draft rows and, for the stand-alone sampling stage, the target rows too.
 __global__ void __launch_bounds__(kSampleThreads)
 sample_stats_kernel(const SampleParams p)
 {
     __shared__ float red_m[kSampleWarps];
     __shared__ float red_s[kSampleWarps];
     __shared__ int red_i[kSampleWarps];
-    __shared__ int s_argmax[kMaxK + 1];
 
     const int chunk = blockIdx.x;
     const int row = blockIdx.y + p.row_begin;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool is_target = row < p.m_rows;
-    int b;
     const float* src;
     const uint32_t* mask_row = nullptr;
     if (is_target) {
-        b = p.row_seq[row];
         src = p.logits + static_cast<int64_t>(row) * p.vocab;
-        if (p.vocab_mask != nullptr) mask_row = p.vocab_mask + static_cast<int64_t>(b) * p.mask_words;
+        if (p.vocab_mask != nullptr) mask_row = p.vocab_mask + static_cast<int64_t>(p.row_seq[row]) * p.mask_words;
     } else {
-        const int dr = row - p.m_rows;
-        int lo = 0, hi = p.batch - 1;                     // largest b with cu_d[b] <= dr: owns draft row dr
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (p.cu_d[mid] <= dr) lo = mid; else hi = mid - 1;
-        }
-        b = lo;
-        src = p.draft_logits + static_cast<int64_t>(dr) * p.vocab;
+        src = p.draft_logits + static_cast<int64_t>(row - p.m_rows) * p.vocab;
     }
 
     const int v0 = chunk * kSampleChunk;
@@ -120,6 +98,7 @@ sample_stats_kernel(const SampleParams p)
 #pragma unroll
     for (int i = 0; i < kElemsPerThread; ++i) mx = fmaxf(mx, z[i]);
     const float c = p.inv_temp_log2;
+    float2* out = p.stats + static_cast<int64_t>(row) * p.n_chunks + chunk;
 
     if (p.greedy) {
         // (max, lowest index holding it)
@@ -136,6 +115,17 @@ sample_stats_kernel(const SampleParams p)
             if (m2 > mx || (m2 == mx && i2 < best)) { mx = m2; best = i2; }
         }
         if (lane == 0) { red_m[warp] = mx; red_i[warp] = best; }
+        __syncthreads();
+        if (warp != 0) return;
+        float m = (lane < kSampleWarps) ? red_m[lane] : -INFINITY;
+        int bi = (lane < kSampleWarps) ? red_i[lane] : 0x7fffffff;
+#pragma unroll
+        for (int o = kSampleWarps / 2; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+            const int i2 = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (m2 > m || (m2 == m && i2 < bi)) { m = m2; bi = i2; }
+        }
+        if (lane == 0) *out = make_float2(m, __int_as_float(bi));
     } else {
         const float base = (mx == -INFINITY) ? 0.f : mx;
         float se = 0.f;
@@ -148,118 +138,21 @@ sample_stats_kernel(const SampleParams p)
             merge_ms(mx, se, m2, s2, c);
         }
         if (lane == 0) { red_m[warp] = mx; red_s[warp] = se; }
-    }
-    __syncthreads();
-    if (warp != 0) return;
-
-    // ---- warp 0: merge the 8 warps, publish, take a ticket
-    {
+        __syncthreads();
+        if (warp != 0) return;
         float m = (lane < kSampleWarps) ? red_m[lane] : -INFINITY;
-        if (p.greedy) {
-            int bi = (lane < kSampleWarps) ? red_i[lane] : 0x7fffffff;
+        float sm = (lane < kSampleWarps) ? red_s[lane] : 0.f;
 #pragma unroll
-            for (int o = kSampleWarps / 2; o > 0; o >>= 1) {
-                const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-                const int i2 = __shfl_xor_sync(0xffffffffu, bi, o);
-                if (m2 > m || (m2 == m && i2 < bi)) { m = m2; bi = i2; }
-            }
-            if (lane == 0 && is_target) {
-                p.stats[static_cast<int64_t>(row) * p.n_chunks + chunk] = make_float2(m, 0.f);
-                p.arg_idx[static_cast<int64_t>(row) * p.n_chunks + chunk] = bi;
-            }
-        } else {
-            float s = (lane < kSampleWarps) ? red_s[lane] : 0.f;
-#pragma unroll
-            for (int o = kSampleWarps / 2; o > 0; o >>= 1) {
-                const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-                const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
-                merge_ms(m, s, m2, s2, c);
-            }
-            if (lane == 0) p.stats[static_cast<int64_t>(row) * p.n_chunks + chunk] = make_float2(m, s);
+        for (int o = kSampleWarps / 2; o > 0; o >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+            const float s2 = __shfl_xor_sync(0xffffffffu, sm, o);
+            merge_ms(m, sm, m2, s2, c);
         }
-    }
-    const int k_b = p.draft_len[b];
-    int is_last = 0;
-    if (lane == 0) {
-        const int expected = (p.greedy ? (k_b + 1) : (2 * k_b + 1)) * p.n_chunks;
-        __threadfence();
-        const int t = atomicAdd(&p.counters[b], 1);
-        is_last = (t == expected - 1);
-        if (is_last) { p.counters[b] = 0; __threadfence(); }      // ready for the next call
-    }
-    is_last = __shfl_sync(0xffffffffu, is_last, 0);
-    if (!is_last) return;
-    __threadfence();
-
-    // ---- the last CTA of sequence b takes the decision
-    const int q0 = p.cu_q[b], d0 = p.cu_d[b];
-    const double scale = static_cast<double>(p.inv_temp_log2);
-    int n = k_b;
-    if (p.greedy) {
-        for (int j = lane; j <= k_b; j += 32) {
-            const float2* st = p.stats + static_cast<int64_t>(q0 + j) * p.n_chunks;
-            const int32_t* ai = p.arg_idx + static_cast<int64_t>(q0 + j) * p.n_chunks;
-            float bm = -INFINITY;
-            int best = 0;
-            for (int cc = 0; cc < p.n_chunks; ++cc)
-                if (cc == 0 || st[cc].x > bm) { bm = st[cc].x; best = ai[cc]; }     // strict: lowest index wins
-            s_argmax[j] = best;
-        }
-        __syncwarp();
-        for (int base = 0; base < k_b; base += 32) {
-            const int j = base + lane;
-            const bool rej = (j < k_b) && (p.draft_tokens[d0 + j] != s_argmax[j]);
-            const unsigned vote = __ballot_sync(0xffffffffu, rej);
-            if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
-        }
-        if (lane == 0) {
-            p.accepted_len[b] = n;
-            p.next_token[b] = s_argmax[n];
-        }
-        return;
-    }
-
-    const uint64_t seed = p.seeds[b];
-    for (int base = 0; base < k_b; base += 32) {
-        const int j = base + lane;
-        bool rej = false;
-        if (j < k_b) {
-            double mp, sp, mq, sq;
-            merge_row_stats(p.stats + static_cast<int64_t>(q0 + j) * p.n_chunks, p.n_chunks, scale, mp, sp);
-            merge_row_stats(p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks, p.n_chunks, scale, mq, sq);
-            int x = p.draft_tokens[d0 + j];
-            x = min(max(x, 0), p.vocab - 1);
-            double zp = static_cast<double>(p.logits[static_cast<int64_t>(q0 + j) * p.vocab + x]);
-            if (p.vocab_mask != nullptr &&
-                !mask_allows(p.vocab_mask + static_cast<int64_t>(b) * p.mask_words, x)) zp = -INFINITY;
-            const double zq = static_cast<double>(p.draft_logits[static_cast<int64_t>(d0 + j) * p.vocab + x]);
-            const double pt = (zp == -INFINITY) ? 0.0 : exp2((zp - mp) * scale) / sp;
-            const double qt = (zq == -INFINITY) ? 0.0 : exp2((zq - mq) * scale) / sq;
-            const double u = philox_uniform(seed, static_cast<uint32_t>(j), 0u);
-            rej = !(u * qt < pt);
-            if (p.dbg_p != nullptr) {
-                p.dbg_p[d0 + j] = pt;
-                p.dbg_q[d0 + j] = qt;
-                p.dbg_u[d0 + j] = static_cast<float>(u);
-            }
-        }
-        const unsigned vote = __ballot_sync(0xffffffffu, rej);
-        if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
-    }
-    if (lane == 0) {
-        p.accepted_len[b] = n;
-        double mp, sp, mq = 0.0, sq = 1.0;
-        merge_row_stats(p.stats + static_cast<int64_t>(q0 + n) * p.n_chunks, p.n_chunks, scale, mp, sp);
-        if (n < k_b)
-            merge_row_stats(p.stats + static_cast<int64_t>(p.m_rows + d0 + n) * p.n_chunks, p.n_chunks, scale, mq, sq);
-        double* ri = p.row_info + static_cast<int64_t>(b) * 4;
-        ri[0] = mp; ri[1] = 1.0 / sp; ri[2] = mq; ri[3] = 1.0 / sq;
+        if (lane == 0) *out = make_float2(m, sm);
     }
 }
 
-// Rows [row_begin, row_begin + row_count) of the (target rows, then draft rows) list.  The launch may
-// be split (draft rows early on another stream, target rows once the logits exist): whichever CTA
-// arrives last for a sequence takes its decision.
+// Rows [row_begin, row_begin + row_count) of the (target rows, then draft rows) list.
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream)
 {
     if (row_count <= 0) return cudaSuccess;
@@ -267,6 +160,175 @@ cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_
     q.row_begin = row_begin;
     dim3 grid(p.n_chunks, row_count);
     sample_stats_kernel<<<grid, kSampleThreads, 0, stream>>>(q);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------ decision
+// grid (row j, sequence b): the CTA merges the parts of target row j (and draft row j) of the
+// sequence -- maximum first, then the sum with fp32 weights accumulated in fp64 -- and leaves
+// (max, sum) per row.  The CTA that arrives last for the sequence (atomic ticket, nobody waits)
+// evaluates the acceptance tests with Philox uniforms, finds the first rejection by warp vote and
+// stores accepted_len; GREEDY compares the draft with the rows' arg-max.
+__device__ __forceinline__ float block_max(float v, float* red, int lane, int warp)
+{
+    v = warp_max(v);
+    __syncthreads();                                   // red may still be read from a previous use
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float r = red[0];
+#pragma unroll
+    for (int w = 1; w < kSampleWarps; ++w) r = fmaxf(r, red[w]);
+    return r;
+}
+__device__ __forceinline__ double block_sum(double v, double* red, int lane, int warp)
+{
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double r = 0.0;
+#pragma unroll
+    for (int w = 0; w < kSampleWarps; ++w) r += red[w];
+    return r;
+}
+
+__global__ void __launch_bounds__(kSampleThreads)
+sample_decide_kernel(const SampleParams p)
+{
+    __shared__ float red_f[kSampleWarps];
+    __shared__ double red_d[kSampleWarps];
+    __shared__ int red_i[kSampleWarps];
+    __shared__ int s_last;
+    const int j = blockIdx.x;
+    const int b = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k_b = p.draft_len[b];
+    if (j > k_b) return;
+    const int q0 = p.cu_q[b], d0 = p.cu_d[b];
+    const double scale = static_cast<double>(p.inv_temp_log2);
+    const float cf = p.inv_temp_log2;
+    double* rs = p.row_stats + (static_cast<int64_t>(b) * (kMaxK + 1) + j) * 4;
+
+    // ---- target row j
+    {
+        const float2* tp = p.tstats + static_cast<int64_t>(q0 + j) * p.n_tparts;
+        const int n = p.n_tparts;
+        if (p.greedy) {
+            float m = -INFINITY;
+            int best = 0x7fffffff;
+#pragma unroll 8
+            for (int i = threadIdx.x; i < n; i += kSampleThreads) {
+                const float2 pt = __ldcg(&tp[i]);
+                const int idx = __float_as_int(pt.y);
+                if (pt.x > m || (pt.x == m && idx < best)) { m = pt.x; best = idx; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+                const int i2 = __shfl_xor_sync(0xffffffffu, best, o);
+                if (m2 > m || (m2 == m && i2 < best)) { m = m2; best = i2; }
+            }
+            if (lane == 0) { red_f[warp] = m; red_i[warp] = best; }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (int w = 1; w < kSampleWarps; ++w)
+                    if (red_f[w] > m || (red_f[w] == m && red_i[w] < best)) { m = red_f[w]; best = red_i[w]; }
+                rs[0] = static_cast<double>(best);
+            }
+        } else {
+            float m = -INFINITY;
+#pragma unroll 8
+            for (int i = threadIdx.x; i < n; i += kSampleThreads) m = fmaxf(m, __ldcg(&tp[i].x));
+            m = block_max(m, red_f, lane, warp);
+            double sm = 0.0;
+#pragma unroll 8
+            for (int i = threadIdx.x; i < n; i += kSampleThreads) {
+                const float2 pt = __ldcg(&tp[i]);
+                if (pt.x != -INFINITY) sm += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - m) * cf));
+            }
+            sm = block_sum(sm, red_d, lane, warp);
+            if (threadIdx.x == 0) { rs[0] = static_cast<double>(m); rs[1] = sm; }
+            // ---- draft row j: few parts, one warp
+            if (j < k_b && warp == 1) {
+                const float2* dp = p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks;
+                float mq = -INFINITY;
+                for (int i = lane; i < p.n_chunks; i += 32) mq = fmaxf(mq, __ldcg(&dp[i].x));
+                mq = warp_max(mq);
+                double sq = 0.0;
+                for (int i = lane; i < p.n_chunks; i += 32) {
+                    const float2 pt = __ldcg(&dp[i]);
+                    if (pt.x != -INFINITY) sq += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - mq) * cf));
+                }
+                sq = warp_sum(sq);
+                if (lane == 0) { rs[2] = static_cast<double>(mq); rs[3] = sq; }
+            }
+        }
+    }
+    // ---- ticket: the last row of the sequence decides
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int tk = atomicAdd(&p.counters[b], 1);
+        s_last = (tk == k_b);
+        if (s_last) { p.counters[b] = 0; __threadfence(); }          // ready for the next call
+    }
+    __syncthreads();
+    if (!s_last || warp != 0) return;
+    __threadfence();
+
+    const double* rs0 = p.row_stats + static_cast<int64_t>(b) * (kMaxK + 1) * 4;
+    int n = k_b;
+    if (p.greedy) {
+        for (int base = 0; base < k_b; base += 32) {
+            const int jj = base + lane;
+            const bool rej = (jj < k_b) && (p.draft_tokens[d0 + jj] != static_cast<int>(__ldcg(rs0 + jj * 4)));
+            const unsigned vote = __ballot_sync(0xffffffffu, rej);
+            if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
+        }
+        if (lane == 0) {
+            p.accepted_len[b] = n;
+            p.next_token[b] = static_cast<int>(__ldcg(rs0 + n * 4));
+        }
+        return;
+    }
+    const uint64_t seed = p.seeds[b];
+    for (int base = 0; base < k_b; base += 32) {
+        const int jj = base + lane;
+        bool rej = false;
+        if (jj < k_b) {
+            const double mp = __ldcg(rs0 + jj * 4), sp = __ldcg(rs0 + jj * 4 + 1);
+            const double mq = __ldcg(rs0 + jj * 4 + 2), sq = __ldcg(rs0 + jj * 4 + 3);
+            int x = p.draft_tokens[d0 + jj];
+            x = min(max(x, 0), p.vocab - 1);
+            double zp = static_cast<double>(p.logits[static_cast<int64_t>(q0 + jj) * p.vocab + x]);
+            if (p.vocab_mask != nullptr &&
+                !mask_allows(p.vocab_mask + static_cast<int64_t>(b) * p.mask_words, x)) zp = -INFINITY;
+            const double zq = static_cast<double>(p.draft_logits[static_cast<int64_t>(d0 + jj) * p.vocab + x]);
+            const double pt = (zp == -INFINITY) ? 0.0 : exp2((zp - mp) * scale) / sp;
+            const double qt = (zq == -INFINITY) ? 0.0 : exp2((zq - mq) * scale) / sq;
+            const double u = philox_uniform(seed, static_cast<uint32_t>(jj), 0u);
+            rej = !(u * qt < pt);
+            if (p.dbg_p != nullptr) {
+                p.dbg_p[d0 + jj] = pt;
+                p.dbg_q[d0 + jj] = qt;
+                p.dbg_u[d0 + jj] = static_cast<float>(u);
+            }
+        }
+        const unsigned vote = __ballot_sync(0xffffffffu, rej);
+        if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
+    }
+    if (lane == 0) {
+        p.accepted_len[b] = n;
+        double* ri = p.row_info + static_cast<int64_t>(b) * 4;
+        ri[0] = __ldcg(rs0 + n * 4); ri[1] = 1.0 / __ldcg(rs0 + n * 4 + 1);
+        ri[2] = (n < k_b) ? __ldcg(rs0 + n * 4 + 2) : 0.0; ri[3] = (n < k_b) ? 1.0 / __ldcg(rs0 + n * 4 + 3) : 1.0;
+    }
+}
+
+cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, cudaStream_t stream)
+{
+    dim3 grid(k_batch_max + 1, p.batch);
+    sample_decide_kernel<<<grid, kSampleThreads, 0, stream>>>(p);
     return cudaGetLastError();
 }
 
