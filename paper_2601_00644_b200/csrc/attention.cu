@@ -22,9 +22,10 @@
 //                                       B = P^T written by the softmax threads ([token][row]:
 //                                       MN-major, unswizzled 8x8 core matrices)
 //
-// Warp roles.  Warp 0: TMA producer (one 16-token K and V page per lane, separate rings of
-// 128-token K and V tiles; the page ids of the next block are fetched one block ahead).  Warp 1:
-// one thread issues every tcgen05.mma; the warp owns the TMEM allocation.  Warps 2..5: softmax,
+// Warp roles.  Warps 0-1: TMA producers, each owning half of every block's pages (a TMA request
+// costs about 55 cycles of the issuing warp, and a block needs 32 of them); separate rings of
+// 128-token K and V tiles; an L2 prefetch of the pages runs several blocks ahead of the copies.
+// Warp 2: one thread issues every tcgen05.mma; the warp owns the TMEM allocation.  Warps 3-6: softmax,
 // thread t = token t of the block (TMEM lane t of S^T).  The maximum of a query row over the
 // block is a column maximum: redux.sync.max over each warp, then over the four warps through
 // shared memory.  The running maximum is only raised when it grew by more than 2^8 (O^T in TMEM
@@ -46,7 +47,8 @@ constexpr int kAttTmemCols = 512;
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column offsets
 constexpr float kRescaleThreshold = 8.f;                             // log2 units
 constexpr int kAttSmemLimit = 232448;                                // 227 KB opt-in maximum per CTA
-constexpr int kAttStaticReserve = 512;                               // __shared__ variables of the kernel
+constexpr int kAttStaticReserve = 1024;                              // __shared__ variables of the kernel
+constexpr int kAttPrefetchBlocks = 6;                                // how far ahead of the copies the L2 prefetch runs
 
 struct AttBars {
     uint64_t k_full[kAttMaxStages], k_empty[kAttMaxStages];
@@ -578,7 +580,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
     }
 }
 
-template <int DH>
+template <int DH, int NCH>
 __global__ void __launch_bounds__(kAttThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
 {
@@ -596,6 +598,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
     AttBars* bars = sm.bars;
     __shared__ int s_warp_tot[32];
     __shared__ AttStart s_start;
+    __shared__ int s_phys[kAttProducerWarps][8][2 * kAttPagesPerStage / kAttProducerWarps];   // per producer warp: page ids
+                                                        // of the blocks between its prefetch cursor and its copies, by lane
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -614,7 +618,7 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         fence_barrier_init();
         tma_prefetch_desc(&kv_map);
     }
-    if (warp == 1) {
+    if (warp == kAttProducerWarps) {
         tmem_alloc(&bars->tmem_slot, kAttTmemCols);
         tmem_relinquish();
     }
@@ -672,16 +676,66 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         cur.blk = s_start.blk_off % cur.nb;
     }
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+    if (warp < kAttProducerWarps) {
+        // ------------------------------------------------------------------ TMA producers
+        // Producer warp w owns pages [w*PW, (w+1)*PW) of every block; lane l < 2*PW issues the K and the
+        // V copy of (page l / 2, 64-column half l % 2).
+        constexpr int PW = kAttPagesPerStage / kAttProducerWarps;          // pages per producer warp
         const uint64_t pol = l2_policy_evict_first();
+        const int my_page = warp * PW + (lane >> 1);                       // page of the block this lane copies
+        const int my_half = lane & 1;
+        const bool copy_lane = lane < 2 * PW && my_half < Cfg::kSlabs;
+        int (*ring)[2 * PW] = s_phys[warp];
         bool new_pair = true;
         bool ok = true;
-        int phys_next = 0;
-        bool have_next = false;
+        // A second cursor runs kAttPrefetchBlocks ahead of the copies.  It looks the page ids up (one
+        // page-table read per block, kept in a small shared-memory ring until the copy needs them;
+        // the read for the next block is always in flight while this block is handled) and asks for
+        // the pages to be brought into L2: a tile's shared-memory slot is then busy for an L2 hit,
+        // not for a trip to HBM, so the rings that fit in shared memory keep HBM streaming.
+        AttCursor pf = cur;
+        int pf_q = 0;
+        auto pf_load = [&](const AttCursor& c) -> int {
+            const int pt_begin = c.blk * kAttBlockTokens;
+            const int pnpg = (min(c.kvl, pt_begin + kAttBlockTokens) - pt_begin + kPageTokens - 1) / kPageTokens;
+            return (lane < 2 * PW && my_page < pnpg)
+                       ? p.page_table[static_cast<int64_t>(c.b) * p.max_pages_per_seq + c.blk * kAttPagesPerStage + my_page] : -1;
+        };
+        const int lines_per_tile_page = kPageTokens * DH * 2 / 128;        // 128-byte lines of one page's K (or V), one kv head
+        auto pf_issue = [&](int ph) {
+            if (lane < 2 * PW) ring[pf_q & 7][lane] = ph;
+            const int pkvh = pf.pair / pf.rbc;
+            // plain per-line prefetches from all lanes: the TMA path is kept for the copies
+#pragma unroll
+            for (int pg = 0; pg < PW; ++pg) {
+                const int id = __shfl_sync(0xffffffffu, ph, 2 * pg);
+                if (id >= 0 && id < p.num_pages && lane < lines_per_tile_page) {
+                    const uint8_t* kb = p.kv_pages + (static_cast<int64_t>(id * 2 + 0) * p.n_kv_heads + pkvh) * (kPageTokens * DH * 2);
+                    const uint8_t* vb = p.kv_pages + (static_cast<int64_t>(id * 2 + 1) * p.n_kv_heads + pkvh) * (kPageTokens * DH * 2);
+                    prefetch_l2(kb + lane * 128);
+                    prefetch_l2(vb + lane * 128);
+                }
+            }
+            ++pf_q;
+            pf.advance(p, pf_q < n_my);
+        };
+        {
+            // the first blocks: all page-table reads first, then the prefetches
+            int ph0[kAttPrefetchBlocks];
+            AttCursor tmp = pf;
+#pragma unroll
+            for (int i = 0; i < kAttPrefetchBlocks; ++i) {
+                ph0[i] = -1;
+                if (i < n_my) { ph0[i] = pf_load(tmp); tmp.advance(p, i + 1 < n_my); }
+            }
+#pragma unroll
+            for (int i = 0; i < kAttPrefetchBlocks; ++i)
+                if (i < n_my) pf_issue(ph0[i]);
+        }
+        int pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
         for (int q = 0; q < n_my && ok; ++q) {
             const int kvh = cur.pair / cur.rbc;
-            if (new_pair) {
+            if (new_pair && warp == 0) {
                 // bring the pair's query rows into L2 ahead of the softmax threads that copy them
                 const int row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
                 const int rows_here = min(kAttRowsPerPair, p.group * (cur.k + 1) - row_lo);
@@ -699,47 +753,32 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             const int t_begin = cur.blk * kAttBlockTokens;
             const int t_end = min(cur.kvl, t_begin + kAttBlockTokens);
             const int npg = (t_end - t_begin + kPageTokens - 1) / kPageTokens;
-            int phys = phys_next;
-            if (!have_next && lane < npg)
-                phys = p.page_table[static_cast<int64_t>(cur.b) * p.max_pages_per_seq + cur.blk * kAttPagesPerStage + lane];
-            if (lane < npg && (phys < 0 || phys >= p.num_pages)) {
+            const bool active = copy_lane && my_page < npg;
+            int phys = (lane < 2 * PW) ? ring[q & 7][lane] : -1;
+            if (active && (phys < 0 || phys >= p.num_pages)) {
                 report_error(p.status, kErrBadPage, phys, 1);
                 phys = 0;                                   // stay inside the pool
             }
             const uint32_t tile_tx = static_cast<uint32_t>(npg * Cfg::kSlabs * kPageTokens * 128);
+            const int smem_off = my_half * Cfg::kSlabBytes + my_page * (kPageTokens * 128);
             // K tile
             if (k_use > 0 && !mbar_wait(&bars->k_empty[ks], (k_use - 1) & 1, p.status, 1)) { ok = false; break; }
-            if (lane == 0) mbar_arrive_expect_tx(&bars->k_full[ks], tile_tx);
-            __syncwarp();
-            if (lane < npg) {
-                uint8_t* dst = sm.k_ring + ks * Cfg::kTileBytes + lane * (kPageTokens * 128);
-                const int row_k = ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens;
-#pragma unroll
-                for (int hf = 0; hf < Cfg::kSlabs; ++hf)
-                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &bars->k_full[ks], hf * 64, row_k, pol);
-            }
+            if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&bars->k_full[ks], tile_tx);
+            if (active)
+                tma_load_2d(sm.k_ring + ks * Cfg::kTileBytes + smem_off, &kv_map, &bars->k_full[ks], my_half * 64,
+                            ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens, pol);
             // V tile
             if (v_use > 0 && !mbar_wait(&bars->v_empty[vs], (v_use - 1) & 1, p.status, 20)) { ok = false; break; }
-            if (lane == 0) mbar_arrive_expect_tx(&bars->v_full[vs], tile_tx);
+            if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&bars->v_full[vs], tile_tx);
+            if (active)
+                tma_load_2d(sm.v_ring + vs * Cfg::kTileBytes + smem_off, &kv_map, &bars->v_full[vs], my_half * 64,
+                            ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens, pol);
             __syncwarp();
-            if (lane < npg) {
-                uint8_t* dst = sm.v_ring + vs * Cfg::kTileBytes + lane * (kPageTokens * 128);
-                const int row_v = ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens;
-#pragma unroll
-                for (int hf = 0; hf < Cfg::kSlabs; ++hf)
-                    tma_load_2d(dst + hf * Cfg::kSlabBytes, &kv_map, &bars->v_full[vs], hf * 64, row_v, pol);
+            if (pf_q < n_my) {
+                pf_issue(pf_ph);
+                pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
             }
-            __syncwarp();
             new_pair = cur.advance(p, q + 1 < n_my);
-            // page ids of the next block, fetched while this block's copies are in flight
-            have_next = false;
-            if (q + 1 < n_my) {
-                const int nt_begin = cur.blk * kAttBlockTokens;
-                const int n_npg = (min(cur.kvl, nt_begin + kAttBlockTokens) - nt_begin + kPageTokens - 1) / kPageTokens;
-                if (lane < n_npg)
-                    phys_next = p.page_table[static_cast<int64_t>(cur.b) * p.max_pages_per_seq + cur.blk * kAttPagesPerStage + lane];
-                have_next = true;
-            }
         }
         // do not leave while a copy of ours may still be landing in shared memory
         if (ok && n_my > 0) {
@@ -747,104 +786,127 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             mbar_wait(&bars->k_full[ql % p.k_stages], (ql / p.k_stages) & 1, p.status, 9);
             mbar_wait(&bars->v_full[ql % p.v_stages], (ql / p.v_stages) & 1, p.status, 9);
         }
-    } else if (warp == 1) {
+    } else if (warp == kAttProducerWarps) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_my > 0) {
+            // This one thread is on the critical path of every block, so its work per block is kept
+            // to a few dozen instructions: descriptors are built once and only advanced by adding
+            // (byte offset >> 4) to their address field, ring positions are carried, not divided.
             const uint32_t idesc_s = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad));
             const uint32_t idesc_o = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad)) | kIdescAMajorMN | kIdescBMajorMN;
-            const uint32_t q_addr = smem_u32(sm.q);
-            const uint32_t q_slab = static_cast<uint32_t>(n_pad) * 128u;
+            const uint64_t dq0 = umma_desc_k_sw128(smem_u32(sm.q));
+            const uint64_t dk0 = umma_desc_k_sw128(smem_u32(sm.k_ring));
+            const uint64_t dv0 = umma_desc_mn_sw128(smem_u32(sm.v_ring), Cfg::kSlabBytes, 1024);
+            const uint64_t dp0 = umma_desc_mn_plain(smem_u32(sm.pt), 2048, 128);
+            const uint32_t q_slab16 = (static_cast<uint32_t>(n_pad) * 128u) >> 4;
+            const uint32_t p_buf16 = static_cast<uint32_t>(Cfg::p_bytes(n_pad)) >> 4;
             bool ok = true;
-            int seg = 0;
-            // S^T[q & 1] = K Q^T of block q (waits: the pair's Q tile, the K tile, the S^T buffer)
-            auto issue_s = [&](int q, bool seg_first, int seg_idx) -> bool {
-                const int ks = q % p.k_stages, buf = q & 1, u = q >> 1;
-                if (seg_first && !mbar_wait(&bars->q_full, seg_idx & 1, p.status, 2)) return false;
-                if (!mbar_wait(&bars->k_full[ks], (q / p.k_stages) & 1, p.status, 3)) return false;
-                if (u > 0 && !mbar_wait(&bars->s_empty[buf], (u - 1) & 1, p.status, 4)) return false;
+            // state of the S^T issue stream (runs one block ahead inside a segment)
+            int s_ks = 0; uint32_t s_kpar = 0;             // K ring slot / parity of its full barrier
+            int s_buf = 0; uint32_t s_spar = 1;            // S^T buffer; parity to wait for on s_empty (previous use)
+            int s_q = 0, s_seg = 0;
+            // S^T[buf] = K Q^T of the next block in order (waits: the pair's Q tile, the K tile, the S^T buffer)
+            auto issue_s = [&](bool seg_first) -> bool {
+                if (seg_first && !mbar_wait(&bars->q_full, s_seg & 1, p.status, 2)) return false;
+                if (!mbar_wait(&bars->k_full[s_ks], s_kpar, p.status, 3)) return false;
+                if (s_q >= 2 && !mbar_wait(&bars->s_empty[s_buf], s_spar, p.status, 4)) return false;
                 tc_fence_after();
-                const uint32_t k_addr = smem_u32(sm.k_ring + ks * Cfg::kTileBytes);
-                const uint32_t acc = tmem_base + (buf ? kTmemS1 : kTmemS0);
+                const uint64_t dk = dk0 + static_cast<uint32_t>((s_ks * Cfg::kTileBytes) >> 4);
+                const uint32_t acc = tmem_base + (s_buf ? kTmemS1 : kTmemS0);
 #pragma unroll
-                for (int kk = 0; kk < DH / 16; ++kk) {
-                    const uint64_t da = umma_desc_k_sw128(k_addr + (kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32);
-                    const uint64_t db = umma_desc_k_sw128(q_addr + (kk >> 2) * q_slab + (kk & 3) * 32);
-                    umma_bf16(acc, da, db, idesc_s, kk > 0 ? 1u : 0u);
-                }
-                umma_commit(&bars->s_full[buf]);
-                umma_commit(&bars->k_empty[ks]);
+                for (int kk = 0; kk < DH / 16; ++kk)
+                    umma_bf16(acc, dk + static_cast<uint32_t>(((kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32) >> 4),
+                              dq0 + ((kk >> 2) * q_slab16 + (kk & 3) * 2), idesc_s, kk > 0 ? 1u : 0u);
+                umma_commit(&bars->s_full[s_buf]);
+                umma_commit(&bars->k_empty[s_ks]);
+                if (++s_ks == p.k_stages) { s_ks = 0; s_kpar ^= 1u; }
+                if (s_buf == 1) s_spar ^= 1u;              // both buffers used once more: next round waits the other parity
+                s_buf ^= 1;
+                ++s_q;
                 return true;
             };
+            int vs = 0; uint32_t vpar = 0;                 // V ring slot / parity
+            int pb = 0; uint32_t ppar = 0;                 // P^T buffer / parity of p_full
             bool seg_first = true;
-            ok = issue_s(0, true, 0);
+            ok = issue_s(true);
             for (int q = 0; q < n_my && ok; ++q) {
                 const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
-                const int vs = q % p.v_stages;
-                if (!seg_last && q + 1 < n_my) { if (!issue_s(q + 1, false, seg)) { ok = false; break; } }   // overlaps the softmax of q
-                const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
-                if (!mbar_wait(&bars->v_full[vs], (q / p.v_stages) & 1, p.status, 21)) { ok = false; break; }
-                if (!mbar_wait(&bars->p_full[pbuf], pu & 1, p.status, 5)) { ok = false; break; }
+                if (!seg_last) { if (!issue_s(false)) { ok = false; break; } }     // overlaps the softmax of q
+                if (!mbar_wait(&bars->v_full[vs], vpar, p.status, 21)) { ok = false; break; }
+                if (!mbar_wait(&bars->p_full[pb], ppar, p.status, 5)) { ok = false; break; }
                 tc_fence_after();
                 {
-                    const uint32_t p_addr = smem_u32(sm.pt + pbuf * Cfg::p_bytes(n_pad));
-                    const uint32_t v_addr = smem_u32(sm.v_ring + vs * Cfg::kTileBytes);
+                    const uint64_t dv = dv0 + static_cast<uint32_t>((vs * Cfg::kTileBytes) >> 4);
+                    const uint64_t dp = dp0 + static_cast<uint32_t>(pb) * p_buf16;
 #pragma unroll
-                    for (int ks = 0; ks < kAttBlockTokens / 16; ++ks) {
-                        // 16 tokens: two groups of 8 k-rows in both operands
-                        const uint64_t da = umma_desc_mn_sw128(v_addr + ks * 2048, Cfg::kSlabBytes, 1024);
-                        const uint64_t db = umma_desc_mn_plain(p_addr + ks * 256, 2048, 128);
-                        umma_bf16(tmem_base + kTmemO, da, db, idesc_o, (seg_first && ks == 0) ? 0u : 1u);
-                    }
+                    for (int ks = 0; ks < kAttBlockTokens / 16; ++ks)      // 16 tokens: two groups of 8 k-rows in both operands
+                        umma_bf16(tmem_base + kTmemO, dv + static_cast<uint32_t>((ks * 2048) >> 4), dp + static_cast<uint32_t>((ks * 256) >> 4),
+                                  idesc_o, (seg_first && ks == 0) ? 0u : 1u);
                 }
                 umma_commit(&bars->v_empty[vs]);
-                umma_commit(&bars->p_empty[pbuf]);
+                umma_commit(&bars->p_empty[pb]);
                 umma_commit(&bars->o_full);
+                if (++vs == p.v_stages) { vs = 0; vpar ^= 1u; }
+                if (++pb == p.p_bufs) { pb = 0; ppar ^= 1u; }
                 cur.advance(p, q + 1 < n_my);
                 seg_first = seg_last;
                 if (seg_last) {
-                    ++seg;
-                    if (q + 1 < n_my && !issue_s(q + 1, true, seg)) { ok = false; break; }
+                    ++s_seg;
+                    if (q + 1 < n_my && !issue_s(true)) { ok = false; break; }
                 }
             }
         }
     } else if (n_my > 0) {
-        if (n_pad <= 32) att_softmax<DH, 1>(p, sm, tmem_base, cur, n_my, total_blocks);
-        else if (n_pad <= 64) att_softmax<DH, 2>(p, sm, tmem_base, cur, n_my, total_blocks);
-        else if (n_pad <= 96) att_softmax<DH, 3>(p, sm, tmem_base, cur, n_my, total_blocks);
-        else att_softmax<DH, 4>(p, sm, tmem_base, cur, n_my, total_blocks);
+        att_softmax<DH, NCH>(p, sm, tmem_base, cur, n_my, total_blocks);
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kAttProducerWarps) {
         tc_fence_after();
         tmem_dealloc(tmem_base, kAttTmemCols);
     }
 }
 
+// one kernel per (head dim, chunks of 32 query rows): each instance keeps only the registers and the
+// code of its own softmax width
+template <int DH, int NCH>
+static cudaError_t att_set_smem()
+{
+    return cudaFuncSetAttribute(attention_kernel<DH, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kAttSmemLimit - kAttStaticReserve);
+}
+template <int DH>
+static cudaError_t att_init_dh()
+{
+    cudaError_t e = att_set_smem<DH, 1>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 2>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 3>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 4>();
+    return e;
+}
 cudaError_t attention_init(int head_dim)
 {
-    if (head_dim == 128)
-        return cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kAttSmemLimit - kAttStaticReserve);
-    return cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                kAttSmemLimit - kAttStaticReserve);
+    return head_dim == 128 ? att_init_dh<128>() : att_init_dh<64>();
+}
+
+template <int DH>
+static void att_launch_dh(const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas, cudaStream_t stream)
+{
+    const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<DH>::kTileBytes +
+                        AttCfg<DH>::fixed_bytes(p.n_pad, p.p_bufs);
+    dim3 grid(n_ctas), block(kAttThreads);
+    if (p.n_pad <= 32) attention_kernel<DH, 1><<<grid, block, smem, stream>>>(kv_map, p);
+    else if (p.n_pad <= 64) attention_kernel<DH, 2><<<grid, block, smem, stream>>>(kv_map, p);
+    else if (p.n_pad <= 96) attention_kernel<DH, 3><<<grid, block, smem, stream>>>(kv_map, p);
+    else attention_kernel<DH, 4><<<grid, block, smem, stream>>>(kv_map, p);
 }
 
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
                              cudaStream_t stream)
 {
-    dim3 grid(n_ctas);
-    dim3 block(kAttThreads);
-    if (h.cfg.head_dim == 128) {
-        const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<128>::kTileBytes +
-                            AttCfg<128>::fixed_bytes(p.n_pad, p.p_bufs);
-        attention_kernel<128><<<grid, block, smem, stream>>>(kv_map, p);
-    } else {
-        const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<64>::kTileBytes +
-                            AttCfg<64>::fixed_bytes(p.n_pad, p.p_bufs);
-        attention_kernel<64><<<grid, block, smem, stream>>>(kv_map, p);
-    }
+    if (h.cfg.head_dim == 128) att_launch_dh<128>(kv_map, p, n_ctas, stream);
+    else att_launch_dh<64>(kv_map, p, n_ctas, stream);
     return cudaGetLastError();
 }
 

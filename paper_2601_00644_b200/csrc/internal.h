@@ -16,7 +16,8 @@ constexpr int kSampleChunk = 8192;        // vocabulary entries per CTA of the s
 constexpr int kDrawChunk = 2048;          // vocabulary entries per CTA of the draw kernel
 constexpr int kAttBlockTokens = 128;      // KV tokens per attention work block / pipeline stage
 constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block (MMA M)
-constexpr int kAttThreads = 192;          // TMA warp + MMA warp + 4 softmax warps
+constexpr int kAttProducerWarps = 2;      // issuing a TMA request costs ~55 cycles of its warp: two warps share a block's 32
+constexpr int kAttThreads = (kAttProducerWarps + 1 + 4) * 32;   // TMA warps + MMA warp + 4 softmax warps
 constexpr int kAttMaxStages = 8;          // K / V ring depth (what fits in shared memory is used)
 constexpr int kNumStageEvents = 7;
 
@@ -27,6 +28,7 @@ struct Plan {                 // device tables written by the plan kernel, read 
 };
 
 struct AttnParams {
+    const uint8_t* kv_pages;  // the pool (also described by the tensor map), for L2 prefetches
     const __nv_bfloat16* hidden;
     const int32_t* page_table;
     const int32_t* kv_len;
