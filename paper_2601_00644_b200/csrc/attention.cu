@@ -48,7 +48,7 @@ constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column of
 constexpr float kRescaleThreshold = 8.f;                             // log2 units
 constexpr int kAttSmemLimit = 232448;                                // 227 KB opt-in maximum per CTA
 constexpr int kAttStaticReserve = 1024;                              // __shared__ variables of the kernel
-constexpr int kAttPrefetchBlocks = 6;                                // how far ahead of the copies the L2 prefetch runs
+constexpr int kAttPrefetchBlocks = 4;                                // how far ahead of the copies the L2 prefetch runs
 
 struct AttBars {
     uint64_t k_full[kAttMaxStages], k_empty[kAttMaxStages];
@@ -96,6 +96,12 @@ void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages)
     *v_stages = vs;
 }
 
+// The attention kernel waits in dozens of places and its code has to stay small enough for the
+// instruction caches (its cold paths run once per CTA): one shared copy of the wait loop.
+static __device__ __noinline__ bool att_wait(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
+{
+    return mbar_wait(bar, parity, status, where);
+}
 __device__ __forceinline__ void prefetch_l2(const void* p)
 {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
@@ -215,6 +221,23 @@ struct AttCursor {
     }
 };
 
+// Sums 32 per-lane values across the warp so that lane i ends up with the total of v[i]:
+// 31 shuffles (halving exchange) instead of 32 full reductions.  v is destroyed.
+__device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const bool up = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < o; ++i) {
+            const float give = up ? v[i] : v[i + o];
+            const float keep = up ? v[i + o] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, give, o);
+        }
+    }
+    return v[0];
+}
+
 struct AttStart { int b, blk_off, q_row0, pair0, blk0, total; };
 
 struct AttSmem {                  // pointers into dynamic shared memory
@@ -251,7 +274,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
     uint32_t group_phase = 0;
     auto group_sync = [&](int where) -> bool {
         mbar_arrive(&bars->group);
-        const bool done = mbar_wait(&bars->group, group_phase, p.status, where);
+        const bool done = att_wait(&bars->group, group_phase, p.status, where);
         group_phase ^= 1u;
         return done;
     };
@@ -297,7 +320,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         const uint32_t col_span = static_cast<uint32_t>(max(0, rows_here - col_min));
         const uint32_t t_s = t_lane + (buf ? kTmemS1 : kTmemS0);
 
-        if (!mbar_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
+        if (!att_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
         tc_fence_after();
 
         // ---- pass 1: column maxima over my warp's 32 tokens, then over the four warps
@@ -340,7 +363,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         }
         if (!seg_first && __any_sync(0xffffffffu, rescale)) {
             // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
-            if (!mbar_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
+            if (!att_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
@@ -363,7 +386,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         }
         // the P^T buffer is free once the product that last read it has completed
         const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
-        if (pu > 0 && !mbar_wait(&bars->p_empty[pbuf], (pu - 1) & 1, p.status, 8)) { ok = false; break; }
+        if (pu > 0 && !att_wait(&bars->p_empty[pbuf], (pu - 1) & 1, p.status, 8)) { ok = false; break; }
         // ---- pass 2: p = 2^(s * scale - m), bf16, into row t of operand B of the second product
         {
             uint8_t* p_row = sm.pt + pbuf * Cfg::p_bytes(n_pad) + t * 16;
@@ -427,12 +450,10 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         for (int ci = 0; ci < NCH; ++ci) {
             l_c[ci] = 0.f;
             if (ci * 32 < n_pad) {
-                float mine = 0.f;
+                float tmp[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float w = warp_sum(lsum[ci * 32 + i]);
-                    if (lane == i) mine = w;
-                }
+                for (int i = 0; i < 32; ++i) tmp[i] = lsum[ci * 32 + i];
+                const float mine = warp_transpose_sum(tmp, lane);
                 if (ci * 32 + lane < n_pad) xl[quarter * n_pad + ci * 32 + lane] = mine;
             }
         }
@@ -442,7 +463,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
             const int col = ci * 32 + lane;
             if (col < n_pad) l_c[ci] = (xl[col] + xl[n_pad + col]) + (xl[2 * n_pad + col] + xl[3 * n_pad + col]);
         }
-        if (!mbar_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
+        if (!att_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
         tc_fence_after();
         if (!o_lane) continue;                                         // nothing of O^T in this warp's lanes
         // which CTAs hold blocks of this pair: CTA c owns blocks [c*T/G, (c+1)*T/G), so the owner of
@@ -453,19 +474,19 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
 
         if (c_first == c_last) {
             // the whole pair was ours: normalise and store; thread t holds element t of every row
+            __nv_bfloat16* out_t = p.attn_out + t;
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
                 if (ci * 32 < n_pad) {
                     uint32_t o[32];
                     tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
                     tmem_ld_wait();
+                    const float inv_l = 1.f / l_c[ci];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        if (ci * 32 + i < rows_here) {                 // uniform
-                            const float l = __shfl_sync(0xffffffffu, l_c[ci], i);
-                            const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
-                            p.attn_out[static_cast<int64_t>(row) * DH + t] = __float2bfloat16_rn(__uint_as_float(o[i]) / l);
-                        }
+                        const float il = __shfl_sync(0xffffffffu, inv_l, i);
+                        const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
+                        if (ci * 32 + i < rows_here) out_t[static_cast<int64_t>(row) * DH] = __float2bfloat16_rn(__uint_as_float(o[i]) * il);
                     }
                 }
             }
@@ -511,70 +532,66 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
 
         // ---- this warp completed its rows of the pair: out = sum_c 2^(m_c - M) O_c / sum_c 2^(m_c - M) l_c,
         // parts taken in CTA order.  The first CTA holds the head of the pair in its last segment unless its
-        // range starts exactly there; every later CTA holds its part in its first segment.
+        // range starts exactly there; every later CTA holds its part in its first segment.  (This path runs
+        // once or twice per CTA and is always cold in the instruction cache: it is kept compact.)
         __threadfence();
         const int blk_begin_c0 = static_cast<int>(static_cast<int64_t>(c_first) * total_blocks / gridDim.x);
         const int slot_c0 = c_first * 2 + ((blk_begin_c0 == pair_blk_first) ? 0 : 1);
         float m_all[NCH], l_all[NCH];
 #pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) {
-            m_all[ci] = -INFINITY;
-            l_all[ci] = 0.f;
-            const int col = ci * 32 + lane;
-            if (col < n_pad) {
-                for (int cc = c_first; cc <= c_last; ++cc) {
-                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
-                    m_all[ci] = fmaxf(m_all[ci], __ldcg(p.part_ml + ((static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair + col) * 2));
-                }
-                for (int cc = c_first; cc <= c_last; ++cc) {
-                    const int slot = (cc == c_first) ? slot_c0 : cc * 2;
-                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(
-                        p.part_ml + ((static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair + col) * 2));
-                    if (ml.x != -INFINITY) l_all[ci] += fast_exp2(ml.x - m_all[ci]) * ml.y;
+        for (int ci = 0; ci < NCH; ++ci) { m_all[ci] = -INFINITY; l_all[ci] = 0.f; }
+#pragma unroll 1
+        for (int cc = c_first; cc <= c_last; ++cc) {               // running (max, sum) of my columns over the parts
+            const int slot = (cc == c_first) ? slot_c0 : cc * 2;
+            const float2* pml = reinterpret_cast<const float2*>(p.part_ml) + (static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 + lane < n_pad) {
+                    const float2 ml = __ldcg(pml + ci * 32 + lane);
+                    const float mn = fmaxf(m_all[ci], ml.x);
+                    const float base = (mn == -INFINITY) ? 0.f : mn;
+                    l_all[ci] = l_all[ci] * fast_exp2(m_all[ci] - base) + ml.y * fast_exp2(ml.x - base);
+                    m_all[ci] = mn;
                 }
             }
         }
 #pragma unroll
         for (int i = 0; i < NCH * 32; ++i) lsum[i] = 0.f;              // reused as the accumulator of my O^T row
+#pragma unroll 1
         for (int cc = c_first; cc <= c_last; ++cc) {
             const int slot = (cc == c_first) ? slot_c0 : cc * 2;
             const float4* po = reinterpret_cast<const float4*>(p.part_o + (static_cast<int64_t>(slot) * DH + t) * kAttRowsPerPair);
+            const float2* pml = reinterpret_cast<const float2*>(p.part_ml) + (static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair;
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
                 if (ci * 32 < n_pad) {
-                    const int col = ci * 32 + lane;
-                    float wgt = 0.f;                                   // weight of this part for my column
-                    if (col < n_pad) {
-                        const float mc = __ldcg(p.part_ml + ((static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair + col) * 2);
+                    float4 v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[i] = __ldcg(po + ci * 8 + i);
+                    float wgt = 0.f;                                   // weight of this part for my column; a part
+                    if (ci * 32 + lane < n_pad) {                      // that saw no visible token has weight 0 and O^T = 0
+                        const float mc = __ldcg(&pml[ci * 32 + lane].x);
                         wgt = (mc == -INFINITY) ? 0.f : fast_exp2(mc - m_all[ci]);
                     }
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        if (ci * 32 + i < rows_here) {                 // uniform
-                            const float4 v = __ldcg(po + ci * 8 + (i >> 2));
-                            const float w0 = __shfl_sync(0xffffffffu, wgt, i), w1 = __shfl_sync(0xffffffffu, wgt, i + 1);
-                            const float w2 = __shfl_sync(0xffffffffu, wgt, i + 2), w3 = __shfl_sync(0xffffffffu, wgt, i + 3);
-                            // a part that saw no visible token has weight 0
-                            if (w0 != 0.f) lsum[ci * 32 + i + 0] += w0 * v.x;
-                            if (w1 != 0.f) lsum[ci * 32 + i + 1] += w1 * v.y;
-                            if (w2 != 0.f) lsum[ci * 32 + i + 2] += w2 * v.z;
-                            if (w3 != 0.f) lsum[ci * 32 + i + 3] += w3 * v.w;
-                        }
+                    for (int i = 0; i < 8; ++i) {
+                        lsum[ci * 32 + 4 * i + 0] += __shfl_sync(0xffffffffu, wgt, 4 * i + 0) * v[i].x;
+                        lsum[ci * 32 + 4 * i + 1] += __shfl_sync(0xffffffffu, wgt, 4 * i + 1) * v[i].y;
+                        lsum[ci * 32 + 4 * i + 2] += __shfl_sync(0xffffffffu, wgt, 4 * i + 2) * v[i].z;
+                        lsum[ci * 32 + 4 * i + 3] += __shfl_sync(0xffffffffu, wgt, 4 * i + 3) * v[i].w;
                     }
                 }
             }
         }
+        __nv_bfloat16* out_t = p.attn_out + t;
 #pragma unroll
         for (int ci = 0; ci < NCH; ++ci) {
-            if (ci * 32 < n_pad) {
+            const float inv_l = 1.f / l_all[ci];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (ci * 32 + i < rows_here) {                     // uniform
-                        const float l = __shfl_sync(0xffffffffu, l_all[ci], i);
-                        const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
-                        p.attn_out[static_cast<int64_t>(row) * DH + t] = __float2bfloat16_rn(lsum[ci * 32 + i] / l);
-                    }
-                }
+            for (int i = 0; i < 32; ++i) {
+                const float il = __shfl_sync(0xffffffffu, inv_l, i);
+                const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
+                if (ci * 32 + i < rows_here) out_t[static_cast<int64_t>(row) * DH] = __float2bfloat16_rn(lsum[ci * 32 + i] * il);
             }
         }
     }
@@ -719,20 +736,16 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             ++pf_q;
             pf.advance(p, pf_q < n_my);
         };
-        {
-            // the first blocks: all page-table reads first, then the prefetches
-            int ph0[kAttPrefetchBlocks];
-            AttCursor tmp = pf;
-#pragma unroll
-            for (int i = 0; i < kAttPrefetchBlocks; ++i) {
-                ph0[i] = -1;
-                if (i < n_my) { ph0[i] = pf_load(tmp); tmp.advance(p, i + 1 < n_my); }
-            }
-#pragma unroll
-            for (int i = 0; i < kAttPrefetchBlocks; ++i)
-                if (i < n_my) pf_issue(ph0[i]);
+        int pf_ph = pf_load(pf);
+#pragma unroll 1
+        for (int i = 0; i < kAttPrefetchBlocks && pf_q < n_my; ++i) {
+            // the page-table read of the next block is in flight while this one is prefetched
+            AttCursor nxt = pf;
+            nxt.advance(p, pf_q + 1 < n_my);
+            const int ph_next = (pf_q + 1 < n_my) ? pf_load(nxt) : -1;
+            pf_issue(pf_ph);
+            pf_ph = ph_next;
         }
-        int pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
         for (int q = 0; q < n_my && ok; ++q) {
             const int kvh = cur.pair / cur.rbc;
             if (new_pair && warp == 0) {
@@ -762,13 +775,13 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             const uint32_t tile_tx = static_cast<uint32_t>(npg * Cfg::kSlabs * kPageTokens * 128);
             const int smem_off = my_half * Cfg::kSlabBytes + my_page * (kPageTokens * 128);
             // K tile
-            if (k_use > 0 && !mbar_wait(&bars->k_empty[ks], (k_use - 1) & 1, p.status, 1)) { ok = false; break; }
+            if (k_use > 0 && !att_wait(&bars->k_empty[ks], (k_use - 1) & 1, p.status, 1)) { ok = false; break; }
             if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&bars->k_full[ks], tile_tx);
             if (active)
                 tma_load_2d(sm.k_ring + ks * Cfg::kTileBytes + smem_off, &kv_map, &bars->k_full[ks], my_half * 64,
                             ((phys * 2 + 0) * p.n_kv_heads + kvh) * kPageTokens, pol);
             // V tile
-            if (v_use > 0 && !mbar_wait(&bars->v_empty[vs], (v_use - 1) & 1, p.status, 20)) { ok = false; break; }
+            if (v_use > 0 && !att_wait(&bars->v_empty[vs], (v_use - 1) & 1, p.status, 20)) { ok = false; break; }
             if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&bars->v_full[vs], tile_tx);
             if (active)
                 tma_load_2d(sm.v_ring + vs * Cfg::kTileBytes + smem_off, &kv_map, &bars->v_full[vs], my_half * 64,
@@ -783,8 +796,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         // do not leave while a copy of ours may still be landing in shared memory
         if (ok && n_my > 0) {
             const int ql = n_my - 1;
-            mbar_wait(&bars->k_full[ql % p.k_stages], (ql / p.k_stages) & 1, p.status, 9);
-            mbar_wait(&bars->v_full[ql % p.v_stages], (ql / p.v_stages) & 1, p.status, 9);
+            att_wait(&bars->k_full[ql % p.k_stages], (ql / p.k_stages) & 1, p.status, 9);
+            att_wait(&bars->v_full[ql % p.v_stages], (ql / p.v_stages) & 1, p.status, 9);
         }
     } else if (warp == kAttProducerWarps) {
         // ------------------------------------------------------------------ MMA issuer
@@ -807,9 +820,9 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             int s_q = 0, s_seg = 0;
             // S^T[buf] = K Q^T of the next block in order (waits: the pair's Q tile, the K tile, the S^T buffer)
             auto issue_s = [&](bool seg_first) -> bool {
-                if (seg_first && !mbar_wait(&bars->q_full, s_seg & 1, p.status, 2)) return false;
-                if (!mbar_wait(&bars->k_full[s_ks], s_kpar, p.status, 3)) return false;
-                if (s_q >= 2 && !mbar_wait(&bars->s_empty[s_buf], s_spar, p.status, 4)) return false;
+                if (seg_first && !att_wait(&bars->q_full, s_seg & 1, p.status, 2)) return false;
+                if (!att_wait(&bars->k_full[s_ks], s_kpar, p.status, 3)) return false;
+                if (s_q >= 2 && !att_wait(&bars->s_empty[s_buf], s_spar, p.status, 4)) return false;
                 tc_fence_after();
                 const uint64_t dk = dk0 + static_cast<uint32_t>((s_ks * Cfg::kTileBytes) >> 4);
                 const uint32_t acc = tmem_base + (s_buf ? kTmemS1 : kTmemS0);
@@ -832,8 +845,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             for (int q = 0; q < n_my && ok; ++q) {
                 const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
                 if (!seg_last) { if (!issue_s(false)) { ok = false; break; } }     // overlaps the softmax of q
-                if (!mbar_wait(&bars->v_full[vs], vpar, p.status, 21)) { ok = false; break; }
-                if (!mbar_wait(&bars->p_full[pb], ppar, p.status, 5)) { ok = false; break; }
+                if (!att_wait(&bars->v_full[vs], vpar, p.status, 21)) { ok = false; break; }
+                if (!att_wait(&bars->p_full[pb], ppar, p.status, 5)) { ok = false; break; }
                 tc_fence_after();
                 {
                     const uint64_t dv = dv0 + static_cast<uint32_t>((vs * Cfg::kTileBytes) >> 4);
