@@ -232,10 +232,10 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
                        accepted_len, next_token);
     if (launch_sample_stats(p, 0, p.greedy ? p.m_rows : p.m_rows + p.s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
-    if (launch_sample_decide(p, g.k_batch_max, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_decide(p, g.k_batch_max, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     if (!p.greedy) {
-        if (launch_sample_draw(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        if (launch_sample_draw(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
     }
     return FLEXSPEC_OK;
@@ -467,18 +467,18 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 2, s);
     mark(h, 3, s);
-    // the vocabulary mask needs the row -> sequence table of the plan kernel
-    if (sp.vocab_mask != nullptr && cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    // the second stream's work is long done by now; joining here keeps LM head -> decision -> draw
+    // back to back on this stream, so that the last two can be launched programmatically
+    if (cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     sp.tstats = h.tstats; sp.n_tparts = 4 * ((h.cfg.vocab + 127) / 128);     // the LM head leaves the target rows' parts
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);
-    if (cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (launch_sample_decide(sp, g.k_batch_max, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_decide(sp, g.k_batch_max, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 5, s);
     if (!sp.greedy) {
-        if (launch_sample_draw(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        if (launch_sample_draw(sp, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
     }
     mark(h, 6, s);

@@ -22,6 +22,13 @@ constexpr int32_t kErrTimeout = -5;
 constexpr int32_t kErrBadPage = -6;
 constexpr int32_t kErrBadToken = -7;
 
+// ---------------------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-serialization attribute may start while its predecessor
+// in the stream still runs; it must not touch the predecessor's results before pdl_wait().
+// Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------- addresses
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {

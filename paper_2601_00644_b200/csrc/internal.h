@@ -128,8 +128,23 @@ cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const A
                              cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
-cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, cudaStream_t stream);
-cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream);
+// pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
+// the stream drains; it waits on the device before touching the predecessor's results)
+cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, bool pdl, cudaStream_t stream);
+cudaError_t launch_sample_draw(const SampleParams& p, bool pdl, cudaStream_t stream);
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    bool pdl, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
 
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
 int attention_p_bufs(int n_pad);

@@ -60,6 +60,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    pdl_launch_dependents();                             // let the next kernel of the stream be set up while this one runs
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }

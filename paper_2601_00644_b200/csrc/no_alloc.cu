@@ -114,7 +114,7 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     p.accepted_len = accepted_len; p.next_token = next_token;
     p.status = status;
     if (launch_sample_stats(p, 0, greedy ? m_rows : m_rows + s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (launch_sample_decide(p, k_batch_max, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (!greedy && launch_sample_draw(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_decide(p, k_batch_max, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (!greedy && launch_sample_draw(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     return FLEXSPEC_OK;
 }

@@ -202,8 +202,10 @@ sample_decide_kernel(const SampleParams p)
     const int j = blockIdx.x;
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int k_b = p.draft_len[b];
+    pdl_launch_dependents();
+    const int k_b = p.draft_len[b];                      // inputs of the step: not written by the preceding kernels
     if (j > k_b) return;
+    pdl_wait();
     const int q0 = p.cu_q[b], d0 = p.cu_d[b];
     const double scale = static_cast<double>(p.inv_temp_log2);
     const float cf = p.inv_temp_log2;
@@ -236,16 +238,16 @@ sample_decide_kernel(const SampleParams p)
                 rs[0] = static_cast<double>(best);
             }
         } else {
-            float m = -INFINITY;
-#pragma unroll 8
-            for (int i = threadIdx.x; i < n; i += kSampleThreads) m = fmaxf(m, __ldcg(&tp[i].x));
-            m = block_max(m, red_f, lane, warp);
-            double sm = 0.0;
+            // one pass: running (max, sum) per thread in fp32, merged across the block with fp64 sums
+            float m = -INFINITY, sf = 0.f;
 #pragma unroll 8
             for (int i = threadIdx.x; i < n; i += kSampleThreads) {
                 const float2 pt = __ldcg(&tp[i]);
-                if (pt.x != -INFINITY) sm += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - m) * cf));
+                merge_ms(m, sf, pt.x, pt.y, cf);
             }
+            const float mt = m;
+            m = block_max(m, red_f, lane, warp);
+            double sm = (mt == -INFINITY) ? 0.0 : static_cast<double>(sf) * static_cast<double>(fast_exp2((mt - m) * cf));
             sm = block_sum(sm, red_d, lane, warp);
             if (threadIdx.x == 0) { rs[0] = static_cast<double>(m); rs[1] = sm; }
             // ---- draft row j: few parts, one warp
@@ -325,11 +327,9 @@ sample_decide_kernel(const SampleParams p)
     }
 }
 
-cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, cudaStream_t stream)
+cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, bool pdl, cudaStream_t stream)
 {
-    dim3 grid(k_batch_max + 1, p.batch);
-    sample_decide_kernel<<<grid, kSampleThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    return launch_kernel_ex(sample_decide_kernel, dim3(k_batch_max + 1, p.batch), dim3(kSampleThreads), 0, stream, pdl, p);
 }
 
 // ------------------------------------------------------------------------------------ draw
@@ -388,6 +388,7 @@ sample_draw_kernel(const SampleParams p)
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int k_b = p.draft_len[b];
+    pdl_wait();                                          // accepted_len and the row statistics come from the decision kernel
     const int n = p.accepted_len[b];
     DrawRow row;
     row.zt = p.logits + static_cast<int64_t>(p.cu_q[b] + n) * p.vocab;
@@ -526,11 +527,9 @@ sample_draw_kernel(const SampleParams p)
     }
 }
 
-cudaError_t launch_sample_draw(const SampleParams& p, cudaStream_t stream)
+cudaError_t launch_sample_draw(const SampleParams& p, bool pdl, cudaStream_t stream)
 {
-    dim3 grid(p.n_dchunks, p.batch);
-    sample_draw_kernel<<<grid, kSampleThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    return launch_kernel_ex(sample_draw_kernel, dim3(p.n_dchunks, p.batch), dim3(kSampleThreads), 0, stream, pdl, p);
 }
 
 }  // namespace fs
