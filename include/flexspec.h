@@ -208,10 +208,12 @@ int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);
  * and returns its first entry (0 or a FLEXSPEC_ERR_* code recorded by a kernel). */
 int flexspec_status(flexspec_handle* h, int32_t* status_host);
 
-/* Per-kernel timing.  With profiling on, verify brackets each kernel with CUDA events on the
- * caller's stream; flexspec_get_stage_ms synchronises those events and writes the last call's
- * durations in milliseconds: [0] plan, [1] attention, [2] attention combine, [3] LM head,
- * [4] sample statistics + decision, [5] sample draw.  Unused stages read 0. */
+/* Per-kernel timing.  With profiling on, verify brackets the kernels of the caller's stream with
+ * CUDA events; flexspec_get_stage_ms synchronises those events and writes the last call's
+ * durations in milliseconds: [0] fork of the second stream, [1] attention, [2] unused,
+ * [3] LM head (with the softmax statistics of the target rows), [4] acceptance decision,
+ * [5] emitted-token draw.  The row-offset kernel and the draft-logit statistics run on a second
+ * stream beside attention and are not timed.  Unused stages read 0. */
 int flexspec_set_profiling(flexspec_handle* h, int32_t on);
 int flexspec_get_stage_ms(flexspec_handle* h, float ms[6]);
 
