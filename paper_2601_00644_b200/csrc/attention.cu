@@ -63,6 +63,7 @@ static_assert(sizeof(AttBars) <= 512, "barrier block");
 // Dynamic shared memory, all offsets from a 1024-byte aligned base:
 //   [k_stages x K slabs] [v_stages x V slabs] [Q: slabs x n_pad x 128 B] [P^T: p_bufs x n_pad x 256 B]
 //   [barriers] [exchange of column maxima / row sums between the warps: 3 x 4 x n_pad floats]
+//   [running maxima: n_pad floats] [overflow flags]
 // K and V travel in separate rings: a K tile is free again after the QK^T product, a V tile only
 // after the softmax and the second product, so V gets the deeper ring.
 template <int DH>
@@ -72,7 +73,7 @@ struct AttCfg {
     static constexpr int kTileBytes = kSlabs * kSlabBytes;     // K (or V) of one 128-token block
     __host__ __device__ static constexpr int q_bytes(int n_pad) { return kSlabs * n_pad * 128; }
     __host__ __device__ static constexpr int p_bytes(int n_pad) { return n_pad * 256; }
-    __host__ __device__ static constexpr int col_bytes(int n_pad) { return 3 * 4 * n_pad * 4; }
+    __host__ __device__ static constexpr int col_bytes(int n_pad) { return (3 * 4 + 1) * n_pad * 4 + 64; }
     __host__ __device__ static constexpr int fixed_bytes(int n_pad, int p_bufs)
     {
         return q_bytes(n_pad) + p_bufs * p_bytes(n_pad) + 512 + col_bytes(n_pad) + 1024;
@@ -247,6 +248,8 @@ struct AttSmem {                  // pointers into dynamic shared memory
     uint8_t* pt;                  // P^T buffers
     AttBars* bars;
     float* xch;                   // [3][4][n_pad]: column maxima (by block parity) and row sums, one row per warp
+    float* m_col;                 // [n_pad] running maximum of every column (query row), log2 units
+    int* flags;                   // [2][4] "a score exceeded its maximum by more than the threshold", by block parity and warp
 };
 
 // ------------------------------------------------------------------------------------ softmax role
@@ -323,71 +326,106 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         if (!att_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
         tc_fence_after();
 
-        // ---- pass 1: column maxima over my warp's 32 tokens, then over the four warps
-        uint32_t sv[32];                                 // kept for pass 2 when there is a single chunk
-        float* xch = sm.xch + (q & 1) * 4 * n_pad;
-#pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) {
-            if (ci * 32 < n_pad) {
-                tmem_ld_x32(t_s + ci * 32, sv);
-                tmem_ld_wait();
-                float mine = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;
-                    const float w = redux_max(masked ? -INFINITY : __uint_as_float(sv[i]));
-                    if (lane == i) mine = w;
-                }
-                if (ci * 32 + lane < n_pad) xch[quarter * n_pad + ci * 32 + lane] = mine;
-            }
-        }
-        if (!group_sync(14)) { ok = false; break; }
-        float alpha[NCH];
-        bool rescale = false;
-#pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) {
-            alpha[ci] = 1.f;
-            const int col = ci * 32 + lane;
-            if (col < n_pad) {
-                const float mx = fmaxf(fmaxf(xch[col], xch[n_pad + col]), fmaxf(xch[2 * n_pad + col], xch[3 * n_pad + col])) *
-                                 p.scale_log2;           // scale > 0: the maximum commutes
-                // ---- raise the running maximum only if it grew by more than the threshold
-                if (seg_first) {
-                    m_used[ci] = mx;
-                } else if (mx > m_used[ci] + kRescaleThreshold) {
-                    alpha[ci] = fast_exp2(m_used[ci] - mx);                // m_used == -inf gives 0
-                    m_used[ci] = mx;
-                    rescale = true;
-                }
-            }
-        }
-        if (!seg_first && __any_sync(0xffffffffu, rescale)) {
-            // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
-            if (!att_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
-            tc_fence_after();
+        // ---- does any score of this block exceed its row's running maximum by more than the threshold?
+        // (cheap: a multiply-add and a max per score against the maxima kept in shared memory; the exact
+        // column maxima below are only needed when the answer is yes, or at the start of a segment)
+        uint32_t sv[32];                                 // kept for the next pass when there is a single chunk
+        bool slow = seg_first;
+        if (!seg_first) {
+            float ex = -INFINITY;
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
                 if (ci * 32 < n_pad) {
-                    uint32_t o[32];
-                    if (o_lane) {
-                        tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
-                        tmem_ld_wait();
-                    }
+                    tmem_ld_x32(t_s + ci * 32, sv);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float a = __shfl_sync(0xffffffffu, alpha[ci], i);
-                        lsum[ci * 32 + i] *= a;
-                        if (o_lane) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
+                    for (int i4 = 0; i4 < 8; ++i4) {
+                        const float4 mv = *reinterpret_cast<const float4*>(sm.m_col + ci * 32 + 4 * i4);
+                        const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int i = 4 * i4 + j;
+                            const float x = fmaf(__uint_as_float(sv[i]), p.scale_log2, -mm[j]);   // -inf maximum: +inf
+                            const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;
+                            ex = fmaxf(ex, masked ? -INFINITY : x);
+                        }
                     }
-                    if (o_lane) tmem_st_x32(t_lane + kTmemO + ci * 32, o);
                 }
             }
-            if (o_lane) tmem_st_wait();
+            const bool hot = __any_sync(0xffffffffu, ex > kRescaleThreshold);
+            if (lane == 0) sm.flags[(q & 1) * 4 + quarter] = hot ? 1 : 0;
+            if (!group_sync(14)) { ok = false; break; }
+            const int* fl = sm.flags + (q & 1) * 4;
+            slow = (fl[0] | fl[1] | fl[2] | fl[3]) != 0;
+        }
+        if (slow) {
+            // ---- exact column maxima over my warp's 32 tokens, then over the four warps
+            float* xch = sm.xch + (q & 1) * 4 * n_pad;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                if (ci * 32 < n_pad) {
+                    tmem_ld_x32(t_s + ci * 32, sv);
+                    tmem_ld_wait();
+                    float mine = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;
+                        const float w = redux_max(masked ? -INFINITY : __uint_as_float(sv[i]));
+                        if (lane == i) mine = w;
+                    }
+                    if (ci * 32 + lane < n_pad) xch[quarter * n_pad + ci * 32 + lane] = mine;
+                }
+            }
+            if (!group_sync(17)) { ok = false; break; }
+            float alpha[NCH];
+            bool rescale = false;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                alpha[ci] = 1.f;
+                const int col = ci * 32 + lane;
+                if (col < n_pad) {
+                    const float mx = fmaxf(fmaxf(xch[col], xch[n_pad + col]), fmaxf(xch[2 * n_pad + col], xch[3 * n_pad + col])) *
+                                     p.scale_log2;       // scale > 0: the maximum commutes
+                    // ---- raise the running maximum only if it grew by more than the threshold
+                    if (seg_first) {
+                        m_used[ci] = mx;
+                    } else if (mx > m_used[ci] + kRescaleThreshold) {
+                        alpha[ci] = fast_exp2(m_used[ci] - mx);            // m_used == -inf gives 0
+                        m_used[ci] = mx;
+                        rescale = true;
+                    }
+                    if (quarter == 0) sm.m_col[col] = m_used[ci];
+                }
+            }
+            if (!seg_first && __any_sync(0xffffffffu, rescale)) {
+                // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
+                if (!att_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ci = 0; ci < NCH; ++ci) {
+                    if (ci * 32 < n_pad) {
+                        uint32_t o[32];
+                        if (o_lane) {
+                            tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
+                            tmem_ld_wait();
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float a = __shfl_sync(0xffffffffu, alpha[ci], i);
+                            lsum[ci * 32 + i] *= a;
+                            if (o_lane) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
+                        }
+                        if (o_lane) tmem_st_x32(t_lane + kTmemO + ci * 32, o);
+                    }
+                }
+                if (o_lane) tmem_st_wait();
+            }
+            if (!group_sync(18)) { ok = false; break; }                // the new maxima are in shared memory
         }
         // the P^T buffer is free once the product that last read it has completed
         const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
         if (pu > 0 && !att_wait(&bars->p_empty[pbuf], (pu - 1) & 1, p.status, 8)) { ok = false; break; }
-        // ---- pass 2: p = 2^(s * scale - m), bf16, into row t of operand B of the second product
+        // ---- p = 2^(s * scale - m), bf16, into row t of operand B of the second product
         {
             uint8_t* p_row = sm.pt + pbuf * Cfg::p_bytes(n_pad) + t * 16;
 #pragma unroll
@@ -397,19 +435,21 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
                         tmem_ld_x32(t_s + ci * 32, sv);
                         tmem_ld_wait();
                     }
-                    const float m_safe = (m_used[ci] == -INFINITY) ? 0.f : m_used[ci];
                     uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float m0 = __shfl_sync(0xffffffffu, m_safe, i);
-                        const float m1 = __shfl_sync(0xffffffffu, m_safe, i + 1);
-                        float e0 = fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -m0));
-                        float e1 = fast_exp2(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -m1));
-                        if (static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span) e0 = 0.f;
-                        if (static_cast<uint32_t>(ci * 32 + i + 1 - col_min) >= col_span) e1 = 0.f;
-                        lsum[ci * 32 + i] += e0;
-                        lsum[ci * 32 + i + 1] += e1;
-                        pk[i >> 1] = pack_bf16(e0, e1);
+                    for (int i4 = 0; i4 < 8; ++i4) {
+                        const float4 mv = *reinterpret_cast<const float4*>(sm.m_col + ci * 32 + 4 * i4);
+                        const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
+                        float e[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int i = 4 * i4 + j;
+                            e[j] = fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -mm[j]));
+                            if (static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span) e[j] = 0.f;   // also rows without a maximum yet
+                            lsum[ci * 32 + i] += e[j];
+                        }
+                        pk[2 * i4] = pack_bf16(e[0], e[1]);
+                        pk[2 * i4 + 1] = pack_bf16(e[2], e[3]);
                     }
 #pragma unroll
                     for (int g8 = 0; g8 < 4; ++g8)
@@ -612,6 +652,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
     sm.pt = sm.q + Cfg::q_bytes(n_pad);
     sm.bars = reinterpret_cast<AttBars*>(sm.pt + p.p_bufs * Cfg::p_bytes(n_pad));
     sm.xch = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sm.bars) + 512);
+    sm.m_col = sm.xch + 12 * n_pad;
+    sm.flags = reinterpret_cast<int*>(sm.m_col + n_pad);
     AttBars* bars = sm.bars;
     __shared__ int s_warp_tot[32];
     __shared__ AttStart s_start;
