@@ -577,24 +577,11 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         __threadfence();
         const int blk_begin_c0 = static_cast<int>(static_cast<int64_t>(c_first) * total_blocks / gridDim.x);
         const int slot_c0 = c_first * 2 + ((blk_begin_c0 == pair_blk_first) ? 0 : 1);
+        // one pass over the parts: the (m, l) of my column and my row of O^T are requested together, and
+        // the accumulator is rescaled whenever a part raises a column's maximum
         float m_all[NCH], l_all[NCH];
 #pragma unroll
         for (int ci = 0; ci < NCH; ++ci) { m_all[ci] = -INFINITY; l_all[ci] = 0.f; }
-#pragma unroll 1
-        for (int cc = c_first; cc <= c_last; ++cc) {               // running (max, sum) of my columns over the parts
-            const int slot = (cc == c_first) ? slot_c0 : cc * 2;
-            const float2* pml = reinterpret_cast<const float2*>(p.part_ml) + (static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair;
-#pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
-                if (ci * 32 + lane < n_pad) {
-                    const float2 ml = __ldcg(pml + ci * 32 + lane);
-                    const float mn = fmaxf(m_all[ci], ml.x);
-                    const float base = (mn == -INFINITY) ? 0.f : mn;
-                    l_all[ci] = l_all[ci] * fast_exp2(m_all[ci] - base) + ml.y * fast_exp2(ml.x - base);
-                    m_all[ci] = mn;
-                }
-            }
-        }
 #pragma unroll
         for (int i = 0; i < NCH * 32; ++i) lsum[i] = 0.f;              // reused as the accumulator of my O^T row
 #pragma unroll 1
@@ -608,17 +595,25 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
                     float4 v[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) v[i] = __ldcg(po + ci * 8 + i);
-                    float wgt = 0.f;                                   // weight of this part for my column; a part
-                    if (ci * 32 + lane < n_pad) {                      // that saw no visible token has weight 0 and O^T = 0
-                        const float mc = __ldcg(&pml[ci * 32 + lane].x);
-                        wgt = (mc == -INFINITY) ? 0.f : fast_exp2(mc - m_all[ci]);
-                    }
+                    float2 ml = make_float2(-INFINITY, 0.f);
+                    if (ci * 32 + lane < n_pad) ml = __ldcg(pml + ci * 32 + lane);
+                    // my column: weight of what is accumulated so far, weight of this part (a part that saw no
+                    // visible token has m = -inf, weight 0 and O^T = 0)
+                    const float mn = fmaxf(m_all[ci], ml.x);
+                    const float base = (mn == -INFINITY) ? 0.f : mn;
+                    const float w_old = fast_exp2(m_all[ci] - base);
+                    const float w_new = fast_exp2(ml.x - base);
+                    l_all[ci] = l_all[ci] * w_old + ml.y * w_new;
+                    m_all[ci] = mn;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        lsum[ci * 32 + 4 * i + 0] += __shfl_sync(0xffffffffu, wgt, 4 * i + 0) * v[i].x;
-                        lsum[ci * 32 + 4 * i + 1] += __shfl_sync(0xffffffffu, wgt, 4 * i + 1) * v[i].y;
-                        lsum[ci * 32 + 4 * i + 2] += __shfl_sync(0xffffffffu, wgt, 4 * i + 2) * v[i].z;
-                        lsum[ci * 32 + 4 * i + 3] += __shfl_sync(0xffffffffu, wgt, 4 * i + 3) * v[i].w;
+                        const float vv[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float wo = __shfl_sync(0xffffffffu, w_old, 4 * i + j);
+                            const float wn = __shfl_sync(0xffffffffu, w_new, 4 * i + j);
+                            lsum[ci * 32 + 4 * i + j] = lsum[ci * 32 + 4 * i + j] * wo + wn * vv[j];
+                        }
                     }
                 }
             }
@@ -778,16 +773,11 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             ++pf_q;
             pf.advance(p, pf_q < n_my);
         };
+        // the cursor starts one block ahead (the first copy must not wait for more than its own page ids)
+        // and gains a block per iteration until it runs kAttPrefetchBlocks ahead
         int pf_ph = pf_load(pf);
-#pragma unroll 1
-        for (int i = 0; i < kAttPrefetchBlocks && pf_q < n_my; ++i) {
-            // the page-table read of the next block is in flight while this one is prefetched
-            AttCursor nxt = pf;
-            nxt.advance(p, pf_q + 1 < n_my);
-            const int ph_next = (pf_q + 1 < n_my) ? pf_load(nxt) : -1;
-            pf_issue(pf_ph);
-            pf_ph = ph_next;
-        }
+        pf_issue(pf_ph);
+        pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
         for (int q = 0; q < n_my && ok; ++q) {
             const int kvh = cur.pair / cur.rbc;
             if (new_pair && warp == 0) {
@@ -829,7 +819,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
                 tma_load_2d(sm.v_ring + vs * Cfg::kTileBytes + smem_off, &kv_map, &bars->v_full[vs], my_half * 64,
                             ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens, pol);
             __syncwarp();
-            if (pf_q < n_my) {
+#pragma unroll 1
+            for (int step = 0; step < 2 && pf_q < n_my && pf_q <= q + kAttPrefetchBlocks; ++step) {
                 pf_issue(pf_ph);
                 pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
             }
