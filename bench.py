@@ -31,6 +31,7 @@ if ROOT not in sys.path:
 # workload, from the ncu capture summarised in profiles/ (None until captured)
 LM_HEAD_TRAFFIC_BYTES = 1051824000 + 8016128
 FALLBACK_HBM_GBS = 6650.0
+REFERENCE_BUDGET_S = 120.0
 
 
 def _peaks():
@@ -98,6 +99,26 @@ def _dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
 
+def shard_for_rank(shape, rank):
+    """Replicas: every rank verifies its own batch of independent sequences (its own seed)."""
+    from paper_2601_00644_b200 import workloads as wl
+    return shape if rank == 0 else wl.scaled(shape, index=shape.index + 100 * rank)
+
+
+def reduce_over_ranks(total_ms, e2e_s, verified, device=None):
+    """Whole-job numbers of a replicated run: the slowest rank's time, the sum of the ranks' tokens.
+    Works on any initialised process group (NCCL on GPUs, gloo in the CPU tests)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return total_ms, e2e_s, float(verified)
+    t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    v = torch.tensor([float(verified)], dtype=torch.float64, device=device)
+    dist.all_reduce(v, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(v[0])
+
+
 # ------------------------------------------------------------------------------ reference arm
 def run_reference(args):
     """The oracle as it stands, on the host cores: each step verifies `sample` whole sequences
@@ -124,19 +145,25 @@ def run_reference(args):
 
     for _ in range(args.warmup):
         step()
+    # the oracle is deliberately slow: the timed loop stops at the requested number of steps or
+    # after REFERENCE_BUDGET_S seconds, whichever comes first (the line reports the steps timed)
     t0 = time.perf_counter()
     verified = 0
+    steps_done = 0
     for _ in range(args.steps):
         res = step()
         verified += int(res["accepted_len"].sum()) + n_seq
+        steps_done += 1
+        if time.perf_counter() - t0 > REFERENCE_BUDGET_S:
+            break
     dt = time.perf_counter() - t0
     value = verified / dt
     cores = oracle.num_threads()
     sample = f"{n_seq} of {shape.batch} sequences of '{shape.name}' per step (whole sequences, k={int(k[0])})"
     line = {
         "impl": "reference", "metric": "verified_tokens_per_s", "value": value, "unit": "tokens/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "n_gpus": args.gpus, "steps": steps_done, "steps_requested": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / steps_done * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": shape.name, "sample": sample},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
@@ -185,8 +212,7 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
 
     shape = wl.CONFIGS[args.config]
-    if world > 1:
-        shape = wl.scaled(shape, index=shape.index + 100 * rank)        # every rank its own batch
+    shape = shard_for_rank(shape, rank)                                  # every rank its own batch
     inp = wl.make_inputs(shape, device=str(dev))
     k_host, kv_host = inp.draft_len.cpu(), inp.kv_len.cpu()
     batch, m_rows, s_rows = inp.batch, inp.m_rows, inp.s_rows
@@ -286,15 +312,7 @@ def run_ours(args):
     assert torch.equal(h_acc.to(dev), acc) and torch.equal(h_nxt.to(dev), nxt)
 
     # ---- reduce over ranks: max time, summed tokens
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_s = float(t[0]), float(t[1])
-        v = torch.tensor([verified], dtype=torch.float64, device=dev)
-        dist.all_reduce(v, op=dist.ReduceOp.SUM)
-        verified_all = float(v[0])
-    else:
-        verified_all = float(verified)
+    total_ms, e2e_s, verified_all = reduce_over_ranks(total_ms, e2e_s, verified, device=dev)
     ms_per_step = total_ms / args.steps
 
     if rank == 0:
