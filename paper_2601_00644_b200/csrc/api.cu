@@ -315,7 +315,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128)));
     A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
     A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 4));
-    A(dev_alloc(&h.row_stats, static_cast<size_t>(c.max_batch) * (kMaxK + 1) * 4));
+    A(dev_alloc(&h.row_stats, static_cast<size_t>(c.max_batch) * (kMaxK + 1) * 8));
     A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * ((c.vocab + kDrawChunk - 1) / kDrawChunk) * 2));
     A(dev_alloc(&h.dbg_p, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.dbg_q, static_cast<size_t>(h.max_s)));

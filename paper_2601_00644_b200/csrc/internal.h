@@ -87,7 +87,7 @@ struct SampleParams {
     const float2* tstats;         // parts of the target rows: [M][n_tparts] (from the LM head), or = stats
     int32_t n_tparts;
     int32_t* counters;            // [2][max_batch] self-resetting tickets (decision, draw)
-    double* row_stats;            // [B][kMaxK+1][4]: (max_p, sum_p, max_q, sum_q) of every row, or the arg-max in [0]
+    double* row_stats;            // [B][kMaxK+1][8]: (max_p, sum_p, max_q, sum_q, rejected) of every row, or the arg-max in [0]
     double* row_info;             // [B][4]: max_p, 1/sum_p, max_q, 1/sum_q of row n
     double* chunk_mass;           // [B][n_dchunks][2]: residual mass, p mass
     int32_t* accepted_len;

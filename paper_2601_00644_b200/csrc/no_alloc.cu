@@ -26,7 +26,7 @@ constexpr size_t kOffRowSeq = kOffCuD + align256(sizeof(int32_t) * (kStaticMaxBa
 constexpr size_t kOffStats = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);
 constexpr size_t kOffRowInfo = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
 constexpr size_t kOffRowStats = kOffRowInfo + align256(sizeof(double) * kStaticMaxBatch * 4);
-constexpr size_t kOffMass = kOffRowStats + align256(sizeof(double) * kStaticMaxBatch * (kMaxK + 1) * 4);
+constexpr size_t kOffMass = kOffRowStats + align256(sizeof(double) * kStaticMaxBatch * (kMaxK + 1) * 8);
 constexpr size_t kScratchBytes = kOffMass + align256(sizeof(double) * kStaticMaxBatch * kStaticDrawChunks * 2);
 
 // In host code this name is only a handle for the runtime: the device address comes from

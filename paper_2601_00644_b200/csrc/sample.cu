@@ -166,9 +166,10 @@ cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_
 // ------------------------------------------------------------------------------------ decision
 // grid (row j, sequence b): the CTA merges the parts of target row j (and draft row j) of the
 // sequence -- maximum first, then the sum with fp32 weights accumulated in fp64 -- and leaves
-// (max, sum) per row.  The CTA that arrives last for the sequence (atomic ticket, nobody waits)
-// evaluates the acceptance tests with Philox uniforms, finds the first rejection by warp vote and
-// stores accepted_len; GREEDY compares the draft with the rows' arg-max.
+// (max, sum) per row together with the outcome of the row's own acceptance test (Philox uniform,
+// u * q(x) < p(x)).  The CTA that arrives last for the sequence (atomic ticket, nobody waits) finds
+// the first rejection by warp vote and stores accepted_len; GREEDY compares the draft with the
+// rows' arg-max.
 __device__ __forceinline__ float block_max(float v, float* red, int lane, int warp)
 {
     v = warp_max(v);
@@ -192,6 +193,8 @@ __device__ __forceinline__ double block_sum(double v, double* red, int lane, int
     return r;
 }
 
+constexpr int kRowStat = 8;       // doubles per (sequence, row): max_p, sum_p, max_q, sum_q, rejected
+
 __global__ void __launch_bounds__(kSampleThreads)
 sample_decide_kernel(const SampleParams p)
 {
@@ -203,15 +206,47 @@ sample_decide_kernel(const SampleParams p)
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     pdl_launch_dependents();
-    const int k_b = p.draft_len[b];                      // inputs of the step: not written by the preceding kernels
+    const int k_b = p.draft_len[b];                      // inputs of the step: not written by the preceding kernel
     if (j > k_b) return;
-    pdl_wait();
     const int q0 = p.cu_q[b], d0 = p.cu_d[b];
     const double scale = static_cast<double>(p.inv_temp_log2);
     const float cf = p.inv_temp_log2;
-    double* rs = p.row_stats + (static_cast<int64_t>(b) * (kMaxK + 1) + j) * 4;
+    double* rs = p.row_stats + (static_cast<int64_t>(b) * (kMaxK + 1) + j) * kRowStat;
+    const bool test_row = !p.greedy && j < k_b;
 
-    // ---- target row j
+    // ---- everything that depends only on the step's inputs and on the draft-logit statistics (second
+    // stream, joined before the preceding kernel started) is done before that kernel's results are
+    // awaited: the draft token, q_j(x_j) and the uniform of this row's acceptance test
+    int x = 0;
+    double mq = 0.0, sq = 1.0, qt = 0.0, u = 0.0;
+    if (test_row && warp == 0) {
+        const float2* dp = p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks;
+        float mqf = -INFINITY;
+        for (int i = lane; i < p.n_chunks; i += 32) mqf = fmaxf(mqf, __ldcg(&dp[i].x));
+        mqf = warp_max(mqf);
+        double acc = 0.0;
+        for (int i = lane; i < p.n_chunks; i += 32) {
+            const float2 pt = __ldcg(&dp[i]);
+            if (pt.x != -INFINITY) acc += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - mqf) * cf));
+        }
+        sq = warp_sum(acc);
+        mq = static_cast<double>(mqf);
+        if (lane == 0) {
+            x = p.draft_tokens[d0 + j];
+            x = min(max(x, 0), p.vocab - 1);
+            const double zq = static_cast<double>(p.draft_logits[static_cast<int64_t>(d0 + j) * p.vocab + x]);
+            qt = (zq == -INFINITY) ? 0.0 : exp2((zq - mq) * scale) / sq;
+            u = philox_uniform(p.seeds[b], static_cast<uint32_t>(j), 0u);
+        }
+    }
+    pdl_wait();
+
+    // ---- target row j: merge the parts (one pass, running (max, sum) per thread in fp32, fp64 sums across the block)
+    double zp = 0.0;
+    if (test_row && threadIdx.x == 0) {
+        zp = static_cast<double>(p.logits[static_cast<int64_t>(q0 + j) * p.vocab + x]);
+        if (p.vocab_mask != nullptr && !mask_allows(p.vocab_mask + static_cast<int64_t>(b) * p.mask_words, x)) zp = -INFINITY;
+    }
     {
         const float2* tp = p.tstats + static_cast<int64_t>(q0 + j) * p.n_tparts;
         const int n = p.n_tparts;
@@ -238,7 +273,6 @@ sample_decide_kernel(const SampleParams p)
                 rs[0] = static_cast<double>(best);
             }
         } else {
-            // one pass: running (max, sum) per thread in fp32, merged across the block with fp64 sums
             float m = -INFINITY, sf = 0.f;
 #pragma unroll 8
             for (int i = threadIdx.x; i < n; i += kSampleThreads) {
@@ -249,24 +283,23 @@ sample_decide_kernel(const SampleParams p)
             m = block_max(m, red_f, lane, warp);
             double sm = (mt == -INFINITY) ? 0.0 : static_cast<double>(sf) * static_cast<double>(fast_exp2((mt - m) * cf));
             sm = block_sum(sm, red_d, lane, warp);
-            if (threadIdx.x == 0) { rs[0] = static_cast<double>(m); rs[1] = sm; }
-            // ---- draft row j: few parts, one warp
-            if (j < k_b && warp == 1) {
-                const float2* dp = p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks;
-                float mq = -INFINITY;
-                for (int i = lane; i < p.n_chunks; i += 32) mq = fmaxf(mq, __ldcg(&dp[i].x));
-                mq = warp_max(mq);
-                double sq = 0.0;
-                for (int i = lane; i < p.n_chunks; i += 32) {
-                    const float2 pt = __ldcg(&dp[i]);
-                    if (pt.x != -INFINITY) sq += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - mq) * cf));
+            if (threadIdx.x == 0) {
+                rs[0] = static_cast<double>(m); rs[1] = sm; rs[2] = mq; rs[3] = sq;
+                double rej = 0.0;
+                if (test_row) {
+                    const double pt = (zp == -INFINITY) ? 0.0 : exp2((zp - static_cast<double>(m)) * scale) / sm;
+                    rej = (u * qt < pt) ? 0.0 : 1.0;
+                    if (p.dbg_p != nullptr) {
+                        p.dbg_p[d0 + j] = pt;
+                        p.dbg_q[d0 + j] = qt;
+                        p.dbg_u[d0 + j] = static_cast<float>(u);
+                    }
                 }
-                sq = warp_sum(sq);
-                if (lane == 0) { rs[2] = static_cast<double>(mq); rs[3] = sq; }
+                rs[4] = rej;
             }
         }
     }
-    // ---- ticket: the last row of the sequence decides
+    // ---- ticket: the last row of the sequence finds the first rejection
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -278,52 +311,27 @@ sample_decide_kernel(const SampleParams p)
     if (!s_last || warp != 0) return;
     __threadfence();
 
-    const double* rs0 = p.row_stats + static_cast<int64_t>(b) * (kMaxK + 1) * 4;
+    const double* rs0 = p.row_stats + static_cast<int64_t>(b) * (kMaxK + 1) * kRowStat;
     int n = k_b;
-    if (p.greedy) {
-        for (int base = 0; base < k_b; base += 32) {
-            const int jj = base + lane;
-            const bool rej = (jj < k_b) && (p.draft_tokens[d0 + jj] != static_cast<int>(__ldcg(rs0 + jj * 4)));
-            const unsigned vote = __ballot_sync(0xffffffffu, rej);
-            if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
-        }
-        if (lane == 0) {
-            p.accepted_len[b] = n;
-            p.next_token[b] = static_cast<int>(__ldcg(rs0 + n * 4));
-        }
-        return;
-    }
-    const uint64_t seed = p.seeds[b];
     for (int base = 0; base < k_b; base += 32) {
         const int jj = base + lane;
         bool rej = false;
-        if (jj < k_b) {
-            const double mp = __ldcg(rs0 + jj * 4), sp = __ldcg(rs0 + jj * 4 + 1);
-            const double mq = __ldcg(rs0 + jj * 4 + 2), sq = __ldcg(rs0 + jj * 4 + 3);
-            int x = p.draft_tokens[d0 + jj];
-            x = min(max(x, 0), p.vocab - 1);
-            double zp = static_cast<double>(p.logits[static_cast<int64_t>(q0 + jj) * p.vocab + x]);
-            if (p.vocab_mask != nullptr &&
-                !mask_allows(p.vocab_mask + static_cast<int64_t>(b) * p.mask_words, x)) zp = -INFINITY;
-            const double zq = static_cast<double>(p.draft_logits[static_cast<int64_t>(d0 + jj) * p.vocab + x]);
-            const double pt = (zp == -INFINITY) ? 0.0 : exp2((zp - mp) * scale) / sp;
-            const double qt = (zq == -INFINITY) ? 0.0 : exp2((zq - mq) * scale) / sq;
-            const double u = philox_uniform(seed, static_cast<uint32_t>(jj), 0u);
-            rej = !(u * qt < pt);
-            if (p.dbg_p != nullptr) {
-                p.dbg_p[d0 + jj] = pt;
-                p.dbg_q[d0 + jj] = qt;
-                p.dbg_u[d0 + jj] = static_cast<float>(u);
-            }
-        }
+        if (jj < k_b)
+            rej = p.greedy ? (p.draft_tokens[d0 + jj] != static_cast<int>(__ldcg(rs0 + jj * kRowStat)))
+                           : (__ldcg(rs0 + jj * kRowStat + 4) != 0.0);
         const unsigned vote = __ballot_sync(0xffffffffu, rej);
         if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
     }
     if (lane == 0) {
         p.accepted_len[b] = n;
-        double* ri = p.row_info + static_cast<int64_t>(b) * 4;
-        ri[0] = __ldcg(rs0 + n * 4); ri[1] = 1.0 / __ldcg(rs0 + n * 4 + 1);
-        ri[2] = (n < k_b) ? __ldcg(rs0 + n * 4 + 2) : 0.0; ri[3] = (n < k_b) ? 1.0 / __ldcg(rs0 + n * 4 + 3) : 1.0;
+        const double* rn = rs0 + n * kRowStat;
+        if (p.greedy) {
+            p.next_token[b] = static_cast<int>(__ldcg(rn));
+        } else {
+            double* ri = p.row_info + static_cast<int64_t>(b) * 4;
+            ri[0] = __ldcg(rn); ri[1] = 1.0 / __ldcg(rn + 1);
+            ri[2] = (n < k_b) ? __ldcg(rn + 2) : 0.0; ri[3] = (n < k_b) ? 1.0 / __ldcg(rn + 3) : 1.0;
+        }
     }
 }
 
