@@ -199,6 +199,48 @@ def cpu_baseline(shape, seconds_target=12.0):
             "sample": f"{reps} x 1 of {shape.batch} sequences of '{shape.name}' (whole sequences), {dt:.1f} s"}
 
 
+def fit_cloud_cost(args, base_shape, dev):
+    """The paper models the cloud-side verification latency as T_base + K * delta_cloud (Section IV-B,
+    refined latency model).  Measure the step at several draft lengths K on the same shape and fit the
+    two constants by least squares."""
+    import numpy as np
+    import torch
+    from paper_2601_00644_b200 import binding, workloads as wl
+    ks, us = [], []
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    for kk in (1, 2, 3, 5, 7, 9, 12):
+        shape = wl.scaled(base_shape, k_min=kk, k_max=kk, name=f"{base_shape.name}_k{kk}")
+        inp = wl.make_inputs(shape, device=str(dev))
+        k_host, kv_host = inp.draft_len.cpu(), inp.kv_len.cpu()
+        ver = binding.Verifier(inp.lm_head_w, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                               max_batch=inp.batch, k_max=kk, max_kv_len=int(kv_host.max()))
+        toks = wl.draw_draft_tokens(inp.noise, shape.temperature, inp.token_uniforms)
+        acc = torch.empty(inp.batch, dtype=torch.int32, device=dev)
+        nxt = torch.empty(inp.batch, dtype=torch.int32, device=dev)
+        stream = torch.cuda.current_stream()
+        t = []
+        for i in range(3 + 20):
+            flush.view(torch.int64).sum()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            ver.verify(inp.kv_pages, inp.page_table, inp.kv_len, kv_host, inp.hidden, toks, inp.noise,
+                       inp.draft_len, k_host, inp.seeds, temperature=shape.temperature,
+                       accepted_len=acc, next_token=nxt, stream=stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                t.append(e0.elapsed_time(e1) * 1e3)
+        ver.close()
+        del inp, toks
+        ks.append(kk); us.append(float(np.median(t)))
+    slope, intercept = np.polyfit(np.array(ks, float), np.array(us), 1)
+    resid = np.array(us) - (intercept + slope * np.array(ks, float))
+    return {"model": "T_cloud(K) = T_base + K * delta_cloud", "T_base_us": float(intercept),
+            "delta_cloud_us_per_token": float(slope), "k": ks, "step_us": us,
+            "max_abs_residual_us": float(np.abs(resid).max()),
+            "note": "median of 20 steps per K, batch and context of the workload; draft logits = noise only"}
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -335,6 +377,8 @@ def run_ours(args):
                        "l2": "read sweep of a 512 MiB buffer between steps, outside the event pairs"},
             "step_us": ms_per_step * 1e3,
             "step_us_median": statistics.median(step_ms) * 1e3,
+            "step_us_p10": sorted(step_ms)[len(step_ms) // 10] * 1e3,
+            "step_us_p90": sorted(step_ms)[(len(step_ms) * 9) // 10] * 1e3,
             "scored_positions_per_s": world * m_rows / (ms_per_step * 1e-3),
             "mean_tau_over_k": accept_rate,
             "algorithmic_bytes_per_step": alg_bytes,
@@ -356,6 +400,9 @@ def run_ours(args):
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl.CONFIGS[args.config])
+        if world == 1 and args.fit_k:
+            del flush
+            line["cloud_cost_fit"] = fit_cloud_cost(args, wl.CONFIGS[args.config], dev)
         print(json.dumps(line))
     ver.close()
     if world > 1:
@@ -370,6 +417,8 @@ def main():
     ap.add_argument("--config", default="llama3_8b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fit-k", action="store_true",
+                    help="also measure the step at several draft lengths and fit the paper's T_base + K*delta_cloud")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
