@@ -174,6 +174,27 @@ int flexspec_sample(flexspec_handle* h, const float* logits,
                     const uint32_t* vocab_mask,
                     int32_t* accepted_len, int32_t* next_token, void* stream);
 
+/* KV session, before the step (Section IV-C: the cloud computes the K/V pairs of the newly received
+ * tokens only).  Writes the K/V rows of the k_b + 1 window positions of every sequence into its
+ * pages: row j of sequence b goes to token position kv_len[b] - (k_b + 1) + j.
+ *   kv_pages    DEVICE bf16 pool as in flexspec_kv (written here, and only here)
+ *   new_k/new_v DEVICE bf16 [M][n_kv_heads][head_dim], rows packed like the query rows, 16-byte aligned
+ *   kv_len      DEVICE int32 [batch] = committed context + k_b + 1 (the length verification will see)
+ * The pages of the window positions must already be in the page table.  Asynchronous on `stream`.
+ * Errors: INVALID_ARG, CUDA; a page id outside the pool is recorded in the status word. */
+int flexspec_kv_append(flexspec_handle* h, void* kv_pages, int32_t num_pages, const int32_t* page_table,
+                       int32_t max_pages_per_seq, const int32_t* kv_len, const int32_t* kv_len_host,
+                       const void* new_k, const void* new_v, const int32_t* draft_len,
+                       const int32_t* draft_len_host, int32_t batch, void* stream);
+
+/* KV session, after the step (Section IV-C: on a rejection the invalid K/V pairs are discarded).
+ * With paged storage the rollback is a new length, computed on the device so that a serving loop
+ * needs no host round trip: kv_len_next[b] = kv_len[b] - (k_b + 1) + accepted_len[b] + 1, i.e. the
+ * committed context plus the accepted drafts plus the position whose K/V the next step appends
+ * first.  All pointers DEVICE int32 [batch]; kv_len_next may alias kv_len. */
+int flexspec_kv_rollback(flexspec_handle* h, const int32_t* kv_len, const int32_t* draft_len,
+                         const int32_t* accepted_len, int32_t batch, int32_t* kv_len_next, void* stream);
+
 /* The acceptance / emitted-token stage (flexspec_sample) without a handle and without any
  * allocation.  (No counterpart in the paper: it exists for how some hosts have to run.)
  * Meant for callers that cannot obtain device memory at call time: a serving process whose

@@ -60,6 +60,10 @@ def lib() -> C.CDLL:
         L.fso_accept.restype = None
         L.fso_accept.argtypes = [i32, vp, vp, vp, vp, vp, i32, i32, f64, vp, vp, i32,
                                  vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fso_kv_append.restype = None
+        L.fso_kv_append.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, vp, vp]
+        L.fso_kv_rollback.restype = None
+        L.fso_kv_rollback.argtypes = [vp, vp, vp, i32, vp]
         L.fso_num_threads.restype = i32
         _lib = L
     return _lib
@@ -184,6 +188,25 @@ def accept(mode, target_logits, draft_logits, draft_tokens, draft_len, seeds, te
                      _p(res["q_tok"]), _p(res["u"]), _p(res["acc_margin"]),
                      _p(res["cdf_margin"]), _p(res["resid_mass"]))
     return res
+
+
+def kv_append(kv_pages, page_table, kv_len, draft_len, new_k, new_v, n_kv_heads, head_dim, page_size=16):
+    """Returns a copy of the pool (uint16 bit patterns) with the window rows written (Section IV-C)."""
+    pool = np.array(kv_pages, dtype=np.uint16, copy=True)
+    page_table = _c(page_table, np.int32)
+    kv_len = _c(kv_len, np.int32)
+    draft_len = _c(draft_len, np.int32)
+    nk, nv = _c(new_k, np.uint16), _c(new_v, np.uint16)
+    lib().fso_kv_append(_p(pool), _p(page_table), int(page_table.shape[1]), _p(kv_len), _p(draft_len),
+                        int(draft_len.shape[0]), n_kv_heads, head_dim, page_size, _p(nk), _p(nv))
+    return pool
+
+
+def kv_rollback(kv_len, draft_len, accepted_len):
+    kv_len, draft_len, accepted_len = _c(kv_len, np.int32), _c(draft_len, np.int32), _c(accepted_len, np.int32)
+    out = np.empty_like(kv_len)
+    lib().fso_kv_rollback(_p(kv_len), _p(draft_len), _p(accepted_len), int(kv_len.shape[0]), _p(out))
+    return out
 
 
 def verify(mode, hidden, kv_pages, page_table, kv_len, draft_len, lm_head_w, draft_tokens,

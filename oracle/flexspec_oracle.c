@@ -358,6 +358,40 @@ void fso_accept(int32_t mode, const double* target_logits, const float* draft_lo
     free(row0); free(tok0);
 }
 
+/* ------------------------------------------------------------ KV session */
+
+void fso_kv_append(uint16_t* kv_pages, const int32_t* page_table, int32_t max_pages_per_seq,
+                   const int32_t* kv_len, const int32_t* draft_len, int32_t batch,
+                   int32_t n_kv_heads, int32_t head_dim, int32_t page_size,
+                   const uint16_t* new_k, const uint16_t* new_v)
+{
+    int64_t row = 0;
+    for (int32_t b = 0; b < batch; ++b) {
+        const int32_t k = draft_len[b];
+        const int32_t ctx = kv_len[b] - (k + 1);
+        for (int32_t j = 0; j <= k; ++j, ++row) {
+            const int32_t t = ctx + j;
+            const int64_t page = page_table[(int64_t)b * max_pages_per_seq + t / page_size];
+            const int32_t slot = t % page_size;
+            for (int32_t h = 0; h < n_kv_heads; ++h)
+                for (int32_t e = 0; e < head_dim; ++e) {
+                    const int64_t src = (row * n_kv_heads + h) * head_dim + e;
+                    kv_pages[(((page * 2 + 0) * n_kv_heads + h) * page_size + slot) * (int64_t)head_dim + e] = new_k[src];
+                    kv_pages[(((page * 2 + 1) * n_kv_heads + h) * page_size + slot) * (int64_t)head_dim + e] = new_v[src];
+                }
+        }
+    }
+}
+
+void fso_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int32_t* accepted_len,
+                     int32_t batch, int32_t* kv_len_next)
+{
+    for (int32_t b = 0; b < batch; ++b) {
+        const int32_t ctx = kv_len[b] - (draft_len[b] + 1);
+        kv_len_next[b] = ctx + accepted_len[b] + 1;
+    }
+}
+
 int32_t fso_num_threads(void)
 {
 #ifdef _OPENMP

@@ -96,6 +96,20 @@ void fso_accept(int32_t mode, const double* target_logits, const float* draft_lo
                 double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
                 double* cdf_margin, double* resid_mass);
 
+/* KV session around the step (Section IV-C).
+ * fso_kv_append: the K/V rows of the k_b + 1 window positions (new_k / new_v, bf16 bit patterns,
+ *   [M][n_kv_heads][head_dim], rows packed by sequence) are written into the pages: row j of
+ *   sequence b is token kv_len[b] - (draft_len[b] + 1) + j.  Bytes are copied, nothing is computed.
+ * fso_kv_rollback: after tau = accepted_len[b] accepted drafts the K/V of the later window
+ *   positions are invalid; the sequence keeps its committed context, the accepted drafts' positions
+ *   and position 0 of the window: kv_len_next = (kv_len - (k+1)) + tau + 1. */
+void fso_kv_append(uint16_t* kv_pages, const int32_t* page_table, int32_t max_pages_per_seq,
+                   const int32_t* kv_len, const int32_t* draft_len, int32_t batch,
+                   int32_t n_kv_heads, int32_t head_dim, int32_t page_size,
+                   const uint16_t* new_k, const uint16_t* new_v);
+void fso_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int32_t* accepted_len,
+                     int32_t batch, int32_t* kv_len_next);
+
 int32_t fso_num_threads(void);
 
 #ifdef __cplusplus

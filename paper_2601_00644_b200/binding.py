@@ -24,7 +24,8 @@ ERR_TIMEOUT, ERR_BAD_PAGE, ERR_BAD_TOKEN, ERR_NO_DEVICE = -5, -6, -7, -8
 
 EXPORTS = [
     "flexspec_create", "flexspec_verify", "flexspec_verify_host", "flexspec_attention",
-    "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_get_debug", "flexspec_status",
+    "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_kv_append",
+    "flexspec_kv_rollback", "flexspec_get_debug", "flexspec_status",
     "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
     "flexspec_destroy", "flexspec_strerror", "flexspec_version",
 ]
@@ -62,6 +63,8 @@ def _load() -> C.CDLL:
     lib.flexspec_lm_head.argtypes = [vp, vp, i32, vp, vp]
     lib.flexspec_sample.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     lib.flexspec_sample_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp]
+    lib.flexspec_kv_append.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.flexspec_kv_rollback.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     lib.flexspec_get_debug.argtypes = [vp, C.POINTER(Debug)]
     lib.flexspec_status.argtypes = [vp, vp]
     lib.flexspec_set_profiling.argtypes = [vp, i32]
@@ -245,6 +248,26 @@ class Verifier:
                                    _ptr(_dev(vocab_mask, torch.int32, "vocab_mask")),
                                    _ptr(accepted_len), _ptr(next_token), _stream_ptr(stream)), "flexspec_sample")
         return accepted_len, next_token
+
+    # ------------------------------------------------------------------ KV session
+    def kv_append(self, kv_pages, page_table, kv_len, kv_len_host, new_k, new_v, draft_len, draft_len_host, stream=None):
+        """Write the K/V rows of the window positions into the pages (before verify)."""
+        batch = int(draft_len_host.numel())
+        _dev(kv_pages, torch.bfloat16, "kv_pages"); _dev(new_k, torch.bfloat16, "new_k"); _dev(new_v, torch.bfloat16, "new_v")
+        _check(LIB.flexspec_kv_append(self._h, _ptr(kv_pages), int(kv_pages.shape[0]), _ptr(_dev(page_table, torch.int32, "page_table")),
+                                      int(page_table.shape[1]), _ptr(_dev(kv_len, torch.int32, "kv_len")),
+                                      _ptr(_host_i32(kv_len_host, "kv_len_host")), _ptr(new_k), _ptr(new_v),
+                                      _ptr(_dev(draft_len, torch.int32, "draft_len")), _ptr(_host_i32(draft_len_host, "draft_len_host")),
+                                      batch, _stream_ptr(stream)), "flexspec_kv_append")
+
+    def kv_rollback(self, kv_len, draft_len, accepted_len, kv_len_next=None, stream=None):
+        """kv_len of the next step after this step's accepted_len (device-side, no host sync)."""
+        if kv_len_next is None:
+            kv_len_next = torch.empty_like(kv_len)
+        _check(LIB.flexspec_kv_rollback(self._h, _ptr(_dev(kv_len, torch.int32, "kv_len")), _ptr(_dev(draft_len, torch.int32, "draft_len")),
+                                        _ptr(_dev(accepted_len, torch.int32, "accepted_len")), int(kv_len.numel()),
+                                        _ptr(_dev(kv_len_next, torch.int32, "kv_len_next")), _stream_ptr(stream)), "flexspec_kv_rollback")
+        return kv_len_next
 
     # ------------------------------------------------------------------ introspection
     def _view(self, ptr, shape, dtype):

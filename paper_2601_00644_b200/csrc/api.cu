@@ -538,6 +538,48 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     return FLEXSPEC_OK;
 }
 
+int flexspec_kv_append(flexspec_handle* fh, void* kv_pages, int32_t num_pages, const int32_t* page_table,
+                       int32_t max_pages_per_seq, const int32_t* kv_len, const int32_t* kv_len_host,
+                       const void* new_k, const void* new_v, const int32_t* draft_len, const int32_t* draft_len_host,
+                       int32_t batch, void* stream)
+{
+    if (fh == nullptr || kv_pages == nullptr || page_table == nullptr || kv_len == nullptr || kv_len_host == nullptr ||
+        new_k == nullptr || new_v == nullptr || draft_len == nullptr)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (num_pages < 1 || max_pages_per_seq < 1) return FLEXSPEC_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(kv_pages) | reinterpret_cast<uintptr_t>(new_k) | reinterpret_cast<uintptr_t>(new_v)) & 15u) != 0)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Geometry g;
+    int rc = check_lengths(h, draft_len_host, kv_len_host, batch, max_pages_per_seq, &g);
+    if (rc != FLEXSPEC_OK) return rc;
+    DeviceGuard guard(h.cfg.device);
+    KvAppendParams p;
+    p.kv_pages = kv_pages; p.page_table = page_table; p.kv_len = kv_len; p.draft_len = draft_len;
+    p.new_k = new_k; p.new_v = new_v;
+    p.batch = batch; p.n_kv_heads = h.cfg.n_kv_heads; p.head_dim = h.cfg.head_dim;
+    p.max_pages_per_seq = max_pages_per_seq; p.num_pages = num_pages;
+    p.status = h.status;
+    h.launches = 0;
+    if (launch_kv_append(p, g.m_rows, static_cast<cudaStream_t>(stream)) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
+    return FLEXSPEC_OK;
+}
+
+int flexspec_kv_rollback(flexspec_handle* fh, const int32_t* kv_len, const int32_t* draft_len,
+                         const int32_t* accepted_len, int32_t batch, int32_t* kv_len_next, void* stream)
+{
+    if (fh == nullptr || kv_len == nullptr || draft_len == nullptr || accepted_len == nullptr || kv_len_next == nullptr)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (batch < 1 || batch > h.cfg.max_batch) return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    if (launch_kv_rollback(kv_len, draft_len, accepted_len, batch, kv_len_next, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return FLEXSPEC_ERR_CUDA;
+    h.launches = 1;
+    return FLEXSPEC_OK;
+}
+
 int flexspec_get_debug(flexspec_handle* fh, flexspec_debug* out)
 {
     if (fh == nullptr || out == nullptr) return FLEXSPEC_ERR_INVALID_ARG;

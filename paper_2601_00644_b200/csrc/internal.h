@@ -47,6 +47,17 @@ struct AttnParams {
     int32_t* status;
 };
 
+struct KvAppendParams {
+    void* kv_pages;               // bf16 [num_pages][2][n_kv_heads][16][head_dim]
+    const int32_t* page_table;
+    const int32_t* kv_len;
+    const int32_t* draft_len;
+    const void* new_k;            // bf16 [M][n_kv_heads][head_dim]
+    const void* new_v;
+    int32_t batch, n_kv_heads, head_dim, max_pages_per_seq, num_pages;
+    int32_t* status;
+};
+
 struct LmHeadParams {
     float* logits;            // [m_rows][vocab]
     int32_t m_rows, vocab, d_model;
@@ -146,6 +157,9 @@ inline cudaError_t launch_kernel_ex(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+cudaError_t launch_kv_append(const KvAppendParams& p, int32_t m_rows, cudaStream_t stream);
+cudaError_t launch_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int32_t* accepted_len, int32_t batch,
+                               int32_t* kv_len_next, cudaStream_t stream);
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
 int attention_p_bufs(int n_pad);
 void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages);

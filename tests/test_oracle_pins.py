@@ -491,3 +491,42 @@ def test_whole_step_composition_and_rollback_contract():
     assert sub["accepted_len"][2] == res["accepted_len"][2]
     assert sub["next_token"][2] == res["next_token"][2]
     assert sub["accepted_len"][0] == -1
+
+
+# ------------------------------------------------------------- KV session
+
+def test_kv_append_and_rollback_against_direct_indexing():
+    """Section IV-C: the window's K/V rows land at positions ctx .. ctx+k of the sequence (checked by
+    reading them back through the page table with plain numpy indexing, and by the fact that attention
+    over the appended pool equals attention over a pool that held those rows all along); the rollback
+    keeps context + accepted drafts + the window's first position."""
+    rng = np.random.RandomState(21)
+    hq, hkv, dh = 4, 2, 16
+    k = np.array([3, 0, 5], np.int32)
+    ctx = np.array([20, 9, 33], np.int32)
+    hidden, kv, pt, kv_len, k2 = _attn_case(rng, 3, hq, hkv, dh, list(k), list(ctx))
+    assert np.array_equal(k, k2)
+    m = int(k.sum()) + 3
+    new_k = rng.randint(0, 2 ** 15, (m, hkv, dh)).astype(np.uint16)
+    new_v = rng.randint(0, 2 ** 15, (m, hkv, dh)).astype(np.uint16)
+    pool = oracle.kv_append(kv, pt, kv_len, k, new_k, new_v, hkv, dh)
+    touched = np.zeros(kv.shape, bool)
+    row = 0
+    for b in range(3):
+        for j in range(k[b] + 1):
+            t = kv_len[b] - (k[b] + 1) + j
+            page, slot = pt[b, t // 16], t % 16
+            assert np.array_equal(pool[page, 0, :, slot, :], new_k[row])
+            assert np.array_equal(pool[page, 1, :, slot, :], new_v[row])
+            touched[page, :, :, slot, :] = True
+            row += 1
+    assert np.array_equal(pool[~touched], kv[~touched])            # nothing else was written
+    # attention sees exactly the appended rows
+    a_new, _ = oracle.attention(hidden, pool, pt, kv_len, k, hq, hkv, dh)
+    a_old, _ = oracle.attention(hidden, kv, pt, kv_len, k, hq, hkv, dh)
+    assert not np.allclose(a_new, a_old)
+    # rollback: all accepted keeps everything but the bonus position's successor; none accepted keeps ctx + 1
+    acc = np.array([3, 0, 2], np.int32)
+    nxt = oracle.kv_rollback(kv_len, k, acc)
+    assert list(nxt) == [20 + 3 + 1, 9 + 0 + 1, 33 + 2 + 1]
+    assert np.all(nxt <= kv_len) and np.all(nxt >= kv_len - k)
