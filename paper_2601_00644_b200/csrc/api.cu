@@ -178,7 +178,8 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, const S
     else { p.n_tile = 256; p.n_blocks = 2; }
     const int rows_per_pass = p.n_tile * p.n_blocks;
     p.n_pass = (m_rows + rows_per_pass - 1) / rows_per_pass;
-    p.n_vtiles = (c.vocab + 127) / 128;
+    if (p.n_pass == 1) { p.n_full_tiles = h.lm_full_tiles; p.last_rows = h.lm_last_rows; p.n_vtiles = h.lm_full_tiles + h.lm_last_tiles; }
+    else { p.n_vtiles = (c.vocab + 127) / 128; p.n_full_tiles = p.n_vtiles; p.last_rows = 128; }
     p.num_stages = lm_head_pick_stages(p.n_tile, p.n_blocks);
     p.acc_stages = (2 * rows_per_pass <= 512) ? 2 : 1;
     p.tstats = nullptr; p.n_tparts = 0; p.inv_temp_log2 = 1.f; p.greedy = 0;
@@ -296,6 +297,20 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     h.w = static_cast<const __nv_bfloat16*>(lm_head_w);
 
     const int n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
+    // LM-head tiling: full waves of 128-row tiles, then one wave of shorter tiles, one per SM, so that
+    // the last wave ends everywhere at the same time
+    {
+        const int tiles128 = (c.vocab + 127) / 128;
+        h.lm_full_tiles = tiles128; h.lm_last_rows = 128; h.lm_last_tiles = 0;
+        if (tiles128 > h.sm_count && tiles128 % h.sm_count != 0) {
+            h.lm_full_tiles = tiles128 / h.sm_count * h.sm_count;
+            const int rows_rem = c.vocab - h.lm_full_tiles * 128;
+            int lr = ((rows_rem + h.sm_count - 1) / h.sm_count + 7) / 8 * 8;
+            if (lr > 128) lr = 128;
+            h.lm_last_rows = lr;
+            h.lm_last_tiles = (rows_rem + lr - 1) / lr;
+        }
+    }
     int rc = FLEXSPEC_OK;
     auto A = [&](int r) { if (rc == FLEXSPEC_OK) rc = r; };
     A(dev_alloc(&h.attn_out, static_cast<size_t>(max_m) * d_model));
@@ -312,7 +327,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
     A(dev_alloc(&h.stats, static_cast<size_t>(max_m + h.max_s) * n_chunks));
-    A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128)));
+    A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128 + h.sm_count)));
     A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
     A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 4));
     A(dev_alloc(&h.row_stats, static_cast<size_t>(c.max_batch) * (kMaxK + 1) * 8));
@@ -343,6 +358,8 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
         rc = FLEXSPEC_ERR_CUDA;
     if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map, lm_head_w, static_cast<uint64_t>(c.vocab),
                                             static_cast<uint64_t>(d_model), 128);
+    if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map_last, lm_head_w, static_cast<uint64_t>(c.vocab),
+                                            static_cast<uint64_t>(d_model), static_cast<uint32_t>(h.lm_last_rows));
     if (rc == FLEXSPEC_OK && (attention_init(c.head_dim) != cudaSuccess || lm_head_init() != cudaSuccess))
         rc = FLEXSPEC_ERR_CUDA;
     if (rc != FLEXSPEC_OK) {
@@ -470,7 +487,8 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     // the second stream's work is long done by now; joining here keeps LM head -> decision -> draw
     // back to back on this stream, so that the last two can be launched programmatically
     if (cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    sp.tstats = h.tstats; sp.n_tparts = 4 * ((h.cfg.vocab + 127) / 128);     // the LM head leaves the target rows' parts
+    sp.tstats = h.tstats;                                                     // the LM head leaves the target rows' parts
+    sp.n_tparts = 4 * (g.m_rows <= 512 ? h.lm_full_tiles + h.lm_last_tiles : (h.cfg.vocab + 127) / 128);
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);

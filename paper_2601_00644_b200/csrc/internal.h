@@ -64,7 +64,9 @@ struct LmHeadParams {
     int32_t n_tile;           // token columns per accumulator block (multiple of 16, <= 256)
     int32_t n_blocks;         // accumulator blocks per pass (1 or 2)
     int32_t n_pass;           // passes over W when m_rows > n_tile * n_blocks
-    int32_t n_vtiles;         // ceil(vocab / 128)
+    int32_t n_vtiles;         // vocabulary tiles: n_full_tiles of 128 rows, then tiles of last_rows rows
+    int32_t n_full_tiles;
+    int32_t last_rows;        // height of the tiles of the last wave (multiple of 8, <= 128)
     int32_t num_stages;       // shared-memory pipeline depth
     int32_t acc_stages;       // TMEM accumulator buffers (1 or 2)
     // optional: softmax statistics of the rows, one part per (row, 32 vocabulary rows), for the
@@ -113,6 +115,8 @@ struct Handle {
     int32_t sm_count;
     const __nv_bfloat16* w;
     CUtensorMap w_map;
+    CUtensorMap w_map_last;   // same tensor, box of lm_last_rows rows (tiles of the last wave)
+    int32_t lm_full_tiles, lm_last_rows, lm_last_tiles;
     // workspace
     __nv_bfloat16* attn_out;
     float* logits;

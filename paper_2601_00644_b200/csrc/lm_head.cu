@@ -45,8 +45,8 @@ size_t lm_head_smem_bytes(int n_tile, int n_blocks, int num_stages)
 }
 
 __global__ void __launch_bounds__(kLmThreads, 1)
-lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
-               const LmHeadParams p)
+lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap w_map_last,
+               const __grid_constant__ CUtensorMap x_map, const LmHeadParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -67,6 +67,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
         for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
         fence_barrier_init();
         tma_prefetch_desc(&w_map);
+        tma_prefetch_desc(&w_map_last);
         tma_prefetch_desc(&x_map);
     }
     if (warp == 1) {
@@ -80,6 +81,11 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 
     const int num_kb = p.d_model / kLmBlockK;
     const int total_tiles = p.n_vtiles * p.n_pass;
+    // Vocabulary tile vt: the first n_full_tiles are 128 rows high; the tiles of the last wave are
+    // last_rows high (one per CTA, so that the wave ends everywhere at the same time).
+    auto tile_row0 = [&](int vt) {
+        return vt < p.n_full_tiles ? vt * kLmBlockV : p.n_full_tiles * kLmBlockV + (vt - p.n_full_tiles) * p.last_rows;
+    };
     const int acc_cols = p.n_blocks * p.n_tile;        // TMEM columns of one accumulator buffer
     const int rows_per_pass = acc_cols;
 
@@ -98,8 +104,10 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, p.status, 2)) { ok = false; break; }
                     uint8_t* st = smem + s * stage_bytes;
-                    mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(stage_bytes));
-                    tma_load_2d(st, &w_map, &full_bar[s], kb * kLmBlockK, vt * kLmBlockV, pol_w);
+                    const bool full_tile = vt < p.n_full_tiles;
+                    mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(full_tile ? stage_bytes
+                                                                                          : p.last_rows * 128 + b_bytes));
+                    tma_load_2d(st, full_tile ? &w_map : &w_map_last, &full_bar[s], kb * kLmBlockK, tile_row0(vt), pol_w);
                     for (int nb = 0; nb < p.n_blocks; ++nb)
                         tma_load_2d(st + kLmATileBytes + nb * p.n_tile * 128, &x_map, &full_bar[s], kb * kLmBlockK,
                                     pass * rows_per_pass + nb * p.n_tile, pol_x);
@@ -154,7 +162,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             const int vt = tile / p.n_pass, pass = tile % p.n_pass;
             if (!mbar_wait(&tmem_full[a], aph, p.status, 6)) { ok = false; break; }
             tc_fence_after();
-            const int v = vt * kLmBlockV + quarter * 32 + lane;
+            const int tile_rows = vt < p.n_full_tiles ? kLmBlockV : p.last_rows;
+            const int v = (quarter * 32 + lane < tile_rows) ? tile_row0(vt) + quarter * 32 + lane : p.vocab;   // past the tile: not a row
             const int row_base = pass * rows_per_pass;
             const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                     static_cast<uint32_t>(a * acc_cols);
@@ -193,7 +202,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const unsigned eq = __ballot_sync(0xffffffffu, zv[i] == mx[i]);
-                            sc[i] = __int_as_float(vt * kLmBlockV + quarter * 32 + __ffs(eq) - 1);
+                            sc[i] = __int_as_float(tile_row0(vt) + quarter * 32 + __ffs(eq) - 1);
                         }
                     } else {
 #pragma unroll
@@ -238,7 +247,7 @@ cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHe
     const int total_tiles = p.n_vtiles * p.n_pass;
     const int grid = total_tiles < h.sm_count ? total_tiles : h.sm_count;
     const size_t smem = lm_head_smem_bytes(p.n_tile, p.n_blocks, p.num_stages);
-    lm_head_kernel<<<grid, kLmThreads, smem, stream>>>(h.w_map, x_map, p);
+    lm_head_kernel<<<grid, kLmThreads, smem, stream>>>(h.w_map, h.w_map_last, x_map, p);
     return cudaGetLastError();
 }
 
