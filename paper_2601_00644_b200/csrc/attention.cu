@@ -24,7 +24,7 @@
 //
 // Warp roles.  Warps 0-1: TMA producers, each owning half of every block's pages (a TMA request
 // costs about 55 cycles of the issuing warp, and a block needs 32 of them); separate rings of
-// 128-token K and V tiles; an L2 prefetch of the pages runs several blocks ahead of the copies.
+// 128-token K and V tiles; the page ids of the next block are looked up one block ahead.
 // Warp 2: one thread issues every tcgen05.mma; the warp owns the TMEM allocation.  Warps 3-6: softmax,
 // thread t = token t of the block (TMEM lane t of S^T).  The maximum of a query row over the
 // block is a column maximum: redux.sync.max over each warp, then over the four warps through
@@ -48,7 +48,6 @@ constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column of
 constexpr float kRescaleThreshold = 8.f;                             // log2 units
 constexpr int kAttSmemLimit = 232448;                                // 227 KB opt-in maximum per CTA
 constexpr int kAttStaticReserve = 1024;                              // __shared__ variables of the kernel
-constexpr int kAttPrefetchBlocks = 4;                                // how far ahead of the copies the L2 prefetch runs
 
 struct AttBars {
     uint64_t k_full[kAttMaxStages], k_empty[kAttMaxStages];
@@ -83,7 +82,7 @@ struct AttCfg {
 // the widest tile leaves room for enough K/V tiles only with a single P^T buffer
 int attention_p_bufs(int n_pad) { return n_pad > 112 ? 1 : 2; }
 
-// ring depths that fit: two K tiles when there is room for at least four tiles, the rest V
+// ring depths that fit: K gets two tiles of four or five, three of six or more; V gets the rest
 void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages)
 {
     const int pb = attention_p_bufs(n_pad);
@@ -91,6 +90,7 @@ void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages)
     const int fixed = head_dim == 128 ? AttCfg<128>::fixed_bytes(n_pad, pb) : AttCfg<64>::fixed_bytes(n_pad, pb);
     const int tiles = (kAttSmemLimit - kAttStaticReserve - fixed) / tile;
     int ks = tiles >= 4 ? 2 : 1;
+    if (tiles >= 6) ks = 3;                       // measured: 3 + 3 beats 2 + 4 by ~0.5 us at the 8B shape
     int vs = tiles - ks;
     if (vs > kAttMaxStages) vs = kAttMaxStages;
     *k_stages = ks;
@@ -742,11 +742,11 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         int (*ring)[2 * PW] = s_phys[warp];
         bool new_pair = true;
         bool ok = true;
-        // A second cursor runs kAttPrefetchBlocks ahead of the copies.  It looks the page ids up (one
-        // page-table read per block, kept in a small shared-memory ring until the copy needs them;
-        // the read for the next block is always in flight while this block is handled) and asks for
-        // the pages to be brought into L2: a tile's shared-memory slot is then busy for an L2 hit,
-        // not for a trip to HBM, so the rings that fit in shared memory keep HBM streaming.
+        // A second cursor runs one block ahead of the copies and looks the page ids up (one page-table
+        // read per block, kept in a small shared-memory ring until the copy needs them; the read for
+        // the next block is in flight while this block is handled).  (Asking for the pages to be
+        // brought into L2 further ahead was measured and did not pay: 4 blocks ahead cost 1.7 us per
+        // step at the 8B shape, 8 blocks 3 us.)
         AttCursor pf = cur;
         int pf_q = 0;
         auto pf_load = [&](const AttCursor& c) -> int {
@@ -755,26 +755,11 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
             return (lane < 2 * PW && my_page < pnpg)
                        ? p.page_table[static_cast<int64_t>(c.b) * p.max_pages_per_seq + c.blk * kAttPagesPerStage + my_page] : -1;
         };
-        const int lines_per_tile_page = kPageTokens * DH * 2 / 128;        // 128-byte lines of one page's K (or V), one kv head
         auto pf_issue = [&](int ph) {
             if (lane < 2 * PW) ring[pf_q & 7][lane] = ph;
-            const int pkvh = pf.pair / pf.rbc;
-            // plain per-line prefetches from all lanes: the TMA path is kept for the copies
-#pragma unroll
-            for (int pg = 0; pg < PW; ++pg) {
-                const int id = __shfl_sync(0xffffffffu, ph, 2 * pg);
-                if (id >= 0 && id < p.num_pages && lane < lines_per_tile_page) {
-                    const uint8_t* kb = p.kv_pages + (static_cast<int64_t>(id * 2 + 0) * p.n_kv_heads + pkvh) * (kPageTokens * DH * 2);
-                    const uint8_t* vb = p.kv_pages + (static_cast<int64_t>(id * 2 + 1) * p.n_kv_heads + pkvh) * (kPageTokens * DH * 2);
-                    prefetch_l2(kb + lane * 128);
-                    prefetch_l2(vb + lane * 128);
-                }
-            }
             ++pf_q;
             pf.advance(p, pf_q < n_my);
         };
-        // the cursor starts one block ahead (the first copy must not wait for more than its own page ids)
-        // and gains a block per iteration until it runs kAttPrefetchBlocks ahead
         int pf_ph = pf_load(pf);
         pf_issue(pf_ph);
         pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
@@ -820,7 +805,7 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
                             ((phys * 2 + 1) * p.n_kv_heads + kvh) * kPageTokens, pol);
             __syncwarp();
 #pragma unroll 1
-            for (int step = 0; step < 2 && pf_q < n_my && pf_q <= q + kAttPrefetchBlocks; ++step) {
+            for (int step = 0; step < 2 && pf_q < n_my && pf_q <= q + 1; ++step) {
                 pf_issue(pf_ph);
                 pf_ph = (pf_q < n_my) ? pf_load(pf) : -1;
             }
