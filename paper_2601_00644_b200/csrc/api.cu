@@ -145,7 +145,6 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     if (rc != FLEXSPEC_OK) return rc;
 
     AttnParams p;
-    p.kv_pages = static_cast<const uint8_t*>(kv->kv_pages);
     p.hidden = static_cast<const __nv_bfloat16*>(hidden);
     p.page_table = kv->page_table;
     p.kv_len = kv->kv_len;

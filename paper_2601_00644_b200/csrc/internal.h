@@ -28,7 +28,6 @@ struct Plan {                 // device tables written by the plan kernel, read 
 };
 
 struct AttnParams {
-    const uint8_t* kv_pages;  // the pool (also described by the tensor map), for L2 prefetches
     const __nv_bfloat16* hidden;
     const int32_t* page_table;
     const int32_t* kv_len;
