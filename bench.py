@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch at the default
 # workload, from the ncu capture summarised in profiles/ (None until captured)
-LM_HEAD_TRAFFIC_BYTES = 1051824000 + 8016128
+LM_HEAD_TRAFFIC_BYTES = 1051930000 + 8530432
 FALLBACK_HBM_GBS = 6650.0
 REFERENCE_BUDGET_S = 120.0
 
