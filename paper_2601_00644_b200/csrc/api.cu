@@ -535,13 +535,23 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     auto H2D = [&](void* dst, const void* src, size_t bytes) {
         if (bytes > 0 && src != nullptr) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
     };
+    // The draft logits are by far the largest input and nothing on the main stream needs them before the
+    // decision: they are copied on the second stream, beside attention and the LM head (the statistics
+    // kernel that reads them runs on that stream, behind the copy).
     H2D(d_hidden, hidden, static_cast<size_t>(g.m_rows) * h.d_model * 2);
-    H2D(d_dlog, draft_logits, static_cast<size_t>(g.s_rows) * h.cfg.vocab * 4);
     H2D(d_tok, draft_tokens, static_cast<size_t>(g.s_rows) * 4);
     H2D(d_len, draft_len, static_cast<size_t>(batch) * 4);
     H2D(d_kvl, kv->kv_len_host, static_cast<size_t>(batch) * 4);
     H2D(d_seed, seeds, static_cast<size_t>(batch) * 8);
     if (!ok) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+    if (draft_logits != nullptr && g.s_rows > 0) {
+        if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess ||
+            cudaMemcpyAsync(d_dlog, draft_logits, static_cast<size_t>(g.s_rows) * h.cfg.vocab * 4, cudaMemcpyHostToDevice,
+                            h.side) != cudaSuccess) {
+            cudaGetLastError();
+            return FLEXSPEC_ERR_CUDA;
+        }
+    }
 
     flexspec_kv kv_dev = *kv;
     kv_dev.kv_len = d_kvl;
