@@ -174,6 +174,7 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, const S
     p.m_rows = m_rows; p.vocab = c.vocab; p.d_model = h.d_model;
     const int m16 = (m_rows + 15) / 16 * 16;
     if (m16 <= 256) { p.n_tile = m16; p.n_blocks = 1; }
+    else if (m16 <= 512) { p.n_blocks = 2; p.n_tile = ((m_rows + 1) / 2 + 15) / 16 * 16; }   // two blocks that just cover the rows
     else { p.n_tile = 256; p.n_blocks = 2; }
     const int rows_per_pass = p.n_tile * p.n_blocks;
     p.n_pass = (m_rows + rows_per_pass - 1) / rows_per_pass;
