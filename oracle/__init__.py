@@ -58,8 +58,10 @@ def lib() -> C.CDLL:
         L.fso_softmax.restype = None
         L.fso_softmax.argtypes = [vp, i32, f64, vp, vp]
         L.fso_accept.restype = None
-        L.fso_accept.argtypes = [i32, vp, vp, vp, vp, vp, i32, i32, f64, vp, vp, i32,
-                                 vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fso_accept.argtypes = [i32, vp, vp, vp, vp, vp, i32, i32, f64, f64, vp, vp, i32,
+                                 vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fso_nucleus.restype = None
+        L.fso_nucleus.argtypes = [vp, i32, f64, vp]
         L.fso_kv_append.restype = None
         L.fso_kv_append.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, vp, vp]
         L.fso_kv_rollback.restype = None
@@ -154,8 +156,16 @@ def softmax(z, temperature=1.0, mask=None):
     return out
 
 
+def nucleus(prob, top_p):
+    """Top-p filtered and renormalised copy of a distribution; returns (prob', margin)."""
+    p = np.array(prob, dtype=np.float64, copy=True)
+    m = np.zeros(1, dtype=np.float64)
+    lib().fso_nucleus(_p(p), int(p.size), float(top_p), _p(m))
+    return p, float(m[0])
+
+
 def accept(mode, target_logits, draft_logits, draft_tokens, draft_len, seeds, temperature=1.0,
-           vocab_mask=None, seq_sel=None):
+           vocab_mask=None, seq_sel=None, top_p=1.0):
     """Acceptance loop + emitted token.  Returns a dict of numpy arrays."""
     zt = _c(target_logits, np.float64)
     zd = _c(draft_logits, np.float32)
@@ -181,12 +191,13 @@ def accept(mode, target_logits, draft_logits, draft_tokens, draft_len, seeds, te
         "acc_margin": np.full(s, np.inf, dtype=np.float64),
         "cdf_margin": np.full(batch, np.inf, dtype=np.float64),
         "resid_mass": np.zeros(batch, dtype=np.float64),
+        "topp_margin": np.full(s + batch, np.inf, dtype=np.float64),
     }
     lib().fso_accept(int(mode), _p(zt), _p(zd), _p(x), _p(k), _p(seeds), batch, vocab,
-                     float(temperature), _p(mask), _p(sel), 0 if sel is None else int(sel.size),
+                     float(temperature), float(top_p), _p(mask), _p(sel), 0 if sel is None else int(sel.size),
                      _p(res["accepted_len"]), _p(res["next_token"]), _p(res["p_tok"]),
                      _p(res["q_tok"]), _p(res["u"]), _p(res["acc_margin"]),
-                     _p(res["cdf_margin"]), _p(res["resid_mass"]))
+                     _p(res["cdf_margin"]), _p(res["resid_mass"]), _p(res["topp_margin"]))
     return res
 
 

@@ -223,6 +223,44 @@ void fso_softmax(const double* z, int32_t vocab, double temperature,
     for (int32_t v = 0; v < vocab; ++v) prob[v] = prob[v] / denom;
 }
 
+/* --------------------------------------------------------------- nucleus */
+
+typedef struct { double p; int32_t v; } fso_pv;
+static int cmp_pv_desc(const void* a, const void* b)
+{
+    const fso_pv* x = (const fso_pv*)a;
+    const fso_pv* y = (const fso_pv*)b;
+    if (x->p > y->p) return -1;
+    if (x->p < y->p) return 1;
+    return (x->v > y->v) - (x->v < y->v);
+}
+
+void fso_nucleus(double* prob, int32_t vocab, double top_p, double* margin)
+{
+    if (margin) *margin = INFINITY;
+    if (!(top_p < 1.0)) return;
+    fso_pv* s = (fso_pv*)malloc(sizeof(fso_pv) * (size_t)vocab);
+    for (int32_t v = 0; v < vocab; ++v) { s[v].p = prob[v]; s[v].v = v; }
+    qsort(s, (size_t)vocab, sizeof(fso_pv), cmp_pv_desc);
+    double c = 0.0, c_prev = 0.0;
+    int32_t m = 0;
+    for (; m < vocab; ++m) {
+        c_prev = c;
+        c += s[m].p;
+        if (c >= top_p) break;
+    }
+    if (m == vocab) m = vocab - 1;
+    const double thr = s[m].p;
+    if (margin) {
+        const double a = fabs(c - top_p), b = fabs(top_p - c_prev);
+        *margin = a < b ? a : b;
+    }
+    double z = 0.0;
+    for (int32_t v = 0; v < vocab; ++v) z += (prob[v] >= thr && prob[v] > 0.0) ? prob[v] : 0.0;
+    for (int32_t v = 0; v < vocab; ++v) prob[v] = (prob[v] >= thr && prob[v] > 0.0) ? prob[v] / z : 0.0;
+    free(s);
+}
+
 /* ------------------------------------------------- acceptance + emission */
 
 static int32_t argmax_lowest(const double* z, int32_t vocab, const uint32_t* mask)
@@ -255,8 +293,8 @@ static int32_t inverse_cdf(const double* r, int32_t vocab, double thr,
 }
 
 static void verify_one(int32_t mode, const double* zt, const float* zd, const int32_t* x,
-                       int32_t k, int32_t vocab, double temperature, uint64_t seed,
-                       const uint32_t* mask,
+                       int32_t k, int32_t vocab, double temperature, double top_p, uint64_t seed,
+                       const uint32_t* mask, double* topp_margin,
                        int32_t* accepted_len, int32_t* next_token,
                        double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
                        double* cdf_margin, double* resid_mass)
@@ -280,6 +318,7 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
     int32_t n = k;
     for (int32_t j = 0; j < k; ++j) {
         fso_softmax(zt + (int64_t)j * vocab, vocab, temperature, mask, p);
+        fso_nucleus(p, vocab, top_p, topp_margin ? topp_margin + j : NULL);
         for (int32_t v = 0; v < vocab; ++v) zq[v] = (double)zd[(int64_t)j * vocab + v];
         fso_softmax(zq, vocab, temperature, NULL, q);
         const double u = fso_uniform(seed, (uint32_t)j, 0u);
@@ -297,6 +336,7 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
 
     /* emitted token: residual at the first rejection, else the bonus row */
     fso_softmax(zt + (int64_t)n * vocab, vocab, temperature, mask, p);
+    fso_nucleus(p, vocab, top_p, topp_margin ? topp_margin + n : NULL);
     double z_mass = 0.0;
     if (n < k) {
         for (int32_t v = 0; v < vocab; ++v) zq[v] = (double)zd[(int64_t)n * vocab + v];
@@ -326,11 +366,11 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
 
 void fso_accept(int32_t mode, const double* target_logits, const float* draft_logits,
                 const int32_t* draft_tokens, const int32_t* draft_len, const uint64_t* seeds,
-                int32_t batch, int32_t vocab, double temperature, const uint32_t* vocab_mask,
+                int32_t batch, int32_t vocab, double temperature, double top_p, const uint32_t* vocab_mask,
                 const int32_t* seq_sel, int32_t n_sel,
                 int32_t* accepted_len, int32_t* next_token,
                 double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
-                double* cdf_margin, double* resid_mass)
+                double* cdf_margin, double* resid_mass, double* topp_margin)
 {
     int64_t* row0 = (int64_t*)malloc(sizeof(int64_t) * (size_t)(batch + 1));
     int64_t* tok0 = (int64_t*)malloc(sizeof(int64_t) * (size_t)(batch + 1));
@@ -348,8 +388,9 @@ void fso_accept(int32_t mode, const double* target_logits, const float* draft_lo
         verify_one(mode,
                    target_logits + row0[b] * vocab,
                    draft_logits ? draft_logits + t0 * vocab : NULL,
-                   draft_tokens + t0, draft_len[b], vocab, temperature, seeds ? seeds[b] : 0,
+                   draft_tokens + t0, draft_len[b], vocab, temperature, top_p, seeds ? seeds[b] : 0,
                    vocab_mask ? vocab_mask + (int64_t)b * mask_words : NULL,
+                   topp_margin ? topp_margin + row0[b] : NULL,
                    accepted_len + b, next_token + b,
                    p_tok ? p_tok + t0 : NULL, q_tok ? q_tok + t0 : NULL,
                    u_acc ? u_acc + t0 : NULL, acc_margin ? acc_margin + t0 : NULL,

@@ -71,7 +71,17 @@ void fso_lm_head(const uint16_t* x, const uint16_t* w, int32_t m, int32_t d, int
 void fso_softmax(const double* z, int32_t vocab, double temperature,
                  const uint32_t* mask, double* prob);
 
-/* Acceptance + emitted token for a batch of sequences.
+/* Nucleus (top-p) filter of a distribution, the sampling rule of the paper's stochastic regime
+ * (Section V: T = 1, top-p 0.9): with the tokens ordered by decreasing probability (ties: lower
+ * index first), m is the smallest prefix length whose mass reaches top_p; every token whose
+ * probability is at least that of the m-th token is kept (so ties with the m-th token are all
+ * kept), the rest get probability 0 and the kept ones are renormalised.  top_p >= 1 leaves prob
+ * untouched.  margin (may be NULL) receives the distance of top_p from the nearer of the two
+ * cumulative sums around the cut, i.e. how close the cut was to falling one token earlier/later. */
+void fso_nucleus(double* prob, int32_t vocab, double top_p, double* margin);
+
+/* Acceptance + emitted token for a batch of sequences.  With top_p < 1 the TARGET distribution of
+ * every row is its nucleus (SAMPLE mode only).
  * mode 0 = SAMPLE: accept x_j iff u_j * q_j(x_j) < p_j(x_j); after n accepted
  *   drafts emit a token from max(0, p_n - q_n)/Z (n < k) or from p_k (n == k)
  *   by inverse CDF in vocabulary order: min{v : sum_{w<=v} r_w > u' * Z}.
@@ -90,11 +100,11 @@ void fso_softmax(const double* z, int32_t vocab, double temperature,
  *     interval, divided by Z;  resid_mass[b] = Z. */
 void fso_accept(int32_t mode, const double* target_logits, const float* draft_logits,
                 const int32_t* draft_tokens, const int32_t* draft_len, const uint64_t* seeds,
-                int32_t batch, int32_t vocab, double temperature, const uint32_t* vocab_mask,
+                int32_t batch, int32_t vocab, double temperature, double top_p, const uint32_t* vocab_mask,
                 const int32_t* seq_sel, int32_t n_sel,
                 int32_t* accepted_len, int32_t* next_token,
                 double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
-                double* cdf_margin, double* resid_mass);
+                double* cdf_margin, double* resid_mass, double* topp_margin /* [M] or NULL */);
 
 /* KV session around the step (Section IV-C).
  * fso_kv_append: the K/V rows of the k_b + 1 window positions (new_k / new_v, bf16 bit patterns,

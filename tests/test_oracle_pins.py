@@ -530,3 +530,60 @@ def test_kv_append_and_rollback_against_direct_indexing():
     nxt = oracle.kv_rollback(kv_len, k, acc)
     assert list(nxt) == [20 + 3 + 1, 9 + 0 + 1, 33 + 2 + 1]
     assert np.all(nxt <= kv_len) and np.all(nxt >= kv_len - k)
+
+
+# ------------------------------------------------------------------ top-p
+
+def test_nucleus_against_numpy_sort_and_its_invariants():
+    rng = np.random.RandomState(31)
+    for v, top_p in [(7, 0.5), (50, 0.9), (1000, 0.9), (1000, 0.3), (64, 0.999)]:
+        p = rng.dirichlet(np.ones(v) * 0.3)
+        got, margin = oracle.nucleus(p, top_p)
+        order = np.lexsort((np.arange(v), -p))                    # decreasing p, ties by index
+        c = np.cumsum(p[order])
+        m = int(np.searchsorted(c, top_p, side="left"))           # first prefix with mass >= top_p
+        keep = p >= p[order[m]]
+        want = np.where(keep, p, 0.0) / p[keep].sum()
+        assert np.allclose(got, want, rtol=0, atol=1e-15)
+        assert abs(got.sum() - 1) < 1e-12
+        assert p[keep].sum() >= top_p and (m == 0 or c[m - 1] < top_p)   # minimal prefix
+        assert np.isclose(margin, min(abs(c[m] - top_p), abs(top_p - (c[m - 1] if m else 0.0))))
+    # ties with the last kept token are all kept; top_p >= 1 is the identity
+    p = np.array([0.4, 0.2, 0.2, 0.2])
+    got, _ = oracle.nucleus(p, 0.5)
+    assert np.allclose(got, [0.4, 0.2, 0.2, 0.2])
+    got, _ = oracle.nucleus(p, 0.3)
+    assert np.allclose(got, [1, 0, 0, 0])
+    got, m = oracle.nucleus(p, 1.0)
+    assert np.array_equal(got, p) and m == np.inf
+
+
+def test_top_p_sampling_is_lossless_with_respect_to_the_nucleus():
+    """With top_p < 1 the emitted token follows the nucleus of the target row (chi-square, 4*10^5
+    trials), a draft token outside the nucleus is always rejected, and top_p = 1 changes nothing."""
+    rng = np.random.RandomState(32)
+    v, n = 12, 400_000
+    p0 = rng.dirichlet(np.ones(v) * 0.7)
+    p1 = rng.dirichlet(np.ones(v) * 0.7)
+    q0 = rng.dirichlet(np.ones(v) * 0.7)
+    top_p = 0.8
+    zt = np.tile(np.stack([_logits_for(p0), _logits_for(p1)]), (n, 1))
+    zd32 = _logits_for(q0).astype(np.float32)
+    q_seen = scipy.special.softmax(zd32.astype(np.float64))
+    zd = np.tile(zd32[None, :], (n, 1))
+    toks = rng.choice(v, size=n, p=q_seen).astype(np.int32)
+    seeds = rng.randint(0, 2 ** 62, n).astype(np.uint64)
+    res = oracle.accept(oracle.SAMPLE, zt, zd, toks, np.ones(n, np.int32), seeds, top_p=top_p)
+    nuc0, _ = oracle.nucleus(p0, top_p)
+    first = np.where(res["accepted_len"] >= 1, toks, res["next_token"])
+    counts = np.bincount(first, minlength=v).astype(np.float64)
+    assert np.all(counts[nuc0 == 0] == 0)                          # nothing outside the nucleus is ever emitted
+    sup = nuc0 > 0
+    chi = ((counts[sup] - n * nuc0[sup]) ** 2 / (n * nuc0[sup])).sum()
+    assert chi < scipy.stats.chi2.ppf(0.999, int(sup.sum()) - 1), chi
+    outside = (nuc0[toks] == 0)
+    assert outside.any() and np.all(res["accepted_len"][outside] == 0)
+    assert np.allclose(res["p_tok"], nuc0[toks])
+    same = oracle.accept(oracle.SAMPLE, zt[:2000], zd[:1000], toks[:1000], np.ones(1000, np.int32), seeds[:1000], top_p=1.0)
+    base = oracle.accept(oracle.SAMPLE, zt[:2000], zd[:1000], toks[:1000], np.ones(1000, np.int32), seeds[:1000])
+    assert np.array_equal(same["next_token"], base["next_token"]) and np.array_equal(same["accepted_len"], base["accepted_len"])
