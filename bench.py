@@ -261,6 +261,8 @@ def run_ours(args):
     ver = binding.Verifier(inp.lm_head_w, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                            max_batch=batch, k_max=int(k_host.max()), max_kv_len=int(kv_host.max()))
 
+    if args.top_p < 1.0:
+        ver.set_top_p(args.top_p)
     # draft logits = target logits (from this library's attention + LM head) + sigma * noise
     attn = ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, kv_host, inp.hidden, inp.draft_len, k_host)
     tgt = ver.lm_head(attn)
@@ -373,7 +375,7 @@ def run_ours(args):
             "config": {"workload": shape.name, "batch_per_gpu": batch, "k": [int(k_host.min()), int(k_host.max())],
                        "context": [shape.ctx_min, shape.ctx_max], "vocab": v, "d_model": d,
                        "heads": [shape.n_q_heads, shape.n_kv_heads, shape.head_dim],
-                       "temperature": shape.temperature, "mode": "sample",
+                       "temperature": shape.temperature, "mode": "sample", "top_p": args.top_p,
                        "l2": "read sweep of a 512 MiB buffer between steps, outside the event pairs"},
             "step_us": ms_per_step * 1e3,
             "step_us_median": statistics.median(step_ms) * 1e3,
@@ -417,6 +419,8 @@ def main():
     ap.add_argument("--config", default="llama3_8b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--top-p", type=float, default=1.0,
+                    help="nucleus sampling of the target (the paper's stochastic regime uses 0.9); 1.0 = off")
     ap.add_argument("--fit-k", action="store_true",
                     help="also measure the step at several draft lengths and fit the paper's T_base + K*delta_cloud")
     args = ap.parse_args()

@@ -222,6 +222,14 @@ int flexspec_sample_static(const float* logits, const int32_t* draft_tokens, con
                            const uint32_t* vocab_mask, int32_t* accepted_len, int32_t* next_token,
                            void* stream);
 
+/* Nucleus (top-p) sampling of the target, the paper's stochastic regime (Section V: T = 1,
+ * top-p 0.9).  From the next verify / sample call on, the target distribution of every row is its
+ * nucleus: the tokens whose probability is at least that of the last token of the smallest
+ * top-probability prefix holding mass >= top_p (ties with that token are all kept), renormalised;
+ * acceptance tests, the residual and the bonus draw use it.  top_p = 1 (the default) switches the
+ * filter off.  SAMPLE mode only; 0 < top_p <= 1, else INVALID_ARG. */
+int flexspec_set_top_p(flexspec_handle* h, float top_p);
+
 /* Workspace pointers for stage-wise comparison. */
 int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);
 

@@ -25,7 +25,7 @@ ERR_TIMEOUT, ERR_BAD_PAGE, ERR_BAD_TOKEN, ERR_NO_DEVICE = -5, -6, -7, -8
 EXPORTS = [
     "flexspec_create", "flexspec_verify", "flexspec_verify_host", "flexspec_attention",
     "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_kv_append",
-    "flexspec_kv_rollback", "flexspec_get_debug", "flexspec_status",
+    "flexspec_kv_rollback", "flexspec_set_top_p", "flexspec_get_debug", "flexspec_status",
     "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
     "flexspec_destroy", "flexspec_strerror", "flexspec_version",
 ]
@@ -65,6 +65,7 @@ def _load() -> C.CDLL:
     lib.flexspec_sample_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp]
     lib.flexspec_kv_append.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.flexspec_kv_rollback.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    lib.flexspec_set_top_p.argtypes = [vp, f32]
     lib.flexspec_get_debug.argtypes = [vp, C.POINTER(Debug)]
     lib.flexspec_status.argtypes = [vp, vp]
     lib.flexspec_set_profiling.argtypes = [vp, i32]
@@ -301,6 +302,10 @@ class Verifier:
             "q_tok": self._view(d.q_tok, (s_rows,), torch.float64),
             "u": self._view(d.u_acc, (s_rows,), torch.float32),
         }
+
+    def set_top_p(self, top_p: float):
+        """Nucleus sampling of the target (1.0 = off) for the following calls."""
+        _check(LIB.flexspec_set_top_p(self._h, float(top_p)), "flexspec_set_top_p")
 
     def status(self):
         st = (C.c_int32 * 4)()

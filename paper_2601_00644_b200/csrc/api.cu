@@ -77,7 +77,7 @@ void free_workspace(Handle& h)
 {
     cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml); cudaFree(h.att_tickets);
     cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq);
-    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.row_stats); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.chunk_mass);
+    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.row_stats); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.topp); cudaFree(h.chunk_mass);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
     for (int i = 0; i < kNumStageEvents; ++i)
@@ -217,6 +217,7 @@ void fill_sample_params(Handle& h, SampleParams& p, const float* logits, const i
     p.stats = h.stats; p.counters = h.counters;
     p.tstats = h.stats; p.n_tparts = p.n_chunks;          // target parts from the statistics kernel unless the LM head wrote them
     p.row_info = h.row_info; p.row_stats = h.row_stats; p.chunk_mass = h.chunk_mass;
+    p.top_p = p.greedy ? 1.f : h.top_p; p.topp = h.topp;
     p.accepted_len = accepted_len; p.next_token = next_token;
     if (c.flags & FLEXSPEC_FLAG_DEBUG) { p.dbg_p = h.dbg_p; p.dbg_q = h.dbg_q; p.dbg_u = h.dbg_u; }
     p.status = h.status;
@@ -233,6 +234,10 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
                        accepted_len, next_token);
     if (launch_sample_stats(p, 0, p.greedy ? p.m_rows : p.m_rows + p.s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
+    if (p.top_p < 1.f) {
+        if (launch_sample_nucleus(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        h.launches++;
+    }
     if (launch_sample_decide(p, g.k_batch_max, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     if (!p.greedy) {
@@ -295,6 +300,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     h.max_s = c.max_batch * c.k_max;
     h.sm_count = prop.multiProcessorCount;
     h.w = static_cast<const __nv_bfloat16*>(lm_head_w);
+    h.top_p = 1.f;
 
     const int n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
     // LM-head tiling: full waves of 128-row tiles, then one wave of shorter tiles, one per SM, so that
@@ -329,7 +335,8 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.stats, static_cast<size_t>(max_m + h.max_s) * n_chunks));
     A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128 + h.sm_count)));
     A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
-    A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 4));
+    A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 8));
+    A(dev_alloc(&h.topp, static_cast<size_t>(max_m) * 2));
     A(dev_alloc(&h.row_stats, static_cast<size_t>(c.max_batch) * (kMaxK + 1) * 8));
     A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * ((c.vocab + kDrawChunk - 1) / kDrawChunk) * 2));
     A(dev_alloc(&h.dbg_p, static_cast<size_t>(h.max_s)));
@@ -492,7 +499,11 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);
-    if (launch_sample_decide(sp, g.k_batch_max, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (sp.top_p < 1.f) {
+        if (launch_sample_nucleus(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;     // needs the row -> sequence table only with a mask: joined above
+        h.launches++;
+    }
+    if (launch_sample_decide(sp, g.k_batch_max, sp.top_p >= 1.f, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 5, s);
     if (!sp.greedy) {
@@ -605,6 +616,13 @@ int flexspec_kv_rollback(flexspec_handle* fh, const int32_t* kv_len, const int32
     if (launch_kv_rollback(kv_len, draft_len, accepted_len, batch, kv_len_next, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
     h.launches = 1;
+    return FLEXSPEC_OK;
+}
+
+int flexspec_set_top_p(flexspec_handle* fh, float top_p)
+{
+    if (fh == nullptr || !(top_p > 0.f) || top_p > 1.f) return FLEXSPEC_ERR_INVALID_ARG;
+    fh->h.top_p = top_p;
     return FLEXSPEC_OK;
 }
 

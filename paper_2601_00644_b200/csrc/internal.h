@@ -100,7 +100,10 @@ struct SampleParams {
     int32_t n_tparts;
     int32_t* counters;            // [2][max_batch] self-resetting tickets (decision, draw)
     double* row_stats;            // [B][kMaxK+1][8]: (max_p, sum_p, max_q, sum_q, rejected) of every row, or the arg-max in [0]
-    double* row_info;             // [B][4]: max_p, 1/sum_p, max_q, 1/sum_q of row n
+    double* row_info;             // [B][8]: max_p, 1/sum_p, max_q, 1/sum_q of row n, [4] its nucleus threshold (logit)
+    float top_p;                  // nucleus mass of the target distribution; >= 1: no filtering
+    double* topp;                 // [M][2]: lowest kept logit of the row's nucleus, mass of the nucleus (in units of
+                                  // 2^((z - max) * c)); written by the nucleus kernel when top_p < 1
     double* chunk_mass;           // [B][n_dchunks][2]: residual mass, p mass
     int32_t* accepted_len;
     int32_t* next_token;
@@ -121,7 +124,7 @@ struct Handle {
     float* logits;
     float* part_o; float* part_ml; int32_t* att_tickets; int32_t att_pairs_max;
     Plan plan;
-    float2* stats; float2* tstats; int32_t* counters; double* row_stats; double* row_info; double* chunk_mass;
+    float2* stats; float2* tstats; int32_t* counters; double* row_stats; double* row_info; double* topp; float top_p; double* chunk_mass;
     double* dbg_p; double* dbg_q; float* dbg_u;
     int32_t* status;
     // host staging for flexspec_verify_host
@@ -144,6 +147,7 @@ cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHe
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
 // pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
 // the stream drains; it waits on the device before touching the predecessor's results)
+cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream);
 cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, bool pdl, cudaStream_t stream);
 cudaError_t launch_sample_draw(const SampleParams& p, bool pdl, cudaStream_t stream);
 

@@ -25,7 +25,7 @@ constexpr size_t kOffCuD = kOffCuQ + align256(sizeof(int32_t) * (kStaticMaxBatch
 constexpr size_t kOffRowSeq = kOffCuD + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));
 constexpr size_t kOffStats = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);
 constexpr size_t kOffRowInfo = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
-constexpr size_t kOffRowStats = kOffRowInfo + align256(sizeof(double) * kStaticMaxBatch * 4);
+constexpr size_t kOffRowStats = kOffRowInfo + align256(sizeof(double) * kStaticMaxBatch * 8);
 constexpr size_t kOffMass = kOffRowStats + align256(sizeof(double) * kStaticMaxBatch * (kMaxK + 1) * 8);
 constexpr size_t kScratchBytes = kOffMass + align256(sizeof(double) * kStaticMaxBatch * kStaticDrawChunks * 2);
 
@@ -107,6 +107,7 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     p.inv_temp_log2 = greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     p.stats = reinterpret_cast<float2*>(base + kOffStats);
     p.tstats = p.stats; p.n_tparts = p.n_chunks;
+    p.top_p = 1.f; p.topp = nullptr;
     p.counters = reinterpret_cast<int32_t*>(base + kOffCounters);
     p.row_info = reinterpret_cast<double*>(base + kOffRowInfo);
     p.row_stats = reinterpret_cast<double*>(base + kOffRowStats);

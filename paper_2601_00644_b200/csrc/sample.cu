@@ -163,6 +163,121 @@ cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------ nucleus (top-p)
+// The paper's stochastic regime samples the target with top-p 0.9.  The nucleus of a row is the set
+// of tokens whose logit is at least tau, where tau is the largest logit value such that the tokens
+// with logit >= tau hold at least top_p of the row's mass (ties with tau are all kept).  One CTA
+// per target row finds tau exactly by a 4-round radix selection over the order-preserving 32-bit
+// keys of the logits, 8 bits per round: a 256-bin histogram of probability MASS over the keys that
+// match the prefix found so far (one private fp32 histogram per warp, filled with the native
+// shared-memory float add -- with flat logits every key of a round falls into one or two bins, and
+// a single shared fp64 histogram serialised to a millisecond --, then summed in fp64), and a walk
+// from the top bin down to the bin in which the cumulative mass reaches the target.
+constexpr int kNucThreads = 1024;
+
+__device__ __forceinline__ uint32_t order_key(float z)       // larger float <-> larger key
+{
+    const uint32_t u = __float_as_uint(z);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_to_float(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+__global__ void __launch_bounds__(kNucThreads)
+sample_nucleus_kernel(const SampleParams p)
+{
+    __shared__ double s_hist[256];
+    __shared__ float s_whist[kNucThreads / 32][256];
+    __shared__ float s_redf[kNucThreads / 32];
+    __shared__ double s_redd[kNucThreads / 32];
+    __shared__ double s_above, s_target, s_binmass;
+    __shared__ uint32_t s_prefix;
+    const int row = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float cf = p.inv_temp_log2;
+    const uint32_t* mask_row = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(p.row_seq[row]) * p.mask_words : nullptr;
+
+    // ---- (max, mass) of the row from its parts
+    const float2* tp = p.tstats + static_cast<int64_t>(row) * p.n_tparts;
+    float m = -INFINITY, sf = 0.f;
+    for (int i = tid; i < p.n_tparts; i += kNucThreads) {
+        const float2 pt = __ldcg(&tp[i]);
+        merge_ms(m, sf, pt.x, pt.y, cf);
+    }
+    const float mt = m;
+    m = warp_max(m);
+    if (lane == 0) s_redf[warp] = m;
+    __syncthreads();
+    for (int w = 0; w < kNucThreads / 32; ++w) m = fmaxf(m, s_redf[w]);
+    double sm = (mt == -INFINITY) ? 0.0 : static_cast<double>(sf) * static_cast<double>(fast_exp2((mt - m) * cf));
+    sm = warp_sum(sm);
+    if (lane == 0) s_redd[warp] = sm;
+    __syncthreads();
+    sm = 0.0;
+    for (int w = 0; w < kNucThreads / 32; ++w) sm += s_redd[w];
+    if (tid == 0) { s_above = 0.0; s_target = static_cast<double>(p.top_p) * sm; s_prefix = 0u; }
+
+    const float* src = p.logits + static_cast<int64_t>(row) * p.vocab;
+    for (int round = 0; round < 4; ++round) {
+        const int shift = 24 - 8 * round;
+        for (int i = tid; i < (kNucThreads / 32) * 256; i += kNucThreads) (&s_whist[0][0])[i] = 0.f;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        const uint32_t hi_mask = (round == 0) ? 0u : (0xffffffffu << (shift + 8));
+        // eight loads in flight per thread (the row comes out of L2: a dependent load per element would
+        // cost its full latency 125 times per round)
+        for (int v0 = 0; v0 < p.vocab; v0 += kNucThreads * 8) {
+            float zz[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int v = v0 + i * kNucThreads + tid;
+                zz[i] = (v < p.vocab) ? __ldg(src + v) : -INFINITY;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int v = v0 + i * kNucThreads + tid;
+                float z = zz[i];
+                if (mask_row != nullptr && v < p.vocab && !mask_allows(mask_row, v)) z = -INFINITY;
+                const uint32_t key = order_key(z);
+                if (z != -INFINITY && (key & hi_mask) == (prefix & hi_mask))
+                    atomicAdd(&s_whist[warp][(key >> shift) & 255u], fast_exp2((z - m) * cf));
+            }
+        }
+        __syncthreads();
+        if (tid < 256) {
+            double acc = 0.0;
+#pragma unroll 8
+            for (int w = 0; w < kNucThreads / 32; ++w) acc += static_cast<double>(s_whist[w][tid]);
+            s_hist[tid] = acc;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double cum = s_above;
+            int bin = 255;
+            for (; bin > 0; --bin) {
+                if (cum + s_hist[bin] >= s_target) break;
+                cum += s_hist[bin];
+            }
+            s_above = cum;
+            s_binmass = s_hist[bin];
+            s_prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(key_to_float(s_prefix));
+        p.topp[static_cast<int64_t>(row) * 2 + 1] = s_above + s_binmass;
+    }
+}
+
+cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream)
+{
+    sample_nucleus_kernel<<<p.m_rows, kNucThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------------------------ decision
 // grid (row j, sequence b): the CTA merges the parts of target row j (and draft row j) of the
 // sequence -- maximum first, then the sum with fp32 weights accumulated in fp64 -- and leaves
@@ -284,10 +399,12 @@ sample_decide_kernel(const SampleParams p)
             double sm = (mt == -INFINITY) ? 0.0 : static_cast<double>(sf) * static_cast<double>(fast_exp2((mt - m) * cf));
             sm = block_sum(sm, red_d, lane, warp);
             if (threadIdx.x == 0) {
-                rs[0] = static_cast<double>(m); rs[1] = sm; rs[2] = mq; rs[3] = sq;
+                double tau = -INFINITY;                   // nucleus of the target row: its lowest kept logit and its mass
+                if (p.top_p < 1.f) { tau = p.topp[static_cast<int64_t>(q0 + j) * 2]; sm = p.topp[static_cast<int64_t>(q0 + j) * 2 + 1]; }
+                rs[0] = static_cast<double>(m); rs[1] = sm; rs[2] = mq; rs[3] = sq; rs[5] = tau;
                 double rej = 0.0;
                 if (test_row) {
-                    const double pt = (zp == -INFINITY) ? 0.0 : exp2((zp - static_cast<double>(m)) * scale) / sm;
+                    const double pt = (zp == -INFINITY || zp < tau) ? 0.0 : exp2((zp - static_cast<double>(m)) * scale) / sm;
                     rej = (u * qt < pt) ? 0.0 : 1.0;
                     if (p.dbg_p != nullptr) {
                         p.dbg_p[d0 + j] = pt;
@@ -328,9 +445,10 @@ sample_decide_kernel(const SampleParams p)
         if (p.greedy) {
             p.next_token[b] = static_cast<int>(__ldcg(rn));
         } else {
-            double* ri = p.row_info + static_cast<int64_t>(b) * 4;
+            double* ri = p.row_info + static_cast<int64_t>(b) * 8;
             ri[0] = __ldcg(rn); ri[1] = 1.0 / __ldcg(rn + 1);
             ri[2] = (n < k_b) ? __ldcg(rn + 2) : 0.0; ri[3] = (n < k_b) ? 1.0 / __ldcg(rn + 3) : 1.0;
+            ri[4] = __ldcg(rn + 5);
         }
     }
 }
@@ -346,12 +464,12 @@ cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, boo
 // and all sums are fp64.
 struct DrawRow {
     const float* zt; const float* zd; const uint32_t* mask;
-    float mp, mq, c;
+    float mp, mq, c, tau;         // tau: lowest logit of the target row's nucleus (-inf: no top-p filter)
     double inv_sp, inv_sq;
     bool residual;
     __device__ __forceinline__ double prob_p(float z, int v) const
     {
-        if (z == -INFINITY || !mask_allows(mask, v)) return 0.0;
+        if (z == -INFINITY || z < tau || !mask_allows(mask, v)) return 0.0;
         return static_cast<double>(fast_exp2((z - mp) * c)) * inv_sp;
     }
     __device__ __forceinline__ double prob_q(float z) const
@@ -403,9 +521,10 @@ sample_draw_kernel(const SampleParams p)
     row.residual = (n < k_b);
     row.zd = row.residual ? p.draft_logits + static_cast<int64_t>(p.cu_d[b] + n) * p.vocab : nullptr;
     row.mask = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(b) * p.mask_words : nullptr;
-    const double* ri = p.row_info + static_cast<int64_t>(b) * 4;
+    const double* ri = p.row_info + static_cast<int64_t>(b) * 8;
     row.mp = static_cast<float>(ri[0]); row.inv_sp = ri[1];
     row.mq = static_cast<float>(ri[2]); row.inv_sq = ri[3];
+    row.tau = static_cast<float>(ri[4]);
     row.c = p.inv_temp_log2;
     const bool vec_ok = ((p.vocab & 3) == 0);
 

@@ -210,3 +210,61 @@ def test_sample_invariants_on_gpu():
     assert np.all(acc.cpu().numpy() == 0)
     assert np.all(nxt.cpu().numpy() % 2 == 0)
     ver.close()
+
+
+# ------------------------------------------------------------------ nucleus (top-p) sampling
+
+@pytest.mark.parametrize("top_p,temperature", [(0.9, 1.0), (0.5, 0.7), (0.999, 1.0)])
+@pytest.mark.parametrize("vocab,batch,k_hi,holes,mask", [
+    (4096, 3, 4, False, False),
+    (777, 9, 7, True, False),
+    (20000, 16, 12, False, True),
+])
+def test_sample_stage_with_top_p_matches_oracle(top_p, temperature, vocab, batch, k_hi, holes, mask):
+    B = _binding()
+    k, zt, zd, toks, seeds, vmask = _sample_case(7 * vocab + batch, batch, vocab, 0, k_hi, 0, temperature,
+                                                 holes=holes, mask=mask)
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=max(k_hi, 1), max_kv_len=64, mode=0, debug=True)
+    ver.set_top_p(top_p)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).cuda()
+    vm_d = None if vmask is None else dev(vmask.view(np.int32), torch.int32)
+    acc, nxt = ver.sample(dev(zt, torch.float32), dev(toks, torch.int32), dev(zd, torch.float32), dev(k, torch.int32),
+                          torch.from_numpy(k), dev(seeds.view(np.int64), torch.int64), temperature=temperature, vocab_mask=vm_d)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    acc, nxt = acc.cpu().numpy(), nxt.cpu().numpy()
+    ref = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, temperature, vmask, top_p=top_p)
+    r0 = np.concatenate([[0], np.cumsum(k + 1)]); t0 = np.concatenate([[0], np.cumsum(k)])
+    dbg = ver.debug(int(k.sum()) + batch, int(k.sum()))
+    p_g = dbg["p_tok"].cpu().numpy()
+    excused = 0
+    for b in range(batch):
+        kb = int(k[b])
+        # a nucleus cut that falls within 1e-6 of top_p may legitimately land one token earlier / later:
+        # only then may an outcome differ beyond the usual near-tie clauses
+        cut_tie = ref["topp_margin"][r0[b]:r0[b + 1]].min() < 1e-6
+        bad = False
+        if kb and np.abs(p_g[t0[b]:t0[b] + kb] - ref["p_tok"][t0[b]:t0[b] + kb]).max() >= 1e-5:
+            bad = True
+        elif acc[b] != ref["accepted_len"][b]:
+            j = min(acc[b], ref["accepted_len"][b])
+            if ref["acc_margin"][t0[b] + j] < 1e-5:
+                excused += 1
+                continue
+            bad = True
+        elif nxt[b] != ref["next_token"][b] and not ref["cdf_margin"][b] < 1e-6:
+            bad = True
+        if bad:
+            assert cut_tie, (b, acc[b], ref["accepted_len"][b], nxt[b], ref["next_token"][b])
+            excused += 1
+    assert excused <= 1
+    # the filter is really on: with top_p = 0.5 some draft token fell outside its row's nucleus
+    if top_p == 0.5 and k.sum() > 0:
+        assert (ref["p_tok"] == 0).any() and (p_g[ref["p_tok"] == 0] == 0).all()
+    ver.set_top_p(1.0)
+    acc1, nxt1 = ver.sample(dev(zt, torch.float32), dev(toks, torch.int32), dev(zd, torch.float32), dev(k, torch.int32),
+                            torch.from_numpy(k), dev(seeds.view(np.int64), torch.int64), temperature=temperature, vocab_mask=vm_d)
+    ref1 = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, temperature, vmask)
+    assert (acc1.cpu().numpy() != ref1["accepted_len"]).sum() <= 1           # switched off again
+    ver.close()

@@ -61,6 +61,32 @@ def test_reduced_8b_shape_flat_and_peaked():
     ver.close()
 
 
+def test_verify_with_top_p_on_peaked_logits():
+    """The whole step with nucleus sampling (the paper's stochastic regime, top-p 0.9): decisions against
+    the oracle fed the GPU's own logits (the filter makes decisions discontinuous in the logits, so the
+    end-to-end comparison through the bf16 rounding of the attention output is left to the unfiltered tests)."""
+    H = _H()
+    shape = wl.peaked(wl.scaled(wl.CONFIGS["llama3_8b"], batch=4, vocab=20000, ctx_min=300, ctx_max=700, index=16))
+    case = H.Case(shape)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    ver.set_top_p(0.9)
+    acc, nxt = H.run_gpu_verify(case, ver)
+    dbg = ver.debug(case.inp.m_rows, case.inp.s_rows)
+    logits_g = dbg["logits"].cpu().numpy().astype(np.float64)
+    import oracle
+    ref = oracle.accept(0, logits_g, case.draft_logits.cpu().numpy(), case.draft_tokens.cpu().numpy(), case.k,
+                        case.h_seeds, shape.temperature, None, top_p=0.9)
+    # rows whose nucleus cut falls within 1e-6 of top_p may legitimately differ; all others must agree
+    ok_rows = [b for b in range(case.batch) if ref["topp_margin"][case.row0[b]:case.row0[b + 1]].min() >= 1e-6]
+    assert len(ok_rows) >= case.batch - 1
+    case.check = ok_rows
+    H.compare_decisions(case, acc, nxt, ref, H.CDF_TIE_TOL, "top-p")
+    drows = case.drows_of(ok_rows)
+    assert np.abs(dbg["p_tok"].cpu().numpy()[drows] - ref["p_tok"][drows]).max() < H.PROB_TOL
+    ver.close()
+
+
 def test_ragged_batch_with_k0_and_greedy():
     shape = wl.scaled(wl.CONFIGS["adaptive_k"], batch=7, vocab=9000, k_min=0, k_max=12, ctx_min=30,
                       ctx_max=900, index=12)
