@@ -311,7 +311,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
         if (tiles128 > h.sm_count && tiles128 % h.sm_count != 0) {
             h.lm_full_tiles = tiles128 / h.sm_count * h.sm_count;
             const int rows_rem = c.vocab - h.lm_full_tiles * 128;
-            int lr = ((rows_rem + h.sm_count - 1) / h.sm_count + 7) / 8 * 8;
+            int lr = (rows_rem + h.sm_count - 1) / h.sm_count;
             if (lr > 128) lr = 128;
             h.lm_last_rows = lr;
             h.lm_last_tiles = (rows_rem + lr - 1) / lr;

@@ -65,7 +65,7 @@ struct LmHeadParams {
     int32_t n_pass;           // passes over W when m_rows > n_tile * n_blocks
     int32_t n_vtiles;         // vocabulary tiles: n_full_tiles of 128 rows, then tiles of last_rows rows
     int32_t n_full_tiles;
-    int32_t last_rows;        // height of the tiles of the last wave (multiple of 8, <= 128)
+    int32_t last_rows;        // height of the tiles of the last wave (<= 128)
     int32_t num_stages;       // shared-memory pipeline depth
     int32_t acc_stages;       // TMEM accumulator buffers (1 or 2)
     // optional: softmax statistics of the rows, one part per (row, 32 vocabulary rows), for the
