@@ -94,6 +94,15 @@ def test_ragged_batch_with_k0_and_greedy():
     _run(shape, mode=1)
 
 
+def test_many_short_sequences_in_one_call():
+    """More sequences than threads in a CTA (the per-CTA range computation then handles several
+    sequences per thread), tiny contexts, k from 0: every sequence against the oracle."""
+    shape = wl.scaled(wl.CONFIGS["tiny"], batch=300, vocab=1000, k_min=0, k_max=3, ctx_min=0, ctx_max=40, index=17)
+    case, rep = _run(wl.peaked(shape))
+    assert rep["iso_ties"] + rep["iso_cdf_ties"] <= 2
+    _run(wl.peaked(shape), mode=1)
+
+
 def test_degenerate_cases_p_equals_q_and_disjoint_support():
     """Long-context config's sub-cases on a reduced shape: a sequence whose draft logits are the
     target's own (every draft accepted) and one whose drafts lie outside the target's support
