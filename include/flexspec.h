@@ -118,7 +118,9 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
  *   hidden        DEVICE bf16 [M][d_model]; row r viewed as [H][head_dim] is the query of
  *                 every head (the attention output feeds the LM head directly)
  *   draft_tokens  DEVICE int32 [S]
- *   draft_logits  DEVICE fp32 [S][vocab]; may be NULL in GREEDY mode
+ *   draft_logits  DEVICE fp32 [S][vocab]; may be NULL in GREEDY mode.  When vocab is a multiple
+ *                 of 4 the rows are read with 16-byte loads and the array must start on a
+ *                 16-byte boundary (else INVALID_ARG); otherwise 4-byte alignment is enough.
  *   draft_len     DEVICE int32 [batch], draft_len_host its HOST copy (launch geometry)
  *   seeds         DEVICE uint64 [batch]; uniforms are Philox4x32-10 with key =
  *                 (lo32, hi32) of the seed, counter = (j, stream, 0, 0), word 0,
@@ -165,8 +167,8 @@ int flexspec_attention(flexspec_handle* h, const flexspec_kv* kv, const void* hi
 int flexspec_lm_head(flexspec_handle* h, const void* x, int32_t m_rows, float* logits, void* stream);
 
 /* Stage 3 alone (Algorithm 2 acceptance loop and correction token; the stochastic rule of
- * the speculative-sampling papers it cites).  logits DEVICE fp32 [M][vocab] (NULL = workspace);
- * other arguments as in flexspec_verify. */
+ * the speculative-sampling papers it cites).  logits DEVICE fp32 [M][vocab] (NULL = workspace),
+ * aligned like draft_logits; other arguments as in flexspec_verify. */
 int flexspec_sample(flexspec_handle* h, const float* logits,
                     const int32_t* draft_tokens, const float* draft_logits,
                     const int32_t* draft_len, const int32_t* draft_len_host,
@@ -213,8 +215,8 @@ int flexspec_kv_rollback(flexspec_handle* h, const int32_t* kv_len, const int32_
  *     call clears the part that has to start at zero on `stream` before its kernels.  Two calls
  *     whose GPU work may overlap (different streams, no ordering) race on the array: serialise
  *     them.
- *   - Arguments as flexspec_sample, all DEVICE pointers except draft_len_host; `mode` is a
- *     FLEXSPEC_MODE_* value.  A draft token outside [0, vocab) is clamped, not reported.
+ *   - Arguments as flexspec_sample (the same alignment of the two logit arrays included), all
+ *     DEVICE pointers except draft_len_host; `mode` is a FLEXSPEC_MODE_* value.  A draft token outside [0, vocab) is clamped, not reported.
  * Errors: INVALID_ARG, UNSUPPORTED (limits above), NO_DEVICE, CUDA. */
 int flexspec_sample_static(const float* logits, const int32_t* draft_tokens, const float* draft_logits,
                            const int32_t* draft_len, const int32_t* draft_len_host, const uint64_t* seeds,

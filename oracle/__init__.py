@@ -60,6 +60,8 @@ def lib() -> C.CDLL:
         L.fso_accept.restype = None
         L.fso_accept.argtypes = [i32, vp, vp, vp, vp, vp, i32, i32, f64, f64, vp, vp, i32,
                                  vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fso_emission.restype = f64
+        L.fso_emission.argtypes = [vp, vp, i32, f64, f64, vp, vp, vp]
         L.fso_nucleus.restype = None
         L.fso_nucleus.argtypes = [vp, i32, f64, vp]
         L.fso_kv_append.restype = None
@@ -162,6 +164,17 @@ def nucleus(prob, top_p):
     m = np.zeros(1, dtype=np.float64)
     lib().fso_nucleus(_p(p), int(p.size), float(top_p), _p(m))
     return p, float(m[0])
+
+
+def emission(target_row, draft_row=None, temperature=1.0, top_p=1.0, mask=None):
+    """Unnormalised weights r[v] of the emitted token and their sum Z for one target row: the residual
+    max(0, p - q) when a draft row is given (first rejection), p itself otherwise (bonus row)."""
+    zt = _c(target_row, np.float64)
+    zd = _c(draft_row, np.float32)
+    mask = _c(mask, np.uint32)
+    r = np.empty(zt.shape[0], dtype=np.float64)
+    z = lib().fso_emission(_p(zt), _p(zd), int(zt.shape[0]), float(temperature), float(top_p), _p(mask), _p(r), None)
+    return r, float(z)
 
 
 def accept(mode, target_logits, draft_logits, draft_tokens, draft_len, seeds, temperature=1.0,

@@ -292,6 +292,35 @@ static int32_t inverse_cdf(const double* r, int32_t vocab, double thr,
     return last_pos;
 }
 
+/* Unnormalised weights of the emitted token and their sum Z: max(0, p - q) when a draft row is
+ * given (the first rejection) and that residual has positive mass, else p (the bonus row, or a
+ * residual that rounding emptied). */
+double fso_emission(const double* zt_row, const float* zd_row, int32_t vocab, double temperature,
+                    double top_p, const uint32_t* mask, double* r, double* topp_margin)
+{
+    double* p = (double*)malloc(sizeof(double) * (size_t)vocab);
+    fso_softmax(zt_row, vocab, temperature, mask, p);
+    fso_nucleus(p, vocab, top_p, topp_margin);
+    double z_mass = 0.0;
+    if (zd_row != NULL) {
+        double* q = (double*)malloc(sizeof(double) * (size_t)vocab);
+        double* zq = (double*)malloc(sizeof(double) * (size_t)vocab);
+        for (int32_t v = 0; v < vocab; ++v) zq[v] = (double)zd_row[v];
+        fso_softmax(zq, vocab, temperature, NULL, q);
+        for (int32_t v = 0; v < vocab; ++v) {
+            r[v] = p[v] - q[v] > 0.0 ? p[v] - q[v] : 0.0;
+            z_mass += r[v];
+        }
+        free(q); free(zq);
+    }
+    if (zd_row == NULL || !(z_mass > 0.0)) {
+        z_mass = 0.0;
+        for (int32_t v = 0; v < vocab; ++v) { r[v] = p[v]; z_mass += r[v]; }
+    }
+    free(p);
+    return z_mass;
+}
+
 static void verify_one(int32_t mode, const double* zt, const float* zd, const int32_t* x,
                        int32_t k, int32_t vocab, double temperature, double top_p, uint64_t seed,
                        const uint32_t* mask, double* topp_margin,
@@ -335,21 +364,8 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
     }
 
     /* emitted token: residual at the first rejection, else the bonus row */
-    fso_softmax(zt + (int64_t)n * vocab, vocab, temperature, mask, p);
-    fso_nucleus(p, vocab, top_p, topp_margin ? topp_margin + n : NULL);
-    double z_mass = 0.0;
-    if (n < k) {
-        for (int32_t v = 0; v < vocab; ++v) zq[v] = (double)zd[(int64_t)n * vocab + v];
-        fso_softmax(zq, vocab, temperature, NULL, q);
-        for (int32_t v = 0; v < vocab; ++v) {
-            r[v] = p[v] - q[v] > 0.0 ? p[v] - q[v] : 0.0;
-            z_mass += r[v];
-        }
-    }
-    if (n == k || !(z_mass > 0.0)) {
-        z_mass = 0.0;
-        for (int32_t v = 0; v < vocab; ++v) { r[v] = p[v]; z_mass += r[v]; }
-    }
+    double z_mass = fso_emission(zt + (int64_t)n * vocab, n < k ? zd + (int64_t)n * vocab : NULL, vocab,
+                                 temperature, top_p, mask, r, topp_margin ? topp_margin + n : NULL);
     const double u2 = fso_uniform(seed, (uint32_t)n, 1u);
     double c_below, c_at;
     const double thr = u2 * z_mass;

@@ -80,6 +80,13 @@ void fso_softmax(const double* z, int32_t vocab, double temperature,
  * cumulative sums around the cut, i.e. how close the cut was to falling one token earlier/later. */
 void fso_nucleus(double* prob, int32_t vocab, double top_p, double* margin);
 
+/* The weights the emitted token is drawn from, for one target row (Algorithm 2: "sample correction
+ * token"): r[v] = max(0, p(v) - q(v)) when zd_row is given (first rejection; p, q the softmaxes of
+ * the two rows at `temperature`, p filtered to its nucleus when top_p < 1), or r = p when zd_row is
+ * NULL (bonus row) or the residual has no mass.  Returns Z = sum_v r[v]; r is not normalised. */
+double fso_emission(const double* zt_row, const float* zd_row, int32_t vocab, double temperature,
+                    double top_p, const uint32_t* mask, double* r, double* topp_margin);
+
 /* Acceptance + emitted token for a batch of sequences.  With top_p < 1 the TARGET distribution of
  * every row is its nucleus (SAMPLE mode only).
  * mode 0 = SAMPLE: accept x_j iff u_j * q_j(x_j) < p_j(x_j); after n accepted

@@ -247,6 +247,13 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
     return FLEXSPEC_OK;
 }
 
+// The sampling kernels read the logit rows with 16-byte loads when the vocabulary is a multiple of
+// four (every row then starts on a 16-byte boundary if the array does); otherwise with 4-byte loads.
+bool logits_aligned(const void* ptr, int32_t vocab)
+{
+    return (reinterpret_cast<uintptr_t>(ptr) & ((vocab & 3) == 0 ? 15u : 3u)) == 0;
+}
+
 bool sample_args_ok(const Handle& h, const int32_t* draft_tokens, const float* draft_logits,
                     const uint64_t* seeds, float temperature, const Geometry& g)
 {
@@ -441,6 +448,7 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
     int rc = check_lengths(h, draft_len_host, nullptr, batch, 0, &g);
     if (rc != FLEXSPEC_OK) return rc;
     if (!sample_args_ok(h, draft_tokens, draft_logits, seeds, temperature, g)) return FLEXSPEC_ERR_INVALID_ARG;
+    if (!logits_aligned(logits, h.cfg.vocab) || !logits_aligned(draft_logits, h.cfg.vocab)) return FLEXSPEC_ERR_INVALID_ARG;
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
@@ -466,6 +474,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     int rc = check_lengths(h, draft_len_host, kv->kv_len_host, batch, kv->max_pages_per_seq, &g);
     if (rc != FLEXSPEC_OK) return rc;
     if (!sample_args_ok(h, draft_tokens, draft_logits, seeds, temperature, g)) return FLEXSPEC_ERR_INVALID_ARG;
+    if (!logits_aligned(draft_logits, h.cfg.vocab)) return FLEXSPEC_ERR_INVALID_ARG;
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;

@@ -64,6 +64,10 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     const bool greedy = (mode == FLEXSPEC_MODE_GREEDY || temperature == 0.f);
     if (s_rows > 0 && draft_tokens == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
     if (!greedy && (seeds == nullptr || (s_rows > 0 && draft_logits == nullptr))) return FLEXSPEC_ERR_INVALID_ARG;
+    // the kernels read logit rows with 16-byte loads when vocab is a multiple of four
+    const uintptr_t align_mask = (vocab & 3) == 0 ? 15u : 3u;
+    if (((reinterpret_cast<uintptr_t>(logits) | reinterpret_cast<uintptr_t>(draft_logits)) & align_mask) != 0)
+        return FLEXSPEC_ERR_INVALID_ARG;
 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_NO_DEVICE; }

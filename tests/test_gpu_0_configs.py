@@ -1,0 +1,57 @@
+"""GPU parity of the whole verification step on the five paper-shaped workloads at their full size,
+in the launch configuration the benchmark times.  The tiny one is compared on its only sequence; the
+four large ones on a subset of whole sequences (sequences are independent, so a subset is exact)
+plus properties that hold for every sequence.
+
+This file sorts first among the GPU tests, so a run that stops at the first failure has shown the
+five workloads before anything else."""
+import math
+
+import numpy as np
+import pytest
+import scipy.stats
+
+from paper_2601_00644_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(shape, check=None, mode=0):
+    import tests.harness as H
+    case = H.Case(shape, check_seqs=check, mode=mode)
+    case.build_drafts()
+    ver = H.make_verifier(case)
+    rep = H.full_parity(case, ver)
+    # same call again: identical outputs (tickets reset, no stale state)
+    acc2, nxt2 = H.run_gpu_verify(case, ver)
+    assert np.array_equal(acc2, rep["accepted_len"]) and np.array_equal(nxt2, rep["next_token"])
+    ver.close()
+    return case, rep
+
+
+def test_tiny_config():
+    case, rep = _run(wl.CONFIGS["tiny"])
+    assert rep["e2e_ties"] + rep["e2e_cdf_ties"] + rep["e2e_explained"] == 0, rep
+
+
+@pytest.mark.parametrize("name,check", [
+    ("llama3_8b", [0, 7, 15]),
+    ("adaptive_k", [1, 20, 41, 63]),
+    ("llama3_70b", [3, 30]),
+    ("long_ctx", [2, 6]),
+])
+def test_full_config_subset_parity_and_properties(name, check):
+    shape = wl.CONFIGS[name]
+    case, rep = _run(shape, check=check)
+    acc = rep["accepted_len"]
+    k = case.k
+    assert np.all((acc >= 0) & (acc <= k))
+    assert np.all((rep["next_token"] >= 0) & (rep["next_token"] < shape.vocab))
+    # per-position acceptance follows the flat-target closed form 2*Phi(-sigma/(2T)):
+    # position j is reached iff all earlier ones were accepted, so count tests actually taken
+    sig = case.inp.sigma.cpu().numpy()
+    taken = np.minimum(acc + 1, k).sum()
+    accepted = acc.sum()
+    want = float(np.sum(np.minimum(acc + 1, k) * 2 * scipy.stats.norm.cdf(-sig / (2 * shape.temperature))) / max(taken, 1))
+    assert abs(accepted / max(taken, 1) - want) < 5 * math.sqrt(0.25 / max(taken, 1)) + 0.02
+    assert rep["e2e_ties"] + rep["e2e_cdf_ties"] + rep["e2e_explained"] <= 1, rep
