@@ -387,7 +387,7 @@ def run_ours(args):
             "hbm_roofline_frac_of_8TBs": alg_bytes / (ms_per_step * 1e-3) / 8e12,
             "hbm_roofline_frac_of_measured": alg_bytes / (ms_per_step * 1e-3) / (peak * 1e9),
             "stage_us": {"attention": stage_ms[1] * 1e3, "lm_head": stage_ms[3] * 1e3,
-                         "decide": stage_ms[4] * 1e3, "draw": stage_ms[5] * 1e3,
+                         "nucleus": stage_ms[4] * 1e3, "accept": stage_ms[5] * 1e3,
                          "note": "CUDA events between the kernels of the main stream (second profiling loop); "
                                  "plan and draft-logit statistics run on a second stream beside attention"},
             "roofline": {"kernel": "lm_head_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,

@@ -72,7 +72,7 @@ typedef struct {
     int32_t  n_q_heads;     /* H; d_model = H * head_dim, must be a multiple of 64           */
     int32_t  n_kv_heads;    /* Hkv, divides H                                                 */
     int32_t  head_dim;      /* 64 or 128                                                      */
-    int32_t  vocab;         /* V >= 1                                                         */
+    int32_t  vocab;         /* 1 <= V <= 1048576                                              */
     int32_t  page_size;     /* tokens per KV page: must be 16                                 */
     int32_t  max_batch;     /* 1..1024 sequences per call                                     */
     int32_t  k_max;         /* largest draft length k_b, 0..63                                */
@@ -134,8 +134,10 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
  *   next_token    DEVICE int32 [batch] out: the token emitted after the accepted prefix
  * Errors: INVALID_ARG (NULLs, batch > max_batch, k_b > k_max, kv_len out of range or
  * smaller than k_b+1, too few pages per sequence), CUDA. Device-side problems
- * (bad page id, bad token id, a wait that gave up) are recorded in the status
- * word, see flexspec_status. */
+ * (bad page id, bad token id, a wait that gave up, a DEVICE draft_len that disagrees
+ * with draft_len_host: INVALID_ARG, and the sampling stage then treats every k_b as 0)
+ * are recorded in the status word, see flexspec_status.  Outputs of a call whose status
+ * word is non-zero are undefined. */
 int flexspec_verify(flexspec_handle* h, const flexspec_kv* kv, const void* hidden,
                     const int32_t* draft_tokens, const float* draft_logits,
                     const int32_t* draft_len, const int32_t* draft_len_host,
@@ -204,15 +206,17 @@ int flexspec_kv_rollback(flexspec_handle* h, const int32_t* kv_len, const int32_
  * fail or eat into the pool's reserve; or a step loop that must never stall on the implicit
  * device synchronisation of an allocation or a free.  Such callers cannot use flexspec_create,
  * which allocates the workspace.
- *   - The working memory is one fixed array inside the loaded library (about 0.5 MB, held on
+ *   - The working memory is one fixed array inside the loaded library (268 032 bytes, held on
  *     every GPU that loads the library until the process exits).  Limits that follow from it:
  *     batch <= 64, sum_b (k_b + 1) <= 1024, vocab <= 131072; larger calls return
  *     FLEXSPEC_ERR_UNSUPPORTED and launch nothing.
  *   - Runs on the CURRENT device of the calling thread.  The first call on a device looks up
  *     the device address of the array (a cheap runtime query, no allocation); make that first
- *     call outside any stream capture.
+ *     call outside any stream capture, and from one thread: the look-up is not synchronised,
+ *     so two threads must not make the first call on a device at the same time.
  *   - All calls on a device share the array, and it keeps the previous call's contents; each
- *     call clears the part that has to start at zero on `stream` before its kernels.  Two calls
+ *     call clears the part that has to start at zero (the status word) on `stream` before its
+ *     kernels, which rewrite everything else before reading it.  Two calls
  *     whose GPU work may overlap (different streams, no ordering) race on the array: serialise
  *     them.
  *   - Arguments as flexspec_sample (the same alignment of the two logit arrays included), all
@@ -242,9 +246,10 @@ int flexspec_status(flexspec_handle* h, int32_t* status_host);
 /* Per-kernel timing.  With profiling on, verify brackets the kernels of the caller's stream with
  * CUDA events; flexspec_get_stage_ms synchronises those events and writes the last call's
  * durations in milliseconds: [0] fork of the second stream, [1] attention, [2] unused,
- * [3] LM head (with the softmax statistics of the target rows), [4] acceptance decision,
- * [5] emitted-token draw.  The row-offset kernel and the draft-logit statistics run on a second
- * stream beside attention and are not timed.  Unused stages read 0. */
+ * [3] LM head (with the softmax statistics of the target rows), [4] nucleus thresholds (top-p
+ * only), [5] acceptance kernel (tests, first rejection, emitted token).  The row-offset kernel
+ * and the draft-logit statistics run on a second stream beside attention and are not timed.
+ * Unused stages read 0. */
 int flexspec_set_profiling(flexspec_handle* h, int32_t on);
 int flexspec_get_stage_ms(flexspec_handle* h, float ms[6]);
 

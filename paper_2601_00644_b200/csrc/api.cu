@@ -76,8 +76,8 @@ struct DeviceGuard {
 void free_workspace(Handle& h)
 {
     cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml); cudaFree(h.att_tickets);
-    cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq);
-    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.row_stats); cudaFree(h.counters); cudaFree(h.row_info); cudaFree(h.topp); cudaFree(h.chunk_mass);
+    cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq); cudaFree(h.plan.k_eff);
+    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.topp);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
     for (int i = 0; i < kNumStageEvents; ++i)
@@ -125,9 +125,11 @@ void mark(Handle& h, int idx, cudaStream_t s)
     if (h.profiling) { cudaEventRecord(h.ev[idx], s); h.ev_used[idx] = 1; }
 }
 
-int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, cudaStream_t s)
+int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, const Geometry& g,
+             cudaStream_t s)
 {
-    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, h.plan, h.status, s) != cudaSuccess)
+    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, g.m_rows, g.s_rows, g.k_batch_max, h.plan, h.status,
+                    s) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
     h.launches++;
     return FLEXSPEC_OK;
@@ -208,15 +210,13 @@ void fill_sample_params(Handle& h, SampleParams& p, const float* logits, const i
     p.greedy = (c.mode == FLEXSPEC_MODE_GREEDY || temperature == 0.f) ? 1 : 0;
     p.logits = logits; p.draft_logits = draft_logits; p.draft_tokens = draft_tokens;
     p.draft_len = draft_len; p.seeds = seeds; p.vocab_mask = vocab_mask;
-    p.cu_q = h.plan.cu_q; p.cu_d = h.plan.cu_d; p.row_seq = h.plan.row_seq;
+    p.cu_q = h.plan.cu_q; p.cu_d = h.plan.cu_d; p.row_seq = h.plan.row_seq; p.k_eff = h.plan.k_eff;
     p.batch = batch; p.vocab = c.vocab; p.m_rows = g.m_rows; p.s_rows = g.s_rows;
     p.n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
-    p.n_dchunks = (c.vocab + kDrawChunk - 1) / kDrawChunk;
     p.mask_words = (c.vocab + 31) / 32;
     p.inv_temp_log2 = p.greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
-    p.stats = h.stats; p.counters = h.counters;
+    p.stats = h.stats;
     p.tstats = h.stats; p.n_tparts = p.n_chunks;          // target parts from the statistics kernel unless the LM head wrote them
-    p.row_info = h.row_info; p.row_stats = h.row_stats; p.chunk_mass = h.chunk_mass;
     p.top_p = p.greedy ? 1.f : h.top_p; p.topp = h.topp;
     p.accepted_len = accepted_len; p.next_token = next_token;
     if (c.flags & FLEXSPEC_FLAG_DEBUG) { p.dbg_p = h.dbg_p; p.dbg_q = h.dbg_q; p.dbg_u = h.dbg_u; }
@@ -238,12 +238,8 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
         if (launch_sample_nucleus(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
     }
-    if (launch_sample_decide(p, g.k_batch_max, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_accept(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
-    if (!p.greedy) {
-        if (launch_sample_draw(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-        h.launches++;
-    }
     return FLEXSPEC_OK;
 }
 
@@ -287,7 +283,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     const int64_t d_model = static_cast<int64_t>(c.n_q_heads) * c.head_dim;
     if (d_model % 64 != 0 || d_model > 65536) return FLEXSPEC_ERR_UNSUPPORTED;
     const int64_t max_m = static_cast<int64_t>(c.max_batch) * (c.k_max + 1);
-    if (max_m * c.vocab > (1LL << 40)) return FLEXSPEC_ERR_UNSUPPORTED;
+    if (max_m * c.vocab > (1LL << 40) || c.vocab > kMaxVocab) return FLEXSPEC_ERR_UNSUPPORTED;
 
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || c.device >= n_dev) { cudaGetLastError(); return FLEXSPEC_ERR_NO_DEVICE; }
@@ -339,13 +335,10 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.plan.cu_q, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
+    A(dev_alloc(&h.plan.k_eff, static_cast<size_t>(c.max_batch)));
     A(dev_alloc(&h.stats, static_cast<size_t>(max_m + h.max_s) * n_chunks));
     A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128 + h.sm_count)));
-    A(dev_alloc(&h.counters, static_cast<size_t>(2) * kMaxBatch));
-    A(dev_alloc(&h.row_info, static_cast<size_t>(c.max_batch) * 8));
     A(dev_alloc(&h.topp, static_cast<size_t>(max_m) * 2));
-    A(dev_alloc(&h.row_stats, static_cast<size_t>(c.max_batch) * (kMaxK + 1) * 8));
-    A(dev_alloc(&h.chunk_mass, static_cast<size_t>(c.max_batch) * ((c.vocab + kDrawChunk - 1) / kDrawChunk) * 2));
     A(dev_alloc(&h.dbg_p, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.dbg_q, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.dbg_u, static_cast<size_t>(h.max_s)));
@@ -358,8 +351,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
         if (cudaMalloc(&h.stage_dev, h.stage_bytes) != cudaSuccess) { cudaGetLastError(); rc = FLEXSPEC_ERR_OOM; }
     }
     if (rc == FLEXSPEC_OK) {
-        if (cudaMemset(h.counters, 0, sizeof(int32_t) * 2 * kMaxBatch) != cudaSuccess ||
-            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 4) != cudaSuccess ||
+        if (cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 4) != cudaSuccess ||
             cudaMemset(h.status, 0, sizeof(int32_t) * 4) != cudaSuccess)
             rc = FLEXSPEC_ERR_CUDA;
     }
@@ -374,7 +366,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
                                             static_cast<uint64_t>(d_model), 128);
     if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map_last, lm_head_w, static_cast<uint64_t>(c.vocab),
                                             static_cast<uint64_t>(d_model), static_cast<uint32_t>(h.lm_last_rows));
-    if (rc == FLEXSPEC_OK && (attention_init(c.head_dim) != cudaSuccess || lm_head_init() != cudaSuccess))
+    if (rc == FLEXSPEC_OK && (attention_init(c.head_dim) != cudaSuccess || lm_head_init() != cudaSuccess || sample_init() != cudaSuccess))
         rc = FLEXSPEC_ERR_CUDA;
     if (rc != FLEXSPEC_OK) {
         cudaGetLastError();
@@ -452,7 +444,7 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    rc = run_plan(h, draft_len, draft_tokens, batch, s);
+    rc = run_plan(h, draft_len, draft_tokens, batch, g, s);
     if (rc != FLEXSPEC_OK) return rc;
     return run_sample(h, logits ? logits : h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch,
                       temperature, vocab_mask, accepted_len, next_token, s);
@@ -487,7 +479,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     // nothing from the target model, so they run beside attention and the LM head
     if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
-    rc = run_plan(h, draft_len, draft_tokens, batch, h.side);
+    rc = run_plan(h, draft_len, draft_tokens, batch, g, h.side);
     if (rc != FLEXSPEC_OK) return rc;
     if (!sp.greedy && sp.s_rows > 0) {
         if (launch_sample_stats(sp, sp.m_rows, sp.s_rows, h.side) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
@@ -512,13 +504,9 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
         if (launch_sample_nucleus(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;     // needs the row -> sequence table only with a mask: joined above
         h.launches++;
     }
-    if (launch_sample_decide(sp, g.k_batch_max, sp.top_p >= 1.f, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    h.launches++;
     mark(h, 5, s);
-    if (!sp.greedy) {
-        if (launch_sample_draw(sp, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-        h.launches++;
-    }
+    if (launch_sample_accept(sp, sp.top_p >= 1.f, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    h.launches++;
     mark(h, 6, s);
     return FLEXSPEC_OK;
 }
@@ -656,7 +644,12 @@ int flexspec_status(flexspec_handle* fh, int32_t* status_host)
     int32_t st[4] = {0, 0, 0, 0};
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
     if (cudaMemcpy(st, h.status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (st[0] != 0 && cudaMemset(h.status, 0, sizeof(st)) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (st[0] != 0) {
+        // a kernel that gave up may have left its arrival tickets half counted: start the next call clean
+        if (cudaMemset(h.status, 0, sizeof(st)) != cudaSuccess ||
+            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 4) != cudaSuccess)
+            return FLEXSPEC_ERR_CUDA;
+    }
     if (status_host != nullptr) memcpy(status_host, st, sizeof(st));
     return st[0];
 }
@@ -677,8 +670,8 @@ int flexspec_get_stage_ms(flexspec_handle* fh, float ms[6])
     if (!h.profiling || !h.ev_used[0] || !h.ev_used[6]) return FLEXSPEC_ERR_INVALID_ARG;
     DeviceGuard guard(h.cfg.device);
     if (cudaEventSynchronize(h.ev[6]) != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
-    // events: 0 start, 1 after plan, 2 after attention split kernel, 3 after combine, 4 after LM head,
-    // 5 after sample statistics, 6 end
+    // events: 0 call start, 1 after the fork of the second stream, 2 = 3 after attention, 4 after the LM head,
+    // 5 after the nucleus kernel (top-p only; else = 4), 6 after the acceptance kernel
     for (int i = 0; i < 6; ++i) {
         if (!h.ev_used[i] || !h.ev_used[i + 1]) continue;
         if (cudaEventElapsedTime(&ms[i], h.ev[i], h.ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }

@@ -18,6 +18,7 @@ __device__ __forceinline__ void report_error(int32_t* status, int32_t code, int3
     }
 }
 
+constexpr int32_t kErrInvalidArg = -1;
 constexpr int32_t kErrTimeout = -5;
 constexpr int32_t kErrBadPage = -6;
 constexpr int32_t kErrBadToken = -7;
@@ -28,6 +29,14 @@ constexpr int32_t kErrBadToken = -7;
 // Without the attribute both are no-ops.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------- thread-block clusters
+// Split barrier over all threads of the cluster.  Every thread of every CTA executes both halves,
+// at points where its warp is converged; arrive has release, wait has acquire semantics, so
+// distributed-shared-memory writes before the arrive are visible after the wait.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync() { cluster_arrive(); cluster_wait(); }
 
 // ---------------------------------------------------------------------------- addresses
 __device__ __forceinline__ uint32_t smem_u32(const void* p)

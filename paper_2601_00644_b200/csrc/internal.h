@@ -13,7 +13,10 @@ namespace fs {
 constexpr int kMaxBatch = 1024;
 constexpr int kMaxK = 63;
 constexpr int kSampleChunk = 8192;        // vocabulary entries per CTA of the statistics kernel
-constexpr int kDrawChunk = 2048;          // vocabulary entries per CTA of the draw kernel
+constexpr int kAcceptCluster = 8;         // CTAs (one thread-block cluster) per sequence in the acceptance kernel
+constexpr int kWarpChunk = 1024;          // vocabulary entries whose mass one warp adds up at a time there
+constexpr int kMaxWarpChunksPerCta = 128; // per-CTA list of warp-chunk masses in shared memory
+constexpr int kMaxVocab = kAcceptCluster * kMaxWarpChunksPerCta * kWarpChunk;   // 1 048 576
 constexpr int kAttBlockTokens = 128;      // KV tokens per attention work block / pipeline stage
 constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block (MMA M)
 constexpr int kAttProducerWarps = 2;      // issuing a TMA request costs ~55 cycles of its warp: two warps share a block's 32
@@ -25,6 +28,8 @@ struct Plan {                 // device tables written by the plan kernel, read 
     int32_t* cu_q;            // [max_batch+1] first query row of each sequence
     int32_t* cu_d;            // [max_batch+1] first draft row of each sequence
     int32_t* row_seq;         // [max_m] sequence of each query row
+    int32_t* k_eff;           // [max_batch] draft length the sampling kernels use: draft_len[b] once it has been
+                              // checked against the geometry the host sized the launches for (0 if it disagrees)
 };
 
 struct AttnParams {
@@ -90,7 +95,7 @@ struct SampleParams {
     const int32_t* cu_q;
     const int32_t* cu_d;
     const int32_t* row_seq;
-    int32_t batch, vocab, m_rows, s_rows, n_chunks, n_dchunks, mask_words;
+    int32_t batch, vocab, m_rows, s_rows, n_chunks, mask_words;
     int32_t row_begin;            // first row of this launch of the statistics kernel
     float inv_temp_log2;          // log2(e) / T
     int32_t greedy;
@@ -98,13 +103,10 @@ struct SampleParams {
                                   // units, sum exp), or (max, arg-max index as int bits) in greedy mode
     const float2* tstats;         // parts of the target rows: [M][n_tparts] (from the LM head), or = stats
     int32_t n_tparts;
-    int32_t* counters;            // [2][max_batch] self-resetting tickets (decision, draw)
-    double* row_stats;            // [B][kMaxK+1][8]: (max_p, sum_p, max_q, sum_q, rejected) of every row, or the arg-max in [0]
-    double* row_info;             // [B][8]: max_p, 1/sum_p, max_q, 1/sum_q of row n, [4] its nucleus threshold (logit)
+    const int32_t* k_eff;         // [B] checked draft lengths (plan kernel)
     float top_p;                  // nucleus mass of the target distribution; >= 1: no filtering
     double* topp;                 // [M][2]: lowest kept logit of the row's nucleus, mass of the nucleus (in units of
                                   // 2^((z - max) * c)); written by the nucleus kernel when top_p < 1
-    double* chunk_mass;           // [B][n_dchunks][2]: residual mass, p mass
     int32_t* accepted_len;
     int32_t* next_token;
     double* dbg_p; double* dbg_q; float* dbg_u;   // [S] or null
@@ -124,7 +126,7 @@ struct Handle {
     float* logits;
     float* part_o; float* part_ml; int32_t* att_tickets; int32_t att_pairs_max;
     Plan plan;
-    float2* stats; float2* tstats; int32_t* counters; double* row_stats; double* row_info; double* topp; float top_p; double* chunk_mass;
+    float2* stats; float2* tstats; double* topp; float top_p;
     double* dbg_p; double* dbg_q; float* dbg_u;
     int32_t* status;
     // host staging for flexspec_verify_host
@@ -139,8 +141,10 @@ struct Handle {
 };
 
 // launch wrappers (each returns a cudaError_t from the launch)
+// m_rows / s_rows / k_cap: the geometry derived from the HOST copy of the lengths; the kernel checks the
+// device copy against it
 cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
-                        Plan plan, int32_t* status, cudaStream_t stream);
+                        int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status, cudaStream_t stream);
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
                              cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
@@ -148,8 +152,7 @@ cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_
 // pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
 // the stream drains; it waits on the device before touching the predecessor's results)
 cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream);
-cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, bool pdl, cudaStream_t stream);
-cudaError_t launch_sample_draw(const SampleParams& p, bool pdl, cudaStream_t stream);
+cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream);
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
@@ -171,6 +174,7 @@ cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
 int attention_p_bufs(int n_pad);
 void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages);
 cudaError_t lm_head_init();
+cudaError_t sample_init();                  // opt-in shared memory size of the acceptance kernel (per device)
 size_t lm_head_smem_bytes(int n_tile, int n_blocks, int num_stages);
 int lm_head_pick_stages(int n_tile, int n_blocks);
 

@@ -13,21 +13,17 @@ constexpr int kStaticMaxBatch = 64;
 constexpr int kStaticMaxRows = 1024;                 // M = sum_b (k_b + 1)
 constexpr int kStaticMaxVocab = 131072;
 constexpr int kStaticChunks = (kStaticMaxVocab + kSampleChunk - 1) / kSampleChunk;       // 16
-constexpr int kStaticDrawChunks = (kStaticMaxVocab + kDrawChunk - 1) / kDrawChunk;       // 64
 
 constexpr size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
-// layout of the scratch array (every piece 256-byte aligned)
+// layout of the scratch array (every piece 256-byte aligned): 268 032 bytes in all
 constexpr size_t kOffStatus = 0;                                                          // int32[4]
-constexpr size_t kOffCounters = kOffStatus + 256;                                         // int32[2][kMaxBatch]
-constexpr size_t kOffCuQ = kOffCounters + align256(sizeof(int32_t) * 2 * kMaxBatch);
+constexpr size_t kOffCuQ = kOffStatus + 256;                                              // int32[batch + 1]
 constexpr size_t kOffCuD = kOffCuQ + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));
-constexpr size_t kOffRowSeq = kOffCuD + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));
-constexpr size_t kOffStats = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);
-constexpr size_t kOffRowInfo = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
-constexpr size_t kOffRowStats = kOffRowInfo + align256(sizeof(double) * kStaticMaxBatch * 8);
-constexpr size_t kOffMass = kOffRowStats + align256(sizeof(double) * kStaticMaxBatch * (kMaxK + 1) * 8);
-constexpr size_t kScratchBytes = kOffMass + align256(sizeof(double) * kStaticMaxBatch * kStaticDrawChunks * 2);
+constexpr size_t kOffKEff = kOffCuD + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));   // int32[batch]
+constexpr size_t kOffRowSeq = kOffKEff + align256(sizeof(int32_t) * kStaticMaxBatch);      // int32[rows]
+constexpr size_t kOffStats = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);      // float2[2 * rows][chunks]
+constexpr size_t kScratchBytes = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
 
 // In host code this name is only a handle for the runtime: the device address comes from
 // cudaGetSymbolAddress (below), once per device.
@@ -79,13 +75,14 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
             cudaGetLastError();
             return FLEXSPEC_ERR_CUDA;
         }
+        if (sample_init() != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }   // a function attribute, no allocation
         g_scratch_ptr[dev] = static_cast<unsigned char*>(ptr);
     }
     unsigned char* base = g_scratch_ptr[dev];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    // the array keeps whatever the previous call left: the status word and the arrival counters
-    // must start at zero
+    // the array keeps whatever the previous call left: the status word must start at zero (the
+    // tables and statistics behind it are fully rewritten by this call's kernels before they are read)
     if (cudaMemsetAsync(base + kOffStatus, 0, kOffCuQ - kOffStatus, s) != cudaSuccess) {
         cudaGetLastError();
         return FLEXSPEC_ERR_CUDA;
@@ -95,31 +92,27 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     Plan plan;
     plan.cu_q = reinterpret_cast<int32_t*>(base + kOffCuQ);
     plan.cu_d = reinterpret_cast<int32_t*>(base + kOffCuD);
+    plan.k_eff = reinterpret_cast<int32_t*>(base + kOffKEff);
     plan.row_seq = reinterpret_cast<int32_t*>(base + kOffRowSeq);
-    if (launch_plan(draft_len, draft_tokens, batch, vocab, plan, status, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_plan(draft_len, draft_tokens, batch, vocab, m_rows, s_rows, k_batch_max, plan, status, s) != cudaSuccess)
+        return FLEXSPEC_ERR_CUDA;
 
     SampleParams p;
     memset(&p, 0, sizeof(p));
     p.greedy = greedy ? 1 : 0;
     p.logits = logits; p.draft_logits = draft_logits; p.draft_tokens = draft_tokens;
     p.draft_len = draft_len; p.seeds = seeds; p.vocab_mask = vocab_mask;
-    p.cu_q = plan.cu_q; p.cu_d = plan.cu_d; p.row_seq = plan.row_seq;
+    p.cu_q = plan.cu_q; p.cu_d = plan.cu_d; p.row_seq = plan.row_seq; p.k_eff = plan.k_eff;
     p.batch = batch; p.vocab = vocab; p.m_rows = m_rows; p.s_rows = s_rows;
     p.n_chunks = (vocab + kSampleChunk - 1) / kSampleChunk;
-    p.n_dchunks = (vocab + kDrawChunk - 1) / kDrawChunk;
     p.mask_words = (vocab + 31) / 32;
     p.inv_temp_log2 = greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     p.stats = reinterpret_cast<float2*>(base + kOffStats);
     p.tstats = p.stats; p.n_tparts = p.n_chunks;
     p.top_p = 1.f; p.topp = nullptr;
-    p.counters = reinterpret_cast<int32_t*>(base + kOffCounters);
-    p.row_info = reinterpret_cast<double*>(base + kOffRowInfo);
-    p.row_stats = reinterpret_cast<double*>(base + kOffRowStats);
-    p.chunk_mass = reinterpret_cast<double*>(base + kOffMass);
     p.accepted_len = accepted_len; p.next_token = next_token;
     p.status = status;
     if (launch_sample_stats(p, 0, greedy ? m_rows : m_rows + s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (launch_sample_decide(p, k_batch_max, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
-    if (!greedy && launch_sample_draw(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_accept(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     return FLEXSPEC_OK;
 }

@@ -1,7 +1,7 @@
 // Plan kernel: the small per-call tables the sampling stage reads.  One CTA; thread b handles
 // sequence b.  Prefix sums of (k_b + 1) and k_b give the packed row offsets of the ragged batch
 // (FlexSpec's channel-aware stride makes k_b differ per sequence, Section IV-B).  Draft tokens
-// are range-checked here.
+// are range-checked here, and the device copy of the lengths is checked against the host's.
 #include "common.cuh"
 #include "internal.h"
 
@@ -33,20 +33,41 @@ __device__ __forceinline__ int block_inclusive_scan(int v, int* warp_tot)
     return v + before;
 }
 
+// The launches of a call are sized on the host from the HOST copy of the draft lengths (m_rows,
+// s_rows, k_cap = the largest k_b), while the kernels index with the DEVICE copy.  If the two
+// disagree -- a length outside [0, k_cap], or totals that differ -- every later index could leave
+// its array, so the call is neutralised instead: an error goes to the status word, every
+// sequence is treated as k_b = 0 on row min(b, m_rows - 1), and all tables stay inside [0, m_rows).
 __global__ void __launch_bounds__(kMaxBatch)
 plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ draft_tokens, int32_t batch,
-            int32_t vocab, Plan plan, int32_t* status)
+            int32_t vocab, int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status)
 {
     __shared__ int warp_tot[32];
     const int t = threadIdx.x;
     const bool live = t < batch;
-    const int k = live ? draft_len[t] : 0;
+    const int k_raw = live ? draft_len[t] : 0;
+    const int k = min(max(k_raw, 0), k_cap);
     if (t < 32) warp_tot[t] = 0;
     __syncthreads();
     const int q_end = block_inclusive_scan(live ? k + 1 : 0, warp_tot);
     const int d_end = block_inclusive_scan(k, warp_tot);
+    int bad = (live && k_raw != k) ? 1 : 0;
+    if (t == batch - 1 && (q_end != m_rows || d_end != s_rows)) bad = 1;
+    bad = __syncthreads_or(bad);
+    if (bad) {
+        if (t == 0) report_error(status, kErrInvalidArg, k_raw, 7);
+        if (live) {
+            plan.k_eff[t] = 0;
+            plan.cu_q[t] = min(t, m_rows - 1);
+            plan.cu_d[t] = 0;
+        }
+        if (t == 0) { plan.cu_q[batch] = m_rows; plan.cu_d[batch] = 0; }
+        for (int r = t; r < m_rows; r += blockDim.x) plan.row_seq[r] = 0;
+        return;
+    }
     if (live) {
         const int q0 = q_end - (k + 1), d0 = d_end - k;
+        plan.k_eff[t] = k;
         plan.cu_q[t] = q0;
         plan.cu_d[t] = d0;
         for (int j = 0; j <= k; ++j) plan.row_seq[q0 + j] = t;
@@ -63,10 +84,10 @@ plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ d
 }
 
 cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
-                        Plan plan, int32_t* status, cudaStream_t stream)
+                        int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status, cudaStream_t stream)
 {
     const int threads = (batch + 31) / 32 * 32;
-    plan_kernel<<<1, threads, 0, stream>>>(draft_len, draft_tokens, batch, vocab, plan, status);
+    plan_kernel<<<1, threads, 0, stream>>>(draft_len, draft_tokens, batch, vocab, m_rows, s_rows, k_cap, plan, status);
     return cudaGetLastError();
 }
 

@@ -13,12 +13,13 @@
 //            by shuffles, one block barrier).  Serves the draft rows (ahead of time, on a second
 //            stream) and, for the stand-alone stage, the target rows; inside flexspec_verify the
 //            LM-head kernel writes the target rows' parts from its epilogue.
-//   decide : one CTA per sequence merges the parts of its rows, evaluates the acceptance tests
-//            with Philox uniforms, finds the first rejection by warp vote, stores accepted_len.
-//   draw   : grid (chunk of 2048, sequence) over row n of each sequence only: probability mass of
-//            the residual (and of p) per chunk, fp32 exponentials accumulated in fp64; the last
-//            CTA of a sequence picks the chunk that holds u' * Z and scans it in vocabulary order
-//            (inverse CDF).
+//   accept : one cluster of eight CTAs per sequence: merges the parts of the sequence's rows,
+//            evaluates the acceptance tests with Philox uniforms, finds the first rejection by warp
+//            vote, and draws the emitted token from row n by inverse CDF in vocabulary order
+//            (fp32 exponentials accumulated in fp64) -- results travel between the CTAs through
+//            distributed shared memory, so the whole decision is one launch.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -27,7 +28,6 @@ namespace fs {
 constexpr int kSampleThreads = 256;
 constexpr int kSampleWarps = kSampleThreads / 32;
 constexpr int kElemsPerThread = kSampleChunk / kSampleThreads;   // 32
-constexpr int kDrawElems = kDrawChunk / kSampleThreads;          // 8
 
 __device__ __forceinline__ bool mask_allows(const uint32_t* mask_row, int v)
 {
@@ -278,99 +278,225 @@ cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream)
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------------------------------------ decision
-// grid (row j, sequence b): the CTA merges the parts of target row j (and draft row j) of the
-// sequence -- maximum first, then the sum with fp32 weights accumulated in fp64 -- and leaves
-// (max, sum) per row together with the outcome of the row's own acceptance test (Philox uniform,
-// u * q(x) < p(x)).  The CTA that arrives last for the sequence (atomic ticket, nobody waits) finds
-// the first rejection by warp vote and stores accepted_len; GREEDY compares the draft with the
-// rows' arg-max.
-__device__ __forceinline__ float block_max(float v, float* red, int lane, int warp)
+// ------------------------------------------------------------------------------------ acceptance
+// One thread-block cluster of eight CTAs per sequence does the whole decision in one launch; the
+// CTAs hand their results to one another through distributed shared memory, so there are no
+// global-memory tickets, fences or second launch on the path from the logits to the outputs.
+//
+//   before the dependency wait (the kernel is launched programmatically behind the LM head): what
+//     needs only the step's inputs and the draft-logit statistics -- the draft token, q_j(x_j) and
+//     the Philox uniform of every acceptance test of this CTA's rows (rows are dealt round-robin).
+//   A  each CTA merges the parts of its target rows (maximum first, then the sum with fp32 weights
+//     accumulated in fp64), evaluates u * q(x) < p(x) (GREEDY: compares x with the arg-max) and
+//     writes the row's result into the shared memory of all eight CTAs.        -- cluster barrier --
+//   B  every CTA finds the first rejection n by warp vote over the row results (GREEDY ends here).
+//   C  row n only: the vocabulary is cut into eight contiguous slices, one per CTA, and a slice into
+//     chunks of 1024 entries, one warp each: the mass of the emission weights of each chunk is
+//     recorded, slice totals go to all CTAs.                                    -- cluster barrier --
+//   D  the CTA whose slice holds u' * Z picks the chunk from its list and one warp scans those
+//     1024 entries in vocabulary order (inverse CDF).  If rounding leaves no entry above the
+//     threshold, the last entry with positive mass is taken, at every level.
+//
+// The kernel runs once per step and is short, and the step streams gigabytes through L2 in between,
+// so its instructions are fetched cold (from DRAM) every time: straight-line code was measured at
+// about a microsecond per few KB on this path.  The loops of C and D are therefore kept rolled and
+// the logits travel to shared memory asynchronously (all copies of a chunk in flight at once) instead
+// of into a long unrolled register tile; D then scans the picked chunk where C left it.
+//
+// Arithmetic of C and D.  The weights are kept in units of 1 / s_p (s = sum of 2^((z - max) c) of a
+// row): w_v = max(0, e_p(v) - rho e_q(v)) at a rejection, rho = s_p / s_q, and w_v = e_p(v) for the
+// bonus row, with e = the same fp32 2^x as in the statistics.  A common factor does not move the
+// inverse CDF, so no entry is ever normalised.  Entries are fp32 (one fused multiply-add); a lane
+// adds 32 of them in fp32 and everything above that -- lanes, chunks, slices, the running sums of
+// the final scan -- is fp64.  (Double-precision arithmetic per entry was measured at 12 us for this
+// phase alone: the vector fp64 rate of this GPU is a small fraction of its fp32 rate.)
+namespace cg = cooperative_groups;
+
+constexpr int kAcceptThreads = 256;        // two CTAs per SM: every cluster of a 16-sequence batch finds room at once
+constexpr int kAcceptWarps = kAcceptThreads / 32;
+constexpr int kAcceptRowsPerCta = (kMaxK + 1 + kAcceptCluster - 1) / kAcceptCluster;   // 8
+
+struct RowResult {
+    double s_p, s_q, tau;             // sum of 2^((z - max) * c) of the target / draft row; lowest kept logit of the nucleus
+    float m_p, m_q;                   // maxima (logit units)
+    int32_t rej;                      // 1: this row's draft token is rejected
+    int32_t argmax;                   // GREEDY: lowest index holding the row's maximum
+};
+
+// Row n of one sequence: the unnormalised weights the emitted token is drawn from.
+struct DrawRow {
+    const float* zt; const float* zd; const uint32_t* mask;
+    float mp, mq, c, tau;             // tau: lowest logit of the target row's nucleus (-inf: no top-p filter)
+    float rho;                        // s_p / s_q
+    bool residual;
+    bool plain;                       // no vocabulary mask and no nucleus: e_p needs no per-entry checks
+    // 2^((z - max) c); a logit of -inf gives 2^-inf = 0 by itself
+    __device__ __forceinline__ float e_p(float z, int v) const
+    {
+        if (!plain && (z < tau || !mask_allows(mask, v))) return 0.f;
+        return fast_exp2((z - mp) * c);
+    }
+    __device__ __forceinline__ float e_q(float z) const { return fast_exp2((z - mq) * c); }
+    // weight of entry v; use_p: draw from p itself (bonus row, or a residual without mass)
+    __device__ __forceinline__ float weight(float zt_v, float zd_v, int v, bool use_p) const
+    {
+        const float ep = e_p(zt_v, v);
+        return use_p ? ep : fmaxf(fmaf(-rho, e_q(zd_v), ep), 0.f);
+    }
+};
+// A chunk of kWarpChunk entries of a logits row in shared memory.  Entry i sits at chunk_pos(i): inside
+// its group of 32 the four-entry (16-byte) pieces are permuted by the group index, so that 16-byte
+// copies stay whole, the lane-interleaved walk (lane l takes entry 32 g + l) is conflict-free and
+// the lane-contiguous one (lane l takes entry 32 l + e) meets at most four lanes per bank.
+__device__ __forceinline__ int chunk_pos(int i) { return i ^ (((i >> 5) & 7) << 2); }
+__device__ __forceinline__ void cp_async_16(float* smem_dst, const float* src)
 {
-    v = warp_max(v);
-    __syncthreads();                                   // red may still be read from a previous use
-    if (lane == 0) red[warp] = v;
-    __syncthreads();
-    float r = red[0];
-#pragma unroll
-    for (int w = 1; w < kSampleWarps; ++w) r = fmaxf(r, red[w]);
-    return r;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
 }
-__device__ __forceinline__ double block_sum(double v, double* red, int lane, int warp)
+__device__ __forceinline__ void cp_async_4(float* smem_dst, const float* src)
 {
-    v = warp_sum(v);
-    __syncthreads();
-    if (lane == 0) red[warp] = v;
-    __syncthreads();
-    double r = 0.0;
-#pragma unroll
-    for (int w = 0; w < kSampleWarps; ++w) r += red[w];
-    return r;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+// One warp requests the entries [base, base + kWarpChunk) of a row (those below vocab); nothing is
+// awaited.  vec_ok: the row starts on a 16-byte boundary and vocab is a multiple of four.
+__device__ __forceinline__ void stage_chunk(float* dst, const float* row, int base, int vocab, bool vec_ok, int lane)
+{
+    if (vec_ok) {
+#pragma unroll 4
+        for (int i = lane * 4; i < kWarpChunk; i += 128)
+            if (base + i < vocab) cp_async_16(dst + chunk_pos(i), row + base + i);
+    } else {
+#pragma unroll 4
+        for (int i = lane; i < kWarpChunk; i += 32)
+            if (base + i < vocab) cp_async_4(dst + chunk_pos(i), row + base + i);
+    }
 }
 
-constexpr int kRowStat = 8;       // doubles per (sequence, row): max_p, sum_p, max_q, sum_q, rejected
-
-__global__ void __launch_bounds__(kSampleThreads)
-sample_decide_kernel(const SampleParams p)
+__device__ __forceinline__ double warp_inclusive_scan(double v, int lane)
 {
-    __shared__ float red_f[kSampleWarps];
-    __shared__ double red_d[kSampleWarps];
-    __shared__ int red_i[kSampleWarps];
-    __shared__ int s_last;
-    const int j = blockIdx.x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// In a list of n masses (vocabulary order) finds the first entry at which the running sum, started
+// at `carry`, exceeds thr; if none does, the last entry with positive mass (-1 if there is none).
+// Called by one full warp; `mass(i)` returns the i-th mass.  Returns the index and the running sum
+// before it.
+template <typename MassFn>
+__device__ __forceinline__ int warp_pick(int n, double carry, double thr, int lane, MassFn mass, double& before)
+{
+    int pick = -1, last_pos = -1;
+    double last_before = 0.0;
+    before = carry;
+    for (int c0 = 0; c0 < n && pick < 0; c0 += 32) {
+        const int cc = c0 + lane;
+        const double m = (cc < n) ? mass(cc) : 0.0;
+        const double incl = warp_inclusive_scan(m, lane) + carry;
+        const unsigned hit = __ballot_sync(0xffffffffu, cc < n && m > 0.0 && incl > thr);
+        const unsigned pos = __ballot_sync(0xffffffffu, m > 0.0);
+        if (hit != 0u) {
+            const int l = __ffs(hit) - 1;
+            pick = c0 + l;
+            before = __shfl_sync(0xffffffffu, incl - m, l);
+        } else if (pos != 0u) {
+            const int l = 31 - __clz(pos);
+            last_pos = c0 + l;
+            last_before = __shfl_sync(0xffffffffu, incl - m, l);
+        }
+        carry = __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (pick < 0) { pick = last_pos; before = last_before; }
+    return pick;
+}
+
+__global__ void __cluster_dims__(kAcceptCluster, 1, 1) __launch_bounds__(kAcceptThreads)
+sample_accept_kernel(const SampleParams p)
+{
+    __shared__ RowResult s_row[kMaxK + 1];               // results of all rows of the sequence (every CTA holds a copy)
+    __shared__ RowResult s_tmp;
+    __shared__ double2 s_wc[kMaxWarpChunksPerCta];       // (residual mass, p mass) of this CTA's chunks
+    __shared__ double s_slice[kAcceptCluster][2];        // slice totals of all CTAs
+    __shared__ float red_f[kAcceptWarps];
+    __shared__ double red_d[kAcceptWarps];
+    __shared__ int red_i[kAcceptWarps];
+    __shared__ int s_x[kAcceptRowsPerCta];
+    __shared__ double s_qt[kAcceptRowsPerCta], s_u[kAcceptRowsPerCta], s_mq[kAcceptRowsPerCta], s_sq[kAcceptRowsPerCta];
+    __shared__ double s_u2[kMaxK + 1];                   // uniform of the emitted token after n accepted drafts, every n
+    __shared__ int s_n;
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = static_cast<int>(cluster.block_rank());
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    pdl_launch_dependents();
-    const int k_b = p.draft_len[b];                      // inputs of the step: not written by the preceding kernel
-    if (j > k_b) return;
+    const int k_b = p.k_eff[b];                            // tables of the plan kernel: complete before the preceding kernel started
     const int q0 = p.cu_q[b], d0 = p.cu_d[b];
     const double scale = static_cast<double>(p.inv_temp_log2);
     const float cf = p.inv_temp_log2;
-    double* rs = p.row_stats + (static_cast<int64_t>(b) * (kMaxK + 1) + j) * kRowStat;
-    const bool test_row = !p.greedy && j < k_b;
+    const int my_rows = (k_b >= rank) ? (k_b - rank) / kAcceptCluster + 1 : 0;      // rows rank, rank + 8, ... <= k_b
+    cluster_arrive();                                      // "this CTA runs": awaited before the first write into a peer's shared memory
 
-    // ---- everything that depends only on the step's inputs and on the draft-logit statistics (second
-    // stream, joined before the preceding kernel started) is done before that kernel's results are
-    // awaited: the draft token, q_j(x_j) and the uniform of this row's acceptance test
-    int x = 0;
-    double mq = 0.0, sq = 1.0, qt = 0.0, u = 0.0;
-    if (test_row && warp == 0) {
-        const float2* dp = p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks;
-        float mqf = -INFINITY;
-        for (int i = lane; i < p.n_chunks; i += 32) mqf = fmaxf(mqf, __ldcg(&dp[i].x));
-        mqf = warp_max(mqf);
-        double acc = 0.0;
-        for (int i = lane; i < p.n_chunks; i += 32) {
-            const float2 pt = __ldcg(&dp[i]);
-            if (pt.x != -INFINITY) acc += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - mqf) * cf));
-        }
-        sq = warp_sum(acc);
-        mq = static_cast<double>(mqf);
-        if (lane == 0) {
-            x = p.draft_tokens[d0 + j];
+    // ---- what needs no target logits.  The uniforms of the emitted token, one per possible n:
+    if (!p.greedy && threadIdx.x <= k_b) s_u2[threadIdx.x] = philox_uniform(p.seeds[b], static_cast<uint32_t>(threadIdx.x), 1u);
+    // ---- draft side of this CTA's acceptance tests: warp i handles row rank + 8 i
+    if (warp < my_rows) {
+        const int j = rank + warp * kAcceptCluster;
+        if (j < k_b) {
+            int x = p.draft_tokens[d0 + j];
             x = min(max(x, 0), p.vocab - 1);
-            const double zq = static_cast<double>(p.draft_logits[static_cast<int64_t>(d0 + j) * p.vocab + x]);
-            qt = (zq == -INFINITY) ? 0.0 : exp2((zq - mq) * scale) / sq;
-            u = philox_uniform(p.seeds[b], static_cast<uint32_t>(j), 0u);
+            if (!p.greedy) {
+                const float2* dp = p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks;
+                float mqf = -INFINITY;
+                for (int i = lane; i < p.n_chunks; i += 32) mqf = fmaxf(mqf, __ldcg(&dp[i].x));
+                mqf = warp_max(mqf);
+                double acc = 0.0;
+                for (int i = lane; i < p.n_chunks; i += 32) {
+                    const float2 pt = __ldcg(&dp[i]);
+                    if (pt.x != -INFINITY) acc += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - mqf) * cf));
+                }
+                const double sq = warp_sum(acc);
+                if (lane == 0) {
+                    const double mq = static_cast<double>(mqf);
+                    const double zq = static_cast<double>(p.draft_logits[static_cast<int64_t>(d0 + j) * p.vocab + x]);
+                    s_mq[warp] = mq; s_sq[warp] = sq;
+                    s_qt[warp] = (zq == -INFINITY) ? 0.0 : static_cast<double>(fast_exp2(static_cast<float>((zq - mq) * scale))) / sq;
+                    s_u[warp] = philox_uniform(p.seeds[b], static_cast<uint32_t>(j), 0u);
+                }
+            }
+            if (lane == 0) s_x[warp] = x;
+        } else if (lane == 0) {
+            s_x[warp] = 0; s_mq[warp] = 0.0; s_sq[warp] = 1.0; s_qt[warp] = 0.0; s_u[warp] = 0.0;
         }
     }
-    pdl_wait();
+    __syncthreads();
+    pdl_wait();                                            // the target logits and their parts come from the preceding kernel
+    cluster_wait();                                        // all eight CTAs of the cluster have started
 
-    // ---- target row j: merge the parts (one pass, running (max, sum) per thread in fp32, fp64 sums across the block)
-    double zp = 0.0;
-    if (test_row && threadIdx.x == 0) {
-        zp = static_cast<double>(p.logits[static_cast<int64_t>(q0 + j) * p.vocab + x]);
-        if (p.vocab_mask != nullptr && !mask_allows(p.vocab_mask + static_cast<int64_t>(b) * p.mask_words, x)) zp = -INFINITY;
-    }
-    {
+    // ---- A: this CTA's target rows
+    for (int i = 0; i < my_rows; ++i) {
+        const int j = rank + i * kAcceptCluster;
+        const bool test_row = j < k_b;
+        const int x = s_x[i];
+        double zp = 0.0;
+        if (test_row && !p.greedy && threadIdx.x == 0) {
+            zp = static_cast<double>(p.logits[static_cast<int64_t>(q0 + j) * p.vocab + x]);
+            if (p.vocab_mask != nullptr && !mask_allows(p.vocab_mask + static_cast<int64_t>(b) * p.mask_words, x)) zp = -INFINITY;
+        }
         const float2* tp = p.tstats + static_cast<int64_t>(q0 + j) * p.n_tparts;
         const int n = p.n_tparts;
         if (p.greedy) {
             float m = -INFINITY;
             int best = 0x7fffffff;
 #pragma unroll 8
-            for (int i = threadIdx.x; i < n; i += kSampleThreads) {
-                const float2 pt = __ldcg(&tp[i]);
+            for (int t = threadIdx.x; t < n; t += kAcceptThreads) {
+                const float2 pt = __ldcg(&tp[t]);
                 const int idx = __float_as_int(pt.y);
                 if (pt.x > m || (pt.x == m && idx < best)) { m = pt.x; best = idx; }
             }
@@ -383,280 +509,215 @@ sample_decide_kernel(const SampleParams p)
             if (lane == 0) { red_f[warp] = m; red_i[warp] = best; }
             __syncthreads();
             if (threadIdx.x == 0) {
-                for (int w = 1; w < kSampleWarps; ++w)
+                for (int w = 1; w < kAcceptWarps; ++w)
                     if (red_f[w] > m || (red_f[w] == m && red_i[w] < best)) { m = red_f[w]; best = red_i[w]; }
-                rs[0] = static_cast<double>(best);
+                s_tmp.argmax = best;
+                s_tmp.rej = (test_row && x != best) ? 1 : 0;
+                s_tmp.m_p = m; s_tmp.m_q = 0.f; s_tmp.s_p = 1.0; s_tmp.s_q = 1.0; s_tmp.tau = -INFINITY;
             }
         } else {
             float m = -INFINITY, sf = 0.f;
-#pragma unroll 8
-            for (int i = threadIdx.x; i < n; i += kSampleThreads) {
-                const float2 pt = __ldcg(&tp[i]);
+#pragma unroll 16
+            for (int t = threadIdx.x; t < n; t += kAcceptThreads) {
+                const float2 pt = __ldcg(&tp[t]);
                 merge_ms(m, sf, pt.x, pt.y, cf);
             }
+            // block-wide (max, sum): maxima through shared memory, then the sums rescaled to the common maximum
             const float mt = m;
-            m = block_max(m, red_f, lane, warp);
+            m = warp_max(m);
+            if (lane == 0) red_f[warp] = m;
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < kAcceptWarps; ++w) m = fmaxf(m, red_f[w]);
             double sm = (mt == -INFINITY) ? 0.0 : static_cast<double>(sf) * static_cast<double>(fast_exp2((mt - m) * cf));
-            sm = block_sum(sm, red_d, lane, warp);
+            sm = warp_sum(sm);
+            if (lane == 0) red_d[warp] = sm;
+            __syncthreads();
             if (threadIdx.x == 0) {
+                sm = 0.0;
+#pragma unroll
+                for (int w = 0; w < kAcceptWarps; ++w) sm += red_d[w];
                 double tau = -INFINITY;                   // nucleus of the target row: its lowest kept logit and its mass
                 if (p.top_p < 1.f) { tau = p.topp[static_cast<int64_t>(q0 + j) * 2]; sm = p.topp[static_cast<int64_t>(q0 + j) * 2 + 1]; }
-                rs[0] = static_cast<double>(m); rs[1] = sm; rs[2] = mq; rs[3] = sq; rs[5] = tau;
-                double rej = 0.0;
+                int rej = 0;
                 if (test_row) {
-                    const double pt = (zp == -INFINITY || zp < tau) ? 0.0 : exp2((zp - static_cast<double>(m)) * scale) / sm;
-                    rej = (u * qt < pt) ? 0.0 : 1.0;
+                    const double u = s_u[i], qt = s_qt[i];
+                    // the same fp32 2^x as in the statistics (the exponent itself is formed in fp64)
+                    const double pt = (zp == -INFINITY || zp < tau) ? 0.0
+                        : static_cast<double>(fast_exp2(static_cast<float>((zp - static_cast<double>(m)) * scale))) / sm;
+                    rej = (u * qt < pt) ? 0 : 1;
                     if (p.dbg_p != nullptr) {
                         p.dbg_p[d0 + j] = pt;
                         p.dbg_q[d0 + j] = qt;
                         p.dbg_u[d0 + j] = static_cast<float>(u);
                     }
                 }
-                rs[4] = rej;
+                s_tmp.m_p = m; s_tmp.s_p = sm; s_tmp.tau = tau;
+                s_tmp.m_q = static_cast<float>(s_mq[i]); s_tmp.s_q = s_sq[i];
+                s_tmp.rej = rej; s_tmp.argmax = 0;
             }
         }
-    }
-    // ---- ticket: the last row of the sequence finds the first rejection
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int tk = atomicAdd(&p.counters[b], 1);
-        s_last = (tk == k_b);
-        if (s_last) { p.counters[b] = 0; __threadfence(); }          // ready for the next call
-    }
-    __syncthreads();
-    if (!s_last || warp != 0) return;
-    __threadfence();
-
-    const double* rs0 = p.row_stats + static_cast<int64_t>(b) * (kMaxK + 1) * kRowStat;
-    int n = k_b;
-    for (int base = 0; base < k_b; base += 32) {
-        const int jj = base + lane;
-        bool rej = false;
-        if (jj < k_b)
-            rej = p.greedy ? (p.draft_tokens[d0 + jj] != static_cast<int>(__ldcg(rs0 + jj * kRowStat)))
-                           : (__ldcg(rs0 + jj * kRowStat + 4) != 0.0);
-        const unsigned vote = __ballot_sync(0xffffffffu, rej);
-        if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
-    }
-    if (lane == 0) {
-        p.accepted_len[b] = n;
-        const double* rn = rs0 + n * kRowStat;
-        if (p.greedy) {
-            p.next_token[b] = static_cast<int>(__ldcg(rn));
-        } else {
-            double* ri = p.row_info + static_cast<int64_t>(b) * 8;
-            ri[0] = __ldcg(rn); ri[1] = 1.0 / __ldcg(rn + 1);
-            ri[2] = (n < k_b) ? __ldcg(rn + 2) : 0.0; ri[3] = (n < k_b) ? 1.0 / __ldcg(rn + 3) : 1.0;
-            ri[4] = __ldcg(rn + 5);
-        }
-    }
-}
-
-cudaError_t launch_sample_decide(const SampleParams& p, int32_t k_batch_max, bool pdl, cudaStream_t stream)
-{
-    return launch_kernel_ex(sample_decide_kernel, dim3(k_batch_max + 1, p.batch), dim3(kSampleThreads), 0, stream, pdl, p);
-}
-
-// ------------------------------------------------------------------------------------ draw
-// Row n of one sequence: p_v and the residual max(0, p_v - q_v).  The exponentials are the same
-// fp32 2^x as in the statistics pass, so numerator and normaliser share their rounding; products
-// and all sums are fp64.
-struct DrawRow {
-    const float* zt; const float* zd; const uint32_t* mask;
-    float mp, mq, c, tau;         // tau: lowest logit of the target row's nucleus (-inf: no top-p filter)
-    double inv_sp, inv_sq;
-    bool residual;
-    __device__ __forceinline__ double prob_p(float z, int v) const
-    {
-        if (z == -INFINITY || z < tau || !mask_allows(mask, v)) return 0.0;
-        return static_cast<double>(fast_exp2((z - mp) * c)) * inv_sp;
-    }
-    __device__ __forceinline__ double prob_q(float z) const
-    {
-        if (z == -INFINITY) return 0.0;
-        return static_cast<double>(fast_exp2((z - mq) * c)) * inv_sq;
-    }
-    // loads the 8 consecutive entries starting at v (v % 8 == 0) of the target / draft row
-    __device__ __forceinline__ void load8(const float* row, int v, int v_end, bool vec_ok, float (&out)[8]) const
-    {
-        if (vec_ok && v + 7 < v_end) {
-            const float4 a = __ldg(reinterpret_cast<const float4*>(row + v));
-            const float4 b = __ldg(reinterpret_cast<const float4*>(row + v + 4));
-            out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
-            out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) out[i] = (v + i < v_end) ? __ldg(row + v + i) : -INFINITY;
-        }
-    }
-};
-
-__device__ __forceinline__ double warp_inclusive_scan(double v, int lane)
-{
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double t = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= o) v += t;
-    }
-    return v;
-}
-
-__global__ void __launch_bounds__(kSampleThreads)
-sample_draw_kernel(const SampleParams p)
-{
-    __shared__ double red_r[kSampleWarps];
-    __shared__ double red_p[kSampleWarps];
-    __shared__ int s_is_last, s_chunk, s_use_p, s_found, s_last;
-    __shared__ double s_before, s_thr;
-
-    const int chunk = blockIdx.x;
-    const int b = blockIdx.y;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int k_b = p.draft_len[b];
-    pdl_wait();                                          // accepted_len and the row statistics come from the decision kernel
-    const int n = p.accepted_len[b];
-    DrawRow row;
-    row.zt = p.logits + static_cast<int64_t>(p.cu_q[b] + n) * p.vocab;
-    row.residual = (n < k_b);
-    row.zd = row.residual ? p.draft_logits + static_cast<int64_t>(p.cu_d[b] + n) * p.vocab : nullptr;
-    row.mask = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(b) * p.mask_words : nullptr;
-    const double* ri = p.row_info + static_cast<int64_t>(b) * 8;
-    row.mp = static_cast<float>(ri[0]); row.inv_sp = ri[1];
-    row.mq = static_cast<float>(ri[2]); row.inv_sq = ri[3];
-    row.tau = static_cast<float>(ri[4]);
-    row.c = p.inv_temp_log2;
-    const bool vec_ok = ((p.vocab & 3) == 0);
-
-    // thread t owns the contiguous entries [v0 + 8t, v0 + 8t + 8): vocabulary order is kept
-    {
-        const int v0 = chunk * kDrawChunk;
-        const int v_end = min(p.vocab, v0 + kDrawChunk);
-        const int my0 = v0 + threadIdx.x * kDrawElems;
-        double mass_r = 0.0, mass_p = 0.0;
-        if (my0 < v_end) {
-            float zt[8], zd[8];
-            row.load8(row.zt, my0, v_end, vec_ok, zt);
-            if (row.residual) row.load8(row.zd, my0, v_end, vec_ok, zd);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const double pv = row.prob_p(zt[i], my0 + i);
-                mass_p += pv;
-                if (row.residual) { const double d = pv - row.prob_q(zd[i]); mass_r += d > 0.0 ? d : 0.0; }
-            }
-        }
-        mass_r = warp_sum(mass_r);
-        mass_p = warp_sum(mass_p);
-        if (lane == 0) { red_r[warp] = mass_r; red_p[warp] = mass_p; }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            double tr = 0.0, tp = 0.0;
-#pragma unroll
-            for (int w = 0; w < kSampleWarps; ++w) { tr += red_r[w]; tp += red_p[w]; }
-            double* cm = p.chunk_mass + (static_cast<int64_t>(b) * p.n_dchunks + chunk) * 2;
-            cm[0] = tr; cm[1] = tp;
-            __threadfence();
-            const int t = atomicAdd(&p.counters[kMaxBatch + b], 1);
-            s_is_last = (t == p.n_dchunks - 1);
-            if (s_is_last) { p.counters[kMaxBatch + b] = 0; __threadfence(); }
-        }
-        __syncthreads();
-        if (!s_is_last) return;
-        __threadfence();
+        if (threadIdx.x < kAcceptCluster) *cluster.map_shared_rank(&s_row[j], threadIdx.x) = s_tmp;
+        __syncthreads();                                   // s_tmp and the reduction arrays are reused by the next row
     }
+    cluster_sync();                                        // every row result is in every CTA's shared memory
 
-    // ---- the last CTA of the sequence: pick the chunk that holds u' * Z ...
-    const double* cm = p.chunk_mass + static_cast<int64_t>(b) * p.n_dchunks * 2;
+    // ---- B: first rejection
     if (warp == 0) {
-        double z_r = 0.0, z_p = 0.0;
-        for (int c0 = 0; c0 < p.n_dchunks; c0 += 32) {
-            const int cc = c0 + lane;
-            z_r += (cc < p.n_dchunks) ? cm[cc * 2] : 0.0;
-            z_p += (cc < p.n_dchunks) ? cm[cc * 2 + 1] : 0.0;
+        int n = k_b;
+        for (int base = 0; base < k_b; base += 32) {
+            const int jj = base + lane;
+            const bool rej = jj < k_b && s_row[jj].rej != 0;
+            const unsigned vote = __ballot_sync(0xffffffffu, rej);
+            if (vote != 0u && n == k_b) n = base + __ffs(vote) - 1;
         }
-        z_r = warp_sum(z_r);
-        z_p = warp_sum(z_p);
-        const int use_p = !(row.residual && z_r > 0.0);       // bonus row, or a residual lost to rounding
-        const double z_mass = use_p ? z_p : z_r;
-        const double thr = philox_uniform(p.seeds[b], static_cast<uint32_t>(n), 1u) * z_mass;
-        double carry = 0.0, last_before = 0.0;
-        int pick = -1, last_pos = 0;
-        double before = 0.0;
-        for (int c0 = 0; c0 < p.n_dchunks && pick < 0; c0 += 32) {
-            const int cc = c0 + lane;
-            const double m = (cc < p.n_dchunks) ? cm[cc * 2 + use_p] : 0.0;
-            const double incl = warp_inclusive_scan(m, lane) + carry;
-            const unsigned hit = __ballot_sync(0xffffffffu, cc < p.n_dchunks && incl > thr);
-            const unsigned pos = __ballot_sync(0xffffffffu, m > 0.0);
-            if (hit != 0u) {
-                const int l = __ffs(hit) - 1;
-                pick = c0 + l;
-                before = __shfl_sync(0xffffffffu, incl - m, l);
-            } else if (pos != 0u) {
-                const int l = 31 - __clz(pos);
-                last_pos = c0 + l;
-                last_before = __shfl_sync(0xffffffffu, incl - m, l);
-            }
-            carry = __shfl_sync(0xffffffffu, incl, 31);
-        }
-        if (pick < 0) { pick = last_pos; before = last_before; }
         if (lane == 0) {
-            s_chunk = pick; s_use_p = use_p; s_before = before; s_thr = thr;
-            s_found = 0x7fffffff; s_last = -1;
-        }
-    }
-    __syncthreads();
-
-    // ... and scan it in vocabulary order
-    const bool use_p = s_use_p != 0;
-    const int w0 = s_chunk * kDrawChunk + threadIdx.x * kDrawElems;
-    const int w_end = min(p.vocab, (s_chunk + 1) * kDrawChunk);
-    double r[8];
-    double mine = 0.0;
-    {
-        float zt[8], zd[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { zt[i] = -INFINITY; zd[i] = -INFINITY; }
-        if (w0 < w_end) {
-            row.load8(row.zt, w0, w_end, vec_ok, zt);
-            if (!use_p) row.load8(row.zd, w0, w_end, vec_ok, zd);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            double v = 0.0;
-            if (w0 + i < w_end) {
-                const double pv = row.prob_p(zt[i], w0 + i);
-                if (use_p) v = pv;
-                else { const double d = pv - row.prob_q(zd[i]); v = d > 0.0 ? d : 0.0; }
+            s_n = n;
+            if (rank == 0) {
+                p.accepted_len[b] = n;
+                if (p.greedy) p.next_token[b] = s_row[n].argmax;
             }
-            r[i] = v;
-            mine += v;
         }
     }
-    const double incl = warp_inclusive_scan(mine, lane);
-    if (lane == 31) red_r[warp] = incl;
     __syncthreads();
-    double run = s_before + (incl - mine);
-    for (int w = 0; w < warp; ++w) run += red_r[w];
-    int found = 0x7fffffff, last_pos = -1;
+    if (p.greedy) return;                                  // uniform over the cluster; no barrier follows
+    const int n = s_n;
+
+    // ---- C: masses of row n over this CTA's slice of the vocabulary
+    extern __shared__ float s_chunks[];                    // [warps][2][kWarpChunk]: target and draft entries of a warp's chunk
+    DrawRow row;
+    row.zt = p.logits + static_cast<int64_t>(q0 + n) * p.vocab;
+    row.residual = (n < k_b);
+    row.zd = row.residual ? p.draft_logits + static_cast<int64_t>(d0 + n) * p.vocab : nullptr;
+    row.mask = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(b) * p.mask_words : nullptr;
+    row.mp = s_row[n].m_p;
+    row.mq = row.residual ? s_row[n].m_q : 0.f;
+    row.rho = row.residual ? static_cast<float>(s_row[n].s_p / s_row[n].s_q) : 0.f;
+    row.tau = static_cast<float>(s_row[n].tau);
+    row.plain = (row.mask == nullptr && row.tau == -INFINITY);
+    row.c = cf;
+    const bool vec_ok = ((p.vocab & 3) == 0);
+    const int wc_total = (p.vocab + kWarpChunk - 1) / kWarpChunk;
+    const int wc_per_cta = (wc_total + kAcceptCluster - 1) / kAcceptCluster;     // <= kMaxWarpChunksPerCta (vocab <= kMaxVocab)
+    const int wc_begin = min(wc_total, rank * wc_per_cta);
+    const int n_wc = min(wc_total, wc_begin + wc_per_cta) - wc_begin;
+    float* my_zt = s_chunks + warp * 2 * kWarpChunk;
+    float* my_zd = my_zt + kWarpChunk;
+#pragma unroll 1
+    for (int i = warp; i < n_wc; i += kAcceptWarps) {
+        const int base = (wc_begin + i) * kWarpChunk;
+        __syncwarp();                                      // the previous chunk of this warp has been read
+        stage_chunk(my_zt, row.zt, base, p.vocab, vec_ok, lane);
+        if (row.residual) stage_chunk(my_zd, row.zd, base, p.vocab, vec_ok, lane);
+        cp_async_wait_all();
+        __syncwarp();
+        float mr = 0.f, mp = 0.f;
+#pragma unroll 4
+        for (int e = lane; e < kWarpChunk; e += 32) {
+            const int v = base + e;
+            if (v < p.vocab) {
+                const float ep = row.e_p(my_zt[chunk_pos(e)], v);
+                mp += ep;
+                if (row.residual) mr += fmaxf(fmaf(-row.rho, row.e_q(my_zd[chunk_pos(e)]), ep), 0.f);
+            }
+        }
+        const double dr = warp_sum(static_cast<double>(mr));
+        const double dp = warp_sum(static_cast<double>(mp));
+        if (lane == 0) s_wc[i] = make_double2(dr, dp);
+    }
+    __syncthreads();
+    if (warp == 0) {
+        double tr = 0.0, tp = 0.0;
+        for (int i = lane; i < n_wc; i += 32) { tr += s_wc[i].x; tp += s_wc[i].y; }
+        tr = warp_sum(tr);
+        tp = warp_sum(tp);
+        if (lane < kAcceptCluster) {
+            double* dst = cluster.map_shared_rank(&s_slice[0][0], lane);
+            dst[rank * 2 + 0] = tr;
+            dst[rank * 2 + 1] = tp;
+        }
+    }
+    cluster_sync();                                        // slice totals are everywhere; no remote access after this
+    if (warp != 0) return;
+
+    // ---- D: which slice holds u' * Z, which chunk of it, which entry
+    double z_r = 0.0, z_p = 0.0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        run += r[i];
-        if (r[i] > 0.0) last_pos = w0 + i;
-        if (run > s_thr && found == 0x7fffffff && r[i] > 0.0) found = w0 + i;
+    for (int c = 0; c < kAcceptCluster; ++c) { z_r += s_slice[c][0]; z_p += s_slice[c][1]; }
+    const bool use_p = !(row.residual && z_r > 0.0);      // bonus row, or a residual lost to rounding
+    const double thr = s_u2[n] * (use_p ? z_p : z_r);
+    // the slice that holds thr (every lane walks the eight totals itself: shorter than a shuffle scan)
+    double before = 0.0;
+    int slice = -1;
+    {
+        double run = 0.0, last_before = 0.0;
+        int last_pos = -1;
+#pragma unroll
+        for (int c = 0; c < kAcceptCluster; ++c) {
+            const double m = s_slice[c][use_p ? 1 : 0];
+            if (slice < 0 && m > 0.0) {
+                if (run + m > thr) { slice = c; before = run; }
+                else { last_pos = c; last_before = run; }
+            }
+            run += m;
+        }
+        if (slice < 0) { slice = last_pos; before = last_before; }
     }
-    if (found != 0x7fffffff) atomicMin(&s_found, found);
-    if (last_pos >= 0) atomicMax(&s_last, last_pos);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        // if rounding left no entry above the threshold: the last entry with positive mass
-        p.next_token[b] = (s_found != 0x7fffffff) ? s_found : (s_last >= 0 ? s_last : 0);
+    if (slice < 0) {                                       // no mass anywhere (every token masked): token 0
+        if (rank == 0 && lane == 0) p.next_token[b] = 0;
+        return;
     }
+    if (slice != rank) return;
+    const int wc = max(0, warp_pick(n_wc, before, thr, lane, [&](int i) { return use_p ? s_wc[i].y : s_wc[i].x; }, before));
+    const int base = (wc_begin + wc) * kWarpChunk;
+    // the chunk's entries: still in the shared memory of the warp that added them up, unless that warp
+    // went on to a later chunk (vocabularies beyond 16 chunks per slice): then they are fetched again
+    const float* c_zt = s_chunks + (wc % kAcceptWarps) * 2 * kWarpChunk;
+    if (wc + kAcceptWarps < n_wc) {
+        stage_chunk(my_zt, row.zt, base, p.vocab, vec_ok, lane);
+        if (row.residual) stage_chunk(my_zd, row.zd, base, p.vocab, vec_ok, lane);
+        cp_async_wait_all();
+        __syncwarp();
+        c_zt = my_zt;
+    }
+    const float* c_zd = c_zt + kWarpChunk;
+    // lane l adds up the 32 consecutive entries [base + 32 l, base + 32 l + 32)
+    double mine = 0.0;
+#pragma unroll 4
+    for (int e = 0; e < 32; ++e) {
+        const int v = base + lane * 32 + e;
+        if (v < p.vocab)
+            mine += static_cast<double>(row.weight(c_zt[chunk_pos(lane * 32 + e)], use_p ? 0.f : c_zd[chunk_pos(lane * 32 + e)], v, use_p));
+    }
+    const double incl = before + warp_inclusive_scan(mine, lane);
+    const unsigned hit = __ballot_sync(0xffffffffu, mine > 0.0 && incl > thr);
+    const unsigned pos = __ballot_sync(0xffffffffu, mine > 0.0);
+    // the group of 32 that holds thr (if rounding left none: the last one with mass), scanned by the whole warp
+    const int grp = hit != 0u ? __ffs(hit) - 1 : (pos != 0u ? 31 - __clz(pos) : 0);
+    const double grp_before = __shfl_sync(0xffffffffu, incl - mine, grp);
+    const int v = base + grp * 32 + lane;
+    const float w = (v < p.vocab) ? row.weight(c_zt[chunk_pos(grp * 32 + lane)], use_p ? 0.f : c_zd[chunk_pos(grp * 32 + lane)], v, use_p) : 0.f;
+    const double run = grp_before + warp_inclusive_scan(static_cast<double>(w), lane);
+    const unsigned hit2 = __ballot_sync(0xffffffffu, w > 0.f && run > thr);
+    const unsigned pos2 = __ballot_sync(0xffffffffu, w > 0.f);
+    // if rounding left no entry above the threshold: the last entry with positive mass
+    const int pick = hit2 != 0u ? __ffs(hit2) - 1 : (pos2 != 0u ? 31 - __clz(pos2) : 0);
+    if (lane == 0) p.next_token[b] = min(base + grp * 32 + pick, p.vocab - 1);
 }
 
-cudaError_t launch_sample_draw(const SampleParams& p, bool pdl, cudaStream_t stream)
+constexpr size_t kAcceptSmemBytes = static_cast<size_t>(kAcceptWarps) * 2 * kWarpChunk * sizeof(float);   // 65 536
+
+cudaError_t sample_init()
 {
-    return launch_kernel_ex(sample_draw_kernel, dim3(p.n_dchunks, p.batch), dim3(kSampleThreads), 0, stream, pdl, p);
+    return cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(kAcceptSmemBytes));
+}
+
+cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream)
+{
+    return launch_kernel_ex(sample_accept_kernel, dim3(kAcceptCluster, p.batch), dim3(kAcceptThreads), kAcceptSmemBytes, stream,
+                            pdl, p);
 }
 
 }  // namespace fs

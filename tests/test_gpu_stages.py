@@ -268,3 +268,32 @@ def test_sample_stage_with_top_p_matches_oracle(top_p, temperature, vocab, batch
     ref1 = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, temperature, vmask)
     assert (acc1.cpu().numpy() != ref1["accepted_len"]).sum() <= 1           # switched off again
     ver.close()
+
+
+def test_device_lengths_that_disagree_with_the_host_copy_are_reported():
+    """The launches are sized from draft_len_host; the kernels index with the device copy.  A device
+    copy that disagrees must not send any index outside its array: the row-offset kernel reports
+    INVALID_ARG through the status word and the stage runs with every k_b = 0."""
+    from paper_2601_00644_b200 import binding as B
+    rng = np.random.RandomState(3)
+    batch, vocab = 5, 4096
+    k = np.array([2, 0, 3, 1, 2], np.int32)
+    m, s = int(k.sum()) + batch, int(k.sum())
+    zt = torch.from_numpy(rng.standard_normal((m, vocab)).astype(np.float32)).cuda()
+    zd = torch.from_numpy(rng.standard_normal((s, vocab)).astype(np.float32)).cuda()
+    toks = torch.from_numpy(rng.randint(0, vocab, s).astype(np.int32)).cuda()
+    seeds = torch.from_numpy(rng.randint(0, 2 ** 62, batch).astype(np.int64)).cuda()
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=8, max_kv_len=64)
+    for bad in ([2, 0, 4, 1, 2], [2, 0, 3, 1, 1], [2, -1, 3, 1, 2], [2, 0, 7, 0, 0]):
+        k_dev = torch.tensor(bad, dtype=torch.int32, device="cuda")
+        acc, nxt = ver.sample(zt, toks, zd, k_dev, torch.from_numpy(k), seeds)
+        torch.cuda.synchronize()
+        code, st = ver.status()
+        assert code == B.ERR_INVALID_ARG, (bad, code, st)
+        assert torch.all(acc == 0) and torch.all((nxt >= 0) & (nxt < vocab))
+    # and the handle is fine afterwards
+    acc, nxt = ver.sample(zt, toks, zd, torch.from_numpy(k).cuda(), torch.from_numpy(k), seeds)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0 and torch.all((acc >= 0) & (acc <= torch.from_numpy(k).cuda()))
+    ver.close()

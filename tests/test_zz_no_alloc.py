@@ -50,6 +50,22 @@ def test_static_entry_matches_handle_entry_on_two_calls_in_a_row(mode, temperatu
         assert torch.equal(got_acc, want_acc)
         assert torch.equal(got_nxt, want_nxt)
         ver.close()
+        # ... and against the fp64 oracle on the same logits: identical except at near-ties
+        # (|u - min(1, p/q)| < 1e-5 for an acceptance test, 1e-6 for the inverse-CDF boundary)
+        import oracle
+        ref = oracle.accept(mode, c["zt"].cpu().numpy().astype(np.float64), c["zd"].cpu().numpy(),
+                            c["toks"].cpu().numpy(), c["k"], c["seeds"].cpu().numpy().view(np.uint64), temperature)
+        t0 = np.concatenate([[0], np.cumsum(c["k"])])
+        acc, nxt = got_acc.cpu().numpy(), got_nxt.cpu().numpy()
+        ties = 0
+        for b in range(len(c["k"])):
+            if acc[b] != ref["accepted_len"][b]:
+                assert ref["acc_margin"][t0[b] + min(acc[b], ref["accepted_len"][b])] < 1e-5
+                ties += 1
+            elif nxt[b] != ref["next_token"][b]:
+                assert ref["cdf_margin"][b] < 1e-6
+                ties += 1
+        assert ties <= 1
 
 
 def test_static_entry_rejects_sizes_beyond_its_array():
