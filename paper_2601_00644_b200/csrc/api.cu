@@ -85,13 +85,14 @@ void free_workspace(Handle& h)
     if (h.ev_fork) cudaEventDestroy(h.ev_fork);
     if (h.ev_join) cudaEventDestroy(h.ev_join);
     if (h.side) cudaStreamDestroy(h.side);
+    free(h.att_seq);
+    h.att_seq = nullptr;
 }
 
 // geometry of one call, derived from the host copies of the lengths
 struct Geometry {
     int32_t m_rows = 0, s_rows = 0, k_batch_max = 0, kv_max = 0;
-    int64_t att_blocks = 0;      // attention work blocks (128 tokens of one pair), as the plan kernel counts them
-    int32_t att_ctas = 0;
+    int64_t att_blocks = 0;      // attention work blocks (128 tokens of one (sequence, kv head, row block) pair)
 };
 
 int check_lengths(const Handle& h, const int32_t* draft_len_host, const int32_t* kv_len_host, int32_t batch,
@@ -116,7 +117,122 @@ int check_lengths(const Handle& h, const int32_t* draft_len_host, const int32_t*
         }
     }
     if (g->att_blocks > 0x7fffffffLL) return FLEXSPEC_ERR_UNSUPPORTED;
-    g->att_ctas = static_cast<int32_t>(g->att_blocks < h.sm_count ? g->att_blocks : h.sm_count);
+    return FLEXSPEC_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention work list.  All 128-token blocks of all (sequence, kv head, row block) pairs, numbered
+// sequence by sequence and pair by pair, are cut into one contiguous range per CTA.  Two cuts are
+// built and the cheaper one is taken:
+//   balanced  : equal ranges (a pair may straddle CTAs; its parts are merged in the kernel);
+//   pair-wise : every CTA takes whole pairs, under the smallest capacity that needs no more CTAs than
+//               there are SMs (no pair is split, so nothing is merged).
+// Cost of a CTA, in microseconds from per-CTA timelines of the kernel: its blocks x the block period
+// for the tile width, a pipeline drain / refill per further segment, and the park-and-merge tail
+// if one of its segments is part of a split pair.
+int32_t pairwise_ctas(const SeqBlocks* sq, int32_t batch, int64_t cap, int32_t* begins, int32_t max_ctas)
+{
+    // greedy: walk the pairs in order, open a new CTA when the next pair does not fit; returns the CTAs used
+    int32_t used = 0;
+    int64_t load = 0, pos = 0;
+    for (int b = 0; b < batch; ++b) {
+        for (int pr = 0; pr < sq[b].pairs; ++pr) {
+            if (used == 0 || load + sq[b].nb > cap) {
+                if (used == max_ctas) return max_ctas + 1;
+                if (begins != nullptr) begins[used] = static_cast<int32_t>(pos);
+                ++used;
+                load = 0;
+            }
+            load += sq[b].nb;
+            pos += sq[b].nb;
+        }
+    }
+    return used;
+}
+
+double cut_cost(const SeqBlocks* sq, int32_t batch, const int32_t* begins, int32_t n_ctas, int64_t total, double t_blk)
+{
+    const double t_seg = 4.0, t_split = 7.5;
+    double worst = 0.0;
+    int b = 0;
+    int64_t seq0 = 0;                                    // first block of sequence b
+    for (int c = 0; c < n_ctas; ++c) {
+        const int64_t lo = begins[c], hi = (c + 1 < n_ctas) ? begins[c + 1] : total;
+        while (seq0 + static_cast<int64_t>(sq[b].pairs) * sq[b].nb <= lo) { seq0 += static_cast<int64_t>(sq[b].pairs) * sq[b].nb; ++b; }
+        // segments of [lo, hi): walk the pairs it touches
+        int segs = 0;
+        bool split = false;
+        int bb = b;
+        int64_t s0 = seq0, x = lo;
+        while (x < hi) {
+            const int64_t in_seq = x - s0;
+            const int64_t pair_lo = s0 + in_seq / sq[bb].nb * sq[bb].nb, pair_hi = pair_lo + sq[bb].nb;
+            ++segs;
+            if (pair_lo < lo || pair_hi > hi) split = true;
+            x = pair_hi < hi ? pair_hi : hi;
+            if (x >= s0 + static_cast<int64_t>(sq[bb].pairs) * sq[bb].nb) { s0 += static_cast<int64_t>(sq[bb].pairs) * sq[bb].nb; ++bb; }
+        }
+        const double cost = static_cast<double>(hi - lo) * t_blk + (segs > 1 ? (segs - 1) * t_seg : 0.0) + (split ? t_split : 0.0);
+        if (cost > worst) worst = cost;
+    }
+    return worst;
+}
+
+int plan_attention(const Handle& h, const int32_t* draft_len_host, const int32_t* kv_len_host, int32_t batch,
+                   const Geometry& g, int32_t n_pad, AttTable* tab, int32_t* n_ctas_out)
+{
+    const flexspec_config& c = h.cfg;
+    const int group = c.n_q_heads / c.n_kv_heads;
+    SeqBlocks* sq = h.att_seq;                           // host scratch of the handle, max_batch entries
+    int32_t max_nb = 0;
+    for (int b = 0; b < batch; ++b) {
+        const int k = draft_len_host[b];
+        sq[b].pairs = c.n_kv_heads * ((group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
+        sq[b].nb = (kv_len_host[b] + kAttBlockTokens - 1) / kAttBlockTokens;
+        sq[b].rows = k + 1;
+        if (sq[b].nb > max_nb) max_nb = sq[b].nb;
+    }
+    const int64_t total = g.att_blocks;
+    int32_t max_ctas = h.sm_count < kAttMaxCtas ? h.sm_count : kAttMaxCtas;
+    if (total < max_ctas) max_ctas = static_cast<int32_t>(total);
+    const double t_blk = n_pad <= 32 ? 1.7 : (n_pad <= 64 ? 2.4 : (n_pad <= 96 ? 3.5 : 4.5));
+
+    int32_t begins_a[kAttMaxCtas], begins_b[kAttMaxCtas];
+    // balanced
+    const int32_t n_a = max_ctas;
+    for (int cta = 0; cta < n_a; ++cta) begins_a[cta] = static_cast<int32_t>(cta * total / n_a);
+    const double cost_a = cut_cost(sq, batch, begins_a, n_a, total, t_blk);
+    // pair-wise: smallest capacity (bisection) that fits into max_ctas CTAs
+    int64_t lo = max_nb, hi = total;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) / 2;
+        if (pairwise_ctas(sq, batch, mid, nullptr, max_ctas) <= max_ctas) hi = mid; else lo = mid + 1;
+    }
+    const int32_t n_b = pairwise_ctas(sq, batch, lo, begins_b, max_ctas);
+    const double cost_b = (n_b <= max_ctas) ? cut_cost(sq, batch, begins_b, n_b, total, t_blk) : 1e300;
+    const bool use_b = cost_b < cost_a;
+    const int32_t* begins = use_b ? begins_b : begins_a;
+    const int32_t n_ctas = use_b ? n_b : n_a;
+
+    // fill the table: one pass over the sequences
+    int b = 0;
+    int64_t seq0 = 0;
+    int32_t row0 = 0, pair0 = 0;
+    for (int cta = 0; cta < n_ctas; ++cta) {
+        const int64_t x = begins[cta];
+        while (seq0 + static_cast<int64_t>(sq[b].pairs) * sq[b].nb <= x) {
+            seq0 += static_cast<int64_t>(sq[b].pairs) * sq[b].nb;
+            row0 += sq[b].rows; pair0 += sq[b].pairs;
+            ++b;
+        }
+        AttCta& e = tab->cta[cta];
+        e.blk_begin = static_cast<int32_t>(x);
+        e.n_my = static_cast<int32_t>(((cta + 1 < n_ctas) ? begins[cta + 1] : total) - x);
+        e.b = b; e.blk_off = static_cast<int32_t>(x - seq0);
+        e.q_row0 = row0; e.pair0 = pair0; e.blk0 = static_cast<int32_t>(seq0);
+        e.k = draft_len_host[b]; e.kvl = kv_len_host[b]; e.pad = 0;
+    }
+    *n_ctas_out = n_ctas;
     return FLEXSPEC_OK;
 }
 
@@ -136,7 +252,7 @@ int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, i
 }
 
 int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const int32_t* draft_len,
-                  const Geometry& g, int32_t batch, void* attn_out, cudaStream_t s)
+                  const int32_t* draft_len_host, const Geometry& g, int32_t batch, void* attn_out, cudaStream_t s)
 {
     const flexspec_config& c = h.cfg;
     const int group = c.n_q_heads / c.n_kv_heads;
@@ -147,6 +263,7 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     if (rc != FLEXSPEC_OK) return rc;
 
     AttnParams p;
+    p.m_rows = g.m_rows; p.k_cap = g.k_batch_max; p.kv_cap = g.kv_max;
     p.hidden = static_cast<const __nv_bfloat16*>(hidden);
     p.page_table = kv->page_table;
     p.kv_len = kv->kv_len;
@@ -163,7 +280,11 @@ int run_attention(Handle& h, const flexspec_kv* kv, const void* hidden, const in
     p.part_o = h.part_o; p.part_ml = h.part_ml; p.tickets = h.att_tickets;
     p.attn_out = static_cast<__nv_bfloat16*>(attn_out);
     p.status = h.status;
-    if (launch_attention(h, kv_map, p, g.att_ctas, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    AttTable tab;
+    int32_t n_ctas = 0;
+    rc = plan_attention(h, draft_len_host, kv->kv_len_host, batch, g, p.n_pad, &tab, &n_ctas);
+    if (rc != FLEXSPEC_OK) return rc;
+    if (launch_attention(h, kv_map, p, tab, n_ctas, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     return FLEXSPEC_OK;
 }
@@ -304,6 +425,8 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     h.sm_count = prop.multiProcessorCount;
     h.w = static_cast<const __nv_bfloat16*>(lm_head_w);
     h.top_p = 1.f;
+    h.att_seq = static_cast<SeqBlocks*>(malloc(sizeof(SeqBlocks) * static_cast<size_t>(c.max_batch)));
+    if (h.att_seq == nullptr) { delete fh; return FLEXSPEC_ERR_OOM; }
 
     const int n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
     // LM-head tiling: full waves of 128-row tiles, then one wave of shorter tiles, one per SM, so that
@@ -414,7 +537,7 @@ int flexspec_attention(flexspec_handle* fh, const flexspec_kv* kv, const void* h
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    return run_attention(h, kv, hidden, draft_len, g, batch, attn_out ? attn_out : h.attn_out, s);
+    return run_attention(h, kv, hidden, draft_len, draft_len_host, g, batch, attn_out ? attn_out : h.attn_out, s);
 }
 
 int flexspec_lm_head(flexspec_handle* fh, const void* x, int32_t m_rows, float* logits, void* stream)
@@ -488,7 +611,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     if (cudaEventRecord(h.ev_join, h.side) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     // ---- main stream
     mark(h, 1, s);
-    rc = run_attention(h, kv, hidden, draft_len, g, batch, h.attn_out, s);
+    rc = run_attention(h, kv, hidden, draft_len, draft_len_host, g, batch, h.attn_out, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 2, s);
     mark(h, 3, s);

@@ -8,8 +8,10 @@
 // (8 pages of 16).  All blocks of the batch, numbered sequence by sequence and pair by pair, are
 // divided into equal contiguous ranges, one per CTA, with one CTA per SM: a single balanced wave
 // whatever the mix of context lengths and draft lengths.  A CTA therefore works on a few
-// "segments" (runs of blocks of one pair).  Every CTA derives its own range from draft_len[] and
-// kv_len[] (a block-wide prefix sum over the sequences), so no planning kernel runs first.
+// "segments" (runs of blocks of one pair).  The host, which has a copy of the lengths, cuts the list
+// -- equal ranges, or whole pairs per CTA when that balances well enough to save every split --
+// and passes each CTA's starting point as a kernel parameter, so a CTA requests its first K/V tile
+// without reading or scanning anything first.
 //
 // Both contractions run on the 5th-generation tensor cores with accumulators in tensor memory
 // (the legacy warp-level MMA path cannot keep up with the KV stream).  A verification step has
@@ -167,40 +169,22 @@ __device__ __forceinline__ uint64_t umma_desc_mn_plain(uint32_t smem_addr, uint3
 constexpr uint32_t kIdescAMajorMN = 1u << 15;
 constexpr uint32_t kIdescBMajorMN = 1u << 16;
 
-// Exclusive prefix sum over the block of one int per thread; returns the block total in `total`.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int& total)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n_warps = (blockDim.x + 31) >> 5;
-    int incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    int before = 0, sum = 0;
-    for (int w = 0; w < n_warps; ++w) {
-        const int t = warp_tot[w];
-        if (w < warp) before += t;
-        sum += t;
-    }
-    __syncthreads();
-    total = sum;
-    return before + incl - v;
-}
-
 // Position in the batch-wide block list; every role walks it in lock step.
 struct AttCursor {
     int b, pair, blk;             // sequence, pair inside it, block inside the pair
     int k, kvl, nb, rbc, pairs;   // of sequence b: draft length, kv length, blocks per pair,
                                   // row blocks per kv head, pairs
     int q_row0, pair0, blk0;      // first query row / first pair / first block of sequence b
+    // the device copies of the lengths are clamped to what the host sized the call for, so that a
+    // device array that disagrees with its host copy cannot send an index outside its buffer
     __device__ __forceinline__ void load_seq(const AttnParams& p)
     {
-        k = p.draft_len[b];
-        kvl = p.kv_len[b];
+        set_seq(p, p.draft_len[b], p.kv_len[b]);
+    }
+    __device__ __forceinline__ void set_seq(const AttnParams& p, int k_in, int kvl_in)
+    {
+        k = min(max(k_in, 0), p.k_cap);
+        kvl = min(max(kvl_in, k + 1), p.kv_cap);
         nb = (kvl + kAttBlockTokens - 1) / kAttBlockTokens;
         rbc = (p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair;
         pairs = p.n_kv_heads * rbc;
@@ -239,8 +223,6 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane)
     return v[0];
 }
 
-struct AttStart { int b, blk_off, q_row0, pair0, blk0, total; };
-
 struct AttSmem {                  // pointers into dynamic shared memory
     uint8_t* k_ring;
     uint8_t* v_ring;
@@ -252,14 +234,24 @@ struct AttSmem {                  // pointers into dynamic shared memory
     int* flags;                   // [2][4] "a score exceeded its maximum by more than the threshold", by block parity and warp
 };
 
+// CTA that holds block x of the batch-wide list: the last one whose range starts at or before x.
+static __device__ __noinline__ int att_owner(const AttTable& tab, int n_ctas, int x)
+{
+    int lo = 0, hi = n_ctas - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (tab.cta[mid].blk_begin <= x) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
 // ------------------------------------------------------------------------------------ softmax role
 // NCH = chunks of 32 columns (query rows) of S^T: n_pad <= 32 * NCH.  Per-column state (running
 // maximum, row sum, output row) lives in lane i of every warp for column 32*ci + i and is
 // broadcast by shuffles, so the four warps only meet once per block (column maxima) and once
 // per segment (row sums).
 template <int DH, int NCH>
-__device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& sm, uint32_t tmem_base, AttCursor cur,
-                                            int n_my, int64_t total_blocks)
+__device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable& tab, const AttSmem& sm, AttCursor cur, int n_my)
 {
     using Cfg = AttCfg<DH>;
     AttBars* bars = sm.bars;
@@ -268,10 +260,14 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
     const int t = quarter * 32 + lane;                  // token of the block (S^T), Dh index (O^T)
     const int cta = blockIdx.x;
     const int n_pad = p.n_pad;
-    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    uint32_t t_lane = 0;                                // set once the TMEM allocation is known (after the first Q tile is staged)
     const int q_slab = n_pad * 128;
     const bool o_lane = quarter * 32 < DH;              // warp-uniform: this warp's lanes hold rows of O^T
 
+    if (n_my <= 0) {                                    // not produced by the host planner; keep the rendezvous whole
+        asm volatile("bar.sync 1, %0;" ::"n"(32 + kAttSoftmaxThreads) : "memory");
+        return;
+    }
     bool ok = true, seg_first = true;
     int seg = 0;
     uint32_t group_phase = 0;
@@ -297,7 +293,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
             for (int idx = t; idx < rows_here * (DH / 8); idx += kAttSoftmaxThreads) {
                 const int row = idx / (DH / 8), ch = idx % (DH / 8);
                 const int rho = row_lo + row;
-                const int64_t src_row = static_cast<int64_t>(cur.q_row0 + rho / p.group) * p.n_q_heads + kvh * p.group + rho % p.group;
+                const int tok_row = min(cur.q_row0 + rho / p.group, p.m_rows - 1);
+                const int64_t src_row = static_cast<int64_t>(tok_row) * p.n_q_heads + kvh * p.group + rho % p.group;
                 const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.hidden + src_row * DH) + ch);
                 *reinterpret_cast<uint4*>(sm.q + (ch >> 3) * q_slab + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = v;
             }
@@ -307,11 +304,17 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
             for (int ci = 0; ci < NCH; ++ci) {
                 m_used[ci] = -INFINITY;
                 const int rho = row_lo + ci * 32 + lane;
-                row_c[ci] = (cur.q_row0 + rho / p.group) * p.n_q_heads + kvh * p.group + rho % p.group;
+                row_c[ci] = min(cur.q_row0 + rho / p.group, p.m_rows - 1) * p.n_q_heads + kvh * p.group + rho % p.group;
             }
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&bars->q_full);
+            if (q == 0) {
+                // the MMA warp allocated tensor memory meanwhile: meet it (warps 2..6) and read the base
+                asm volatile("bar.sync 1, %0;" ::"n"(32 + kAttSoftmaxThreads) : "memory");
+                tc_fence_after();
+                t_lane = bars->tmem_slot + (static_cast<uint32_t>(quarter * 32) << 16);
+            }
         }
         const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
         const int buf = q & 1, u = q >> 1;
@@ -475,7 +478,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         mbar_arrive(&bars->s_empty[buf]);
 
         const int pair_global = cur.pair0 + cur.pair;
-        const int64_t pair_blk_first = static_cast<int64_t>(cur.blk0) + static_cast<int64_t>(cur.pair) * cur.nb;
+        const int pair_blk_first = cur.blk0 + cur.pair * cur.nb;
         const int pair_nb = cur.nb;
         cur.advance(p, q + 1 < n_my);
         seg_first = seg_last;
@@ -506,13 +509,11 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         if (!att_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
         tc_fence_after();
         if (!o_lane) continue;                                         // nothing of O^T in this warp's lanes
-        // which CTAs hold blocks of this pair: CTA c owns blocks [c*T/G, (c+1)*T/G), so the owner of
-        // block x is ceil((x+1)*G/T) - 1
-        const int64_t pair_blk_last = pair_blk_first + pair_nb - 1;
-        const int c_first = static_cast<int>(((pair_blk_first + 1) * gridDim.x - 1) / total_blocks);
-        const int c_last = static_cast<int>(((pair_blk_last + 1) * gridDim.x - 1) / total_blocks);
+        // does the pair reach into another CTA's range?  (this CTA holds blocks [blk_begin, blk_begin + n_my))
+        const int pair_blk_last = pair_blk_first + pair_nb - 1;
+        const bool whole = pair_blk_first >= tab.cta[cta].blk_begin && pair_blk_last < tab.cta[cta].blk_begin + n_my;
 
-        if (c_first == c_last) {
+        if (whole) {
             // the whole pair was ours: normalise and store; thread t holds element t of every row
             __nv_bfloat16* out_t = p.attn_out + t;
 #pragma unroll
@@ -534,6 +535,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
             continue;
         }
 
+        const int c_first = att_owner(tab, gridDim.x, pair_blk_first);
+        const int c_last = att_owner(tab, gridDim.x, pair_blk_last);
         // ---- the pair spans CTAs c_first..c_last: every warp parks its 32 rows of O^T with its own copy
         // of (m, l) and takes its own ticket; the warp that arrives last for (pair, warp) merges those
         // rows.  A CTA's parts are its first and its last segment.
@@ -575,8 +578,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
         // range starts exactly there; every later CTA holds its part in its first segment.  (This path runs
         // once or twice per CTA and is always cold in the instruction cache: it is kept compact.)
         __threadfence();
-        const int blk_begin_c0 = static_cast<int>(static_cast<int64_t>(c_first) * total_blocks / gridDim.x);
-        const int slot_c0 = c_first * 2 + ((blk_begin_c0 == pair_blk_first) ? 0 : 1);
+        const int slot_c0 = c_first * 2 + ((tab.cta[c_first].blk_begin == pair_blk_first) ? 0 : 1);
         // one pass over the parts: the (m, l) of my column and my row of O^T are requested together, and
         // the accumulator is rescaled whenever a part raises a column's maximum
         float m_all[NCH], l_all[NCH];
@@ -634,7 +636,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttSmem& 
 
 template <int DH, int NCH>
 __global__ void __launch_bounds__(kAttThreads, 1)
-attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
+attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ AttnParams p,
+                 const __grid_constant__ AttTable tab)
 {
     using Cfg = AttCfg<DH>;
     extern __shared__ uint8_t smem_raw[];
@@ -650,8 +653,6 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
     sm.m_col = sm.xch + 12 * n_pad;
     sm.flags = reinterpret_cast<int*>(sm.m_col + n_pad);
     AttBars* bars = sm.bars;
-    __shared__ int s_warp_tot[32];
-    __shared__ AttStart s_start;
     __shared__ int s_phys[kAttProducerWarps][8][2 * kAttPagesPerStage / kAttProducerWarps];   // per producer warp: page ids
                                                         // of the blocks between its prefetch cursor and its copies, by lane
 
@@ -672,63 +673,17 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         fence_barrier_init();
         tma_prefetch_desc(&kv_map);
     }
-    if (warp == kAttProducerWarps) {
-        tmem_alloc(&bars->tmem_slot, kAttTmemCols);
-        tmem_relinquish();
-    }
+    __syncthreads();                                    // barriers are initialised: the producers may start
 
-    // ---- where this CTA starts: prefix sums of blocks / pairs / rows over the sequences
-    int blk_begin, n_my;
-    {
-        const int per = (p.batch + blockDim.x - 1) / blockDim.x;
-        const int b_lo = min(p.batch, static_cast<int>(threadIdx.x) * per);
-        const int b_hi = min(p.batch, b_lo + per);
-        int my_blocks = 0, my_pairs = 0, my_rows = 0;
-        for (int b = b_lo; b < b_hi; ++b) {
-            const int k = p.draft_len[b];
-            const int nb = (p.kv_len[b] + kAttBlockTokens - 1) / kAttBlockTokens;
-            const int pairs = p.n_kv_heads * ((p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
-            my_blocks += pairs * nb;
-            my_pairs += pairs;
-            my_rows += k + 1;
-        }
-        int total, unused;
-        const int ex_blocks = block_exclusive_scan(my_blocks, s_warp_tot, total);
-        const int ex_pairs = block_exclusive_scan(my_pairs, s_warp_tot, unused);
-        const int ex_rows = block_exclusive_scan(my_rows, s_warp_tot, unused);
-        const int64_t t64 = total;
-        blk_begin = static_cast<int>(cta * t64 / gridDim.x);
-        n_my = static_cast<int>((cta + 1) * t64 / gridDim.x) - blk_begin;
-        if (n_my > 0 && blk_begin >= ex_blocks && blk_begin < ex_blocks + my_blocks) {
-            int blk0 = ex_blocks, pair0 = ex_pairs, row0 = ex_rows;
-            for (int b = b_lo; b < b_hi; ++b) {
-                const int k = p.draft_len[b];
-                const int nb = (p.kv_len[b] + kAttBlockTokens - 1) / kAttBlockTokens;
-                const int pairs = p.n_kv_heads * ((p.group * (k + 1) + kAttRowsPerPair - 1) / kAttRowsPerPair);
-                if (blk_begin < blk0 + pairs * nb) {
-                    s_start.b = b; s_start.blk_off = blk_begin - blk0;
-                    s_start.q_row0 = row0; s_start.pair0 = pair0; s_start.blk0 = blk0;
-                    break;
-                }
-                blk0 += pairs * nb; pair0 += pairs; row0 += k + 1;
-            }
-        }
-        if (threadIdx.x == 0) s_start.total = total;
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = bars->tmem_slot;
-    const int64_t total_blocks = s_start.total;
-
+    // ---- where this CTA starts (host-computed)
+    const int n_my = tab.cta[cta].n_my;
     AttCursor cur;
-    if (n_my > 0) {
-        cur.b = s_start.b;
-        cur.q_row0 = s_start.q_row0; cur.pair0 = s_start.pair0; cur.blk0 = s_start.blk0;
-        cur.load_seq(p);
-        cur.pair = s_start.blk_off / cur.nb;
-        cur.blk = s_start.blk_off % cur.nb;
-    }
+    cur.b = tab.cta[cta].b;
+    cur.q_row0 = tab.cta[cta].q_row0; cur.pair0 = tab.cta[cta].pair0; cur.blk0 = tab.cta[cta].blk0;
+    cur.set_seq(p, tab.cta[cta].k, tab.cta[cta].kvl);
+    cur.pair = tab.cta[cta].blk_off / cur.nb;
+    cur.blk = tab.cta[cta].blk_off % cur.nb;
+    uint32_t tmem_base = 0;
 
     if (warp < kAttProducerWarps) {
         // ------------------------------------------------------------------ TMA producers
@@ -819,6 +774,14 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
         }
     } else if (warp == kAttProducerWarps) {
         // ------------------------------------------------------------------ MMA issuer
+        // The warp owns the tensor memory: it allocates while the producers already request K/V and the
+        // softmax warps stage the first Q tile, then meets the softmax warps (named barrier 1).
+        tmem_alloc(&bars->tmem_slot, kAttTmemCols);
+        tmem_relinquish();
+        tc_fence_before();
+        asm volatile("bar.sync 1, %0;" ::"n"(32 + kAttSoftmaxThreads) : "memory");
+        tc_fence_after();
+        tmem_base = bars->tmem_slot;
         if (lane == 0 && n_my > 0) {
             // This one thread is on the critical path of every block, so its work per block is kept
             // to a few dozen instructions: descriptors are built once and only advanced by adding
@@ -887,8 +850,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p)
                 }
             }
         }
-    } else if (n_my > 0) {
-        att_softmax<DH, NCH>(p, sm, tmem_base, cur, n_my, total_blocks);
+    } else {
+        att_softmax<DH, NCH>(p, tab, sm, cur, n_my);
     }
 
     tc_fence_before();
@@ -922,22 +885,22 @@ cudaError_t attention_init(int head_dim)
 }
 
 template <int DH>
-static void att_launch_dh(const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas, cudaStream_t stream)
+static void att_launch_dh(const CUtensorMap& kv_map, const AttnParams& p, const AttTable& tab, int32_t n_ctas, cudaStream_t stream)
 {
     const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<DH>::kTileBytes +
                         AttCfg<DH>::fixed_bytes(p.n_pad, p.p_bufs);
     dim3 grid(n_ctas), block(kAttThreads);
-    if (p.n_pad <= 32) attention_kernel<DH, 1><<<grid, block, smem, stream>>>(kv_map, p);
-    else if (p.n_pad <= 64) attention_kernel<DH, 2><<<grid, block, smem, stream>>>(kv_map, p);
-    else if (p.n_pad <= 96) attention_kernel<DH, 3><<<grid, block, smem, stream>>>(kv_map, p);
-    else attention_kernel<DH, 4><<<grid, block, smem, stream>>>(kv_map, p);
+    if (p.n_pad <= 32) attention_kernel<DH, 1><<<grid, block, smem, stream>>>(kv_map, p, tab);
+    else if (p.n_pad <= 64) attention_kernel<DH, 2><<<grid, block, smem, stream>>>(kv_map, p, tab);
+    else if (p.n_pad <= 96) attention_kernel<DH, 3><<<grid, block, smem, stream>>>(kv_map, p, tab);
+    else attention_kernel<DH, 4><<<grid, block, smem, stream>>>(kv_map, p, tab);
 }
 
-cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
-                             cudaStream_t stream)
+cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, const AttTable& tab,
+                             int32_t n_ctas, cudaStream_t stream)
 {
-    if (h.cfg.head_dim == 128) att_launch_dh<128>(kv_map, p, n_ctas, stream);
-    else att_launch_dh<64>(kv_map, p, n_ctas, stream);
+    if (h.cfg.head_dim == 128) att_launch_dh<128>(kv_map, p, tab, n_ctas, stream);
+    else att_launch_dh<64>(kv_map, p, tab, n_ctas, stream);
     return cudaGetLastError();
 }
 

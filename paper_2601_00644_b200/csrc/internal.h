@@ -39,6 +39,7 @@ struct AttnParams {
     const int32_t* draft_len;
     int32_t batch, n_q_heads, n_kv_heads, group;
     int32_t max_pages_per_seq, num_pages;
+    int32_t m_rows, k_cap, kv_cap;   // geometry the host sized the call for: device lengths are clamped to it
     int32_t n_pad;            // MMA N: the largest pair's query rows rounded up to 16 (<= 128)
     int32_t k_stages;         // depth of the K ring (128-token tiles)
     int32_t v_stages;         // depth of the V ring
@@ -49,6 +50,23 @@ struct AttnParams {
     int32_t* tickets;         // [pairs][4 warps] self-resetting arrival counters of the split merge
     __nv_bfloat16* attn_out;  // [M][d_model]
     int32_t* status;
+};
+
+// Where every CTA of the attention kernel starts in the batch-wide list of 128-token blocks, computed
+// on the host from the host copies of the lengths and passed with the launch as a kernel parameter
+// (nothing has to be read or scanned on the device before the first K/V request).
+constexpr int kAttMaxCtas = 160;
+struct AttCta {
+    int32_t blk_begin;        // first block of this CTA in the batch-wide list
+    int32_t n_my;             // blocks of this CTA (> 0)
+    int32_t b;                // sequence of the first block ...
+    int32_t blk_off;          // ... and the block's offset inside that sequence's blocks
+    int32_t q_row0, pair0, blk0;   // first query row / first pair / first block of sequence b
+    int32_t k, kvl;           // draft length and kv length of sequence b (host copy)
+    int32_t pad;
+};
+struct AttTable {
+    AttCta cta[kAttMaxCtas];
 };
 
 struct KvAppendParams {
@@ -113,8 +131,11 @@ struct SampleParams {
     int32_t* status;
 };
 
+struct SeqBlocks { int32_t pairs, nb, rows; };   // attention planner, per sequence: pairs, blocks per pair, query rows
+
 struct Handle {
     flexspec_config cfg;
+    SeqBlocks* att_seq;       // HOST [max_batch]
     int32_t d_model, max_m, max_s;
     int32_t sm_count;
     const __nv_bfloat16* w;
@@ -145,8 +166,8 @@ struct Handle {
 // device copy against it
 cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
                         int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status, cudaStream_t stream);
-cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, int32_t n_ctas,
-                             cudaStream_t stream);
+cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, const AttTable& table,
+                             int32_t n_ctas, cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
 // pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
