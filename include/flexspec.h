@@ -243,6 +243,14 @@ int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);
  * and returns its first entry (0 or a FLEXSPEC_ERR_* code recorded by a kernel). */
 int flexspec_status(flexspec_handle* h, int32_t* status_host);
 
+/* Diagnostic for the bounded waits (no counterpart in the paper).  Every device-side wait of the
+ * library (TMA arrivals, tensor-core completions, hand-overs between warps) gives up after a fixed
+ * wall time, records FLEXSPEC_ERR_TIMEOUT in the status word and lets its kernel return, so a stalled
+ * pipeline never turns into a hung GPU.  This call launches a one-thread kernel that waits, with that
+ * same routine, on a barrier nobody ever signals: after limit_ns (1 us .. 50 ms, else INVALID_ARG)
+ * the wait runs out and flexspec_status returns FLEXSPEC_ERR_TIMEOUT; the handle stays usable. */
+int flexspec_selftest_wait_timeout(flexspec_handle* h, int64_t limit_ns, void* stream);
+
 /* Per-kernel timing.  With profiling on, verify brackets the kernels of the caller's stream with
  * CUDA events; flexspec_get_stage_ms synchronises those events and writes the last call's
  * durations in milliseconds: [0] fork of the second stream, [1] attention, [2] unused,

@@ -26,7 +26,7 @@ EXPORTS = [
     "flexspec_create", "flexspec_verify", "flexspec_verify_host", "flexspec_attention",
     "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_kv_append",
     "flexspec_kv_rollback", "flexspec_set_top_p", "flexspec_get_debug", "flexspec_status",
-    "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
+    "flexspec_selftest_wait_timeout", "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
     "flexspec_destroy", "flexspec_strerror", "flexspec_version",
 ]
 
@@ -68,6 +68,7 @@ def _load() -> C.CDLL:
     lib.flexspec_set_top_p.argtypes = [vp, f32]
     lib.flexspec_get_debug.argtypes = [vp, C.POINTER(Debug)]
     lib.flexspec_status.argtypes = [vp, vp]
+    lib.flexspec_selftest_wait_timeout.argtypes = [vp, C.c_int64, vp]
     lib.flexspec_set_profiling.argtypes = [vp, i32]
     lib.flexspec_get_stage_ms.argtypes = [vp, vp]
     lib.flexspec_last_launches.argtypes = [vp]
@@ -311,6 +312,11 @@ class Verifier:
         st = (C.c_int32 * 4)()
         code = LIB.flexspec_status(self._h, st)
         return code, list(st)
+
+    def selftest_wait_timeout(self, limit_ns: int, stream=None):
+        """Launch the diagnostic kernel whose bounded wait runs out after limit_ns (see the header)."""
+        _check(LIB.flexspec_selftest_wait_timeout(self._h, int(limit_ns), _stream_ptr(stream)),
+               "flexspec_selftest_wait_timeout")
 
     def set_profiling(self, on: bool):
         _check(LIB.flexspec_set_profiling(self._h, 1 if on else 0), "flexspec_set_profiling")

@@ -777,6 +777,17 @@ int flexspec_status(flexspec_handle* fh, int32_t* status_host)
     return st[0];
 }
 
+int flexspec_selftest_wait_timeout(flexspec_handle* fh, int64_t limit_ns, void* stream)
+{
+    if (fh == nullptr || limit_ns < 1000 || limit_ns > 50ll * 1000 * 1000) return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    DeviceGuard guard(h.cfg.device);
+    if (launch_wait_timeout(h.status, static_cast<uint64_t>(limit_ns), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return FLEXSPEC_ERR_CUDA;
+    h.launches = 1;
+    return FLEXSPEC_OK;
+}
+
 int flexspec_set_profiling(flexspec_handle* fh, int32_t on)
 {
     if (fh == nullptr) return FLEXSPEC_ERR_INVALID_ARG;

@@ -24,10 +24,11 @@
 //                                       B = P^T written by the softmax threads ([token][row]:
 //                                       MN-major, unswizzled 8x8 core matrices)
 //
-// Warp roles.  Warps 0-1: TMA producers, each owning half of every block's pages (a TMA request
+// Warp roles (8 warps).  Warps 0-1: TMA producers, each owning half of every block's pages (a TMA request
 // costs about 55 cycles of the issuing warp, and a block needs 32 of them); separate rings of
 // 128-token K and V tiles; the page ids of the next block are looked up one block ahead.
-// Warp 2: one thread issues every tcgen05.mma; the warp owns the TMEM allocation.  Warps 3-6: softmax,
+// Warp 2: one thread issues the QK^T products; the warp owns the TMEM allocation.  Warp 7: one thread
+// issues the PV products (one thread issuing both bounded the kernel).  Warps 3-6: softmax,
 // thread t = token t of the block (TMEM lane t of S^T).  The maximum of a query row over the
 // block is a column maximum: redux.sync.max over each warp, then over the four warps through
 // shared memory.  The running maximum is only raised when it grew by more than 2^8 (O^T in TMEM
@@ -45,6 +46,8 @@ namespace fs {
 constexpr int kPageTokens = 16;
 constexpr int kAttPagesPerStage = kAttBlockTokens / kPageTokens;    // 8
 constexpr int kAttSoftmaxThreads = 128;
+constexpr int kAttPvWarp = kAttProducerWarps + 5;                   // warp order: TMA producers, S^T issuer, 4 softmax warps, PV issuer
+constexpr int kAttConsumerThreads = kAttThreads - kAttProducerWarps * 32;   // everyone who touches tensor memory (named barrier 1)
 constexpr int kAttTmemCols = 512;
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column offsets
 constexpr float kRescaleThreshold = 8.f;                             // log2 units
@@ -101,9 +104,15 @@ void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages)
 
 // The attention kernel waits in dozens of places and its code has to stay small enough for the
 // instruction caches (its cold paths run once per CTA): one shared copy of the wait loop.
-static __device__ __noinline__ bool att_wait(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
+static __device__ __noinline__ bool att_wait_slow(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
 {
     return mbar_wait(bar, parity, status, where);
+}
+// a barrier that has already completed costs one non-blocking test
+__device__ __forceinline__ bool att_wait(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
+{
+    if (mbar_test_wait(bar, parity)) return true;
+    return att_wait_slow(bar, parity, status, where);
 }
 __device__ __forceinline__ void prefetch_l2(const void* p)
 {
@@ -265,7 +274,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
     const bool o_lane = quarter * 32 < DH;              // warp-uniform: this warp's lanes hold rows of O^T
 
     if (n_my <= 0) {                                    // not produced by the host planner; keep the rendezvous whole
-        asm volatile("bar.sync 1, %0;" ::"n"(32 + kAttSoftmaxThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
         return;
     }
     bool ok = true, seg_first = true;
@@ -311,7 +320,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             mbar_arrive(&bars->q_full);
             if (q == 0) {
                 // the MMA warp allocated tensor memory meanwhile: meet it (warps 2..6) and read the base
-                asm volatile("bar.sync 1, %0;" ::"n"(32 + kAttSoftmaxThreads) : "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
                 tc_fence_after();
                 t_lane = bars->tmem_slot + (static_cast<uint32_t>(quarter * 32) << 16);
             }
@@ -773,81 +782,80 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             att_wait(&bars->v_full[ql % p.v_stages], (ql / p.v_stages) & 1, p.status, 9);
         }
     } else if (warp == kAttProducerWarps) {
-        // ------------------------------------------------------------------ MMA issuer
-        // The warp owns the tensor memory: it allocates while the producers already request K/V and the
-        // softmax warps stage the first Q tile, then meets the softmax warps (named barrier 1).
+        // ------------------------------------------------------------------ MMA issuer of S^T = K Q^T
+        // The two products are issued by two threads in two warps: one thread issuing both, with its
+        // barrier waits and commits, took 1.7 us per block and was what bounded the kernel.
+        // This warp also owns the tensor memory: it allocates while the producers already request K/V
+        // and the softmax warps stage the first Q tile, then meets the other consumers (named barrier 1).
         tmem_alloc(&bars->tmem_slot, kAttTmemCols);
         tmem_relinquish();
         tc_fence_before();
-        asm volatile("bar.sync 1, %0;" ::"n"(32 + kAttSoftmaxThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
         tc_fence_after();
         tmem_base = bars->tmem_slot;
         if (lane == 0 && n_my > 0) {
-            // This one thread is on the critical path of every block, so its work per block is kept
-            // to a few dozen instructions: descriptors are built once and only advanced by adding
-            // (byte offset >> 4) to their address field, ring positions are carried, not divided.
+            // descriptors are built once and only advanced by adding (byte offset >> 4) to their address
+            // field, ring positions are carried, not divided
             const uint32_t idesc_s = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad));
-            const uint32_t idesc_o = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad)) | kIdescAMajorMN | kIdescBMajorMN;
             const uint64_t dq0 = umma_desc_k_sw128(smem_u32(sm.q));
             const uint64_t dk0 = umma_desc_k_sw128(smem_u32(sm.k_ring));
-            const uint64_t dv0 = umma_desc_mn_sw128(smem_u32(sm.v_ring), Cfg::kSlabBytes, 1024);
-            const uint64_t dp0 = umma_desc_mn_plain(smem_u32(sm.pt), 2048, 128);
             const uint32_t q_slab16 = (static_cast<uint32_t>(n_pad) * 128u) >> 4;
-            const uint32_t p_buf16 = static_cast<uint32_t>(Cfg::p_bytes(n_pad)) >> 4;
-            bool ok = true;
-            // state of the S^T issue stream (runs one block ahead inside a segment)
-            int s_ks = 0; uint32_t s_kpar = 0;             // K ring slot / parity of its full barrier
-            int s_buf = 0; uint32_t s_spar = 1;            // S^T buffer; parity to wait for on s_empty (previous use)
-            int s_q = 0, s_seg = 0;
-            // S^T[buf] = K Q^T of the next block in order (waits: the pair's Q tile, the K tile, the S^T buffer)
-            auto issue_s = [&](bool seg_first) -> bool {
-                if (seg_first && !att_wait(&bars->q_full, s_seg & 1, p.status, 2)) return false;
-                if (!att_wait(&bars->k_full[s_ks], s_kpar, p.status, 3)) return false;
-                if (s_q >= 2 && !att_wait(&bars->s_empty[s_buf], s_spar, p.status, 4)) return false;
+            int ks = 0; uint32_t kpar = 0;                 // K ring slot / parity of its full barrier
+            int buf = 0; uint32_t spar = 1;                // S^T buffer; parity to wait for on s_empty (previous use)
+            int seg = 0;
+            bool seg_first = true;
+            for (int q = 0; q < n_my; ++q) {
+                // waits: the pair's Q tile (new segment), the K tile, the S^T buffer (two blocks back)
+                if (seg_first && !att_wait(&bars->q_full, seg & 1, p.status, 2)) break;
+                if (!att_wait(&bars->k_full[ks], kpar, p.status, 3)) break;
+                if (q >= 2 && !att_wait(&bars->s_empty[buf], spar, p.status, 4)) break;
                 tc_fence_after();
-                const uint64_t dk = dk0 + static_cast<uint32_t>((s_ks * Cfg::kTileBytes) >> 4);
-                const uint32_t acc = tmem_base + (s_buf ? kTmemS1 : kTmemS0);
+                const uint64_t dk = dk0 + static_cast<uint32_t>((ks * Cfg::kTileBytes) >> 4);
+                const uint32_t acc = tmem_base + (buf ? kTmemS1 : kTmemS0);
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk)
                     umma_bf16(acc, dk + static_cast<uint32_t>(((kk >> 2) * Cfg::kSlabBytes + (kk & 3) * 32) >> 4),
                               dq0 + ((kk >> 2) * q_slab16 + (kk & 3) * 2), idesc_s, kk > 0 ? 1u : 0u);
-                umma_commit(&bars->s_full[s_buf]);
-                umma_commit(&bars->k_empty[s_ks]);
-                if (++s_ks == p.k_stages) { s_ks = 0; s_kpar ^= 1u; }
-                if (s_buf == 1) s_spar ^= 1u;              // both buffers used once more: next round waits the other parity
-                s_buf ^= 1;
-                ++s_q;
-                return true;
-            };
+                umma_commit(&bars->s_full[buf]);
+                umma_commit(&bars->k_empty[ks]);
+                if (++ks == p.k_stages) { ks = 0; kpar ^= 1u; }
+                if (buf == 1) spar ^= 1u;                  // both buffers used once more: next round waits the other parity
+                buf ^= 1;
+                seg_first = (cur.blk == cur.nb - 1);       // the next block opens a segment
+                if (seg_first) ++seg;
+                cur.advance(p, q + 1 < n_my);
+            }
+        }
+    } else if (warp == kAttPvWarp) {
+        // ------------------------------------------------------------------ MMA issuer of O^T += V^T P^T
+        asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
+        tc_fence_after();
+        tmem_base = bars->tmem_slot;
+        if (lane == 0 && n_my > 0) {
+            const uint32_t idesc_o = umma_idesc_bf16(128, static_cast<uint32_t>(n_pad)) | kIdescAMajorMN | kIdescBMajorMN;
+            const uint64_t dv0 = umma_desc_mn_sw128(smem_u32(sm.v_ring), Cfg::kSlabBytes, 1024);
+            const uint64_t dp0 = umma_desc_mn_plain(smem_u32(sm.pt), 2048, 128);
+            const uint32_t p_buf16 = static_cast<uint32_t>(Cfg::p_bytes(n_pad)) >> 4;
             int vs = 0; uint32_t vpar = 0;                 // V ring slot / parity
             int pb = 0; uint32_t ppar = 0;                 // P^T buffer / parity of p_full
             bool seg_first = true;
-            ok = issue_s(true);
-            for (int q = 0; q < n_my && ok; ++q) {
-                const bool seg_last = (cur.blk == cur.nb - 1) || (q + 1 == n_my);
-                if (!seg_last) { if (!issue_s(false)) { ok = false; break; } }     // overlaps the softmax of q
-                if (!att_wait(&bars->v_full[vs], vpar, p.status, 21)) { ok = false; break; }
-                if (!att_wait(&bars->p_full[pb], ppar, p.status, 5)) { ok = false; break; }
+            for (int q = 0; q < n_my; ++q) {
+                if (!att_wait(&bars->v_full[vs], vpar, p.status, 21)) break;
+                if (!att_wait(&bars->p_full[pb], ppar, p.status, 5)) break;
                 tc_fence_after();
-                {
-                    const uint64_t dv = dv0 + static_cast<uint32_t>((vs * Cfg::kTileBytes) >> 4);
-                    const uint64_t dp = dp0 + static_cast<uint32_t>(pb) * p_buf16;
+                const uint64_t dv = dv0 + static_cast<uint32_t>((vs * Cfg::kTileBytes) >> 4);
+                const uint64_t dp = dp0 + static_cast<uint32_t>(pb) * p_buf16;
 #pragma unroll
-                    for (int ks = 0; ks < kAttBlockTokens / 16; ++ks)      // 16 tokens: two groups of 8 k-rows in both operands
-                        umma_bf16(tmem_base + kTmemO, dv + static_cast<uint32_t>((ks * 2048) >> 4), dp + static_cast<uint32_t>((ks * 256) >> 4),
-                                  idesc_o, (seg_first && ks == 0) ? 0u : 1u);
-                }
+                for (int ks = 0; ks < kAttBlockTokens / 16; ++ks)      // 16 tokens: two groups of 8 k-rows in both operands
+                    umma_bf16(tmem_base + kTmemO, dv + static_cast<uint32_t>((ks * 2048) >> 4), dp + static_cast<uint32_t>((ks * 256) >> 4),
+                              idesc_o, (seg_first && ks == 0) ? 0u : 1u);
                 umma_commit(&bars->v_empty[vs]);
                 umma_commit(&bars->p_empty[pb]);
                 umma_commit(&bars->o_full);
                 if (++vs == p.v_stages) { vs = 0; vpar ^= 1u; }
                 if (++pb == p.p_bufs) { pb = 0; ppar ^= 1u; }
+                seg_first = (cur.blk == cur.nb - 1);       // the next block opens a segment
                 cur.advance(p, q + 1 < n_my);
-                seg_first = seg_last;
-                if (seg_last) {
-                    ++s_seg;
-                    if (q + 1 < n_my && !issue_s(true)) { ok = false; break; }
-                }
             }
         }
     } else {

@@ -78,19 +78,48 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls, records a timeout in the status word and
-// returns false; the caller carries on to its normal teardown so nothing is left waiting.
-// try_wait itself suspends the thread for a hardware-chosen interval, so the loop neither
-// burns issue slots (a non-blocking test_wait spin measurably slowed the other warps of the
-// SM) nor adds the wake-up latency of a sleep.
-constexpr uint32_t kWaitLimit = 1u << 24;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
+// Non-blocking test of a phase: true if it has completed.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
 {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-    }
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up once `limit_ns` of wall time (the GPU's nanosecond timer) have passed,
+// records a timeout in the status word and returns false; the caller carries on to its normal
+// teardown so nothing is left waiting.  try_wait itself suspends the thread for a hardware-chosen
+// interval, so the loop neither burns issue slots (a non-blocking test_wait spin measurably slowed
+// the other warps of the SM) nor adds the wake-up latency of a sleep; the clock is read once per
+// 32 polls.
+constexpr uint64_t kWaitLimitNs = 200ull * 1000ull * 1000ull;       // 200 ms: far beyond any wait of a healthy kernel
+__device__ __forceinline__ uint64_t globaltimer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool mbar_wait_ns(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where,
+                                             uint64_t limit_ns)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    do {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+    } while (globaltimer_ns() - t0 <= limit_ns);
     report_error(status, kErrTimeout, static_cast<int32_t>(parity), where);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status, int32_t where)
+{
+    return mbar_wait_ns(bar, parity, status, where, kWaitLimitNs);
 }
 
 // ---------------------------------------------------------------------------- TMA

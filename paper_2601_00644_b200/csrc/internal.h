@@ -20,7 +20,7 @@ constexpr int kMaxVocab = kAcceptCluster * kMaxWarpChunksPerCta * kWarpChunk;   
 constexpr int kAttBlockTokens = 128;      // KV tokens per attention work block / pipeline stage
 constexpr int kAttRowsPerPair = 128;      // query rows per (sequence, kv head) row block (MMA M)
 constexpr int kAttProducerWarps = 2;      // issuing a TMA request costs ~55 cycles of its warp: two warps share a block's 32
-constexpr int kAttThreads = (kAttProducerWarps + 1 + 4) * 32;   // TMA warps + MMA warp + 4 softmax warps
+constexpr int kAttThreads = (kAttProducerWarps + 1 + 4 + 1) * 32;   // TMA warps, QK^T issuer, 4 softmax warps, PV issuer
 constexpr int kAttMaxStages = 8;          // K / V ring depth (what fits in shared memory is used)
 constexpr int kNumStageEvents = 7;
 
@@ -191,6 +191,7 @@ inline cudaError_t launch_kernel_ex(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 cudaError_t launch_kv_append(const KvAppendParams& p, int32_t m_rows, cudaStream_t stream);
 cudaError_t launch_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int32_t* accepted_len, int32_t batch,
                                int32_t* kv_len_next, cudaStream_t stream);
+cudaError_t launch_wait_timeout(int32_t* status, uint64_t limit_ns, cudaStream_t stream);
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
 int attention_p_bufs(int n_pad);
 void attention_stages(int head_dim, int n_pad, int* k_stages, int* v_stages);

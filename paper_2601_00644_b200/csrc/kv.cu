@@ -55,6 +55,24 @@ __global__ void kv_rollback_kernel(const int32_t* __restrict__ kv_len, const int
     if (b < batch) kv_len_next[b] = kv_len[b] - (draft_len[b] + 1) + accepted_len[b] + 1;
 }
 
+// Diagnostic: one thread waits on a barrier on which nobody ever arrives, with the bounded wait every
+// pipeline of the library uses; the wait runs out after limit_ns, the timeout lands in the status
+// word and the kernel returns normally.
+__global__ void wait_timeout_kernel(int32_t* status, uint64_t limit_ns)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+        mbar_wait_ns(&bar, 0u, status, 99, limit_ns);
+    }
+}
+cudaError_t launch_wait_timeout(int32_t* status, uint64_t limit_ns, cudaStream_t stream)
+{
+    wait_timeout_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_kv_append(const KvAppendParams& p, int32_t m_rows, cudaStream_t stream)
 {
     if (m_rows <= 0) return cudaSuccess;

@@ -297,3 +297,24 @@ def test_device_lengths_that_disagree_with_the_host_copy_are_reported():
     torch.cuda.synchronize()
     assert ver.status()[0] == 0 and torch.all((acc >= 0) & (acc <= torch.from_numpy(k).cuda()))
     ver.close()
+
+
+def test_a_bounded_wait_runs_out_and_is_reported():
+    """The wait routine of every pipeline, on a barrier nobody signals, with a limit of two
+    milliseconds: the kernel returns by itself, the status word holds the timeout, and the handle
+    goes on working."""
+    import time
+    from paper_2601_00644_b200 import binding as B
+    w = torch.zeros(256, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=1, k_max=1, max_kv_len=64)
+    t0 = time.perf_counter()
+    ver.selftest_wait_timeout(2_000_000)
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    code, st = ver.status()
+    assert code == B.ERR_TIMEOUT and st[2] == 99
+    assert 0.0015 < waited < 1.0
+    assert ver.status()[0] == 0                    # cleared by the read
+    with pytest.raises(B.FlexSpecError):
+        ver.selftest_wait_timeout(10 ** 9)         # limits beyond 50 ms are refused on the host
+    ver.close()
