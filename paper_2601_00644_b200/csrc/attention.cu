@@ -280,8 +280,11 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
     bool ok = true, seg_first = true;
     int seg = 0;
     uint32_t group_phase = 0;
+    // the four softmax warps meet on an mbarrier, one arrival per warp (128 arrivals on one shared-memory
+    // word serialise: measured ~0.2 us per barrier and block)
     auto group_sync = [&](int where) -> bool {
-        mbar_arrive(&bars->group);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->group);
         const bool done = att_wait(&bars->group, group_phase, p.status, where);
         group_phase ^= 1u;
         return done;
@@ -293,8 +296,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
     int rows_here = 0, row_lo = 0, ctx = 0;
 
     for (int q = 0; q < n_my && ok; ++q) {
-        const int kvh = cur.pair / cur.rbc;
         if (seg_first) {
+            const int kvh = cur.pair / cur.rbc;
             // ---- the pair's query rows -> shared memory, K-major swizzled rows of operand B
             row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
             rows_here = min(kAttRowsPerPair, p.group * (cur.k + 1) - row_lo);
@@ -317,7 +320,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             }
             fence_proxy_async();
             tc_fence_before();
-            mbar_arrive(&bars->q_full);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->q_full);
             if (q == 0) {
                 // the MMA warp allocated tensor memory meanwhile: meet it (warps 2..6) and read the base
                 asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
@@ -338,141 +342,137 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         if (!att_wait(&bars->s_full[buf], u & 1, p.status, 6)) { ok = false; break; }
         tc_fence_after();
 
-        // ---- does any score of this block exceed its row's running maximum by more than the threshold?
-        // (cheap: a multiply-add and a max per score against the maxima kept in shared memory; the exact
-        // column maxima below are only needed when the answer is yes, or at the start of a segment)
-        uint32_t sv[32];                                 // kept for the next pass when there is a single chunk
-        bool slow = seg_first;
-        if (!seg_first) {
-            float ex = -INFINITY;
+        // the P^T buffer is free once the product that last read it has completed
+        const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
+        if (pu > 0 && !att_wait(&bars->p_empty[pbuf], (pu - 1) & 1, p.status, 8)) { ok = false; break; }
+
+        // ---- One pass per block in the common case: p = 2^(s * scale - m) against the running maxima kept
+        // in shared memory, written as bf16 into row t of operand B of the second product, while noting
+        // whether any score exceeded its row's maximum by more than the threshold.  The four warps then
+        // agree; only if one of them saw such a score (or at the start of a segment, where there is no
+        // maximum yet) are the exact column maxima taken, O^T and the row sums rescaled -- this block's
+        // contribution to the row sums included -- and the block's P^T written again against the new maxima.
+        bool fresh = seg_first;                          // the maxima are (re)computed before the pass
+        bool add = true;                                 // the pass adds to the row sums
+#pragma unroll 1
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+            if (fresh) {
+                // ---- exact column maxima over my warp's 32 tokens, then over the four warps
+                float* xch = sm.xch + (q & 1) * 4 * n_pad;
 #pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
-                if (ci * 32 < n_pad) {
-                    tmem_ld_x32(t_s + ci * 32, sv);
-                    tmem_ld_wait();
+                for (int ci = 0; ci < NCH; ++ci) {
+                    if (ci * 32 < n_pad) {
+                        uint32_t sv[32];
+                        tmem_ld_x32(t_s + ci * 32, sv);
+                        tmem_ld_wait();
+                        float mine = -INFINITY;
 #pragma unroll
-                    for (int i4 = 0; i4 < 8; ++i4) {
-                        const float4 mv = *reinterpret_cast<const float4*>(sm.m_col + ci * 32 + 4 * i4);
-                        const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int i = 4 * i4 + j;
-                            const float x = fmaf(__uint_as_float(sv[i]), p.scale_log2, -mm[j]);   // -inf maximum: +inf
+                        for (int i = 0; i < 32; ++i) {
                             const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;
-                            ex = fmaxf(ex, masked ? -INFINITY : x);
+                            const float w = redux_max(masked ? -INFINITY : __uint_as_float(sv[i]));
+                            if (lane == i) mine = w;
                         }
+                        if (ci * 32 + lane < n_pad) xch[quarter * n_pad + ci * 32 + lane] = mine;
+                    }
+                }
+                if (!group_sync(17)) { ok = false; break; }
+                float alpha[NCH];
+                bool rescale = false;
+#pragma unroll
+                for (int ci = 0; ci < NCH; ++ci) {
+                    alpha[ci] = 1.f;
+                    const int col = ci * 32 + lane;
+                    if (col < n_pad) {
+                        const float mx = fmaxf(fmaxf(xch[col], xch[n_pad + col]), fmaxf(xch[2 * n_pad + col], xch[3 * n_pad + col])) *
+                                         p.scale_log2;       // scale > 0: the maximum commutes
+                        // ---- raise the running maximum only if it grew by more than the threshold
+                        if (seg_first) {
+                            m_used[ci] = mx;
+                        } else if (mx > m_used[ci] + kRescaleThreshold) {
+                            alpha[ci] = fast_exp2(m_used[ci] - mx);            // m_used == -inf gives 0
+                            m_used[ci] = mx;
+                            rescale = true;
+                        }
+                        if (quarter == 0) sm.m_col[col] = m_used[ci];
+                    }
+                }
+                if (!seg_first && __any_sync(0xffffffffu, rescale)) {
+                    // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
+                    if (!att_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int ci = 0; ci < NCH; ++ci) {
+                        if (ci * 32 < n_pad) {
+                            uint32_t o[32];
+                            if (o_lane) {
+                                tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
+                                tmem_ld_wait();
+                            }
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                const float a = __shfl_sync(0xffffffffu, alpha[ci], i);
+                                lsum[ci * 32 + i] *= a;
+                                if (o_lane) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
+                            }
+                            if (o_lane) tmem_st_x32(t_lane + kTmemO + ci * 32, o);
+                        }
+                    }
+                    if (o_lane) tmem_st_wait();
+                }
+                if (!group_sync(18)) { ok = false; break; }                // the new maxima are in shared memory
+            }
+            // ---- p = 2^(s * scale - m)
+            float ex = -INFINITY;
+            {
+                uint8_t* p_row = sm.pt + pbuf * Cfg::p_bytes(n_pad) + t * 16;
+#pragma unroll
+                for (int ci = 0; ci < NCH; ++ci) {
+                    if (ci * 32 < n_pad) {
+                        uint32_t sv[32];
+                        tmem_ld_x32(t_s + ci * 32, sv);
+                        tmem_ld_wait();
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 mv = *reinterpret_cast<const float4*>(sm.m_col + ci * 32 + 4 * i4);
+                            const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
+                            float e[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int i = 4 * i4 + j;
+                                const float x = fmaf(__uint_as_float(sv[i]), p.scale_log2, -mm[j]);
+                                const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;   // also rows without a maximum yet
+                                e[j] = masked ? 0.f : fast_exp2(x);
+                                ex = fmaxf(ex, masked ? -INFINITY : x);
+                                if (add) lsum[ci * 32 + i] += e[j];
+                            }
+                            pk[2 * i4] = pack_bf16(e[0], e[1]);
+                            pk[2 * i4 + 1] = pack_bf16(e[2], e[3]);
+                        }
+#pragma unroll
+                        for (int g8 = 0; g8 < 4; ++g8)
+                            if (ci * 32 + g8 * 8 < n_pad)
+                                *reinterpret_cast<uint4*>(p_row + (ci * 4 + g8) * 2048) =
+                                    make_uint4(pk[4 * g8], pk[4 * g8 + 1], pk[4 * g8 + 2], pk[4 * g8 + 3]);
                     }
                 }
             }
+            if (fresh) break;                            // written against maxima taken from this very block
             const bool hot = __any_sync(0xffffffffu, ex > kRescaleThreshold);
             if (lane == 0) sm.flags[(q & 1) * 4 + quarter] = hot ? 1 : 0;
             if (!group_sync(14)) { ok = false; break; }
             const int* fl = sm.flags + (q & 1) * 4;
-            slow = (fl[0] | fl[1] | fl[2] | fl[3]) != 0;
+            if ((fl[0] | fl[1] | fl[2] | fl[3]) == 0) break;
+            fresh = true;                                // second round: new maxima, then P^T again, the row sums
+            add = false;                                 // already hold this block (they are rescaled with the rest)
         }
-        if (slow) {
-            // ---- exact column maxima over my warp's 32 tokens, then over the four warps
-            float* xch = sm.xch + (q & 1) * 4 * n_pad;
-#pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
-                if (ci * 32 < n_pad) {
-                    tmem_ld_x32(t_s + ci * 32, sv);
-                    tmem_ld_wait();
-                    float mine = -INFINITY;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;
-                        const float w = redux_max(masked ? -INFINITY : __uint_as_float(sv[i]));
-                        if (lane == i) mine = w;
-                    }
-                    if (ci * 32 + lane < n_pad) xch[quarter * n_pad + ci * 32 + lane] = mine;
-                }
-            }
-            if (!group_sync(17)) { ok = false; break; }
-            float alpha[NCH];
-            bool rescale = false;
-#pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
-                alpha[ci] = 1.f;
-                const int col = ci * 32 + lane;
-                if (col < n_pad) {
-                    const float mx = fmaxf(fmaxf(xch[col], xch[n_pad + col]), fmaxf(xch[2 * n_pad + col], xch[3 * n_pad + col])) *
-                                     p.scale_log2;       // scale > 0: the maximum commutes
-                    // ---- raise the running maximum only if it grew by more than the threshold
-                    if (seg_first) {
-                        m_used[ci] = mx;
-                    } else if (mx > m_used[ci] + kRescaleThreshold) {
-                        alpha[ci] = fast_exp2(m_used[ci] - mx);            // m_used == -inf gives 0
-                        m_used[ci] = mx;
-                        rescale = true;
-                    }
-                    if (quarter == 0) sm.m_col[col] = m_used[ci];
-                }
-            }
-            if (!seg_first && __any_sync(0xffffffffu, rescale)) {
-                // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
-                if (!att_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int ci = 0; ci < NCH; ++ci) {
-                    if (ci * 32 < n_pad) {
-                        uint32_t o[32];
-                        if (o_lane) {
-                            tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
-                            tmem_ld_wait();
-                        }
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float a = __shfl_sync(0xffffffffu, alpha[ci], i);
-                            lsum[ci * 32 + i] *= a;
-                            if (o_lane) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
-                        }
-                        if (o_lane) tmem_st_x32(t_lane + kTmemO + ci * 32, o);
-                    }
-                }
-                if (o_lane) tmem_st_wait();
-            }
-            if (!group_sync(18)) { ok = false; break; }                // the new maxima are in shared memory
-        }
-        // the P^T buffer is free once the product that last read it has completed
-        const int pbuf = q % p.p_bufs, pu = q / p.p_bufs;
-        if (pu > 0 && !att_wait(&bars->p_empty[pbuf], (pu - 1) & 1, p.status, 8)) { ok = false; break; }
-        // ---- p = 2^(s * scale - m), bf16, into row t of operand B of the second product
-        {
-            uint8_t* p_row = sm.pt + pbuf * Cfg::p_bytes(n_pad) + t * 16;
-#pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
-                if (ci * 32 < n_pad) {
-                    if (NCH > 1) {
-                        tmem_ld_x32(t_s + ci * 32, sv);
-                        tmem_ld_wait();
-                    }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i4 = 0; i4 < 8; ++i4) {
-                        const float4 mv = *reinterpret_cast<const float4*>(sm.m_col + ci * 32 + 4 * i4);
-                        const float mm[4] = {mv.x, mv.y, mv.z, mv.w};
-                        float e[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int i = 4 * i4 + j;
-                            e[j] = fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -mm[j]));
-                            if (static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span) e[j] = 0.f;   // also rows without a maximum yet
-                            lsum[ci * 32 + i] += e[j];
-                        }
-                        pk[2 * i4] = pack_bf16(e[0], e[1]);
-                        pk[2 * i4 + 1] = pack_bf16(e[2], e[3]);
-                    }
-#pragma unroll
-                    for (int g8 = 0; g8 < 4; ++g8)
-                        if (ci * 32 + g8 * 8 < n_pad)
-                            *reinterpret_cast<uint4*>(p_row + (ci * 4 + g8) * 2048) =
-                                make_uint4(pk[4 * g8], pk[4 * g8 + 1], pk[4 * g8 + 2], pk[4 * g8 + 3]);
-                }
-            }
-        }
+        if (!ok) break;
         // rows of V past the end of the sequence may hold anything (the pool is the caller's, or
         // the page was never loaded): their weight is exactly 0, but 0 * NaN is NaN, so clear them
+        if (t_begin + kAttBlockTokens > cur.kvl) {
+            // (the tile must have landed first, or the copy would overwrite the zeros)
+            if (!att_wait(&bars->v_full[q % p.v_stages], (q / p.v_stages) & 1, p.status, 22)) { ok = false; break; }
+        }
         if (t_begin + kAttBlockTokens > cur.kvl && t >= cur.kvl - t_begin) {
             uint8_t* v_row = sm.v_ring + (q % p.v_stages) * Cfg::kTileBytes + t * 128;
 #pragma unroll
@@ -483,8 +483,11 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         }
         fence_proxy_async();
         tc_fence_before();
-        mbar_arrive(&bars->p_full[pbuf]);
-        mbar_arrive(&bars->s_empty[buf]);
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(&bars->p_full[pbuf]);
+            mbar_arrive(&bars->s_empty[buf]);
+        }
 
         const int pair_global = cur.pair0 + cur.pair;
         const int pair_blk_first = cur.blk0 + cur.pair * cur.nb;
@@ -673,12 +676,12 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         for (int s = 0; s < p.k_stages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
         for (int s = 0; s < p.v_stages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int a = 0; a < 2; ++a) {
-            mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], kAttSoftmaxThreads);
-            mbar_init(&bars->p_full[a], kAttSoftmaxThreads); mbar_init(&bars->p_empty[a], 1);
+            mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], kAttSoftmaxThreads / 32);   // one arrival per softmax warp
+            mbar_init(&bars->p_full[a], kAttSoftmaxThreads / 32); mbar_init(&bars->p_empty[a], 1);
         }
-        mbar_init(&bars->q_full, kAttSoftmaxThreads);
+        mbar_init(&bars->q_full, kAttSoftmaxThreads / 32);
         mbar_init(&bars->o_full, 1);
-        mbar_init(&bars->group, kAttSoftmaxThreads);
+        mbar_init(&bars->group, kAttSoftmaxThreads / 32);
         fence_barrier_init();
         tma_prefetch_desc(&kv_map);
     }
