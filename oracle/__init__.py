@@ -58,10 +58,14 @@ def lib() -> C.CDLL:
         L.fso_softmax.restype = None
         L.fso_softmax.argtypes = [vp, i32, f64, vp, vp]
         L.fso_accept.restype = None
-        L.fso_accept.argtypes = [i32, vp, vp, vp, vp, vp, i32, i32, f64, f64, vp, vp, i32,
+        L.fso_accept.argtypes = [i32, vp, vp, vp, vp, vp, i32, i32, f64, vp, i32, f64, vp, vp, i32,
                                  vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.fso_emission.restype = f64
-        L.fso_emission.argtypes = [vp, vp, i32, f64, f64, vp, vp, vp]
+        L.fso_emission.argtypes = [vp, vp, i32, f64, i32, f64, vp, vp, vp]
+        L.fso_topk.restype = None
+        L.fso_topk.argtypes = [vp, i32, i32]
+        L.fso_kv_release.restype = None
+        L.fso_kv_release.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp]
         L.fso_nucleus.restype = None
         L.fso_nucleus.argtypes = [vp, i32, f64, vp]
         L.fso_kv_append.restype = None
@@ -166,20 +170,28 @@ def nucleus(prob, top_p):
     return p, float(m[0])
 
 
-def emission(target_row, draft_row=None, temperature=1.0, top_p=1.0, mask=None):
+def topk(prob, top_k):
+    """Top-k filtered and renormalised copy of a distribution (ties with the k-th token are all kept)."""
+    p = np.array(prob, dtype=np.float64, copy=True)
+    lib().fso_topk(_p(p), int(p.size), int(top_k))
+    return p
+
+
+def emission(target_row, draft_row=None, temperature=1.0, top_p=1.0, mask=None, top_k=0):
     """Unnormalised weights r[v] of the emitted token and their sum Z for one target row: the residual
     max(0, p - q) when a draft row is given (first rejection), p itself otherwise (bonus row)."""
     zt = _c(target_row, np.float64)
     zd = _c(draft_row, np.float32)
     mask = _c(mask, np.uint32)
     r = np.empty(zt.shape[0], dtype=np.float64)
-    z = lib().fso_emission(_p(zt), _p(zd), int(zt.shape[0]), float(temperature), float(top_p), _p(mask), _p(r), None)
+    z = lib().fso_emission(_p(zt), _p(zd), int(zt.shape[0]), float(temperature), int(top_k), float(top_p), _p(mask), _p(r), None)
     return r, float(z)
 
 
 def accept(mode, target_logits, draft_logits, draft_tokens, draft_len, seeds, temperature=1.0,
-           vocab_mask=None, seq_sel=None, top_p=1.0):
-    """Acceptance loop + emitted token.  Returns a dict of numpy arrays."""
+           vocab_mask=None, seq_sel=None, top_p=1.0, top_k=0, temperatures=None):
+    """Acceptance loop + emitted token.  Returns a dict of numpy arrays.  `temperatures`: one value per
+    sequence (overrides `temperature`); top_k / top_p filter the target distribution."""
     zt = _c(target_logits, np.float64)
     zd = _c(draft_logits, np.float32)
     x = _c(draft_tokens, np.int32)
@@ -206,8 +218,10 @@ def accept(mode, target_logits, draft_logits, draft_tokens, draft_len, seeds, te
         "resid_mass": np.zeros(batch, dtype=np.float64),
         "topp_margin": np.full(s + batch, np.inf, dtype=np.float64),
     }
+    temps = _c(temperatures, np.float64)
+    assert temps is None or temps.size == batch
     lib().fso_accept(int(mode), _p(zt), _p(zd), _p(x), _p(k), _p(seeds), batch, vocab,
-                     float(temperature), float(top_p), _p(mask), _p(sel), 0 if sel is None else int(sel.size),
+                     float(temperature), _p(temps), int(top_k), float(top_p), _p(mask), _p(sel), 0 if sel is None else int(sel.size),
                      _p(res["accepted_len"]), _p(res["next_token"]), _p(res["p_tok"]),
                      _p(res["q_tok"]), _p(res["u"]), _p(res["acc_margin"]),
                      _p(res["cdf_margin"]), _p(res["resid_mass"]), _p(res["topp_margin"]))
@@ -233,9 +247,19 @@ def kv_rollback(kv_len, draft_len, accepted_len):
     return out
 
 
+def kv_release(page_table, kv_len_prev, kv_len_next, page_size=16):
+    """Returns (page table with the released entries set to -1, released page ids in order)."""
+    pt = np.array(page_table, dtype=np.int32, copy=True)
+    prev, nxt = _c(kv_len_prev, np.int32), _c(kv_len_next, np.int32)
+    free = np.full(pt.size, -1, dtype=np.int32)
+    cnt = np.zeros(1, dtype=np.int32)
+    lib().fso_kv_release(_p(pt), int(pt.shape[1]), _p(prev), _p(nxt), int(pt.shape[0]), page_size, _p(free), _p(cnt))
+    return pt, free[:int(cnt[0])]
+
+
 def verify(mode, hidden, kv_pages, page_table, kv_len, draft_len, lm_head_w, draft_tokens,
            draft_logits, seeds, n_q_heads, n_kv_heads, head_dim, page_size=16, temperature=1.0,
-           vocab_mask=None, seq_sel=None):
+           vocab_mask=None, seq_sel=None, top_p=1.0, top_k=0, temperatures=None):
     """The whole step in the order of Algorithm 2, Step 2: attention over the
     restored KV session -> bf16 -> LM head -> acceptance loop -> emitted token."""
     draft_len = _c(draft_len, np.int32)
@@ -247,7 +271,7 @@ def verify(mode, hidden, kv_pages, page_table, kv_len, draft_len, lm_head_w, dra
         row_sel = np.concatenate([np.arange(row0[b], row0[b + 1]) for b in seq_sel]).astype(np.int32)
     logits = lm_head(attn16, lm_head_w, row_sel)
     res = accept(mode, logits, draft_logits, draft_tokens, draft_len, seeds, temperature,
-                 vocab_mask, seq_sel)
+                 vocab_mask, seq_sel, top_p=top_p, top_k=top_k, temperatures=temperatures)
     res["attn_f64"] = attn64
     res["attn_bf16"] = attn16
     res["logits"] = logits

@@ -261,6 +261,30 @@ void fso_nucleus(double* prob, int32_t vocab, double top_p, double* margin)
     free(s);
 }
 
+/* ------------------------------------------------------------------ top-k */
+
+void fso_topk(double* prob, int32_t vocab, int32_t top_k)
+{
+    if (top_k <= 0 || top_k >= vocab) return;
+    fso_pv* s = (fso_pv*)malloc(sizeof(fso_pv) * (size_t)vocab);
+    for (int32_t v = 0; v < vocab; ++v) { s[v].p = prob[v]; s[v].v = v; }
+    qsort(s, (size_t)vocab, sizeof(fso_pv), cmp_pv_desc);
+    const double thr = s[top_k - 1].p;                    /* probability of the k-th largest */
+    double z = 0.0;
+    for (int32_t v = 0; v < vocab; ++v) z += (prob[v] >= thr && prob[v] > 0.0) ? prob[v] : 0.0;
+    for (int32_t v = 0; v < vocab; ++v) prob[v] = (prob[v] >= thr && prob[v] > 0.0) ? prob[v] / z : 0.0;
+    free(s);
+}
+
+/* the target distribution of one row: softmax at the temperature, then top-k, then top-p */
+static void target_dist(const double* zt_row, int32_t vocab, double temperature, int32_t top_k, double top_p,
+                        const uint32_t* mask, double* p, double* topp_margin)
+{
+    fso_softmax(zt_row, vocab, temperature, mask, p);
+    fso_topk(p, vocab, top_k);
+    fso_nucleus(p, vocab, top_p, topp_margin);
+}
+
 /* ------------------------------------------------- acceptance + emission */
 
 static int32_t argmax_lowest(const double* z, int32_t vocab, const uint32_t* mask)
@@ -296,11 +320,10 @@ static int32_t inverse_cdf(const double* r, int32_t vocab, double thr,
  * given (the first rejection) and that residual has positive mass, else p (the bonus row, or a
  * residual that rounding emptied). */
 double fso_emission(const double* zt_row, const float* zd_row, int32_t vocab, double temperature,
-                    double top_p, const uint32_t* mask, double* r, double* topp_margin)
+                    int32_t top_k, double top_p, const uint32_t* mask, double* r, double* topp_margin)
 {
     double* p = (double*)malloc(sizeof(double) * (size_t)vocab);
-    fso_softmax(zt_row, vocab, temperature, mask, p);
-    fso_nucleus(p, vocab, top_p, topp_margin);
+    target_dist(zt_row, vocab, temperature, top_k, top_p, mask, p, topp_margin);
     double z_mass = 0.0;
     if (zd_row != NULL) {
         double* q = (double*)malloc(sizeof(double) * (size_t)vocab);
@@ -322,7 +345,7 @@ double fso_emission(const double* zt_row, const float* zd_row, int32_t vocab, do
 }
 
 static void verify_one(int32_t mode, const double* zt, const float* zd, const int32_t* x,
-                       int32_t k, int32_t vocab, double temperature, double top_p, uint64_t seed,
+                       int32_t k, int32_t vocab, double temperature, int32_t top_k, double top_p, uint64_t seed,
                        const uint32_t* mask, double* topp_margin,
                        int32_t* accepted_len, int32_t* next_token,
                        double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
@@ -346,8 +369,7 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
     /* the acceptance test at every draft position; n = first failure */
     int32_t n = k;
     for (int32_t j = 0; j < k; ++j) {
-        fso_softmax(zt + (int64_t)j * vocab, vocab, temperature, mask, p);
-        fso_nucleus(p, vocab, top_p, topp_margin ? topp_margin + j : NULL);
+        target_dist(zt + (int64_t)j * vocab, vocab, temperature, top_k, top_p, mask, p, topp_margin ? topp_margin + j : NULL);
         for (int32_t v = 0; v < vocab; ++v) zq[v] = (double)zd[(int64_t)j * vocab + v];
         fso_softmax(zq, vocab, temperature, NULL, q);
         const double u = fso_uniform(seed, (uint32_t)j, 0u);
@@ -365,7 +387,7 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
 
     /* emitted token: residual at the first rejection, else the bonus row */
     double z_mass = fso_emission(zt + (int64_t)n * vocab, n < k ? zd + (int64_t)n * vocab : NULL, vocab,
-                                 temperature, top_p, mask, r, topp_margin ? topp_margin + n : NULL);
+                                 temperature, top_k, top_p, mask, r, topp_margin ? topp_margin + n : NULL);
     const double u2 = fso_uniform(seed, (uint32_t)n, 1u);
     double c_below, c_at;
     const double thr = u2 * z_mass;
@@ -382,7 +404,8 @@ static void verify_one(int32_t mode, const double* zt, const float* zd, const in
 
 void fso_accept(int32_t mode, const double* target_logits, const float* draft_logits,
                 const int32_t* draft_tokens, const int32_t* draft_len, const uint64_t* seeds,
-                int32_t batch, int32_t vocab, double temperature, double top_p, const uint32_t* vocab_mask,
+                int32_t batch, int32_t vocab, double temperature, const double* temperatures, int32_t top_k,
+                double top_p, const uint32_t* vocab_mask,
                 const int32_t* seq_sel, int32_t n_sel,
                 int32_t* accepted_len, int32_t* next_token,
                 double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
@@ -404,7 +427,8 @@ void fso_accept(int32_t mode, const double* target_logits, const float* draft_lo
         verify_one(mode,
                    target_logits + row0[b] * vocab,
                    draft_logits ? draft_logits + t0 * vocab : NULL,
-                   draft_tokens + t0, draft_len[b], vocab, temperature, top_p, seeds ? seeds[b] : 0,
+                   draft_tokens + t0, draft_len[b], vocab, temperatures ? temperatures[b] : temperature, top_k, top_p,
+                   seeds ? seeds[b] : 0,
                    vocab_mask ? vocab_mask + (int64_t)b * mask_words : NULL,
                    topp_margin ? topp_margin + row0[b] : NULL,
                    accepted_len + b, next_token + b,
@@ -446,6 +470,21 @@ void fso_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int3
     for (int32_t b = 0; b < batch; ++b) {
         const int32_t ctx = kv_len[b] - (draft_len[b] + 1);
         kv_len_next[b] = ctx + accepted_len[b] + 1;
+    }
+}
+
+void fso_kv_release(int32_t* page_table, int32_t max_pages_per_seq, const int32_t* kv_len_prev,
+                    const int32_t* kv_len_next, int32_t batch, int32_t page_size,
+                    int32_t* free_list, int32_t* free_count)
+{
+    for (int32_t b = 0; b < batch; ++b) {
+        const int32_t keep = (kv_len_next[b] + page_size - 1) / page_size;   /* pages that still hold valid tokens */
+        const int32_t had = (kv_len_prev[b] + page_size - 1) / page_size;
+        for (int32_t i = keep; i < had; ++i) {
+            int32_t* e = page_table + (int64_t)b * max_pages_per_seq + i;
+            free_list[(*free_count)++] = *e;
+            *e = -1;
+        }
     }
 }
 

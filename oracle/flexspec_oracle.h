@@ -80,15 +80,24 @@ void fso_softmax(const double* z, int32_t vocab, double temperature,
  * cumulative sums around the cut, i.e. how close the cut was to falling one token earlier/later. */
 void fso_nucleus(double* prob, int32_t vocab, double top_p, double* margin);
 
+/* Top-k filter of a distribution (the usual companion of top-p in sampling stacks; the paper's
+ * stochastic regime names top-p only): every token whose probability is at least that of the k-th
+ * most probable one is kept (ties with it are all kept, so the set is defined by a threshold and not
+ * by a sort's tie order), the rest get probability 0, the kept ones are renormalised.
+ * top_k <= 0 or >= vocab leaves prob untouched.  Applied BEFORE the nucleus filter. */
+void fso_topk(double* prob, int32_t vocab, int32_t top_k);
+
 /* The weights the emitted token is drawn from, for one target row (Algorithm 2: "sample correction
  * token"): r[v] = max(0, p(v) - q(v)) when zd_row is given (first rejection; p, q the softmaxes of
- * the two rows at `temperature`, p filtered to its nucleus when top_p < 1), or r = p when zd_row is
+ * the two rows at `temperature`, p filtered by top-k and then to its nucleus), or r = p when zd_row is
  * NULL (bonus row) or the residual has no mass.  Returns Z = sum_v r[v]; r is not normalised. */
 double fso_emission(const double* zt_row, const float* zd_row, int32_t vocab, double temperature,
-                    double top_p, const uint32_t* mask, double* r, double* topp_margin);
+                    int32_t top_k, double top_p, const uint32_t* mask, double* r, double* topp_margin);
 
-/* Acceptance + emitted token for a batch of sequences.  With top_p < 1 the TARGET distribution of
- * every row is its nucleus (SAMPLE mode only).
+/* Acceptance + emitted token for a batch of sequences.  The TARGET distribution of every row is
+ * softmax(z / T) filtered by top-k (if 0 < top_k < vocab) and then to its nucleus (if top_p < 1),
+ * SAMPLE mode only.  T is `temperature`, or temperatures[b] per sequence when that array is given
+ * (both logit sets of the sequence are divided by it).
  * mode 0 = SAMPLE: accept x_j iff u_j * q_j(x_j) < p_j(x_j); after n accepted
  *   drafts emit a token from max(0, p_n - q_n)/Z (n < k) or from p_k (n == k)
  *   by inverse CDF in vocabulary order: min{v : sum_{w<=v} r_w > u' * Z}.
@@ -107,7 +116,8 @@ double fso_emission(const double* zt_row, const float* zd_row, int32_t vocab, do
  *     interval, divided by Z;  resid_mass[b] = Z. */
 void fso_accept(int32_t mode, const double* target_logits, const float* draft_logits,
                 const int32_t* draft_tokens, const int32_t* draft_len, const uint64_t* seeds,
-                int32_t batch, int32_t vocab, double temperature, double top_p, const uint32_t* vocab_mask,
+                int32_t batch, int32_t vocab, double temperature, const double* temperatures /* [batch] or NULL */,
+                int32_t top_k, double top_p, const uint32_t* vocab_mask,
                 const int32_t* seq_sel, int32_t n_sel,
                 int32_t* accepted_len, int32_t* next_token,
                 double* p_tok, double* q_tok, double* u_acc, double* acc_margin,
@@ -126,6 +136,14 @@ void fso_kv_append(uint16_t* kv_pages, const int32_t* page_table, int32_t max_pa
                    const uint16_t* new_k, const uint16_t* new_v);
 void fso_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int32_t* accepted_len,
                      int32_t batch, int32_t* kv_len_next);
+
+/* fso_kv_release: after the rollback the pages that hold no valid token any more are given back
+ *   (Section IV-C: the invalid KV pairs are discarded): for every sequence the page-table entries
+ *   ceil(kv_len_next / page_size) .. ceil(kv_len_prev / page_size) - 1 are appended to free_list
+ *   (sequence by sequence, ascending entry index), *free_count is advanced and the entries become -1. */
+void fso_kv_release(int32_t* page_table, int32_t max_pages_per_seq, const int32_t* kv_len_prev,
+                    const int32_t* kv_len_next, int32_t batch, int32_t page_size,
+                    int32_t* free_list, int32_t* free_count);
 
 int32_t fso_num_threads(void);
 

@@ -587,3 +587,101 @@ def test_top_p_sampling_is_lossless_with_respect_to_the_nucleus():
     same = oracle.accept(oracle.SAMPLE, zt[:2000], zd[:1000], toks[:1000], np.ones(1000, np.int32), seeds[:1000], top_p=1.0)
     base = oracle.accept(oracle.SAMPLE, zt[:2000], zd[:1000], toks[:1000], np.ones(1000, np.int32), seeds[:1000])
     assert np.array_equal(same["next_token"], base["next_token"]) and np.array_equal(same["accepted_len"], base["accepted_len"])
+
+
+# ------------------------------------------------------------------ top-k, per-sequence temperature, page release
+
+def test_top_k_filter_against_a_numpy_sort():
+    rng = np.random.RandomState(41)
+    for v, k in [(7, 3), (50, 1), (1000, 40), (1000, 999), (64, 64), (64, 0), (64, 200)]:
+        p = rng.dirichlet(np.full(v, 0.3))
+        got = oracle.topk(p, k)
+        if k <= 0 or k >= v:
+            assert np.array_equal(got, p)
+            continue
+        order = np.lexsort((np.arange(v), -p))
+        keep = order[:k]
+        want = np.zeros(v)
+        want[keep] = p[keep] / p[keep].sum()
+        assert np.allclose(got, want, rtol=0, atol=1e-15)
+        assert np.count_nonzero(got) == k and abs(got.sum() - 1.0) < 1e-12
+    # ties with the k-th token are all kept
+    p = np.array([0.3, 0.2, 0.2, 0.2, 0.1])
+    assert np.count_nonzero(oracle.topk(p, 2)) == 4
+    assert np.count_nonzero(oracle.topk(p, 1)) == 1
+    # top-k comes before top-p: the nucleus is taken of the renormalised top-k distribution
+    p = np.array([0.4, 0.3, 0.2, 0.1])
+    both, _ = oracle.nucleus(oracle.topk(p, 2), 0.6)           # top-2 -> (4/7, 3/7); mass 0.6 needs both
+    assert np.allclose(both, [4 / 7, 3 / 7, 0, 0])
+    r, z = oracle.emission(np.log(p), None, top_k=2, top_p=0.6)
+    assert np.allclose(r, both) and abs(z - 1.0) < 1e-12
+
+
+def test_top_k_sampling_follows_the_filtered_target():
+    """With top_k the emitted token follows the top-k filtered target row (chi-square over 3*10^5
+    trials) and a draft token outside the top-k set is always rejected."""
+    rng = np.random.RandomState(43)
+    v, n, top_k = 12, 300000, 5
+    z_t = rng.standard_normal(v) * 1.5
+    z_d = (z_t + rng.standard_normal(v)).astype(np.float32)
+    p0 = np.exp(z_t - z_t.max()); p0 /= p0.sum()
+    pk = oracle.topk(p0, top_k)
+    q0 = np.exp(z_d.astype(np.float64) - z_d.max()); q0 /= q0.sum()
+    toks = rng.choice(v, size=n, p=q0).astype(np.int32)
+    zt = np.tile(z_t, (2 * n, 1))
+    zd = np.tile(z_d, (n, 1))
+    seeds = rng.randint(0, 2 ** 62, n).astype(np.uint64)
+    res = oracle.accept(oracle.SAMPLE, zt, zd, toks, np.ones(n, np.int32), seeds, top_k=top_k)
+    outside = pk[toks] == 0.0
+    assert outside.any() and np.all(res["accepted_len"][outside] == 0)
+    first = np.where(res["accepted_len"] >= 1, toks, res["next_token"])
+    counts = np.bincount(first, minlength=v).astype(np.float64)
+    assert np.all(counts[pk == 0.0] == 0)
+    sup = pk > 0
+    chi2 = float((((counts[sup] - n * pk[sup]) ** 2) / (n * pk[sup])).sum())
+    assert chi2 < scipy.stats.chi2.ppf(0.999, sup.sum() - 1)
+
+
+def test_per_sequence_temperatures_equal_separate_runs():
+    rng = np.random.RandomState(47)
+    v, batch = 300, 6
+    k = rng.randint(0, 5, batch).astype(np.int32)
+    m, s = int(k.sum()) + batch, int(k.sum())
+    zt = rng.standard_normal((m, v)) * 2
+    zd = (rng.standard_normal((s, v)) * 2).astype(np.float32)
+    toks = rng.randint(0, v, s).astype(np.int32)
+    seeds = rng.randint(0, 2 ** 62, batch).astype(np.uint64)
+    temps = np.array([0.5, 1.0, 0.7, 1.3, 2.0, 0.9])
+    res = oracle.accept(oracle.SAMPLE, zt, zd, toks, k, seeds, temperature=123.0, temperatures=temps)
+    for b in range(batch):
+        one = oracle.accept(oracle.SAMPLE, zt, zd, toks, k, seeds, temperature=float(temps[b]), seq_sel=[b])
+        assert one["accepted_len"][b] == res["accepted_len"][b] and one["next_token"][b] == res["next_token"][b]
+    t0 = np.concatenate([[0], np.cumsum(k)])
+    r0 = np.concatenate([[0], np.cumsum(k + 1)])
+    for b in range(batch):                       # p(x_j) against scipy at the sequence's own temperature
+        for j in range(k[b]):
+            want = scipy.special.softmax(zt[r0[b] + j] / temps[b])[toks[t0[b] + j]]
+            assert abs(res["p_tok"][t0[b] + j] - want) < 1e-14
+
+
+def test_kv_release_returns_exactly_the_pages_past_the_new_length():
+    rng = np.random.RandomState(53)
+    batch, max_pages = 5, 12
+    prev = np.array([100, 33, 16, 48, 17], np.int32)           # lengths before the rollback
+    nxt = np.array([96, 33, 1, 31, 16], np.int32)              # after: pages kept = ceil(next / 16)
+    pt = np.full((batch, max_pages), -1, np.int32)
+    ids = rng.permutation(200).astype(np.int32)
+    c = 0
+    for b in range(batch):
+        n = -(-int(prev[b]) // 16)
+        pt[b, :n] = ids[c:c + n]; c += n
+    new_pt, freed = oracle.kv_release(pt, prev, nxt)
+    want = []
+    for b in range(batch):
+        keep, had = -(-int(nxt[b]) // 16), -(-int(prev[b]) // 16)
+        want += list(pt[b, keep:had])
+        assert np.array_equal(new_pt[b, :keep], pt[b, :keep]) and np.all(new_pt[b, keep:] == -1)
+    assert list(freed) == want and len(freed) == (7 - 6) + 0 + 0 + (3 - 2) + (2 - 1)
+    # nothing to release when nothing was rejected
+    same_pt, none = oracle.kv_release(pt, prev, prev)
+    assert np.array_equal(same_pt, pt) and len(none) == 0
