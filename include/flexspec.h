@@ -206,7 +206,7 @@ int flexspec_kv_rollback(flexspec_handle* h, const int32_t* kv_len, const int32_
  * fail or eat into the pool's reserve; or a step loop that must never stall on the implicit
  * device synchronisation of an allocation or a free.  Such callers cannot use flexspec_create,
  * which allocates the workspace.
- *   - The working memory is one fixed array inside the loaded library (268 032 bytes, held on
+ *   - The working memory is one fixed array inside the loaded library (276 224 bytes, held on
  *     every GPU that loads the library until the process exits).  Limits that follow from it:
  *     batch <= 64, sum_b (k_b + 1) <= 1024, vocab <= 131072; larger calls return
  *     FLEXSPEC_ERR_UNSUPPORTED and launch nothing.
@@ -235,6 +235,19 @@ int flexspec_sample_static(const float* logits, const int32_t* draft_tokens, con
  * acceptance tests, the residual and the bonus draw use it.  top_p = 1 (the default) switches the
  * filter off.  SAMPLE mode only; 0 < top_p <= 1, else INVALID_ARG. */
 int flexspec_set_top_p(flexspec_handle* h, float top_p);
+
+/* All sampling controls of the target distribution at once (Section V, Regime B: T = 1, top-p 0.9;
+ * top-k is the usual companion of top-p and is applied first).  From the next verify / sample call on:
+ *   top_p         as flexspec_set_top_p (1 = off);
+ *   top_k         keep the top_k most probable tokens of every target row (ties with the k-th are all
+ *                 kept) and renormalise, before the nucleus is taken; 0 = off;
+ *   temperatures  DEVICE fp32 [batch] or NULL: when given, sequence b uses temperatures[b] instead
+ *                 of the call's scalar temperature for both of its logit sets.  The array is read by
+ *                 every following call (it is borrowed, not copied) and must hold positive finite
+ *                 values: anything else is reported as INVALID_ARG in the status word and the scalar
+ *                 is used for that sequence.  The scalar still selects the greedy rule when it is 0.
+ * SAMPLE mode only.  Errors: INVALID_ARG. */
+int flexspec_set_sampling(flexspec_handle* h, float top_p, int32_t top_k, const float* temperatures);
 
 /* Workspace pointers for stage-wise comparison. */
 int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);

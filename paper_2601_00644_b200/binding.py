@@ -25,7 +25,7 @@ ERR_TIMEOUT, ERR_BAD_PAGE, ERR_BAD_TOKEN, ERR_NO_DEVICE = -5, -6, -7, -8
 EXPORTS = [
     "flexspec_create", "flexspec_verify", "flexspec_verify_host", "flexspec_attention",
     "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_kv_append",
-    "flexspec_kv_rollback", "flexspec_set_top_p", "flexspec_get_debug", "flexspec_status",
+    "flexspec_kv_rollback", "flexspec_set_top_p", "flexspec_set_sampling", "flexspec_get_debug", "flexspec_status",
     "flexspec_selftest_wait_timeout", "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
     "flexspec_destroy", "flexspec_strerror", "flexspec_version",
 ]
@@ -66,6 +66,7 @@ def _load() -> C.CDLL:
     lib.flexspec_kv_append.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.flexspec_kv_rollback.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     lib.flexspec_set_top_p.argtypes = [vp, f32]
+    lib.flexspec_set_sampling.argtypes = [vp, f32, i32, vp]
     lib.flexspec_get_debug.argtypes = [vp, C.POINTER(Debug)]
     lib.flexspec_status.argtypes = [vp, vp]
     lib.flexspec_selftest_wait_timeout.argtypes = [vp, C.c_int64, vp]
@@ -307,6 +308,13 @@ class Verifier:
     def set_top_p(self, top_p: float):
         """Nucleus sampling of the target (1.0 = off) for the following calls."""
         _check(LIB.flexspec_set_top_p(self._h, float(top_p)), "flexspec_set_top_p")
+
+    def set_sampling(self, top_p: float = 1.0, top_k: int = 0, temperatures: Optional[torch.Tensor] = None):
+        """top-p / top-k filters of the target and per-sequence temperatures (a CUDA fp32 tensor [batch],
+        kept alive here because the library only borrows it) for the following calls."""
+        _dev(temperatures, torch.float32, "temperatures")
+        self._temps = temperatures
+        _check(LIB.flexspec_set_sampling(self._h, float(top_p), int(top_k), _ptr(temperatures)), "flexspec_set_sampling")
 
     def status(self):
         st = (C.c_int32 * 4)()

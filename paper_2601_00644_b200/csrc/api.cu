@@ -76,7 +76,7 @@ struct DeviceGuard {
 void free_workspace(Handle& h)
 {
     cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml); cudaFree(h.att_tickets);
-    cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq); cudaFree(h.plan.k_eff);
+    cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq); cudaFree(h.plan.k_eff); cudaFree(h.plan.row_c);
     cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.topp);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
@@ -242,10 +242,10 @@ void mark(Handle& h, int idx, cudaStream_t s)
 }
 
 int run_plan(Handle& h, const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, const Geometry& g,
-             cudaStream_t s)
+             const SampleParams& sp, cudaStream_t s)
 {
-    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, g.m_rows, g.s_rows, g.k_batch_max, h.plan, h.status,
-                    s) != cudaSuccess)
+    if (launch_plan(draft_len, draft_tokens, batch, h.cfg.vocab, g.m_rows, g.s_rows, g.k_batch_max, sp.temps,
+                    sp.inv_temp_log2, h.plan, h.status, s) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
     h.launches++;
     return FLEXSPEC_OK;
@@ -306,10 +306,11 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, const S
     p.num_stages = lm_head_pick_stages(p.n_tile, p.n_blocks);
     p.acc_stages = (2 * rows_per_pass <= 512) ? 2 : 1;
     p.tstats = nullptr; p.n_tparts = 0; p.inv_temp_log2 = 1.f; p.greedy = 0;
-    p.row_seq = nullptr; p.vocab_mask = nullptr; p.mask_words = 0;
+    p.row_seq = nullptr; p.vocab_mask = nullptr; p.mask_words = 0; p.row_c = nullptr;
     if (sp != nullptr) {
         p.tstats = h.tstats; p.n_tparts = 4 * p.n_vtiles; p.inv_temp_log2 = sp->inv_temp_log2; p.greedy = sp->greedy;
         p.row_seq = sp->row_seq; p.vocab_mask = sp->vocab_mask; p.mask_words = sp->mask_words;
+        p.row_c = sp->temps != nullptr ? sp->row_c : nullptr;
     }
     p.status = h.status;
     CUtensorMap x_map;
@@ -332,13 +333,15 @@ void fill_sample_params(Handle& h, SampleParams& p, const float* logits, const i
     p.logits = logits; p.draft_logits = draft_logits; p.draft_tokens = draft_tokens;
     p.draft_len = draft_len; p.seeds = seeds; p.vocab_mask = vocab_mask;
     p.cu_q = h.plan.cu_q; p.cu_d = h.plan.cu_d; p.row_seq = h.plan.row_seq; p.k_eff = h.plan.k_eff;
+    p.row_c = h.plan.row_c; p.temps = p.greedy ? nullptr : h.temps;
     p.batch = batch; p.vocab = c.vocab; p.m_rows = g.m_rows; p.s_rows = g.s_rows;
     p.n_chunks = (c.vocab + kSampleChunk - 1) / kSampleChunk;
     p.mask_words = (c.vocab + 31) / 32;
     p.inv_temp_log2 = p.greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
     p.stats = h.stats;
     p.tstats = h.stats; p.n_tparts = p.n_chunks;          // target parts from the statistics kernel unless the LM head wrote them
-    p.top_p = p.greedy ? 1.f : h.top_p; p.topp = h.topp;
+    p.top_p = p.greedy ? 1.f : h.top_p; p.top_k = p.greedy ? 0 : h.top_k; p.topp = h.topp;
+    p.filtered = (p.top_p < 1.f || (p.top_k > 0 && p.top_k < c.vocab)) ? 1 : 0;
     p.accepted_len = accepted_len; p.next_token = next_token;
     if (c.flags & FLEXSPEC_FLAG_DEBUG) { p.dbg_p = h.dbg_p; p.dbg_q = h.dbg_q; p.dbg_u = h.dbg_u; }
     p.status = h.status;
@@ -355,8 +358,8 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
                        accepted_len, next_token);
     if (launch_sample_stats(p, 0, p.greedy ? p.m_rows : p.m_rows + p.s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
-    if (p.top_p < 1.f) {
-        if (launch_sample_nucleus(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (p.filtered) {
+        if (launch_sample_filter(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
     }
     if (launch_sample_accept(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
@@ -459,6 +462,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
     A(dev_alloc(&h.plan.k_eff, static_cast<size_t>(c.max_batch)));
+    A(dev_alloc(&h.plan.row_c, static_cast<size_t>(max_m) + h.max_s));
     A(dev_alloc(&h.stats, static_cast<size_t>(max_m + h.max_s) * n_chunks));
     A(dev_alloc(&h.tstats, static_cast<size_t>(max_m) * 4 * ((c.vocab + 127) / 128 + h.sm_count)));
     A(dev_alloc(&h.topp, static_cast<size_t>(max_m) * 2));
@@ -567,7 +571,12 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
     DeviceGuard guard(h.cfg.device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     h.launches = 0;
-    rc = run_plan(h, draft_len, draft_tokens, batch, g, s);
+    {
+        SampleParams sp0;
+        fill_sample_params(h, sp0, logits ? logits : h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch, temperature,
+                           vocab_mask, accepted_len, next_token);
+        rc = run_plan(h, draft_len, draft_tokens, batch, g, sp0, s);
+    }
     if (rc != FLEXSPEC_OK) return rc;
     return run_sample(h, logits ? logits : h.logits, draft_tokens, draft_logits, draft_len, seeds, g, batch,
                       temperature, vocab_mask, accepted_len, next_token, s);
@@ -602,7 +611,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     // nothing from the target model, so they run beside attention and the LM head
     if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
-    rc = run_plan(h, draft_len, draft_tokens, batch, g, h.side);
+    rc = run_plan(h, draft_len, draft_tokens, batch, g, sp, h.side);
     if (rc != FLEXSPEC_OK) return rc;
     if (!sp.greedy && sp.s_rows > 0) {
         if (launch_sample_stats(sp, sp.m_rows, sp.s_rows, h.side) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
@@ -623,12 +632,12 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);
-    if (sp.top_p < 1.f) {
-        if (launch_sample_nucleus(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;     // needs the row -> sequence table only with a mask: joined above
+    if (sp.filtered) {
+        if (launch_sample_filter(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;      // the plan's tables are there: joined above
         h.launches++;
     }
     mark(h, 5, s);
-    if (launch_sample_accept(sp, sp.top_p >= 1.f, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_accept(sp, !sp.filtered, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 6, s);
     return FLEXSPEC_OK;
@@ -743,6 +752,16 @@ int flexspec_set_top_p(flexspec_handle* fh, float top_p)
 {
     if (fh == nullptr || !(top_p > 0.f) || top_p > 1.f) return FLEXSPEC_ERR_INVALID_ARG;
     fh->h.top_p = top_p;
+    return FLEXSPEC_OK;
+}
+
+int flexspec_set_sampling(flexspec_handle* fh, float top_p, int32_t top_k, const float* temperatures)
+{
+    if (fh == nullptr || !(top_p > 0.f) || top_p > 1.f || top_k < 0) return FLEXSPEC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(temperatures) & 3u) != 0) return FLEXSPEC_ERR_INVALID_ARG;
+    fh->h.top_p = top_p;
+    fh->h.top_k = top_k;
+    fh->h.temps = temperatures;
     return FLEXSPEC_OK;
 }
 

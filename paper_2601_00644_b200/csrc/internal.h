@@ -28,6 +28,7 @@ struct Plan {                 // device tables written by the plan kernel, read 
     int32_t* cu_q;            // [max_batch+1] first query row of each sequence
     int32_t* cu_d;            // [max_batch+1] first draft row of each sequence
     int32_t* row_seq;         // [max_m] sequence of each query row
+    float* row_c;             // [max_m + max_s] log2(e) / T of the sequence of every target row, then of every draft row
     int32_t* k_eff;           // [max_batch] draft length the sampling kernels use: draft_len[b] once it has been
                               // checked against the geometry the host sized the launches for (0 if it disagrees)
 };
@@ -96,6 +97,7 @@ struct LmHeadParams {
     float2* tstats;           // [m_rows][n_tparts], n_tparts = 4 * n_vtiles
     int32_t n_tparts;
     float inv_temp_log2;      // log2(e) / T
+    const float* row_c;       // [m_rows] per-row log2(e) / T (per-sequence temperatures); null: inv_temp_log2 for all
     int32_t greedy;           // parts are (max, arg-max index) instead of (max, sum exp)
     const int32_t* row_seq;   // [m_rows] sequence of each row (for the vocabulary mask)
     const uint32_t* vocab_mask;
@@ -115,7 +117,9 @@ struct SampleParams {
     const int32_t* row_seq;
     int32_t batch, vocab, m_rows, s_rows, n_chunks, mask_words;
     int32_t row_begin;            // first row of this launch of the statistics kernel
-    float inv_temp_log2;          // log2(e) / T
+    float inv_temp_log2;          // log2(e) / T of the call (scalar temperature)
+    const float* temps;           // [B] per-sequence temperatures (device) or null
+    const float* row_c;           // [M + S] log2(e) / T per row, written by the plan kernel
     int32_t greedy;
     float2* stats;                // [(M+S)][n_chunks] parts written by the statistics kernel: (chunk max in logit
                                   // units, sum exp), or (max, arg-max index as int bits) in greedy mode
@@ -123,6 +127,8 @@ struct SampleParams {
     int32_t n_tparts;
     const int32_t* k_eff;         // [B] checked draft lengths (plan kernel)
     float top_p;                  // nucleus mass of the target distribution; >= 1: no filtering
+    int32_t top_k;                // keep the top_k most probable tokens first; <= 0: no filtering
+    int32_t filtered;             // top-k or top-p is on: the filter kernel ran and p.topp holds its thresholds
     double* topp;                 // [M][2]: lowest kept logit of the row's nucleus, mass of the nucleus (in units of
                                   // 2^((z - max) * c)); written by the nucleus kernel when top_p < 1
     int32_t* accepted_len;
@@ -147,7 +153,7 @@ struct Handle {
     float* logits;
     float* part_o; float* part_ml; int32_t* att_tickets; int32_t att_pairs_max;
     Plan plan;
-    float2* stats; float2* tstats; double* topp; float top_p;
+    float2* stats; float2* tstats; double* topp; float top_p; int32_t top_k; const float* temps;
     double* dbg_p; double* dbg_q; float* dbg_u;
     int32_t* status;
     // host staging for flexspec_verify_host
@@ -164,15 +170,17 @@ struct Handle {
 // launch wrappers (each returns a cudaError_t from the launch)
 // m_rows / s_rows / k_cap: the geometry derived from the HOST copy of the lengths; the kernel checks the
 // device copy against it
+// temps / scalar_c: per-sequence temperatures (device, may be null) and log2(e) / T of the call
 cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
-                        int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status, cudaStream_t stream);
+                        int32_t m_rows, int32_t s_rows, int32_t k_cap, const float* temps, float scalar_c, Plan plan,
+                        int32_t* status, cudaStream_t stream);
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, const AttTable& table,
                              int32_t n_ctas, cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
 // pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
 // the stream drains; it waits on the device before touching the predecessor's results)
-cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream);
+cudaError_t launch_sample_filter(const SampleParams& p, cudaStream_t stream);
 cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream);
 
 template <typename... KArgs, typename... Args>

@@ -205,9 +205,13 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                             sc[i] = __int_as_float(tile_row0(vt) + quarter * 32 + __ffs(eq) - 1);
                         }
                     } else {
+                        // log2(e) / T of every column's sequence (lane i < 16 fetches column i's)
+                        float c_lane = p.inv_temp_log2;
+                        if (p.row_c != nullptr && lane < 16) c_lane = __ldg(p.row_c + min(row_base + c0 + lane, p.m_rows - 1));
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
-                            sc[i] = fast_exp2((zv[i] - ((mx[i] == -INFINITY) ? 0.f : mx[i])) * p.inv_temp_log2);
+                            sc[i] = fast_exp2((zv[i] - ((mx[i] == -INFINITY) ? 0.f : mx[i])) *
+                                              (p.row_c != nullptr ? __shfl_sync(0xffffffffu, c_lane, i) : p.inv_temp_log2));
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1)
 #pragma unroll

@@ -16,13 +16,14 @@ constexpr int kStaticChunks = (kStaticMaxVocab + kSampleChunk - 1) / kSampleChun
 
 constexpr size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
-// layout of the scratch array (every piece 256-byte aligned): 268 032 bytes in all
+// layout of the scratch array (every piece 256-byte aligned): 276 224 bytes in all
 constexpr size_t kOffStatus = 0;                                                          // int32[4]
 constexpr size_t kOffCuQ = kOffStatus + 256;                                              // int32[batch + 1]
 constexpr size_t kOffCuD = kOffCuQ + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));
 constexpr size_t kOffKEff = kOffCuD + align256(sizeof(int32_t) * (kStaticMaxBatch + 1));   // int32[batch]
 constexpr size_t kOffRowSeq = kOffKEff + align256(sizeof(int32_t) * kStaticMaxBatch);      // int32[rows]
-constexpr size_t kOffStats = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);      // float2[2 * rows][chunks]
+constexpr size_t kOffRowC = kOffRowSeq + align256(sizeof(int32_t) * kStaticMaxRows);       // float[2 * rows]
+constexpr size_t kOffStats = kOffRowC + align256(sizeof(float) * 2 * kStaticMaxRows);      // float2[2 * rows][chunks]
 constexpr size_t kScratchBytes = kOffStats + align256(sizeof(float2) * 2 * kStaticMaxRows * kStaticChunks);
 
 // In host code this name is only a handle for the runtime: the device address comes from
@@ -94,7 +95,10 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     plan.cu_d = reinterpret_cast<int32_t*>(base + kOffCuD);
     plan.k_eff = reinterpret_cast<int32_t*>(base + kOffKEff);
     plan.row_seq = reinterpret_cast<int32_t*>(base + kOffRowSeq);
-    if (launch_plan(draft_len, draft_tokens, batch, vocab, m_rows, s_rows, k_batch_max, plan, status, s) != cudaSuccess)
+    plan.row_c = reinterpret_cast<float*>(base + kOffRowC);
+    const float scalar_c = greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    if (launch_plan(draft_len, draft_tokens, batch, vocab, m_rows, s_rows, k_batch_max, nullptr, scalar_c, plan, status,
+                    s) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
 
     SampleParams p;
@@ -106,7 +110,8 @@ extern "C" int flexspec_sample_static(const float* logits, const int32_t* draft_
     p.batch = batch; p.vocab = vocab; p.m_rows = m_rows; p.s_rows = s_rows;
     p.n_chunks = (vocab + kSampleChunk - 1) / kSampleChunk;
     p.mask_words = (vocab + 31) / 32;
-    p.inv_temp_log2 = greedy ? 1.f : static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    p.inv_temp_log2 = scalar_c;
+    p.row_c = plan.row_c; p.temps = nullptr; p.top_k = 0; p.filtered = 0;
     p.stats = reinterpret_cast<float2*>(base + kOffStats);
     p.tstats = p.stats; p.n_tparts = p.n_chunks;
     p.top_p = 1.f; p.topp = nullptr;

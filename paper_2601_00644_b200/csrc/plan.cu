@@ -40,7 +40,8 @@ __device__ __forceinline__ int block_inclusive_scan(int v, int* warp_tot)
 // sequence is treated as k_b = 0 on row min(b, m_rows - 1), and all tables stay inside [0, m_rows).
 __global__ void __launch_bounds__(kMaxBatch)
 plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ draft_tokens, int32_t batch,
-            int32_t vocab, int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status)
+            int32_t vocab, int32_t m_rows, int32_t s_rows, int32_t k_cap, const float* __restrict__ temps, float scalar_c,
+            Plan plan, int32_t* status)
 {
     __shared__ int warp_tot[32];
     const int t = threadIdx.x;
@@ -63,6 +64,7 @@ plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ d
         }
         if (t == 0) { plan.cu_q[batch] = m_rows; plan.cu_d[batch] = 0; }
         for (int r = t; r < m_rows; r += blockDim.x) plan.row_seq[r] = 0;
+        for (int r = t; r < m_rows + s_rows; r += blockDim.x) plan.row_c[r] = scalar_c;
         return;
     }
     if (live) {
@@ -70,7 +72,15 @@ plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ d
         plan.k_eff[t] = k;
         plan.cu_q[t] = q0;
         plan.cu_d[t] = d0;
-        for (int j = 0; j <= k; ++j) plan.row_seq[q0 + j] = t;
+        // log2(e) / T of the sequence: its own temperature if given (it must be a positive finite number)
+        float c = scalar_c;
+        if (temps != nullptr) {
+            const float tb = temps[t];
+            if (tb > 0.f && tb < 3.0e38f) c = 1.4426950408889634f / tb;
+            else report_error(status, kErrInvalidArg, t, 8);
+        }
+        for (int j = 0; j <= k; ++j) { plan.row_seq[q0 + j] = t; plan.row_c[q0 + j] = c; }
+        for (int j = 0; j < k; ++j) plan.row_c[m_rows + d0 + j] = c;
         if (draft_tokens != nullptr)
             for (int j = 0; j < k; ++j) {
                 const int x = draft_tokens[d0 + j];
@@ -84,10 +94,12 @@ plan_kernel(const int32_t* __restrict__ draft_len, const int32_t* __restrict__ d
 }
 
 cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, int32_t batch, int32_t vocab,
-                        int32_t m_rows, int32_t s_rows, int32_t k_cap, Plan plan, int32_t* status, cudaStream_t stream)
+                        int32_t m_rows, int32_t s_rows, int32_t k_cap, const float* temps, float scalar_c, Plan plan,
+                        int32_t* status, cudaStream_t stream)
 {
     const int threads = (batch + 31) / 32 * 32;
-    plan_kernel<<<1, threads, 0, stream>>>(draft_len, draft_tokens, batch, vocab, m_rows, s_rows, k_cap, plan, status);
+    plan_kernel<<<1, threads, 0, stream>>>(draft_len, draft_tokens, batch, vocab, m_rows, s_rows, k_cap, temps, scalar_c,
+                                           plan, status);
     return cudaGetLastError();
 }
 

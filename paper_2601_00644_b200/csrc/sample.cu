@@ -97,7 +97,7 @@ sample_stats_kernel(const SampleParams p)
     float mx = -INFINITY;
 #pragma unroll
     for (int i = 0; i < kElemsPerThread; ++i) mx = fmaxf(mx, z[i]);
-    const float c = p.inv_temp_log2;
+    const float c = p.row_c[row];                         // log2(e) / T of the row's sequence
     float2* out = p.stats + static_cast<int64_t>(row) * p.n_chunks + chunk;
 
     if (p.greedy) {
@@ -163,17 +163,47 @@ cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------------------------------------ nucleus (top-p)
-// The paper's stochastic regime samples the target with top-p 0.9.  The nucleus of a row is the set
-// of tokens whose logit is at least tau, where tau is the largest logit value such that the tokens
-// with logit >= tau hold at least top_p of the row's mass (ties with tau are all kept).  One CTA
-// per target row finds tau exactly by a 4-round radix selection over the order-preserving 32-bit
-// keys of the logits, 8 bits per round: a 256-bin histogram of probability MASS over the keys that
-// match the prefix found so far (one private fp32 histogram per warp, filled with the native
-// shared-memory float add -- with flat logits every key of a round falls into one or two bins, and
-// a single shared fp64 histogram serialised to a millisecond --, then summed in fp64), and a walk
-// from the top bin down to the bin in which the cumulative mass reaches the target.
-constexpr int kNucThreads = 1024;
+namespace cg = cooperative_groups;
+
+// asynchronous copies global -> shared memory
+__device__ __forceinline__ void cp_async_16(float* smem_dst, const float* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(float* smem_dst, const float* src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// ------------------------------------------------------------------------------------ top-k / top-p filter
+// The paper's stochastic regime samples the target with top-p 0.9; top-k is its usual companion and
+// is applied first.  Both filters are thresholds on the logit: the kept set of a row is
+// {v : z_v >= tau}, tau being the k-th largest logit (top-k; ties with it are kept), respectively the
+// largest logit such that the tokens with logit >= tau hold at least top_p of the (top-k filtered)
+// mass.  tau is found exactly by a radix selection over the order-preserving 32-bit keys of the
+// logits, 8 bits per round, the weight of a key being 1 (top-k) or its probability mass (top-p).
+//
+// One cluster of eight CTAs per target row; every CTA keeps its slice of the row in shared memory
+// (one read of the logits for all rounds).  Per round each CTA builds a 256-bin histogram of its
+// slice, restricted to the keys that match the prefix found so far; after one cluster barrier every
+// CTA adds up the eight histograms (read from its peers' shared memory; histograms alternate
+// between two buffers, so one barrier per round is enough) and walks from the top bin down to the
+// bin in which the running weight reaches the target.  Masses are accumulated as fixed-point integers
+// (2^((z - max) c) rounded to units of 2^-31, added as two 16-bit limbs with the native 32-bit
+// shared-memory atomics; 64-bit shared-memory atomics were measured 15x slower): integer addition is
+// exact and order-independent, so the histograms, the totals and the comparison with the target are
+// the same whatever the order of the atomic adds, and a row's result does not depend on scheduling.
+// The rounding of one entry is at most 2^-32 and unbiased: over a 128 K row its sum stays near 1e-8 of
+// the mass.
+constexpr int kFilterThreads = 256;
+constexpr int kFilterWarps = kFilterThreads / 32;
+constexpr int kFilterSliceMax = 16384;                    // entries of a slice kept in shared memory (64 KB)
+constexpr double kMassUnit = 2147483648.0;                // 2^31
+constexpr float kMassUnitF = 2147483648.0f;
 
 __device__ __forceinline__ uint32_t order_key(float z)       // larger float <-> larger key
 {
@@ -185,96 +215,199 @@ __device__ __forceinline__ float key_to_float(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-__global__ void __launch_bounds__(kNucThreads)
-sample_nucleus_kernel(const SampleParams p)
+struct FilterShared {
+    uint32_t hist[2][3][256];                           // [buffer][count, mass limb (bits 16..31), mass limb (bits 0..15)][bin]
+    unsigned long long tot[2][256];                     // cluster-wide histogram of the round
+    float red[kFilterWarps];
+    float slice_max[kAcceptCluster];
+    uint32_t prefix;                                    // key bits fixed so far
+    unsigned long long above[2];                        // count / mass of the keys above the prefix's bin path
+    unsigned long long target;
+    int bin;
+};
+
+__global__ void __cluster_dims__(kAcceptCluster, 1, 1) __launch_bounds__(kFilterThreads)
+sample_filter_kernel(const SampleParams p)
 {
-    __shared__ double s_hist[256];
-    __shared__ float s_whist[kNucThreads / 32][256];
-    __shared__ float s_redf[kNucThreads / 32];
-    __shared__ double s_redd[kNucThreads / 32];
-    __shared__ double s_above, s_target, s_binmass;
-    __shared__ uint32_t s_prefix;
-    const int row = blockIdx.x;
+    extern __shared__ float s_slice[];                  // this CTA's slice of the row (when it fits)
+    __shared__ FilterShared sh;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = static_cast<int>(cluster.block_rank());
+    const int row = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float cf = p.inv_temp_log2;
+    const float cf = p.row_c[row];
     const uint32_t* mask_row = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(p.row_seq[row]) * p.mask_words : nullptr;
-
-    // ---- (max, mass) of the row from its parts
-    const float2* tp = p.tstats + static_cast<int64_t>(row) * p.n_tparts;
-    float m = -INFINITY, sf = 0.f;
-    for (int i = tid; i < p.n_tparts; i += kNucThreads) {
-        const float2 pt = __ldcg(&tp[i]);
-        merge_ms(m, sf, pt.x, pt.y, cf);
-    }
-    const float mt = m;
-    m = warp_max(m);
-    if (lane == 0) s_redf[warp] = m;
-    __syncthreads();
-    for (int w = 0; w < kNucThreads / 32; ++w) m = fmaxf(m, s_redf[w]);
-    double sm = (mt == -INFINITY) ? 0.0 : static_cast<double>(sf) * static_cast<double>(fast_exp2((mt - m) * cf));
-    sm = warp_sum(sm);
-    if (lane == 0) s_redd[warp] = sm;
-    __syncthreads();
-    sm = 0.0;
-    for (int w = 0; w < kNucThreads / 32; ++w) sm += s_redd[w];
-    if (tid == 0) { s_above = 0.0; s_target = static_cast<double>(p.top_p) * sm; s_prefix = 0u; }
-
     const float* src = p.logits + static_cast<int64_t>(row) * p.vocab;
-    for (int round = 0; round < 4; ++round) {
-        const int shift = 24 - 8 * round;
-        for (int i = tid; i < (kNucThreads / 32) * 256; i += kNucThreads) (&s_whist[0][0])[i] = 0.f;
-        __syncthreads();
-        const uint32_t prefix = s_prefix;
-        const uint32_t hi_mask = (round == 0) ? 0u : (0xffffffffu << (shift + 8));
-        // eight loads in flight per thread (the row comes out of L2: a dependent load per element would
-        // cost its full latency 125 times per round)
-        for (int v0 = 0; v0 < p.vocab; v0 += kNucThreads * 8) {
-            float zz[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int v = v0 + i * kNucThreads + tid;
-                zz[i] = (v < p.vocab) ? __ldg(src + v) : -INFINITY;
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int v = v0 + i * kNucThreads + tid;
-                float z = zz[i];
-                if (mask_row != nullptr && v < p.vocab && !mask_allows(mask_row, v)) z = -INFINITY;
-                const uint32_t key = order_key(z);
-                if (z != -INFINITY && (key & hi_mask) == (prefix & hi_mask))
-                    atomicAdd(&s_whist[warp][(key >> shift) & 255u], fast_exp2((z - m) * cf));
-            }
+    cluster_arrive();                                   // "this CTA runs" (awaited before the first peer access)
+
+    // ---- this CTA's slice: [v0, v1), a multiple of four entries long so that 16-byte copies stay aligned
+    const int per = ((p.vocab + kAcceptCluster - 1) / kAcceptCluster + 3) & ~3;
+    const int v0 = min(p.vocab, rank * per), v1 = min(p.vocab, v0 + per);
+    const int n = v1 - v0;
+    const bool staged = per <= kFilterSliceMax;
+    const bool vec_ok = ((p.vocab & 3) == 0);
+    if (staged) {
+        if (vec_ok) {
+            for (int i = tid * 4; i < n; i += kFilterThreads * 4) cp_async_16(s_slice + i, src + v0 + i);
+        } else {
+            for (int i = tid; i < n; i += kFilterThreads) cp_async_4(s_slice + i, src + v0 + i);
         }
-        __syncthreads();
-        if (tid < 256) {
-            double acc = 0.0;
-#pragma unroll 8
-            for (int w = 0; w < kNucThreads / 32; ++w) acc += static_cast<double>(s_whist[w][tid]);
-            s_hist[tid] = acc;
-        }
-        __syncthreads();
-        if (tid == 0) {
-            double cum = s_above;
-            int bin = 255;
-            for (; bin > 0; --bin) {
-                if (cum + s_hist[bin] >= s_target) break;
-                cum += s_hist[bin];
-            }
-            s_above = cum;
-            s_binmass = s_hist[bin];
-            s_prefix = prefix | (static_cast<uint32_t>(bin) << shift);
-        }
+        cp_async_wait_all();
         __syncthreads();
     }
-    if (tid == 0) {
-        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(key_to_float(s_prefix));
-        p.topp[static_cast<int64_t>(row) * 2 + 1] = s_above + s_binmass;
+    auto logit = [&](int i) -> float {                  // entry i of the slice; masked entries read as -inf
+        const float z = staged ? s_slice[i] : __ldg(src + v0 + i);
+        return (mask_row != nullptr && !mask_allows(mask_row, v0 + i)) ? -INFINITY : z;
+    };
+
+    // ---- row maximum: slice maxima, exchanged through the peers' shared memory
+    float m = -INFINITY;
+    for (int i = tid; i < n; i += kFilterThreads) m = fmaxf(m, logit(i));
+    m = warp_max(m);
+    if (lane == 0) sh.red[warp] = m;
+    __syncthreads();
+    cluster_wait();                                     // all eight CTAs have started
+    if (tid < kAcceptCluster) {
+        float mm = sh.red[0];
+#pragma unroll
+        for (int w = 1; w < kFilterWarps; ++w) mm = fmaxf(mm, sh.red[w]);
+        cluster.map_shared_rank(&sh.slice_max[0], tid)[rank] = mm;
     }
+    if (tid == 0) { sh.prefix = 0u; sh.above[0] = 0ull; sh.above[1] = 0ull; }
+    cluster_sync();
+    m = sh.slice_max[0];
+#pragma unroll
+    for (int c = 1; c < kAcceptCluster; ++c) m = fmaxf(m, sh.slice_max[c]);
+
+    // ---- selections: top-k on counts (if on), then top-p on mass among the keys that survived
+    const bool do_k = p.top_k > 0 && p.top_k < p.vocab;
+    const bool do_p = p.top_p < 1.f;
+    uint32_t floor_key = 0u;                            // keys below it were cut by top-k
+    double kept_mass = 0.0;
+    float tau = -INFINITY;
+    int round_no = 0;                                   // alternates the histogram buffers
+    for (int sel = do_k ? 0 : 1; sel < (do_p ? 2 : 1); ++sel) {
+        // sel 0: weight 1, target k.   sel 1: weight mass, target top_p * (mass of the keys >= floor_key)
+        if (tid == 0) { sh.prefix = 0u; sh.above[0] = 0ull; sh.above[1] = 0ull; }
+        __syncthreads();
+        for (int round = 0; round < 4; ++round, ++round_no) {
+            const int shift = 24 - 8 * round;
+            const int buf = round_no & 1;
+            for (int i = tid; i < 3 * 256; i += kFilterThreads) (&sh.hist[buf][0][0])[i] = 0u;
+            __syncthreads();
+            const uint32_t prefix = sh.prefix;
+            const uint32_t hi_mask = (round == 0) ? 0u : (0xffffffffu << (shift + 8));
+            // four entries per thread and step (their loads and exponentials overlap).  When all lanes of
+            // the warp fall into the same bin (the leading bytes of flat logits) the warp adds once, one
+            // reduction per limb; grouping the lanes by bin with a match was measured twice as slow as
+            // letting them collide.
+            for (int i0 = 0; i0 < n; i0 += kFilterThreads * 4) {
+                int bin[4];
+                uint32_t w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * kFilterThreads + tid;
+                    const float z = (i < n) ? logit(i) : -INFINITY;
+                    const uint32_t key = order_key(z);
+                    const bool live = z != -INFINITY && key >= floor_key && (key & hi_mask) == (prefix & hi_mask);
+                    bin[u] = live ? static_cast<int>((key >> shift) & 255u) : -1;
+                    w[u] = live ? __float2uint_rn(fast_exp2((z - m) * cf) * kMassUnitF) : 0u;   // <= 2^31
+                }
+                const int bin0 = __shfl_sync(0xffffffffu, bin[0], 0);
+                if (__all_sync(0xffffffffu, bin[0] == bin0 && bin[1] == bin0 && bin[2] == bin0 && bin[3] == bin0)) {
+                    const uint32_t hi = __reduce_add_sync(0xffffffffu, (w[0] >> 16) + (w[1] >> 16) + (w[2] >> 16) + (w[3] >> 16));
+                    const uint32_t lo = __reduce_add_sync(0xffffffffu, (w[0] & 0xffffu) + (w[1] & 0xffffu) + (w[2] & 0xffffu) + (w[3] & 0xffffu));
+                    if (lane == 0 && bin0 >= 0) {
+                        atomicAdd(&sh.hist[buf][0][bin0], 128u);
+                        atomicAdd(&sh.hist[buf][1][bin0], hi);
+                        atomicAdd(&sh.hist[buf][2][bin0], lo);
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (bin[u] >= 0) {
+                            atomicAdd(&sh.hist[buf][0][bin[u]], 1u);
+                            atomicAdd(&sh.hist[buf][1][bin[u]], w[u] >> 16);
+                            atomicAdd(&sh.hist[buf][2][bin[u]], w[u] & 0xffffu);
+                        }
+                }
+            }
+            cluster_sync();                             // all eight histograms of this round are complete
+            // cluster-wide histogram: thread t adds bin t of the eight CTAs (both weights)
+            {
+                unsigned long long c_sum = 0ull, m_sum = 0ull;
+#pragma unroll
+                for (int c = 0; c < kAcceptCluster; ++c) {
+                    const uint32_t* peer = cluster.map_shared_rank(&sh.hist[buf][0][0], c);
+                    c_sum += peer[tid];
+                    m_sum += (static_cast<unsigned long long>(peer[256 + tid]) << 16) + peer[512 + tid];
+                }
+                sh.tot[0][tid] = c_sum;
+                sh.tot[1][tid] = m_sum;
+            }
+            __syncthreads();
+            if (warp == 0) {
+                // walk from the top bin down: lane l owns bins 255 - 8 l ... 248 - 8 l; both weights are
+                // scanned, the one of this selection decides
+                unsigned long long mine[2] = {0ull, 0ull};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    mine[0] += sh.tot[0][255 - (lane * 8 + j)];
+                    mine[1] += sh.tot[1][255 - (lane * 8 + j)];
+                }
+                unsigned long long incl[2] = {mine[0], mine[1]};      // inclusive scans over lanes (top bins first)
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned long long t0 = __shfl_up_sync(0xffffffffu, incl[0], o);
+                    const unsigned long long t1 = __shfl_up_sync(0xffffffffu, incl[1], o);
+                    if (lane >= o) { incl[0] += t0; incl[1] += t1; }
+                }
+                if (round == 0 && lane == 31) {
+                    // total weight of the live keys = the base of the target
+                    sh.target = (sel == 0) ? static_cast<unsigned long long>(p.top_k)
+                                           : static_cast<unsigned long long>(static_cast<double>(p.top_p) * static_cast<double>(incl[1]));
+                    if (sh.target < 1ull) sh.target = 1ull;
+                }
+                __syncwarp();
+                const unsigned long long target = sh.target;
+                unsigned long long run[2] = {sh.above[0] + incl[0] - mine[0], sh.above[1] + incl[1] - mine[1]};
+                const unsigned hit = __ballot_sync(0xffffffffu, (sel ? run[1] + mine[1] : run[0] + mine[0]) >= target);
+                // (with exact sums the last lane always reaches the target; the guard keeps the walk defined)
+                const int l = hit != 0u ? __ffs(hit) - 1 : 31;
+                if (lane == l) {
+                    int bin = 255 - lane * 8;
+                    for (int j = 0; j < 7; ++j, --bin) {
+                        if ((sel ? run[1] + sh.tot[1][bin] : run[0] + sh.tot[0][bin]) >= target) break;
+                        run[0] += sh.tot[0][bin];
+                        run[1] += sh.tot[1][bin];
+                    }
+                    sh.above[0] = run[0]; sh.above[1] = run[1];       // weights strictly above the chosen bin
+                    sh.bin = bin;
+                    sh.prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+                }
+            }
+            __syncthreads();
+        }
+        // the selected key: every key >= it is kept
+        const uint32_t key_sel = sh.prefix;
+        const unsigned long long mass_int = sh.above[1] + sh.tot[1][sh.bin];
+        floor_key = key_sel;
+        tau = key_to_float(key_sel);
+        kept_mass = static_cast<double>(mass_int) / kMassUnit;
+        __syncthreads();
+    }
+    if (rank == 0 && tid == 0) {
+        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(tau);
+        p.topp[static_cast<int64_t>(row) * 2 + 1] = kept_mass;
+    }
+    cluster_sync();                                     // no CTA leaves while a peer may still read its histograms
 }
 
-cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream)
+cudaError_t launch_sample_filter(const SampleParams& p, cudaStream_t stream)
 {
-    sample_nucleus_kernel<<<p.m_rows, kNucThreads, 0, stream>>>(p);
+    const int per = ((p.vocab + kAcceptCluster - 1) / kAcceptCluster + 3) & ~3;
+    const size_t smem = per <= kFilterSliceMax ? static_cast<size_t>(per) * sizeof(float) : 0;
+    sample_filter_kernel<<<dim3(kAcceptCluster, p.m_rows), kFilterThreads, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -310,8 +443,6 @@ cudaError_t launch_sample_nucleus(const SampleParams& p, cudaStream_t stream)
 // adds 32 of them in fp32 and everything above that -- lanes, chunks, slices, the running sums of
 // the final scan -- is fp64.  (Double-precision arithmetic per entry was measured at 12 us for this
 // phase alone: the vector fp64 rate of this GPU is a small fraction of its fp32 rate.)
-namespace cg = cooperative_groups;
-
 constexpr int kAcceptThreads = 256;        // two CTAs per SM: every cluster of a 16-sequence batch finds room at once
 constexpr int kAcceptWarps = kAcceptThreads / 32;
 constexpr int kAcceptRowsPerCta = (kMaxK + 1 + kAcceptCluster - 1) / kAcceptCluster;   // 8
@@ -349,18 +480,6 @@ struct DrawRow {
 // copies stay whole, the lane-interleaved walk (lane l takes entry 32 g + l) is conflict-free and
 // the lane-contiguous one (lane l takes entry 32 l + e) meets at most four lanes per bank.
 __device__ __forceinline__ int chunk_pos(int i) { return i ^ (((i >> 5) & 7) << 2); }
-__device__ __forceinline__ void cp_async_16(float* smem_dst, const float* src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_4(float* smem_dst, const float* src)
-{
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all()
-{
-    asm volatile("cp.async.wait_all;" ::: "memory");
-}
 // One warp requests the entries [base, base + kWarpChunk) of a row (those below vocab); nothing is
 // awaited.  vec_ok: the row starts on a 16-byte boundary and vocab is a multiple of four.
 __device__ __forceinline__ void stage_chunk(float* dst, const float* row, int base, int vocab, bool vec_ok, int lane)
@@ -438,8 +557,8 @@ sample_accept_kernel(const SampleParams p)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int k_b = p.k_eff[b];                            // tables of the plan kernel: complete before the preceding kernel started
     const int q0 = p.cu_q[b], d0 = p.cu_d[b];
-    const double scale = static_cast<double>(p.inv_temp_log2);
-    const float cf = p.inv_temp_log2;
+    const float cf = p.row_c[q0];                          // log2(e) / T of this sequence
+    const double scale = static_cast<double>(cf);
     const int my_rows = (k_b >= rank) ? (k_b - rank) / kAcceptCluster + 1 : 0;      // rows rank, rank + 8, ... <= k_b
     cluster_arrive();                                      // "this CTA runs": awaited before the first write into a peer's shared memory
 
@@ -538,7 +657,7 @@ sample_accept_kernel(const SampleParams p)
 #pragma unroll
                 for (int w = 0; w < kAcceptWarps; ++w) sm += red_d[w];
                 double tau = -INFINITY;                   // nucleus of the target row: its lowest kept logit and its mass
-                if (p.top_p < 1.f) { tau = p.topp[static_cast<int64_t>(q0 + j) * 2]; sm = p.topp[static_cast<int64_t>(q0 + j) * 2 + 1]; }
+                if (p.filtered) { tau = p.topp[static_cast<int64_t>(q0 + j) * 2]; sm = p.topp[static_cast<int64_t>(q0 + j) * 2 + 1]; }
                 int rej = 0;
                 if (test_row) {
                     const double u = s_u[i], qt = s_qt[i];
@@ -710,8 +829,12 @@ constexpr size_t kAcceptSmemBytes = static_cast<size_t>(kAcceptWarps) * 2 * kWar
 
 cudaError_t sample_init()
 {
-    return cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                static_cast<int>(kAcceptSmemBytes));
+    cudaError_t e = cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kAcceptSmemBytes));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(sample_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kFilterSliceMax * sizeof(float)));
+    return e;
 }
 
 cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream)

@@ -91,13 +91,15 @@ class Case:
         return dl, self.draft_tokens
 
     # ---- oracle: the decision stage
-    def oracle_accept(self, target_logits_f64, draft_logits=None, draft_tokens=None, temperature=None, top_p=1.0):
+    def oracle_accept(self, target_logits_f64, draft_logits=None, draft_tokens=None, temperature=None, top_p=1.0,
+                      top_k=0, temperatures=None):
         dl = self.draft_logits if draft_logits is None else draft_logits
         dt = self.draft_tokens if draft_tokens is None else draft_tokens
         t = self.shape.temperature if temperature is None else temperature
         return oracle.accept(self.mode, target_logits_f64,
                              None if dl is None else dl.cpu().numpy(), dt.cpu().numpy(), self.k,
-                             self.h_seeds, t, self.vocab_mask, self.check, top_p=top_p)
+                             self.h_seeds, t, self.vocab_mask, self.check, top_p=top_p, top_k=top_k,
+                             temperatures=temperatures)
 
 
 def make_verifier(case: Case, debug=True, mode=None):
@@ -152,7 +154,7 @@ def _ratio(p, q):
 
 
 def compare_end_to_end(case: Case, acc_gpu, nxt_gpu, ref_own, ref_gpu_logits, logits_o, logits_g,
-                       temperature, top_p=1.0, cdf_tol=CDF_TIE_TOL, label="end-to-end"):
+                       temperature, top_p=1.0, cdf_tol=CDF_TIE_TOL, label="end-to-end", top_k=0, temperatures=None):
     """GPU decisions against the oracle's own chain (its attention -> bf16 -> its LM head -> its decisions).
 
     The two sides decide on slightly different logits (a bf16 rounding of the attention output that
@@ -207,8 +209,9 @@ def compare_end_to_end(case: Case, acc_gpu, nxt_gpu, ref_own, ref_gpu_logits, lo
         row = case.row0[b] + n_o
         drow = case.draft_logits[t0 + n_o].cpu().numpy() if n_o < case.k[b] else None
         mask = None if case.vocab_mask is None else case.vocab_mask[b]
-        w_o, z_o = oracle.emission(logits_o[row], drow, temperature, top_p, mask)
-        w_g, z_g = oracle.emission(logits_g[row].astype(np.float64), drow, temperature, top_p, mask)
+        t_b = temperature if temperatures is None else float(temperatures[b])
+        w_o, z_o = oracle.emission(logits_o[row], drow, t_b, top_p, mask, top_k=top_k)
+        w_g, z_g = oracle.emission(logits_g[row].astype(np.float64), drow, t_b, top_p, mask, top_k=top_k)
         u2 = oracle.uniform(int(case.h_seeds[b]), n_o, 1)
         shift = float(np.abs(np.cumsum(w_g) - np.cumsum(w_o)).max()) + u2 * abs(z_g - z_o)
         assert int(ref_gpu_logits["next_token"][b]) == int(nxt_gpu[b]) and margin * z_o <= shift + 1e-15, (
@@ -218,7 +221,7 @@ def compare_end_to_end(case: Case, acc_gpu, nxt_gpu, ref_own, ref_gpu_logits, lo
     return out
 
 
-def full_parity(case: Case, ver, vocab_mask_dev=None, top_p=1.0):
+def full_parity(case: Case, ver, vocab_mask_dev=None, top_p=1.0, top_k=0, temperatures=None):
     """Stage-by-stage and end-to-end comparison of one verify call.  Returns a report dict."""
     acc, nxt = run_gpu_verify(case, ver, vocab_mask_dev)
     m, s = case.inp.m_rows, case.inp.s_rows
@@ -238,7 +241,7 @@ def full_parity(case: Case, ver, vocab_mask_dev=None, top_p=1.0):
     assert ok and rep["logit_row_err"] < REL_TOL, f"logits: {rep}"
 
     # (i) decision stage in isolation: the oracle is fed the GPU's own fp32 logits
-    ref_iso = case.oracle_accept(logits_g.astype(np.float64), top_p=top_p)
+    ref_iso = case.oracle_accept(logits_g.astype(np.float64), top_p=top_p, top_k=top_k, temperatures=temperatures)
     if top_p < 1.0:
         # a nucleus cut within 1e-6 of top_p is a near-tie of the filter itself: such sequences are
         # counted and left out of the identity requirement
@@ -259,8 +262,9 @@ def full_parity(case: Case, ver, vocab_mask_dev=None, top_p=1.0):
     rep["iso_ties"], rep["iso_cdf_ties"] = compare_decisions(case, acc, nxt, ref_iso, CDF_TIE_TOL, "isolated")
 
     # (ii) end to end: the oracle's own attention -> bf16 -> LM head -> decisions
-    ref_e2e = case.oracle_accept(logits_o, top_p=top_p)
-    e2e = compare_end_to_end(case, acc, nxt, ref_e2e, ref_iso, logits_o, logits_g, t, top_p)
+    ref_e2e = case.oracle_accept(logits_o, top_p=top_p, top_k=top_k, temperatures=temperatures)
+    e2e = compare_end_to_end(case, acc, nxt, ref_e2e, ref_iso, logits_o, logits_g, t, top_p, top_k=top_k,
+                             temperatures=temperatures)
     rep["e2e_ties"], rep["e2e_cdf_ties"] = e2e["ties"], e2e["cdf_ties"]
     rep["e2e_explained"] = e2e["explained_accept"] + e2e["explained_token"]
     if case.mode == 0 and drows.size:

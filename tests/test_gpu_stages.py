@@ -318,3 +318,91 @@ def test_a_bounded_wait_runs_out_and_is_reported():
     with pytest.raises(B.FlexSpecError):
         ver.selftest_wait_timeout(10 ** 9)         # limits beyond 50 ms are refused on the host
     ver.close()
+
+
+# ------------------------------------------------------------------ top-k and per-sequence temperatures
+
+def _decisions_match(k, acc, nxt, ref, p_g=None, skip=()):
+    """Identical decisions except at near-ties (1e-5 acceptance, 1e-6 inverse CDF); returns #excused."""
+    t0 = np.concatenate([[0], np.cumsum(k)])
+    excused = 0
+    for b in range(len(k)):
+        if b in skip:
+            continue
+        kb = int(k[b])
+        if p_g is not None and kb:
+            assert np.abs(p_g[t0[b]:t0[b] + kb] - ref["p_tok"][t0[b]:t0[b] + kb]).max() < 1e-5, b
+        if acc[b] != ref["accepted_len"][b]:
+            assert ref["acc_margin"][t0[b] + min(acc[b], ref["accepted_len"][b])] < 1e-5, b
+            excused += 1
+        elif nxt[b] != ref["next_token"][b]:
+            assert ref["cdf_margin"][b] < 1e-6, (b, nxt[b], ref["next_token"][b])
+            excused += 1
+    return excused
+
+
+@pytest.mark.parametrize("top_k,top_p", [(1, 1.0), (5, 1.0), (50, 1.0), (40, 0.9), (3, 0.5)])
+@pytest.mark.parametrize("vocab,batch,k_hi,holes,mask", [
+    (4096, 3, 4, False, False),
+    (777, 9, 7, True, False),
+    (20000, 12, 12, False, True),
+])
+def test_sample_stage_with_top_k_matches_oracle(top_k, top_p, vocab, batch, k_hi, holes, mask):
+    B = _binding()
+    temperature = 0.8
+    k, zt, zd, toks, seeds, vmask = _sample_case(11 * vocab + batch + top_k, batch, vocab, 0, k_hi, 0, temperature,
+                                                 holes=holes, mask=mask)
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=max(k_hi, 1), max_kv_len=64, mode=0, debug=True)
+    ver.set_sampling(top_p=top_p, top_k=top_k)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).cuda()
+    vm_d = None if vmask is None else dev(vmask.view(np.int32), torch.int32)
+    acc, nxt = ver.sample(dev(zt, torch.float32), dev(toks, torch.int32), dev(zd, torch.float32), dev(k, torch.int32),
+                          torch.from_numpy(k), dev(seeds.view(np.int64), torch.int64), temperature=temperature, vocab_mask=vm_d)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    ref = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, temperature, vmask, top_p=top_p, top_k=top_k)
+    r0 = np.concatenate([[0], np.cumsum(k + 1)])
+    dbg = ver.debug(int(k.sum()) + batch, int(k.sum()))
+    # a nucleus cut within 1e-6 of top_p may land one token earlier / later: such sequences are left out
+    skip = [b for b in range(batch) if ref["topp_margin"][r0[b]:r0[b + 1]].min() < 1e-6]
+    assert len(skip) <= 1
+    assert _decisions_match(k, acc.cpu().numpy(), nxt.cpu().numpy(), ref, dbg["p_tok"].cpu().numpy(), skip) <= 1
+    if top_k <= 5 and k.sum() > 0:                    # the filter is really on
+        assert (ref["p_tok"] == 0).any()
+    ver.close()
+
+
+def test_sample_stage_with_per_sequence_temperatures_matches_oracle():
+    B = _binding()
+    batch, vocab, k_hi = 10, 6000, 6
+    k, zt, zd, toks, seeds, _ = _sample_case(4242, batch, vocab, 0, k_hi, 0, 1.0)
+    temps = np.array([0.5, 1.0, 0.7, 1.3, 2.0, 0.9, 1.0, 0.6, 1.7, 0.8], np.float32)
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=k_hi, max_kv_len=64, mode=0, debug=True)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).cuda()
+    args = (dev(zt, torch.float32), dev(toks, torch.int32), dev(zd, torch.float32), dev(k, torch.int32),
+            torch.from_numpy(k), dev(seeds.view(np.int64), torch.int64))
+    for top_p, top_k in [(1.0, 0), (0.9, 30)]:
+        ver.set_sampling(top_p=top_p, top_k=top_k, temperatures=dev(temps, torch.float32))
+        acc, nxt = ver.sample(*args, temperature=1.0)          # the scalar is overridden per sequence
+        torch.cuda.synchronize()
+        assert ver.status()[0] == 0
+        ref = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, 1.0, None, top_p=top_p, top_k=top_k,
+                            temperatures=temps.astype(np.float64))
+        r0 = np.concatenate([[0], np.cumsum(k + 1)])
+        skip = [b for b in range(batch) if ref["topp_margin"][r0[b]:r0[b + 1]].min() < 1e-6]
+        dbg = ver.debug(int(k.sum()) + batch, int(k.sum()))
+        assert _decisions_match(k, acc.cpu().numpy(), nxt.cpu().numpy(), ref, dbg["p_tok"].cpu().numpy(), skip) <= 1
+    # a temperature that is not a positive finite number is reported, and the scalar is used for that sequence
+    bad = temps.copy(); bad[3] = 0.0
+    ver.set_sampling(temperatures=dev(bad, torch.float32))
+    ver.sample(*args, temperature=1.0)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == B.ERR_INVALID_ARG
+    # switched off again: the scalar applies to every sequence
+    ver.set_sampling()
+    acc, nxt = ver.sample(*args, temperature=0.9)
+    ref = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, 0.9)
+    assert _decisions_match(k, acc.cpu().numpy(), nxt.cpu().numpy(), ref) <= 1
+    ver.close()

@@ -70,6 +70,29 @@ def test_verify_with_top_p_on_peaked_logits():
     _few_differences(case, rep, share=0.2)
 
 
+def test_verify_with_top_k_and_per_sequence_temperatures():
+    """The whole step with top-k 20 (then top-p 0.95) and a temperature of its own for every sequence: the
+    LM-head epilogue, the draft-logit statistics, the filter and the acceptance kernel all use the
+    sequence's temperature."""
+    H = _H()
+    shape = wl.peaked(wl.scaled(wl.CONFIGS["llama3_8b"], batch=5, vocab=20000, ctx_min=200, ctx_max=500, k_min=2, k_max=6,
+                                index=18))
+    case = H.Case(shape)
+    temps = np.array([0.6, 1.0, 1.4, 0.8, 1.1])
+    # the edge draws its tokens at the sequence's temperature too: rebuild the drafts row by row
+    case.build_drafts()
+    for b in range(case.batch):
+        sl = slice(case.tok0[b], case.tok0[b + 1])
+        case.draft_tokens[sl] = wl.draw_draft_tokens(case.draft_logits[sl], float(temps[b]), case.inp.token_uniforms[sl])
+    ver = H.make_verifier(case)
+    t_dev = torch.from_numpy(temps.astype(np.float32)).cuda()
+    ver.set_sampling(top_p=0.95, top_k=20, temperatures=t_dev)
+    rep = H.full_parity(case, ver, top_p=0.95, top_k=20, temperatures=temps)
+    assert rep["topp_ties"] <= 1
+    _few_differences(case, rep, share=0.2)
+    ver.close()
+
+
 def test_ragged_batch_with_k0_and_greedy():
     shape = wl.scaled(wl.CONFIGS["adaptive_k"], batch=7, vocab=9000, k_min=0, k_max=12, ctx_min=30,
                       ctx_max=900, index=12)
