@@ -27,9 +27,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch at the default
-# workload, from the ncu capture summarised in profiles/ (None until captured)
-LM_HEAD_TRAFFIC_BYTES = 1051930000 + 8530432
+# dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch, per workload, from the ncu
+# captures summarised in profiles/ (a workload without a capture of the current kernel reports null)
+LM_HEAD_TRAFFIC_BYTES = {}
 FALLBACK_HBM_GBS = 6650.0
 REFERENCE_BUDGET_S = 120.0
 
@@ -44,7 +44,10 @@ def _peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks / throttle reasons sampled every 100 ms from before the warm-up until after the
+    end-to-end leg (a 20-step timed region lasts a few milliseconds: alone it would see no sample).
+    The median clock is taken over the samples drawn under load: board power at least half of the
+    run's highest sample (between phases the GPU idles and clocks down)."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -58,7 +61,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "200"],
+                 "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -77,22 +80,25 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        rows, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
                 continue
             try:
-                sm.append(float(parts[0])); smax.append(float(parts[1]))
+                rows.append((float(parts[0]), float(parts[2]))); smax.append(float(parts[1]))
             except ValueError:
                 continue
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None,
+        p_max = max((p for _, p in rows), default=0.0)
+        loaded = [c for c, p in rows if p >= 0.5 * p_max]
+        return {"sm_mhz": statistics.median(loaded) if loaded else None,
                 "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(loaded), "samples_total": len(rows),
+                "power_w_max": p_max}
 
 
 def _dist_env():
@@ -241,11 +247,23 @@ def fit_cloud_cost(args, base_shape, dev):
             "note": "median of 20 steps per K, batch and context of the workload; draft logits = noise only"}
 
 
+def _free_port():
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
 def run_ours(args):
     import numpy as np
     import torch
     from paper_2601_00644_b200 import binding, workloads as wl
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: become the launcher of N ranks (one per GPU) of this same command
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     rank, local_rank, world = _dist_env()
     if world > 1:
         import torch.distributed as dist
@@ -261,8 +279,11 @@ def run_ours(args):
     ver = binding.Verifier(inp.lm_head_w, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                            max_batch=batch, k_max=int(k_host.max()), max_kv_len=int(kv_host.max()))
 
-    if args.top_p < 1.0:
-        ver.set_top_p(args.top_p)
+    if args.top_p < 1.0 or args.top_k > 0:
+        ver.set_sampling(top_p=args.top_p, top_k=args.top_k)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
     # draft logits = target logits (from this library's attention + LM head) + sigma * noise
     attn = ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, kv_host, inp.hidden, inp.draft_len, k_host)
     tgt = ver.lm_head(attn)
@@ -303,9 +324,6 @@ def run_ours(args):
     # sweep between steps is outside the event pairs
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     barrier()
     t_wall0 = time.perf_counter()
     for i in range(args.steps):
@@ -329,7 +347,31 @@ def run_ours(args):
         stage_acc += np.array(ver.stage_ms())
     ver.set_profiling(False)
     stage_ms = (stage_acc / n_prof).tolist()
-    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- the attention stage of a real model runs once per layer: time L launches of it, each on its own KV pool
+    layers_info = None
+    if args.layers > 1:
+        pools = [inp.kv_pages] + [torch.randn_like(inp.kv_pages) * shape.input_std for _ in range(min(args.layers, 8) - 1)]
+        out = torch.empty(m_rows, shape.d_model, dtype=torch.bfloat16, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_layers = []
+        for it in range(3 + 10):
+            flush_l2()
+            e0.record(stream)
+            for l in range(args.layers):
+                ver.attention(pools[l % len(pools)], inp.page_table, inp.kv_len, kv_host, inp.hidden, inp.draft_len, k_host,
+                              attn_out=out, stream=stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                t_layers.append(e0.elapsed_time(e1))
+        att_ms = statistics.median(t_layers)
+        layers_info = {"layers": args.layers, "attention_ms_all_layers": att_ms,
+                       "attention_us_per_layer": att_ms / args.layers * 1e3,
+                       "distinct_kv_pools": len(pools),
+                       "note": "K1 launched once per layer back to back (pools rotate, so no layer finds its K/V in L2); "
+                               "the other per-layer work of a real model (projections, MLP) is outside this library"}
+        del pools, out
 
     # ---- end to end through the host-buffer entry point (H2D of the step's inputs, D2H of results)
     pin = lambda t: t.cpu().pin_memory()
@@ -351,6 +393,16 @@ def run_ours(args):
         step_host()
     barrier()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
+    # the same bytes as one plain pinned host-to-device copy, in the same run: what the link alone costs
+    stage_dev = torch.empty(h_dlog.numel() + 16, dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        stage_dev[:h_dlog.numel()].view_as(h_dlog).copy_(h_dlog, non_blocking=True)
+        torch.cuda.synchronize()
+    copy_s = (time.perf_counter() - t0) / e2e_steps
+    del stage_dev
+    clocks = sampler.stop() if rank == 0 else None
     h2d = h_hidden.numel() * 2 + h_tok.numel() * 4 + h_dlog.numel() * 4 + h_len.numel() * 4 * 2 + h_seeds.numel() * 8
     d2h = 2 * batch * 4
     assert torch.equal(h_acc.to(dev), acc) and torch.equal(h_nxt.to(dev), nxt)
@@ -366,6 +418,7 @@ def run_ours(args):
         alg_bytes = v * d * 2 + kv_bytes + 3 * m_rows * d * 2 + s_rows * v * 4
         lm_bytes = v * d * 2                                             # 2*d bytes per vocabulary row
         lm_ms = stage_ms[3]
+        step_sum_ms = ms_per_step
         achieved = lm_bytes / (lm_ms * 1e-3) / 1e9 if lm_ms > 0 else 0.0
         line = {
             "metric": "verified_tokens_per_s", "value": verified_all / (ms_per_step * 1e-3), "unit": "tokens/s",
@@ -375,7 +428,7 @@ def run_ours(args):
             "config": {"workload": shape.name, "batch_per_gpu": batch, "k": [int(k_host.min()), int(k_host.max())],
                        "context": [shape.ctx_min, shape.ctx_max], "vocab": v, "d_model": d,
                        "heads": [shape.n_q_heads, shape.n_kv_heads, shape.head_dim],
-                       "temperature": shape.temperature, "mode": "sample", "top_p": args.top_p,
+                       "temperature": shape.temperature, "mode": "sample", "top_p": args.top_p, "top_k": args.top_k,
                        "l2": "read sweep of a 512 MiB buffer between steps, outside the event pairs"},
             "step_us": ms_per_step * 1e3,
             "step_us_median": statistics.median(step_ms) * 1e3,
@@ -392,19 +445,33 @@ def run_ours(args):
                                  "plan and draft-logit statistics run on a second stream beside attention"},
             "roofline": {"kernel": "lm_head_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-                         "traffic": LM_HEAD_TRAFFIC_BYTES, "algorithmic_bytes": lm_bytes},
+                         "traffic": LM_HEAD_TRAFFIC_BYTES.get(shape.name), "algorithmic_bytes": lm_bytes,
+                         "step_share": lm_ms / step_sum_ms},
             "e2e": {"value": verified_all / e2e_s, "unit": "tokens/s", "ms_per_step": e2e_s * 1e3,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "note": "flexspec_verify_host: per-step inputs from pinned host memory; KV pool and W resident"},
+                    "plain_h2d_copy_ms": copy_s * 1e3, "copy_share_of_e2e": copy_s / e2e_s,
+                    "note": "flexspec_verify_host: per-step inputs from pinned host memory; KV pool and W resident; "
+                            "plain_h2d_copy_ms = the draft logits alone as one pinned cudaMemcpyAsync in the same run"},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
             "wall_s_timed_region": t_wall,
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl.CONFIGS[args.config])
+        if layers_info is not None:
+            step_l = ms_per_step + layers_info["attention_ms_all_layers"] - stage_ms[1]
+            layers_info["attention_share_of_step"] = layers_info["attention_ms_all_layers"] / step_l
+            layers_info["step_ms_with_all_layers"] = step_l
+            line["layers"] = layers_info
         if world == 1 and args.fit_k:
             del flush
-            line["cloud_cost_fit"] = fit_cloud_cost(args, wl.CONFIGS[args.config], dev)
+            fit = fit_cloud_cost(args, wl.CONFIGS[args.config], dev)
+            line["cloud_cost_fit"] = fit
+            # the paper's objective (Eq. 2) with the fitted cloud constants: adaptive stride against fixed strides
+            from paper_2601_00644_b200 import policy
+            lat = policy.default_latency_model(fit["T_base_us"] * 1e-6, max(fit["delta_cloud_us_per_token"], 0.0) * 1e-6)
+            line["etgr_tokens_per_s"] = {k: {a: round(float(b), 3) for a, b in v.items()}
+                                         for k, v in policy.etgr_table(lat).items()}
         print(json.dumps(line))
     ver.close()
     if world > 1:
@@ -421,6 +488,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--top-p", type=float, default=1.0,
                     help="nucleus sampling of the target (the paper's stochastic regime uses 0.9); 1.0 = off")
+    ap.add_argument("--top-k", type=int, default=0, help="top-k filter of the target before the nucleus; 0 = off")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="also time the attention stage L times back to back (one launch per layer of a real model)")
     ap.add_argument("--fit-k", action="store_true",
                     help="also measure the step at several draft lengths and fit the paper's T_base + K*delta_cloud")
     args = ap.parse_args()

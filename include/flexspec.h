@@ -38,9 +38,10 @@
  *     read from row j judges draft token x_j; row k_b is the bonus row.  Draft
  *     rows (tokens, draft logits) are packed the same way with k_b per sequence.
  *   - M = sum_b (k_b+1) query rows, S = sum_b k_b draft positions.
- *   - The library never writes to the KV pages.  KV rollback after a rejection
- *     (Section IV-C) is the caller's: the next call passes a kv_len truncated
- *     according to accepted_len.
+ *   - flexspec_verify and the stage calls never write to the KV pages; the session
+ *     calls around the step do (Section IV-C): flexspec_kv_append writes the window's
+ *     K/V rows before it, flexspec_kv_rollback computes the truncated kv_len after a
+ *     rejection and flexspec_kv_release hands the pages past it back.
  */
 #ifndef FLEXSPEC_H
 #define FLEXSPEC_H
@@ -105,7 +106,8 @@ typedef struct {            /* DEVICE pointers into the handle's workspace, vali
     const int32_t* status;     /* int32 [4] device status word: [0] first error code, [1] detail  */
 } flexspec_debug;
 
-/* Create a handle: validates the shape, allocates the workspace on cfg->device
+/* Create a handle for one target model's verification step (the frozen head and the KV-session
+ * layout of Sections IV-A and IV-C): validates the shape, allocates the workspace on cfg->device
  * (logits [max_batch*(k_max+1)][vocab] fp32, attention partials, small tables)
  * and builds the TMA descriptor of the LM-head weights.
  *   lm_head_w : DEVICE bf16 [vocab][d_model] (row v is the output embedding of
@@ -145,17 +147,18 @@ int flexspec_verify(flexspec_handle* h, const flexspec_kv* kv, const void* hidde
                     const uint32_t* vocab_mask,
                     int32_t* accepted_len, int32_t* next_token, void* stream);
 
-/* The same step for callers whose per-step inputs live in HOST memory: copies
- * hidden, draft tokens, draft logits, lengths and seeds to the device, runs
- * flexspec_verify, copies accepted_len / next_token back and synchronises.
- * The KV pool and page table stay on the device (they are the persistent
- * session state); kv->kv_len may be NULL here (taken from kv->kv_len_host).
- * Every other pointer argument is a HOST pointer. */
+/* The same step (Algorithm 2, Step 2: the cloud receives the draft block over the uplink and
+ * returns the verified tokens) for callers whose per-step inputs live in HOST memory: copies
+ * hidden, draft tokens, draft logits, lengths, seeds and the optional vocabulary mask to the
+ * device, runs flexspec_verify, copies accepted_len / next_token back and synchronises.
+ * The KV pool and page table stay on the device (they are the persistent session state of
+ * Section IV-C); kv->kv_len may be NULL here (taken from kv->kv_len_host).
+ * Every other pointer argument is a HOST pointer (vocab_mask may be NULL). */
 int flexspec_verify_host(flexspec_handle* h, const flexspec_kv* kv, const void* hidden,
                          const int32_t* draft_tokens, const float* draft_logits,
                          const int32_t* draft_len, const uint64_t* seeds, int32_t batch,
-                         float temperature, int32_t* accepted_len, int32_t* next_token,
-                         void* stream);
+                         float temperature, const uint32_t* vocab_mask,
+                         int32_t* accepted_len, int32_t* next_token, void* stream);
 
 /* Stage 1 alone (Section IV-C; Algorithm 2 "restore KV cache" + target forward over the block):
  * attn_out DEVICE bf16 [M][d_model] out, or NULL to write the handle's workspace. */
@@ -198,6 +201,23 @@ int flexspec_kv_append(flexspec_handle* h, void* kv_pages, int32_t num_pages, co
  * first.  All pointers DEVICE int32 [batch]; kv_len_next may alias kv_len. */
 int flexspec_kv_rollback(flexspec_handle* h, const int32_t* kv_len, const int32_t* draft_len,
                          const int32_t* accepted_len, int32_t batch, int32_t* kv_len_next, void* stream);
+
+/* KV session, after the rollback: the pages that hold no valid token any more are handed back
+ * (Section IV-C: "discarding" the invalid K/V pairs -- with paged storage that is a free list).
+ * For every sequence the page-table entries ceil(kv_len_next[b] / 16) .. ceil(kv_len_prev[b] / 16) - 1
+ * are appended to free_list (one reservation per sequence: its pages stay together, in ascending
+ * entry order; the order of the sequences in the list is not defined) and set to -1.
+ *   page_table   DEVICE int32 [batch][max_pages_per_seq], modified in place
+ *   kv_len_prev  DEVICE int32 [batch]: the length the pages were allocated for (before the rollback)
+ *   kv_len_next  DEVICE int32 [batch]: e.g. the output of flexspec_kv_rollback
+ *   free_list    DEVICE int32 [free_capacity]; free_count DEVICE int32 [1], advanced atomically (the
+ *                caller sets it, usually to the list's current fill)
+ * Note that the next step's window positions then need pages again: release only what the serving
+ * loop will not re-use at once.  Asynchronous on `stream`.  Errors: INVALID_ARG, CUDA; an entry
+ * outside [0, num_pages) or a list that is too short is recorded in the status word. */
+int flexspec_kv_release(flexspec_handle* h, int32_t* page_table, int32_t max_pages_per_seq, int32_t num_pages,
+                        const int32_t* kv_len_prev, const int32_t* kv_len_next, int32_t batch, int32_t* free_list,
+                        int32_t free_capacity, int32_t* free_count, void* stream);
 
 /* The acceptance / emitted-token stage (flexspec_sample) without a handle and without any
  * allocation.  (No counterpart in the paper: it exists for how some hosts have to run.)
@@ -249,10 +269,11 @@ int flexspec_set_top_p(flexspec_handle* h, float top_p);
  * SAMPLE mode only.  Errors: INVALID_ARG. */
 int flexspec_set_sampling(flexspec_handle* h, float top_p, int32_t top_k, const float* temperatures);
 
-/* Workspace pointers for stage-wise comparison. */
+/* Workspace pointers for stage-wise comparison with an independent implementation of Algorithm 2,
+ * Step 2 (attention output, logits, p_j(x_j), q_j(x_j), u_j of the last call). */
 int flexspec_get_debug(flexspec_handle* h, flexspec_debug* out);
 
-/* Synchronises the device, copies the status word to status_host[4] (may be NULL), clears it
+/* Device-side error reporting (no counterpart in the paper).  Synchronises the device, copies the status word to status_host[4] (may be NULL), clears it
  * and returns its first entry (0 or a FLEXSPEC_ERR_* code recorded by a kernel). */
 int flexspec_status(flexspec_handle* h, int32_t* status_host);
 
@@ -277,7 +298,8 @@ int flexspec_get_stage_ms(flexspec_handle* h, float ms[6]);
 /* Number of kernels the last verify / stage call launched. */
 int flexspec_last_launches(flexspec_handle* h);
 
-/* Releases the workspace.  NULL is accepted. */
+/* Releases the workspace (the KV sessions and the LM-head weights are the caller's and are not
+ * touched).  NULL is accepted. */
 int flexspec_destroy(flexspec_handle* h);
 
 const char* flexspec_strerror(int code);

@@ -25,7 +25,7 @@ ERR_TIMEOUT, ERR_BAD_PAGE, ERR_BAD_TOKEN, ERR_NO_DEVICE = -5, -6, -7, -8
 EXPORTS = [
     "flexspec_create", "flexspec_verify", "flexspec_verify_host", "flexspec_attention",
     "flexspec_lm_head", "flexspec_sample", "flexspec_sample_static", "flexspec_kv_append",
-    "flexspec_kv_rollback", "flexspec_set_top_p", "flexspec_set_sampling", "flexspec_get_debug", "flexspec_status",
+    "flexspec_kv_rollback", "flexspec_kv_release", "flexspec_set_top_p", "flexspec_set_sampling", "flexspec_get_debug", "flexspec_status",
     "flexspec_selftest_wait_timeout", "flexspec_set_profiling", "flexspec_get_stage_ms", "flexspec_last_launches",
     "flexspec_destroy", "flexspec_strerror", "flexspec_version",
 ]
@@ -58,13 +58,14 @@ def _load() -> C.CDLL:
     vp, i32, f32 = C.c_void_p, C.c_int32, C.c_float
     lib.flexspec_create.argtypes = [C.POINTER(Config), vp, C.POINTER(vp)]
     lib.flexspec_verify.argtypes = [vp, C.POINTER(KV), vp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
-    lib.flexspec_verify_host.argtypes = [vp, C.POINTER(KV), vp, vp, vp, vp, vp, i32, f32, vp, vp, vp]
+    lib.flexspec_verify_host.argtypes = [vp, C.POINTER(KV), vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     lib.flexspec_attention.argtypes = [vp, C.POINTER(KV), vp, vp, vp, i32, vp, vp]
     lib.flexspec_lm_head.argtypes = [vp, vp, i32, vp, vp]
     lib.flexspec_sample.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp]
     lib.flexspec_sample_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp]
     lib.flexspec_kv_append.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.flexspec_kv_rollback.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    lib.flexspec_kv_release.argtypes = [vp, vp, i32, i32, vp, vp, i32, vp, i32, vp, vp]
     lib.flexspec_set_top_p.argtypes = [vp, f32]
     lib.flexspec_set_sampling.argtypes = [vp, f32, i32, vp]
     lib.flexspec_get_debug.argtypes = [vp, C.POINTER(Debug)]
@@ -200,18 +201,18 @@ class Verifier:
         return accepted_len, next_token
 
     def verify_host(self, kv_pages, page_table, kv_len_host, hidden, draft_tokens, draft_logits,
-                    draft_len, seeds, accepted_len, next_token, temperature=1.0, stream=None):
+                    draft_len, seeds, accepted_len, next_token, temperature=1.0, stream=None, vocab_mask=None):
         """Per-step inputs and outputs are HOST tensors (pinned for speed); KV stays on the device."""
         batch = int(draft_len.numel())
         kv = self._kv(kv_pages, page_table, None, kv_len_host)
         for t, name in ((hidden, "hidden"), (draft_tokens, "draft_tokens"), (draft_logits, "draft_logits"),
                         (draft_len, "draft_len"), (seeds, "seeds"), (accepted_len, "accepted_len"),
-                        (next_token, "next_token")):
+                        (next_token, "next_token"), (vocab_mask, "vocab_mask")):
             if t is not None and (t.is_cuda or not t.is_contiguous()):
                 raise TypeError(f"{name}: expected a contiguous CPU tensor")
         _check(LIB.flexspec_verify_host(self._h, C.byref(kv), _ptr(hidden), _ptr(draft_tokens),
                                         _ptr(draft_logits), _ptr(draft_len), _ptr(seeds), batch,
-                                        float(temperature), _ptr(accepted_len), _ptr(next_token),
+                                        float(temperature), _ptr(vocab_mask), _ptr(accepted_len), _ptr(next_token),
                                         _stream_ptr(stream)), "flexspec_verify_host")
         return accepted_len, next_token
 
@@ -271,6 +272,15 @@ class Verifier:
                                         _ptr(_dev(accepted_len, torch.int32, "accepted_len")), int(kv_len.numel()),
                                         _ptr(_dev(kv_len_next, torch.int32, "kv_len_next")), _stream_ptr(stream)), "flexspec_kv_rollback")
         return kv_len_next
+
+    def kv_release(self, page_table, num_pages, kv_len_prev, kv_len_next, free_list, free_count, stream=None):
+        """Push the pages past kv_len_next onto free_list (advancing free_count) and clear their table entries."""
+        _check(LIB.flexspec_kv_release(self._h, _ptr(_dev(page_table, torch.int32, "page_table")), int(page_table.shape[1]),
+                                       int(num_pages), _ptr(_dev(kv_len_prev, torch.int32, "kv_len_prev")),
+                                       _ptr(_dev(kv_len_next, torch.int32, "kv_len_next")), int(kv_len_prev.numel()),
+                                       _ptr(_dev(free_list, torch.int32, "free_list")), int(free_list.numel()),
+                                       _ptr(_dev(free_count, torch.int32, "free_count")), _stream_ptr(stream)),
+               "flexspec_kv_release")
 
     # ------------------------------------------------------------------ introspection
     def _view(self, ptr, shape, dtype):

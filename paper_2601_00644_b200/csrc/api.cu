@@ -474,7 +474,8 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     if (rc == FLEXSPEC_OK) {
         // staging for flexspec_verify_host: hidden | draft logits | tokens | lengths (2) | seeds
         h.stage_bytes = static_cast<size_t>(max_m) * d_model * 2 + static_cast<size_t>(h.max_s) * c.vocab * 4 +
-                        static_cast<size_t>(h.max_s) * 4 + static_cast<size_t>(c.max_batch) * (4 + 4 + 8) + 4096;
+                        static_cast<size_t>(h.max_s) * 4 + static_cast<size_t>(c.max_batch) * (4 + 4 + 8) +
+                        static_cast<size_t>(c.max_batch) * ((c.vocab + 31) / 32) * 4 + 4096;
         if (cudaMalloc(&h.stage_dev, h.stage_bytes) != cudaSuccess) { cudaGetLastError(); rc = FLEXSPEC_ERR_OOM; }
     }
     if (rc == FLEXSPEC_OK) {
@@ -645,7 +646,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
 
 int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
                          const int32_t* draft_tokens, const float* draft_logits, const int32_t* draft_len,
-                         const uint64_t* seeds, int32_t batch, float temperature,
+                         const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
                          int32_t* accepted_len, int32_t* next_token, void* stream)
 {
     if (fh == nullptr || hidden == nullptr || draft_len == nullptr || accepted_len == nullptr ||
@@ -670,6 +671,8 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     int32_t* d_len = reinterpret_cast<int32_t*>(carve(static_cast<size_t>(batch) * 4));
     int32_t* d_kvl = reinterpret_cast<int32_t*>(carve(static_cast<size_t>(batch) * 4));
     uint64_t* d_seed = reinterpret_cast<uint64_t*>(carve(static_cast<size_t>(batch) * 8));
+    const size_t mask_bytes = vocab_mask != nullptr ? static_cast<size_t>(batch) * ((h.cfg.vocab + 31) / 32) * 4 : 0;
+    uint32_t* d_mask = reinterpret_cast<uint32_t*>(carve(mask_bytes));
     if (off > h.stage_bytes) return FLEXSPEC_ERR_INVALID_ARG;
 
     bool ok = true;
@@ -684,6 +687,7 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     H2D(d_len, draft_len, static_cast<size_t>(batch) * 4);
     H2D(d_kvl, kv->kv_len_host, static_cast<size_t>(batch) * 4);
     H2D(d_seed, seeds, static_cast<size_t>(batch) * 8);
+    H2D(d_mask, vocab_mask, mask_bytes);
     if (!ok) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
     if (draft_logits != nullptr && g.s_rows > 0) {
         if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess ||
@@ -697,7 +701,8 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     flexspec_kv kv_dev = *kv;
     kv_dev.kv_len = d_kvl;
     rc = flexspec_verify(fh, &kv_dev, d_hidden, d_tok, draft_logits ? d_dlog : nullptr, d_len, draft_len,
-                         seeds ? d_seed : nullptr, batch, temperature, nullptr, h.out_dev, h.out_dev + batch, s);
+                         seeds ? d_seed : nullptr, batch, temperature, vocab_mask ? d_mask : nullptr, h.out_dev,
+                         h.out_dev + batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     ok = cudaMemcpyAsync(accepted_len, h.out_dev, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(next_token, h.out_dev + batch, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
@@ -743,6 +748,24 @@ int flexspec_kv_rollback(flexspec_handle* fh, const int32_t* kv_len, const int32
     if (batch < 1 || batch > h.cfg.max_batch) return FLEXSPEC_ERR_INVALID_ARG;
     DeviceGuard guard(h.cfg.device);
     if (launch_kv_rollback(kv_len, draft_len, accepted_len, batch, kv_len_next, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return FLEXSPEC_ERR_CUDA;
+    h.launches = 1;
+    return FLEXSPEC_OK;
+}
+
+int flexspec_kv_release(flexspec_handle* fh, int32_t* page_table, int32_t max_pages_per_seq, int32_t num_pages,
+                        const int32_t* kv_len_prev, const int32_t* kv_len_next, int32_t batch, int32_t* free_list,
+                        int32_t free_capacity, int32_t* free_count, void* stream)
+{
+    if (fh == nullptr || page_table == nullptr || kv_len_prev == nullptr || kv_len_next == nullptr || free_list == nullptr ||
+        free_count == nullptr)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    Handle& h = fh->h;
+    if (batch < 1 || batch > h.cfg.max_batch || max_pages_per_seq < 1 || num_pages < 1 || free_capacity < 0)
+        return FLEXSPEC_ERR_INVALID_ARG;
+    DeviceGuard guard(h.cfg.device);
+    if (launch_kv_release(page_table, max_pages_per_seq, kv_len_prev, kv_len_next, batch, num_pages, free_list, free_capacity,
+                          free_count, h.status, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return FLEXSPEC_ERR_CUDA;
     h.launches = 1;
     return FLEXSPEC_OK;

@@ -199,6 +199,9 @@ inline cudaError_t launch_kernel_ex(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 cudaError_t launch_kv_append(const KvAppendParams& p, int32_t m_rows, cudaStream_t stream);
 cudaError_t launch_kv_rollback(const int32_t* kv_len, const int32_t* draft_len, const int32_t* accepted_len, int32_t batch,
                                int32_t* kv_len_next, cudaStream_t stream);
+cudaError_t launch_kv_release(int32_t* page_table, int32_t max_pages_per_seq, const int32_t* kv_len_prev,
+                              const int32_t* kv_len_next, int32_t batch, int32_t num_pages, int32_t* free_list,
+                              int32_t free_capacity, int32_t* free_count, int32_t* status, cudaStream_t stream);
 cudaError_t launch_wait_timeout(int32_t* status, uint64_t limit_ns, cudaStream_t stream);
 cudaError_t attention_init(int head_dim);   // opt-in shared memory sizes
 int attention_p_bufs(int n_pad);

@@ -55,6 +55,44 @@ __global__ void kv_rollback_kernel(const int32_t* __restrict__ kv_len, const int
     if (b < batch) kv_len_next[b] = kv_len[b] - (draft_len[b] + 1) + accepted_len[b] + 1;
 }
 
+// Page release after a rollback (Section IV-C: the invalid KV pairs are discarded).  One warp per
+// sequence: the page-table entries that hold no valid token any more -- indices
+// ceil(kv_len_next / 16) .. ceil(kv_len_prev / 16) - 1 -- are pushed onto a free list (one atomic
+// reservation per sequence, so a sequence's pages stay together and in order) and set to -1.
+__global__ void kv_release_kernel(int32_t* __restrict__ page_table, int32_t max_pages_per_seq,
+                                  const int32_t* __restrict__ kv_len_prev, const int32_t* __restrict__ kv_len_next,
+                                  int32_t batch, int32_t num_pages, int32_t* __restrict__ free_list, int32_t free_capacity,
+                                  int32_t* __restrict__ free_count, int32_t* status)
+{
+    const int b = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (b >= batch) return;
+    const int had = min((max(kv_len_prev[b], 0) + 15) / 16, max_pages_per_seq);
+    const int keep = min((max(kv_len_next[b], 0) + 15) / 16, had);
+    const int n = had - keep;
+    if (n <= 0) return;
+    int base = 0;
+    if (lane == 0) base = atomicAdd(free_count, n);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    for (int i = lane; i < n; i += 32) {
+        int32_t* e = page_table + static_cast<int64_t>(b) * max_pages_per_seq + keep + i;
+        const int phys = *e;
+        if (phys < 0 || phys >= num_pages) report_error(status, kErrBadPage, phys, 9);
+        if (base + i < free_capacity) free_list[base + i] = phys;
+        else report_error(status, kErrInvalidArg, base + i, 9);          // the caller's list is too short
+        *e = -1;
+    }
+}
+cudaError_t launch_kv_release(int32_t* page_table, int32_t max_pages_per_seq, const int32_t* kv_len_prev,
+                              const int32_t* kv_len_next, int32_t batch, int32_t num_pages, int32_t* free_list,
+                              int32_t free_capacity, int32_t* free_count, int32_t* status, cudaStream_t stream)
+{
+    const int threads = 128;
+    kv_release_kernel<<<(batch * 32 + threads - 1) / threads, threads, 0, stream>>>(
+        page_table, max_pages_per_seq, kv_len_prev, kv_len_next, batch, num_pages, free_list, free_capacity, free_count, status);
+    return cudaGetLastError();
+}
+
 // Diagnostic: one thread waits on a barrier on which nobody ever arrives, with the bounded wait every
 // pipeline of the library uses; the wait runs out after limit_ns, the timeout lands in the status
 // word and the kernel returns normally.

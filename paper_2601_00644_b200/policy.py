@@ -103,3 +103,66 @@ def draft_len_trace(rates_per_user: Sequence[Sequence[float]], lat: LatencyModel
     """Ragged draft lengths of a verification batch over time: [steps][users]."""
     cols = [simulate(r, lat, g, k_max=k_max, seed=i, **kw)["k"] for i, (r, g) in enumerate(zip(rates_per_user, gammas))]
     return np.stack(cols, axis=1)
+
+
+# ------------------------------------------------------------------ link traces and the ETGR table
+
+#: stylised uplinks (bit/s): median rate, log-normal spread, probability and depth of a fade per step.
+#: They stand in for the 5G / 4G / WiFi conditions of the paper's evaluation (Section V), whose traces are not public.
+LINKS = {
+    "5g": dict(median=50e6, sigma=0.35, fade_prob=0.02, fade_factor=0.05),
+    "4g": dict(median=8e6, sigma=0.50, fade_prob=0.05, fade_factor=0.03),
+    "wifi": dict(median=1.5e6, sigma=0.80, fade_prob=0.15, fade_factor=0.02),
+}
+
+
+def link_rate_trace(kind: str, steps: int, seed: int = 0) -> np.ndarray:
+    """A seeded trace of uplink rates R_n (bit/s): an AR(1) log-normal around the link's median with
+    occasional deep fades (the weak-signal regime in which the paper's policy shortens or lengthens K)."""
+    cfg = LINKS[kind]
+    rng = np.random.RandomState(seed)
+    x = np.zeros(steps)
+    for n in range(1, steps):
+        x[n] = 0.8 * x[n - 1] + rng.standard_normal() * cfg["sigma"] * 0.6
+    rate = cfg["median"] * np.exp(x)
+    fades = rng.random_sample(steps) < cfg["fade_prob"]
+    rate[fades] *= cfg["fade_factor"]
+    return rate
+
+
+def default_latency_model(t_base_s: float = 232e-6, delta_cloud_s: float = 8.4e-6) -> LatencyModel:
+    """Edge and link constants of the order the paper reports (Table V: 8.5 .. 12 ms per drafted token on
+    a phone- or Jetson-class device; end-to-end latencies of a few hundred ms, so tens of ms each way),
+    with the cloud constants measured by this library."""
+    return LatencyModel(alpha_edge=8.5e-3, beta_edge=2e-3, t_prop=40e-3, bits_per_token=17.0, header_bits=400.0,
+                        t_base=t_base_s, delta_cloud=delta_cloud_s, t_down=40e-3)
+
+
+def etgr_table(lat: LatencyModel, gamma: float = 0.7, steps: int = 400, k_max: int = 12,
+               fixed=(1, 3, 5, 7), seed: int = 0):
+    """Effective token generation rate (Eq. 2: tokens committed per second of wall time) of the adaptive
+    stride against fixed strides, per link kind -- the comparison of the paper's stride ablation."""
+    out = {}
+    for i, kind in enumerate(LINKS):
+        rates = link_rate_trace(kind, steps, seed + i)
+        row = {"adaptive": simulate(rates, lat, gamma, k_max=k_max, seed=seed)["etgr"]}
+        row["mean_k_adaptive"] = float(simulate(rates, lat, gamma, k_max=k_max, seed=seed)["k"].mean())
+        for k in fixed:
+            row[f"fixed_{k}"] = simulate(rates, lat, gamma, k_max=k_max, fixed_k=k, seed=seed)["etgr"]
+        out[kind] = row
+    return out
+
+
+def batch_draft_lengths(batch: int, lat: LatencyModel, k_max: int = 12, seed: int = 0, warm_steps: int = 30):
+    """Draft lengths of one verification batch as the policy produces them: user b sits on a 5G, 4G or
+    WiFi-like link (round-robin), has its own true acceptance rate in 0.4 .. 0.9, and has run the policy
+    for warm_steps steps (so its EMA has left the prior); the stride it picks at the next step is its k_b."""
+    kinds = list(LINKS)
+    rng = np.random.RandomState(seed)
+    ks = np.zeros(batch, np.int32)
+    gammas = rng.uniform(0.4, 0.9, batch)
+    for b in range(batch):
+        rates = link_rate_trace(kinds[b % len(kinds)], warm_steps + 1, seed * 1000 + b)
+        sim = simulate(rates[:warm_steps], lat, float(gammas[b]), k_max=k_max, seed=seed * 1000 + b)
+        ks[b] = optimal_stride(float(rates[warm_steps]), sim["gamma_hat"], lat, k_max)
+    return ks, gammas

@@ -68,6 +68,17 @@ CONFIGS: Dict[str, VerifyShape] = {
     "llama3_70b": _shape("llama3_70b", 3, batch=32, n_q_heads=64, n_kv_heads=8, head_dim=128,
                          vocab=128256, k_min=8, k_max=8, ctx_min=8192, ctx_max=8192,
                          sigma_min=0.77, sigma_max=0.77),
+    # the paper's own targets (Section V: Llama-2-70B is the main model; Table VI adds Mixtral 8x7B): smaller
+    # vocabulary, so attention weighs more against the LM head than at the Llama-3 shapes
+    "llama2_70b": _shape("llama2_70b", 5, batch=16, n_q_heads=64, n_kv_heads=8, head_dim=128, vocab=32000,
+                         k_min=5, k_max=5, ctx_min=2048, ctx_max=2048, sigma_min=0.77, sigma_max=0.77),
+    "mixtral_8x7b": _shape("mixtral_8x7b", 6, batch=16, n_q_heads=32, n_kv_heads=8, head_dim=128, vocab=32000,
+                           k_min=5, k_max=5, ctx_min=2048, ctx_max=2048, sigma_min=0.77, sigma_max=0.77),
+    # the ragged batch with its draft lengths chosen by the paper's channel-aware policy (Section IV-B)
+    # instead of uniformly: users on 5G / 4G / WiFi-like links, each with its own acceptance history
+    "adaptive_k_policy": _shape("adaptive_k_policy", 7, batch=64, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                                vocab=128256, k_min=1, k_max=12, ctx_min=512, ctx_max=4096,
+                                sigma_min=0.2, sigma_max=1.5, notes="k from policy"),
     "long_ctx": _shape("long_ctx", 4, batch=8, n_q_heads=32, n_kv_heads=8, head_dim=128,
                        vocab=128256, k_min=16, k_max=16, ctx_min=32768, ctx_max=32768,
                        sigma_min=0.77 * 0.7, sigma_max=0.77 * 0.7, temperature=0.7),
@@ -145,6 +156,10 @@ def make_inputs(shape: VerifyShape, device: str = "cpu", spare_pages: int = 3,
 
     b = shape.batch
     k = host_rng.randint(shape.k_min, shape.k_max + 1, size=b).astype(np.int32)
+    if shape.notes == "k from policy":
+        from . import policy
+        k, _ = policy.batch_draft_lengths(b, policy.default_latency_model(), k_max=shape.k_max, seed=seed & 0xFFFF)
+        k = np.clip(k, shape.k_min, shape.k_max).astype(np.int32)
     ctx = host_rng.randint(shape.ctx_min, shape.ctx_max + 1, size=b).astype(np.int32)
     sigma = host_rng.uniform(shape.sigma_min, shape.sigma_max, size=b).astype(np.float32)
     kv_len = (ctx + k + 1).astype(np.int32)

@@ -39,6 +39,10 @@ def test_tiny_config():
     ("adaptive_k", [1, 20, 41, 63]),
     ("llama3_70b", [3, 30]),
     ("long_ctx", [2, 6]),
+    # the paper's own targets (smaller vocabulary, attention weighs more) and the policy-driven ragged batch
+    ("llama2_70b", [1, 14]),
+    ("mixtral_8x7b", [0, 9]),
+    ("adaptive_k_policy", [5, 33, 60]),
 ])
 def test_full_config_subset_parity_and_properties(name, check):
     shape = wl.CONFIGS[name]

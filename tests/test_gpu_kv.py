@@ -44,3 +44,50 @@ def test_kv_append_and_rollback_match_oracle(kw):
     nxt = ver.kv_rollback(inp.kv_len, inp.draft_len, torch.from_numpy(acc).cuda())
     assert np.array_equal(nxt.cpu().numpy(), oracle.kv_rollback(kv_host.numpy(), k_host.numpy(), acc))
     ver.close()
+
+
+def test_kv_release_matches_oracle():
+    """Pages past the rolled-back length go to the free list and leave the table: the same set per
+    sequence, in the same order, as the oracle's (the order of the sequences in the list is free)."""
+    import oracle
+    from paper_2601_00644_b200 import binding as B
+    rng = np.random.RandomState(77)
+    batch, max_pages, num_pages = 37, 40, 2000
+    prev = rng.randint(1, max_pages * 16 + 1, batch).astype(np.int32)
+    nxt = np.array([rng.randint(1, p + 1) for p in prev], np.int32)
+    nxt[3] = prev[3]                                       # nothing rejected
+    ids = rng.permutation(num_pages).astype(np.int32)
+    pt = np.full((batch, max_pages), -1, np.int32)
+    c = 0
+    for b in range(batch):
+        n = -(-int(prev[b]) // 16)
+        pt[b, :n] = ids[c:c + n]; c += n
+    want_pt, want_free = oracle.kv_release(pt, prev, nxt)
+    w = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=batch, k_max=1, max_kv_len=max_pages * 16)
+    pt_d = torch.from_numpy(pt).cuda()
+    free = torch.full((num_pages,), -7, dtype=torch.int32, device="cuda")
+    count = torch.tensor([5], dtype=torch.int32, device="cuda")            # the list already holds five entries
+    ver.kv_release(pt_d, num_pages, torch.from_numpy(prev).cuda(), torch.from_numpy(nxt).cuda(), free, count)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    assert np.array_equal(pt_d.cpu().numpy(), want_pt)
+    n_free = int(count.item()) - 5
+    assert n_free == len(want_free)
+    got = free.cpu().numpy()
+    assert np.all(got[:5] == -7) and np.all(got[5 + n_free:] == -7)
+    assert sorted(got[5:5 + n_free].tolist()) == sorted(want_free.tolist())
+    # a sequence's pages are contiguous in the list and in ascending entry order
+    pos = {int(p): i for i, p in enumerate(got[5:5 + n_free])}
+    for b in range(batch):
+        keep, had = -(-int(nxt[b]) // 16), -(-int(prev[b]) // 16)
+        idx = [pos[int(p)] for p in pt[b, keep:had]]
+        assert idx == list(range(idx[0], idx[0] + len(idx))) if idx else True
+    # a list that is too short is reported, nothing is written past it
+    pt_d = torch.from_numpy(pt).cuda()
+    small = torch.full((3,), -7, dtype=torch.int32, device="cuda")
+    count.zero_()
+    ver.kv_release(pt_d, num_pages, torch.from_numpy(prev).cuda(), torch.from_numpy(nxt).cuda(), small, count)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == B.ERR_INVALID_ARG
+    ver.close()

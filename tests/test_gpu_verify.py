@@ -217,4 +217,14 @@ def test_verify_host_entry_matches_device_entry():
                     pin(case.draft_logits), pin(inp.draft_len), pin(inp.seeds), acc_h, nxt_h,
                     temperature=shape.temperature)
     assert np.array_equal(acc_h.numpy(), acc) and np.array_equal(nxt_h.numpy(), nxt)
+    # with a vocabulary mask (host memory as well): the same as the device entry with the mask on the device
+    words = (shape.vocab + 31) // 32
+    mask = np.full((case.batch, words), 0xFFFFFFFF, np.uint32)
+    mask[1] = 0x55555555
+    mask_t = torch.from_numpy(mask.view(np.int32))
+    acc_m, nxt_m = H.run_gpu_verify(case, ver, vocab_mask_dev=mask_t.cuda())
+    ver.verify_host(inp.kv_pages, inp.page_table, inp.kv_len.cpu(), pin(inp.hidden), pin(case.draft_tokens),
+                    pin(case.draft_logits), pin(inp.draft_len), pin(inp.seeds), acc_h, nxt_h,
+                    temperature=shape.temperature, vocab_mask=mask_t.pin_memory())
+    assert np.array_equal(acc_h.numpy(), acc_m) and np.array_equal(nxt_h.numpy(), nxt_m) and nxt_m[1] % 2 == 0
     ver.close()

@@ -59,3 +59,32 @@ def test_ema_update_and_simulation_bookkeeping():
     assert slow["etgr"] >= fixed["etgr"] * 0.999
     trace = P.draft_len_trace([rates[:50], np.full(50, 2e3)], LAT, [0.7, 0.5], k_max=12)
     assert trace.shape == (50, 2) and trace.min() >= 1 and trace.max() <= 12
+
+
+def test_link_traces_and_etgr_table():
+    """The three stylised links are seeded and ordered (5G fastest), and on each of them the adaptive
+    stride beats the shortest and the longest fixed stride and stays within a few percent of the best one
+    (its acceptance estimate, the EMA of tau / K of Algorithm 2, sits below the per-token rate the
+    geometric model wants, so it drafts a little short)."""
+    from paper_2601_00644_b200 import policy as P
+    r5, r4, rw = (P.link_rate_trace(k, 500, seed=3) for k in ("5g", "4g", "wifi"))
+    assert np.array_equal(r5, P.link_rate_trace("5g", 500, seed=3))
+    assert np.median(r5) > np.median(r4) > np.median(rw) > 0
+    tab = P.etgr_table(P.default_latency_model(), gamma=0.7, steps=600)
+    for kind, row in tab.items():
+        best_fixed = max(v for k, v in row.items() if k.startswith("fixed_"))
+        assert row["adaptive"] >= 0.93 * best_fixed, (kind, row)
+        assert row["adaptive"] > row["fixed_1"] and row["adaptive"] > row["fixed_7"], (kind, row)
+        assert 1.0 <= row["mean_k_adaptive"] <= 12.0
+
+
+def test_policy_driven_batch_is_ragged_and_seeded():
+    from paper_2601_00644_b200 import policy as P, workloads as wl
+    ks, gammas = P.batch_draft_lengths(64, P.default_latency_model(), k_max=12, seed=5)
+    assert ks.min() >= 1 and ks.max() <= 12 and len(set(ks.tolist())) >= 3
+    # users with a better acceptance history draft longer strides on average
+    assert ks[gammas > 0.75].mean() > ks[gammas < 0.55].mean()
+    shape = wl.scaled(wl.CONFIGS["adaptive_k_policy"], vocab=64, ctx_min=1, ctx_max=8, n_q_heads=2, n_kv_heads=1, head_dim=64)
+    a = wl.make_inputs(shape, with_noise=False).draft_len.numpy()
+    b = wl.make_inputs(shape, with_noise=False).draft_len.numpy()
+    assert np.array_equal(a, b) and len(set(a.tolist())) >= 3
