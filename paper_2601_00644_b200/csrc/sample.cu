@@ -424,11 +424,12 @@ cudaError_t launch_sample_filter(const SampleParams& p, cudaStream_t stream)
 //     writes the row's result into the shared memory of all eight CTAs.        -- cluster barrier --
 //   B  every CTA finds the first rejection n by warp vote over the row results (GREEDY ends here).
 //   C  row n only: the vocabulary is cut into eight contiguous slices, one per CTA, and a slice into
-//     chunks of 1024 entries, one warp each: the mass of the emission weights of each chunk is
-//     recorded, slice totals go to all CTAs.                                    -- cluster barrier --
-//   D  the CTA whose slice holds u' * Z picks the chunk from its list and one warp scans those
-//     1024 entries in vocabulary order (inverse CDF).  If rounding leaves no entry above the
-//     threshold, the last entry with positive mass is taken, at every level.
+//     chunks of 1024 entries, one warp each, streamed through shared memory in halves; the mass of
+//     the emission weights of every group of 16 entries and of every chunk is recorded, slice
+//     totals go to all CTAs.                                                    -- cluster barrier --
+//   D  the CTA whose slice holds u' * Z picks the chunk, then the group of 16, from its lists and
+//     scans those 16 entries in vocabulary order (inverse CDF).  If rounding leaves no entry above
+//     the threshold, the last entry with positive mass is taken, at every level.
 //
 // The kernel runs once per step and is short, and the step streams gigabytes through L2 in between,
 // so its instructions are fetched cold (from DRAM) every time: straight-line code was measured at
@@ -440,8 +441,8 @@ cudaError_t launch_sample_filter(const SampleParams& p, cudaStream_t stream)
 // row): w_v = max(0, e_p(v) - rho e_q(v)) at a rejection, rho = s_p / s_q, and w_v = e_p(v) for the
 // bonus row, with e = the same fp32 2^x as in the statistics.  A common factor does not move the
 // inverse CDF, so no entry is ever normalised.  Entries are fp32 (one fused multiply-add); a lane
-// adds 32 of them in fp32 and everything above that -- lanes, chunks, slices, the running sums of
-// the final scan -- is fp64.  (Double-precision arithmetic per entry was measured at 12 us for this
+// adds the 16 of a group in fp32 and everything above that -- groups, chunks, slices, the running
+// sums of the final scan -- is fp64.  (Double-precision arithmetic per entry was measured at 12 us for this
 // phase alone: the vector fp64 rate of this GPU is a small fraction of its fp32 rate.)
 constexpr int kAcceptThreads = 256;        // two CTAs per SM: every cluster of a 16-sequence batch finds room at once
 constexpr int kAcceptWarps = kAcceptThreads / 32;
@@ -475,23 +476,32 @@ struct DrawRow {
         return use_p ? ep : fmaxf(fmaf(-rho, e_q(zd_v), ep), 0.f);
     }
 };
-// A chunk of kWarpChunk entries of a logits row in shared memory.  Entry i sits at chunk_pos(i): inside
-// its group of 32 the four-entry (16-byte) pieces are permuted by the group index, so that 16-byte
-// copies stay whole, the lane-interleaved walk (lane l takes entry 32 g + l) is conflict-free and
-// the lane-contiguous one (lane l takes entry 32 l + e) meets at most four lanes per bank.
-__device__ __forceinline__ int chunk_pos(int i) { return i ^ (((i >> 5) & 7) << 2); }
-// One warp requests the entries [base, base + kWarpChunk) of a row (those below vocab); nothing is
+// Streaming of row n through shared memory.  A chunk (kWarpChunk = 1024 entries) is two sub-chunks of
+// 512; a sub-chunk is 32 groups of 16 consecutive entries, group g being added up by lane g.  Inside a
+// group the four 16-byte pieces are permuted by (g >> 1) & 3, so that the lanes' 16-byte reads of
+// their own groups (64 bytes apart) fall into different banks.
+constexpr int kSubChunk = 512;
+constexpr int kGroup = 16;
+constexpr int kGroupsPerChunk = kWarpChunk / kGroup;                    // 64
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_group_1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+// One warp requests the entries [base, base + kSubChunk) of a row (those below vocab); nothing is
 // awaited.  vec_ok: the row starts on a 16-byte boundary and vocab is a multiple of four.
-__device__ __forceinline__ void stage_chunk(float* dst, const float* row, int base, int vocab, bool vec_ok, int lane)
+__device__ __forceinline__ void stage_sub(float* dst, const float* row, int base, int vocab, bool vec_ok, int lane)
 {
     if (vec_ok) {
-#pragma unroll 4
-        for (int i = lane * 4; i < kWarpChunk; i += 128)
-            if (base + i < vocab) cp_async_16(dst + chunk_pos(i), row + base + i);
+#pragma unroll
+        for (int it = 0; it < kSubChunk / 128; ++it) {
+            const int q = it * 32 + lane;                               // 16-byte piece of the sub-chunk
+            const int g = q >> 2, j = q & 3;
+            if (base + 4 * q < vocab) cp_async_16(dst + g * kGroup + ((j ^ ((g >> 1) & 3)) << 2), row + base + 4 * q);
+        }
     } else {
 #pragma unroll 4
-        for (int i = lane; i < kWarpChunk; i += 32)
-            if (base + i < vocab) cp_async_4(dst + chunk_pos(i), row + base + i);
+        for (int e = lane; e < kSubChunk; e += 32) {
+            const int g = e >> 4, j = (e >> 2) & 3;
+            if (base + e < vocab) cp_async_4(dst + g * kGroup + ((j ^ ((g >> 1) & 3)) << 2) + (e & 3), row + base + e);
+        }
     }
 }
 
@@ -704,7 +714,7 @@ sample_accept_kernel(const SampleParams p)
     const int n = s_n;
 
     // ---- C: masses of row n over this CTA's slice of the vocabulary
-    extern __shared__ float s_chunks[];                    // [warps][2][kWarpChunk]: target and draft entries of a warp's chunk
+    extern __shared__ float s_dyn[];                       // [warps][2 buffers][target | draft][kSubChunk], then the group masses
     DrawRow row;
     row.zt = p.logits + static_cast<int64_t>(q0 + n) * p.vocab;
     row.residual = (n < k_b);
@@ -721,29 +731,60 @@ sample_accept_kernel(const SampleParams p)
     const int wc_per_cta = (wc_total + kAcceptCluster - 1) / kAcceptCluster;     // <= kMaxWarpChunksPerCta (vocab <= kMaxVocab)
     const int wc_begin = min(wc_total, rank * wc_per_cta);
     const int n_wc = min(wc_total, wc_begin + wc_per_cta) - wc_begin;
-    float* my_zt = s_chunks + warp * 2 * kWarpChunk;
-    float* my_zd = my_zt + kWarpChunk;
+    float* my_buf = s_dyn + warp * (4 * kSubChunk);        // two buffers of (target, draft) sub-chunks
+    float2* s_grp = reinterpret_cast<float2*>(s_dyn + kAcceptWarps * 4 * kSubChunk);   // [n_wc][kGroupsPerChunk] (residual, p) masses
+    {
+        // A warp streams its chunks (warp, warp + 8, ...) as sub-chunks of 512 entries through two small
+        // buffers: the copy of sub-chunk s + 2 is requested as soon as s has been added up, so transfer
+        // and arithmetic overlap.  Lane l adds the 16 consecutive entries [16 l, 16 l + 16) of a sub-chunk
+        // (a "group"): its sum is the group's mass, the warp's sum the chunk's.
+        const int n_sub = 2 * ((n_wc - warp + kAcceptWarps - 1) / kAcceptWarps);      // of this warp (0 if it has no chunk)
+        auto sub_base = [&](int sidx) { return (wc_begin + warp + kAcceptWarps * (sidx >> 1)) * kWarpChunk + (sidx & 1) * kSubChunk; };
+        auto issue = [&](int sidx) {
+            float* dst = my_buf + (sidx & 1) * (2 * kSubChunk);
+            stage_sub(dst, row.zt, sub_base(sidx), p.vocab, vec_ok, lane);
+            if (row.residual) stage_sub(dst + kSubChunk, row.zd, sub_base(sidx), p.vocab, vec_ok, lane);
+            cp_async_commit();
+        };
+        if (n_sub > 0) { issue(0); issue(1); }
+        double cr = 0.0, cp = 0.0;
 #pragma unroll 1
-    for (int i = warp; i < n_wc; i += kAcceptWarps) {
-        const int base = (wc_begin + i) * kWarpChunk;
-        __syncwarp();                                      // the previous chunk of this warp has been read
-        stage_chunk(my_zt, row.zt, base, p.vocab, vec_ok, lane);
-        if (row.residual) stage_chunk(my_zd, row.zd, base, p.vocab, vec_ok, lane);
-        cp_async_wait_all();
-        __syncwarp();
-        float mr = 0.f, mp = 0.f;
-#pragma unroll 4
-        for (int e = lane; e < kWarpChunk; e += 32) {
-            const int v = base + e;
-            if (v < p.vocab) {
-                const float ep = row.e_p(my_zt[chunk_pos(e)], v);
-                mp += ep;
-                if (row.residual) mr += fmaxf(fmaf(-row.rho, row.e_q(my_zd[chunk_pos(e)]), ep), 0.f);
+        for (int sidx = 0; sidx < n_sub; ++sidx) {
+            if (sidx + 1 < n_sub) cp_async_wait_group_1(); else cp_async_wait_all();
+            __syncwarp();
+            const float* zt_s = my_buf + (sidx & 1) * (2 * kSubChunk);
+            const float* zd_s = zt_s + kSubChunk;
+            const int v0 = sub_base(sidx) + lane * kGroup;
+            float mr = 0.f, mp = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int pos = lane * kGroup + ((j ^ ((lane >> 1) & 3)) << 2);
+                const float4 a = *reinterpret_cast<const float4*>(zt_s + pos);
+                float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row.residual) d = *reinterpret_cast<const float4*>(zd_s + pos);
+                const float za[4] = {a.x, a.y, a.z, a.w}, zq[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int v = v0 + 4 * j + e;
+                    if (v < p.vocab) {
+                        const float ep = row.e_p(za[e], v);
+                        mp += ep;
+                        if (row.residual) mr += fmaxf(fmaf(-row.rho, row.e_q(zq[e]), ep), 0.f);
+                    }
+                }
+            }
+            const int chunk = warp + kAcceptWarps * (sidx >> 1);
+            s_grp[chunk * kGroupsPerChunk + (sidx & 1) * 32 + lane] = make_float2(mr, mp);
+            cr += static_cast<double>(mr);
+            cp += static_cast<double>(mp);
+            __syncwarp();                                  // everyone has read the buffer
+            if (sidx + 2 < n_sub) issue(sidx + 2);
+            if (sidx & 1) {                                // the chunk is complete
+                const double dr = warp_sum(cr), dp = warp_sum(cp);
+                if (lane == 0) s_wc[chunk] = make_double2(dr, dp);
+                cr = 0.0; cp = 0.0;
             }
         }
-        const double dr = warp_sum(static_cast<double>(mr));
-        const double dp = warp_sum(static_cast<double>(mp));
-        if (lane == 0) s_wc[i] = make_double2(dr, dp);
     }
     __syncthreads();
     if (warp == 0) {
@@ -760,7 +801,7 @@ sample_accept_kernel(const SampleParams p)
     cluster_sync();                                        // slice totals are everywhere; no remote access after this
     if (warp != 0) return;
 
-    // ---- D: which slice holds u' * Z, which chunk of it, which entry
+    // ---- D: which slice holds u' * Z, which chunk of it, which group of 16, which entry
     double z_r = 0.0, z_p = 0.0;
 #pragma unroll
     for (int c = 0; c < kAcceptCluster; ++c) { z_r += s_slice[c][0]; z_p += s_slice[c][1]; }
@@ -789,48 +830,35 @@ sample_accept_kernel(const SampleParams p)
     }
     if (slice != rank) return;
     const int wc = max(0, warp_pick(n_wc, before, thr, lane, [&](int i) { return use_p ? s_wc[i].y : s_wc[i].x; }, before));
-    const int base = (wc_begin + wc) * kWarpChunk;
-    // the chunk's entries: still in the shared memory of the warp that added them up, unless that warp
-    // went on to a later chunk (vocabularies beyond 16 chunks per slice): then they are fetched again
-    const float* c_zt = s_chunks + (wc % kAcceptWarps) * 2 * kWarpChunk;
-    if (wc + kAcceptWarps < n_wc) {
-        stage_chunk(my_zt, row.zt, base, p.vocab, vec_ok, lane);
-        if (row.residual) stage_chunk(my_zd, row.zd, base, p.vocab, vec_ok, lane);
-        cp_async_wait_all();
-        __syncwarp();
-        c_zt = my_zt;
-    }
-    const float* c_zd = c_zt + kWarpChunk;
-    // lane l adds up the 32 consecutive entries [base + 32 l, base + 32 l + 32)
-    double mine = 0.0;
-#pragma unroll 4
-    for (int e = 0; e < 32; ++e) {
-        const int v = base + lane * 32 + e;
-        if (v < p.vocab)
-            mine += static_cast<double>(row.weight(c_zt[chunk_pos(lane * 32 + e)], use_p ? 0.f : c_zd[chunk_pos(lane * 32 + e)], v, use_p));
-    }
-    const double incl = before + warp_inclusive_scan(mine, lane);
-    const unsigned hit = __ballot_sync(0xffffffffu, mine > 0.0 && incl > thr);
-    const unsigned pos = __ballot_sync(0xffffffffu, mine > 0.0);
-    // the group of 32 that holds thr (if rounding left none: the last one with mass), scanned by the whole warp
-    const int grp = hit != 0u ? __ffs(hit) - 1 : (pos != 0u ? 31 - __clz(pos) : 0);
-    const double grp_before = __shfl_sync(0xffffffffu, incl - mine, grp);
-    const int v = base + grp * 32 + lane;
-    const float w = (v < p.vocab) ? row.weight(c_zt[chunk_pos(grp * 32 + lane)], use_p ? 0.f : c_zd[chunk_pos(grp * 32 + lane)], v, use_p) : 0.f;
-    const double run = grp_before + warp_inclusive_scan(static_cast<double>(w), lane);
-    const unsigned hit2 = __ballot_sync(0xffffffffu, w > 0.f && run > thr);
-    const unsigned pos2 = __ballot_sync(0xffffffffu, w > 0.f);
+    const float2* grp_mass = s_grp + wc * kGroupsPerChunk;
+    const int grp = max(0, warp_pick(kGroupsPerChunk, before, thr, lane, [&](int g) {
+        return static_cast<double>(use_p ? grp_mass[g].y : grp_mass[g].x); }, before));
+    // the group's 16 entries come from L2 once more (lane e takes entry e); same fp32 weights as above
+    const int v = (wc_begin + wc) * kWarpChunk + grp * kGroup + lane;
+    float w = 0.f;
+    if (lane < kGroup && v < p.vocab) w = row.weight(__ldg(row.zt + v), use_p ? 0.f : __ldg(row.zd + v), v, use_p);
+    const double run = before + warp_inclusive_scan(static_cast<double>(w), lane);
+    const unsigned hit = __ballot_sync(0xffffffffu, w > 0.f && run > thr);
+    const unsigned pos = __ballot_sync(0xffffffffu, w > 0.f);
     // if rounding left no entry above the threshold: the last entry with positive mass
-    const int pick = hit2 != 0u ? __ffs(hit2) - 1 : (pos2 != 0u ? 31 - __clz(pos2) : 0);
-    if (lane == 0) p.next_token[b] = min(base + grp * 32 + pick, p.vocab - 1);
+    const int pick = hit != 0u ? __ffs(hit) - 1 : (pos != 0u ? 31 - __clz(pos) : 0);
+    if (lane == 0) p.next_token[b] = min((wc_begin + wc) * kWarpChunk + grp * kGroup + pick, p.vocab - 1);
 }
 
-constexpr size_t kAcceptSmemBytes = static_cast<size_t>(kAcceptWarps) * 2 * kWarpChunk * sizeof(float);   // 65 536
+// dynamic shared memory of the acceptance kernel: the streaming buffers plus the group masses of the slice
+static size_t accept_smem_bytes(int vocab)
+{
+    const int wc_total = (vocab + kWarpChunk - 1) / kWarpChunk;
+    const int wc_per_cta = (wc_total + kAcceptCluster - 1) / kAcceptCluster;
+    return static_cast<size_t>(kAcceptWarps) * 4 * kSubChunk * sizeof(float) + static_cast<size_t>(wc_per_cta) * kGroupsPerChunk * sizeof(float2);
+}
+constexpr size_t kAcceptSmemMax = static_cast<size_t>(kAcceptWarps) * 4 * kSubChunk * sizeof(float) +
+                                  static_cast<size_t>(kMaxWarpChunksPerCta) * kGroupsPerChunk * sizeof(float2);   // 131 072
 
 cudaError_t sample_init()
 {
     cudaError_t e = cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kAcceptSmemBytes));
+                                         static_cast<int>(kAcceptSmemMax));
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(sample_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kFilterSliceMax * sizeof(float)));
@@ -839,8 +867,8 @@ cudaError_t sample_init()
 
 cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream)
 {
-    return launch_kernel_ex(sample_accept_kernel, dim3(kAcceptCluster, p.batch), dim3(kAcceptThreads), kAcceptSmemBytes, stream,
-                            pdl, p);
+    return launch_kernel_ex(sample_accept_kernel, dim3(kAcceptCluster, p.batch), dim3(kAcceptThreads), accept_smem_bytes(p.vocab),
+                            stream, pdl, p);
 }
 
 }  // namespace fs
