@@ -45,9 +45,8 @@ namespace fs {
 
 constexpr int kPageTokens = 16;
 constexpr int kAttPagesPerStage = kAttBlockTokens / kPageTokens;    // 8
-constexpr int kAttSoftmaxThreads = 128;
-constexpr int kAttPvWarp = kAttProducerWarps + 5;                   // warp order: TMA producers, S^T issuer, 4 softmax warps, PV issuer
-constexpr int kAttConsumerThreads = kAttThreads - kAttProducerWarps * 32;   // everyone who touches tensor memory (named barrier 1)
+// warp order: 2 TMA producers, the S^T issuer, 4 or 8 softmax warps (HALVES = 1 or 2), the PV issuer;
+// named barrier 1 joins everyone who touches tensor memory: 64 + 128 * HALVES threads
 constexpr int kAttTmemCols = 512;
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column offsets
 constexpr float kRescaleThreshold = 8.f;                             // log2 units
@@ -59,7 +58,7 @@ struct AttBars {
     uint64_t v_full[kAttMaxStages], v_empty[kAttMaxStages];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_full[2], p_empty[2];
-    uint64_t q_full, o_full, group;
+    uint64_t q_full, o_full[2], group[2];       // o_full alternates with the block parity (see the PV issuer)
     uint32_t tmem_slot;
 };
 static_assert(sizeof(AttBars) <= 512, "barrier block");
@@ -259,13 +258,19 @@ static __device__ __noinline__ int att_owner(const AttTable& tab, int n_ctas, in
 // maximum, row sum, output row) lives in lane i of every warp for column 32*ci + i and is
 // broadcast by shuffles, so the four warps only meet once per block (column maxima) and once
 // per segment (row sums).
-template <int DH, int NCH>
+template <int DH, int NCHT, int HALVES>
 __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable& tab, const AttSmem& sm, AttCursor cur, int n_my)
 {
     using Cfg = AttCfg<DH>;
+    constexpr int NCH = (NCHT + HALVES - 1) / HALVES;   // chunks of 32 columns this thread may own
+    constexpr int kSoftmaxThreads = 128 * HALVES;
     AttBars* bars = sm.bars;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
+    // HALVES == 2: two warps share every quarter (the same 32 tokens) and split the columns (query rows)
+    // chunk-wise: warp half h owns chunks h, h + 2.  Column state, exchanges and barriers of the two halves
+    // are separate; they only meet in the hand-overs to the MMA warps.
+    const int half = HALVES == 2 ? ((warp - (kAttProducerWarps + 1)) >> 2) : 0;
     const int t = quarter * 32 + lane;                  // token of the block (S^T), Dh index (O^T)
     const int cta = blockIdx.x;
     const int n_pad = p.n_pad;
@@ -274,7 +279,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
     const bool o_lane = quarter * 32 < DH;              // warp-uniform: this warp's lanes hold rows of O^T
 
     if (n_my <= 0) {                                    // not produced by the host planner; keep the rendezvous whole
-        asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(64 + 128 * HALVES) : "memory");
         return;
     }
     bool ok = true, seg_first = true;
@@ -284,8 +289,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
     // word serialise: measured ~0.2 us per barrier and block)
     auto group_sync = [&](int where) -> bool {
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->group);
-        const bool done = att_wait(&bars->group, group_phase, p.status, where);
+        if (lane == 0) mbar_arrive(&bars->group[half]);
+        const bool done = att_wait(&bars->group[half], group_phase, p.status, where);
         group_phase ^= 1u;
         return done;
     };
@@ -302,7 +307,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             row_lo = (cur.pair % cur.rbc) * kAttRowsPerPair;
             rows_here = min(kAttRowsPerPair, p.group * (cur.k + 1) - row_lo);
             ctx = cur.kvl - (cur.k + 1);
-            for (int idx = t; idx < rows_here * (DH / 8); idx += kAttSoftmaxThreads) {
+            for (int idx = half * 128 + t; idx < rows_here * (DH / 8); idx += kSoftmaxThreads) {
                 const int row = idx / (DH / 8), ch = idx % (DH / 8);
                 const int rho = row_lo + row;
                 const int tok_row = min(cur.q_row0 + rho / p.group, p.m_rows - 1);
@@ -313,10 +318,10 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
 #pragma unroll
             for (int i = 0; i < NCH * 32; ++i) lsum[i] = 0.f;
 #pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
-                m_used[ci] = -INFINITY;
+            for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
+                m_used[cs] = -INFINITY;
                 const int rho = row_lo + ci * 32 + lane;
-                row_c[ci] = min(cur.q_row0 + rho / p.group, p.m_rows - 1) * p.n_q_heads + kvh * p.group + rho % p.group;
+                row_c[cs] = min(cur.q_row0 + rho / p.group, p.m_rows - 1) * p.n_q_heads + kvh * p.group + rho % p.group;
             }
             fence_proxy_async();
             tc_fence_before();
@@ -324,7 +329,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             if (lane == 0) mbar_arrive(&bars->q_full);
             if (q == 0) {
                 // the MMA warp allocated tensor memory meanwhile: meet it (warps 2..6) and read the base
-                asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(64 + 128 * HALVES) : "memory");
                 tc_fence_after();
                 t_lane = bars->tmem_slot + (static_cast<uint32_t>(quarter * 32) << 16);
             }
@@ -360,7 +365,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                 // ---- exact column maxima over my warp's 32 tokens, then over the four warps
                 float* xch = sm.xch + (q & 1) * 4 * n_pad;
 #pragma unroll
-                for (int ci = 0; ci < NCH; ++ci) {
+                for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
                     if (ci * 32 < n_pad) {
                         uint32_t sv[32];
                         tmem_ld_x32(t_s + ci * 32, sv);
@@ -379,29 +384,29 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                 float alpha[NCH];
                 bool rescale = false;
 #pragma unroll
-                for (int ci = 0; ci < NCH; ++ci) {
-                    alpha[ci] = 1.f;
+                for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
+                    alpha[cs] = 1.f;
                     const int col = ci * 32 + lane;
                     if (col < n_pad) {
                         const float mx = fmaxf(fmaxf(xch[col], xch[n_pad + col]), fmaxf(xch[2 * n_pad + col], xch[3 * n_pad + col])) *
                                          p.scale_log2;       // scale > 0: the maximum commutes
                         // ---- raise the running maximum only if it grew by more than the threshold
                         if (seg_first) {
-                            m_used[ci] = mx;
-                        } else if (mx > m_used[ci] + kRescaleThreshold) {
-                            alpha[ci] = fast_exp2(m_used[ci] - mx);            // m_used == -inf gives 0
-                            m_used[ci] = mx;
+                            m_used[cs] = mx;
+                        } else if (mx > m_used[cs] + kRescaleThreshold) {
+                            alpha[cs] = fast_exp2(m_used[cs] - mx);            // m_used == -inf gives 0
+                            m_used[cs] = mx;
                             rescale = true;
                         }
-                        if (quarter == 0) sm.m_col[col] = m_used[ci];
+                        if (quarter == 0) sm.m_col[col] = m_used[cs];
                     }
                 }
                 if (!seg_first && __any_sync(0xffffffffu, rescale)) {
                     // O^T += V^T P^T of the previous block must have landed before O^T is rescaled
-                    if (!att_wait(&bars->o_full, (q - 1) & 1, p.status, 7)) { ok = false; break; }
+                    if (!att_wait(&bars->o_full[(q - 1) & 1], ((q - 1) >> 1) & 1, p.status, 7)) { ok = false; break; }
                     tc_fence_after();
 #pragma unroll
-                    for (int ci = 0; ci < NCH; ++ci) {
+                    for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
                         if (ci * 32 < n_pad) {
                             uint32_t o[32];
                             if (o_lane) {
@@ -410,8 +415,8 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                             }
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
-                                const float a = __shfl_sync(0xffffffffu, alpha[ci], i);
-                                lsum[ci * 32 + i] *= a;
+                                const float a = __shfl_sync(0xffffffffu, alpha[cs], i);
+                                lsum[cs * 32 + i] *= a;
                                 if (o_lane) o[i] = __float_as_uint(__uint_as_float(o[i]) * a);
                             }
                             if (o_lane) tmem_st_x32(t_lane + kTmemO + ci * 32, o);
@@ -426,7 +431,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             {
                 uint8_t* p_row = sm.pt + pbuf * Cfg::p_bytes(n_pad) + t * 16;
 #pragma unroll
-                for (int ci = 0; ci < NCH; ++ci) {
+                for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
                     if (ci * 32 < n_pad) {
                         uint32_t sv[32];
                         tmem_ld_x32(t_s + ci * 32, sv);
@@ -444,7 +449,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                                 const bool masked = static_cast<uint32_t>(ci * 32 + i - col_min) >= col_span;   // also rows without a maximum yet
                                 e[j] = masked ? 0.f : fast_exp2(x);
                                 ex = fmaxf(ex, masked ? -INFINITY : x);
-                                if (add) lsum[ci * 32 + i] += e[j];
+                                if (add) lsum[cs * 32 + i] += e[j];
                             }
                             pk[2 * i4] = pack_bf16(e[0], e[1]);
                             pk[2 * i4 + 1] = pack_bf16(e[2], e[3]);
@@ -459,9 +464,9 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             }
             if (fresh) break;                            // written against maxima taken from this very block
             const bool hot = __any_sync(0xffffffffu, ex > kRescaleThreshold);
-            if (lane == 0) sm.flags[(q & 1) * 4 + quarter] = hot ? 1 : 0;
+            if (lane == 0) sm.flags[half * 8 + (q & 1) * 4 + quarter] = hot ? 1 : 0;
             if (!group_sync(14)) { ok = false; break; }
-            const int* fl = sm.flags + (q & 1) * 4;
+            const int* fl = sm.flags + half * 8 + (q & 1) * 4;
             if ((fl[0] | fl[1] | fl[2] | fl[3]) == 0) break;
             fresh = true;                                // second round: new maxima, then P^T again, the row sums
             add = false;                                 // already hold this block (they are rescaled with the rest)
@@ -473,7 +478,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             // (the tile must have landed first, or the copy would overwrite the zeros)
             if (!att_wait(&bars->v_full[q % p.v_stages], (q / p.v_stages) & 1, p.status, 22)) { ok = false; break; }
         }
-        if (t_begin + kAttBlockTokens > cur.kvl && t >= cur.kvl - t_begin) {
+        if (half == 0 && t_begin + kAttBlockTokens > cur.kvl && t >= cur.kvl - t_begin) {
             uint8_t* v_row = sm.v_ring + (q % p.v_stages) * Cfg::kTileBytes + t * 128;
 #pragma unroll
             for (int hf = 0; hf < Cfg::kSlabs; ++hf)
@@ -502,23 +507,23 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         float* xl = sm.xch + 2 * 4 * n_pad;
         float l_c[NCH];
 #pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) {
-            l_c[ci] = 0.f;
+        for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
+            l_c[cs] = 0.f;
             if (ci * 32 < n_pad) {
                 float tmp[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) tmp[i] = lsum[ci * 32 + i];
+                for (int i = 0; i < 32; ++i) tmp[i] = lsum[cs * 32 + i];
                 const float mine = warp_transpose_sum(tmp, lane);
                 if (ci * 32 + lane < n_pad) xl[quarter * n_pad + ci * 32 + lane] = mine;
             }
         }
         if (!group_sync(15)) { ok = false; break; }
 #pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) {
+        for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
             const int col = ci * 32 + lane;
-            if (col < n_pad) l_c[ci] = (xl[col] + xl[n_pad + col]) + (xl[2 * n_pad + col] + xl[3 * n_pad + col]);
+            if (col < n_pad) l_c[cs] = (xl[col] + xl[n_pad + col]) + (xl[2 * n_pad + col] + xl[3 * n_pad + col]);
         }
-        if (!att_wait(&bars->o_full, q & 1, p.status, 10)) { ok = false; break; }
+        if (!att_wait(&bars->o_full[q & 1], (q >> 1) & 1, p.status, 10)) { ok = false; break; }
         tc_fence_after();
         if (!o_lane) continue;                                         // nothing of O^T in this warp's lanes
         // does the pair reach into another CTA's range?  (this CTA holds blocks [blk_begin, blk_begin + n_my))
@@ -529,16 +534,16 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             // the whole pair was ours: normalise and store; thread t holds element t of every row
             __nv_bfloat16* out_t = p.attn_out + t;
 #pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
+            for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
                 if (ci * 32 < n_pad) {
                     uint32_t o[32];
                     tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
                     tmem_ld_wait();
-                    const float inv_l = 1.f / l_c[ci];
+                    const float inv_l = 1.f / l_c[cs];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const float il = __shfl_sync(0xffffffffu, inv_l, i);
-                        const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
+                        const int row = __shfl_sync(0xffffffffu, row_c[cs], i);
                         if (ci * 32 + i < rows_here) out_t[static_cast<int64_t>(row) * DH] = __float2bfloat16_rn(__uint_as_float(o[i]) * il);
                     }
                 }
@@ -557,7 +562,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             float* po = p.part_o + (static_cast<int64_t>(my_slot) * DH + t) * kAttRowsPerPair;
             float* pml = p.part_ml + (static_cast<int64_t>(my_slot) * 4 + quarter) * kAttRowsPerPair * 2;
 #pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
+            for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
                 if (ci * 32 < n_pad) {
                     uint32_t o[32];
                     tmem_ld_x32(t_lane + kTmemO + ci * 32, o);
@@ -569,7 +574,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                                    make_float4(__uint_as_float(o[i]), __uint_as_float(o[i + 1]),
                                                __uint_as_float(o[i + 2]), __uint_as_float(o[i + 3])));
                     if (ci * 32 + lane < n_pad)
-                        __stcg(reinterpret_cast<float2*>(pml + (ci * 32 + lane) * 2), make_float2(m_used[ci], l_c[ci]));
+                        __stcg(reinterpret_cast<float2*>(pml + (ci * 32 + lane) * 2), make_float2(m_used[cs], l_c[cs]));
                 }
             }
         }
@@ -578,7 +583,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         __syncwarp();
         int last = 0;
         if (lane == 0) {
-            int32_t* tk = p.tickets + static_cast<int64_t>(pair_global) * 4 + quarter;
+            int32_t* tk = p.tickets + (static_cast<int64_t>(pair_global) * 4 + quarter) * 2 + half;
             last = (atomicAdd(tk, 1) == c_last - c_first);
             if (last) *tk = 0;                                         // ready for the next call
         }
@@ -595,7 +600,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         // the accumulator is rescaled whenever a part raises a column's maximum
         float m_all[NCH], l_all[NCH];
 #pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) { m_all[ci] = -INFINITY; l_all[ci] = 0.f; }
+        for (int cs = 0; cs < NCH; ++cs) { m_all[cs] = -INFINITY; l_all[cs] = 0.f; }
 #pragma unroll
         for (int i = 0; i < NCH * 32; ++i) lsum[i] = 0.f;              // reused as the accumulator of my O^T row
 #pragma unroll 1
@@ -604,7 +609,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
             const float4* po = reinterpret_cast<const float4*>(p.part_o + (static_cast<int64_t>(slot) * DH + t) * kAttRowsPerPair);
             const float2* pml = reinterpret_cast<const float2*>(p.part_ml) + (static_cast<int64_t>(slot) * 4 + quarter) * kAttRowsPerPair;
 #pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) {
+            for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
                 if (ci * 32 < n_pad) {
                     float4 v[8];
 #pragma unroll
@@ -613,12 +618,12 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                     if (ci * 32 + lane < n_pad) ml = __ldcg(pml + ci * 32 + lane);
                     // my column: weight of what is accumulated so far, weight of this part (a part that saw no
                     // visible token has m = -inf, weight 0 and O^T = 0)
-                    const float mn = fmaxf(m_all[ci], ml.x);
+                    const float mn = fmaxf(m_all[cs], ml.x);
                     const float base = (mn == -INFINITY) ? 0.f : mn;
-                    const float w_old = fast_exp2(m_all[ci] - base);
+                    const float w_old = fast_exp2(m_all[cs] - base);
                     const float w_new = fast_exp2(ml.x - base);
-                    l_all[ci] = l_all[ci] * w_old + ml.y * w_new;
-                    m_all[ci] = mn;
+                    l_all[cs] = l_all[cs] * w_old + ml.y * w_new;
+                    m_all[cs] = mn;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float vv[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
@@ -626,7 +631,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
                         for (int j = 0; j < 4; ++j) {
                             const float wo = __shfl_sync(0xffffffffu, w_old, 4 * i + j);
                             const float wn = __shfl_sync(0xffffffffu, w_new, 4 * i + j);
-                            lsum[ci * 32 + 4 * i + j] = lsum[ci * 32 + 4 * i + j] * wo + wn * vv[j];
+                            lsum[cs * 32 + 4 * i + j] = lsum[cs * 32 + 4 * i + j] * wo + wn * vv[j];
                         }
                     }
                 }
@@ -634,20 +639,20 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         }
         __nv_bfloat16* out_t = p.attn_out + t;
 #pragma unroll
-        for (int ci = 0; ci < NCH; ++ci) {
-            const float inv_l = 1.f / l_all[ci];
+        for (int cs = 0; cs < NCH; ++cs) { const int ci = half + cs * HALVES;
+            const float inv_l = 1.f / l_all[cs];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const float il = __shfl_sync(0xffffffffu, inv_l, i);
-                const int row = __shfl_sync(0xffffffffu, row_c[ci], i);
-                if (ci * 32 + i < rows_here) out_t[static_cast<int64_t>(row) * DH] = __float2bfloat16_rn(lsum[ci * 32 + i] * il);
+                const int row = __shfl_sync(0xffffffffu, row_c[cs], i);
+                if (ci * 32 + i < rows_here) out_t[static_cast<int64_t>(row) * DH] = __float2bfloat16_rn(lsum[cs * 32 + i] * il);
             }
         }
     }
 }
 
-template <int DH, int NCH>
-__global__ void __launch_bounds__(kAttThreads, 1)
+template <int DH, int NCHT, int HALVES>
+__global__ void __launch_bounds__((4 + 4 * HALVES) * 32, 1)
 attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ AttnParams p,
                  const __grid_constant__ AttTable tab)
 {
@@ -676,12 +681,13 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         for (int s = 0; s < p.k_stages; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
         for (int s = 0; s < p.v_stages; ++s) { mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1); }
         for (int a = 0; a < 2; ++a) {
-            mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], kAttSoftmaxThreads / 32);   // one arrival per softmax warp
-            mbar_init(&bars->p_full[a], kAttSoftmaxThreads / 32); mbar_init(&bars->p_empty[a], 1);
+            mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], 4 * HALVES);   // one arrival per softmax warp
+            mbar_init(&bars->p_full[a], 4 * HALVES); mbar_init(&bars->p_empty[a], 1);
+            mbar_init(&bars->group[a], 4);                                              // the four warps of one half
         }
-        mbar_init(&bars->q_full, kAttSoftmaxThreads / 32);
-        mbar_init(&bars->o_full, 1);
-        mbar_init(&bars->group, kAttSoftmaxThreads / 32);
+        mbar_init(&bars->q_full, 4 * HALVES);
+        mbar_init(&bars->o_full[0], 1);
+        mbar_init(&bars->o_full[1], 1);
         fence_barrier_init();
         tma_prefetch_desc(&kv_map);
     }
@@ -793,7 +799,7 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         tmem_alloc(&bars->tmem_slot, kAttTmemCols);
         tmem_relinquish();
         tc_fence_before();
-        asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(64 + 128 * HALVES) : "memory");
         tc_fence_after();
         tmem_base = bars->tmem_slot;
         if (lane == 0 && n_my > 0) {
@@ -829,9 +835,9 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                 cur.advance(p, q + 1 < n_my);
             }
         }
-    } else if (warp == kAttPvWarp) {
+    } else if (warp == kAttProducerWarps + 1 + 4 * HALVES) {
         // ------------------------------------------------------------------ MMA issuer of O^T += V^T P^T
-        asm volatile("bar.sync 1, %0;" ::"n"(kAttConsumerThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(64 + 128 * HALVES) : "memory");
         tc_fence_after();
         tmem_base = bars->tmem_slot;
         if (lane == 0 && n_my > 0) {
@@ -854,7 +860,11 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                               idesc_o, (seg_first && ks == 0) ? 0u : 1u);
                 umma_commit(&bars->v_empty[vs]);
                 umma_commit(&bars->p_empty[pb]);
-                umma_commit(&bars->o_full);
+                // "O^T holds block q": two barriers, alternating with q.  A softmax warp that waits for block q
+                // only knows that the product of block q - 2 has completed (it waited for that P^T buffer); with
+                // one barrier its parity could not tell block q - 1 still pending from block q done, with two
+                // each barrier is exactly one phase ahead of what the waiter has seen.
+                umma_commit(&bars->o_full[q & 1]);
                 if (++vs == p.v_stages) { vs = 0; vpar ^= 1u; }
                 if (++pb == p.p_bufs) { pb = 0; ppar ^= 1u; }
                 seg_first = (cur.blk == cur.nb - 1);       // the next block opens a segment
@@ -862,7 +872,7 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             }
         }
     } else {
-        att_softmax<DH, NCH>(p, tab, sm, cur, n_my);
+        att_softmax<DH, NCHT, HALVES>(p, tab, sm, cur, n_my);
     }
 
     tc_fence_before();
@@ -875,19 +885,19 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
 
 // one kernel per (head dim, chunks of 32 query rows): each instance keeps only the registers and the
 // code of its own softmax width
-template <int DH, int NCH>
+template <int DH, int NCHT, int HALVES>
 static cudaError_t att_set_smem()
 {
-    return cudaFuncSetAttribute(attention_kernel<DH, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(attention_kernel<DH, NCHT, HALVES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 kAttSmemLimit - kAttStaticReserve);
 }
 template <int DH>
 static cudaError_t att_init_dh()
 {
-    cudaError_t e = att_set_smem<DH, 1>();
-    if (e == cudaSuccess) e = att_set_smem<DH, 2>();
-    if (e == cudaSuccess) e = att_set_smem<DH, 3>();
-    if (e == cudaSuccess) e = att_set_smem<DH, 4>();
+    cudaError_t e = att_set_smem<DH, 1, 1>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 2, 2>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 3, 2>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 4, 2>();
     return e;
 }
 cudaError_t attention_init(int head_dim)
@@ -900,11 +910,13 @@ static void att_launch_dh(const CUtensorMap& kv_map, const AttnParams& p, const 
 {
     const size_t smem = static_cast<size_t>(p.k_stages + p.v_stages) * AttCfg<DH>::kTileBytes +
                         AttCfg<DH>::fixed_bytes(p.n_pad, p.p_bufs);
-    dim3 grid(n_ctas), block(kAttThreads);
-    if (p.n_pad <= 32) attention_kernel<DH, 1><<<grid, block, smem, stream>>>(kv_map, p, tab);
-    else if (p.n_pad <= 64) attention_kernel<DH, 2><<<grid, block, smem, stream>>>(kv_map, p, tab);
-    else if (p.n_pad <= 96) attention_kernel<DH, 3><<<grid, block, smem, stream>>>(kv_map, p, tab);
-    else attention_kernel<DH, 4><<<grid, block, smem, stream>>>(kv_map, p, tab);
+    // up to 32 query rows per kv head: four softmax warps, one thread per token; beyond: eight, two threads
+    // per token that split the rows (one warp per scheduler could not hide the latencies of a wide tile)
+    dim3 grid(n_ctas);
+    if (p.n_pad <= 32) attention_kernel<DH, 1, 1><<<grid, 256, smem, stream>>>(kv_map, p, tab);
+    else if (p.n_pad <= 64) attention_kernel<DH, 2, 2><<<grid, 384, smem, stream>>>(kv_map, p, tab);
+    else if (p.n_pad <= 96) attention_kernel<DH, 3, 2><<<grid, 384, smem, stream>>>(kv_map, p, tab);
+    else attention_kernel<DH, 4, 2><<<grid, 384, smem, stream>>>(kv_map, p, tab);
 }
 
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, const AttTable& tab,
