@@ -304,7 +304,7 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, const S
     if (p.n_pass == 1) { p.n_full_tiles = h.lm_full_tiles; p.last_rows = h.lm_last_rows; p.n_vtiles = h.lm_full_tiles + h.lm_last_tiles; }
     else { p.n_vtiles = (c.vocab + 127) / 128; p.n_full_tiles = p.n_vtiles; p.last_rows = 128; }
     p.num_stages = lm_head_pick_stages(p.n_tile, p.n_blocks);
-    p.acc_stages = (2 * rows_per_pass <= 512) ? 2 : 1;
+    p.n_bufs = 512 / p.n_tile < 4 ? 512 / p.n_tile : 4;       // what fits into the 512 TMEM columns, four at most
     p.tstats = nullptr; p.n_tparts = 0; p.inv_temp_log2 = 1.f; p.greedy = 0;
     p.row_seq = nullptr; p.vocab_mask = nullptr; p.mask_words = 0; p.row_c = nullptr;
     if (sp != nullptr) {

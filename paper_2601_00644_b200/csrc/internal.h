@@ -91,7 +91,7 @@ struct LmHeadParams {
     int32_t n_full_tiles;
     int32_t last_rows;        // height of the tiles of the last wave (<= 128)
     int32_t num_stages;       // shared-memory pipeline depth
-    int32_t acc_stages;       // TMEM accumulator buffers (1 or 2)
+    int32_t n_bufs;           // accumulator ring: buffers of n_tile TMEM columns (n_blocks <= n_bufs <= 8)
     // optional: softmax statistics of the rows, one part per (row, 32 vocabulary rows), for the
     // sampling stage (null = not wanted)
     float2* tstats;           // [m_rows][n_tparts], n_tparts = 4 * n_vtiles

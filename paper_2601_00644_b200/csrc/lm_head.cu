@@ -28,6 +28,7 @@ constexpr int kLmThreads = 192;
 constexpr int kLmMaxStages = 12;
 constexpr int kLmATileBytes = kLmBlockV * kLmBlockK * 2;     // 16 KB
 constexpr int kLmTmemCols = 512;
+constexpr int kLmMaxAccBufs = 8;        // accumulator ring (buffers of n_tile TMEM columns)
 constexpr int kLmSmemLimit = 232448;    // 227 KB opt-in maximum per CTA
 constexpr int kLmBarBytes = 512;
 
@@ -55,8 +56,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + p.num_stages * stage_bytes);
     uint64_t* empty_bar = full_bar + kLmMaxStages;
     uint64_t* tmem_full = empty_bar + kLmMaxStages;
-    uint64_t* tmem_empty = tmem_full + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    uint64_t* tmem_empty = tmem_full + kLmMaxAccBufs;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + kLmMaxAccBufs);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -64,7 +65,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+        for (int a = 0; a < p.n_bufs; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
         fence_barrier_init();
         tma_prefetch_desc(&w_map);
         tma_prefetch_desc(&w_map_last);
@@ -86,8 +87,11 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
     auto tile_row0 = [&](int vt) {
         return vt < p.n_full_tiles ? vt * kLmBlockV : p.n_full_tiles * kLmBlockV + (vt - p.n_full_tiles) * p.last_rows;
     };
-    const int acc_cols = p.n_blocks * p.n_tile;        // TMEM columns of one accumulator buffer
-    const int rows_per_pass = acc_cols;
+    // Accumulators: a ring of n_bufs buffers of n_tile TMEM columns; a tile takes n_blocks consecutive
+    // buffers, one per block of token columns.  With a buffer to spare the MMAs of the next tile start
+    // (and, where two blocks share the ring with one spare, continue as soon as the epilogue has
+    // drained the first block) while the epilogue still drains this tile.
+    const int rows_per_pass = p.n_blocks * p.n_tile;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -124,13 +128,18 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             const uint32_t idesc = umma_idesc_bf16(kLmBlockV, static_cast<uint32_t>(p.n_tile));
             int s = 0;
             uint32_t ph = 0;
-            int a = 0;
-            uint32_t aph = 0;
+            int seq = 0;                                 // accumulator buffers handed out so far
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                if (!mbar_wait(&tmem_empty[a], aph ^ 1u, p.status, 4)) { ok = false; break; }
+                // the tile's accumulator buffers: their previous contents must have been drained (use u of a
+                // buffer waits for the epilogue of use u - 1; a fresh barrier lets use 0 through)
+                const int slot0 = seq % p.n_bufs, slot1 = (seq + 1) % p.n_bufs;
+                if (!mbar_wait(&tmem_empty[slot0], (static_cast<uint32_t>(seq / p.n_bufs) & 1u) ^ 1u, p.status, 4)) { ok = false; break; }
+                if (p.n_blocks > 1 &&
+                    !mbar_wait(&tmem_empty[slot1], (static_cast<uint32_t>((seq + 1) / p.n_bufs) & 1u) ^ 1u, p.status, 4)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t acc = tmem_base + static_cast<uint32_t>(a * acc_cols);
+                const uint32_t acc0 = tmem_base + static_cast<uint32_t>(slot0 * p.n_tile);
+                const uint32_t acc1 = tmem_base + static_cast<uint32_t>(slot1 * p.n_tile);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, p.status, 5)) { ok = false; break; }
                     tc_fence_after();
@@ -141,33 +150,36 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                         for (int k = 0; k < kLmBlockK / kLmUmmaK; ++k) {
                             const uint64_t da = umma_desc_k_sw128(a_addr + k * kLmUmmaK * 2);
                             const uint64_t db = umma_desc_k_sw128(b_addr + nb * p.n_tile * 128 + k * kLmUmmaK * 2);
-                            umma_bf16(acc + static_cast<uint32_t>(nb * p.n_tile), da, db, idesc,
-                                      (kb > 0 || k > 0) ? 1u : 0u);
+                            umma_bf16(nb ? acc1 : acc0, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
                         }
                     }
                     umma_commit(&empty_bar[s]);          // stage is free once these MMAs have read it
                     if (++s == p.num_stages) { s = 0; ph ^= 1u; }
                 }
-                if (ok) umma_commit(&tmem_full[a]);      // accumulator complete
-                if (++a == p.acc_stages) { a = 0; aph ^= 1u; }
+                if (ok) {                                // accumulators complete
+                    umma_commit(&tmem_full[slot0]);
+                    if (p.n_blocks > 1) umma_commit(&tmem_full[slot1]);
+                }
+                seq += p.n_blocks;
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (4 warps)
         const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31
-        int a = 0;
-        uint32_t aph = 0;
+        int seq = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            const int vt = tile / p.n_pass, pass = tile % p.n_pass;
-            if (!mbar_wait(&tmem_full[a], aph, p.status, 6)) { ok = false; break; }
+          const int vt = tile / p.n_pass, pass = tile % p.n_pass;
+          const int tile_rows = vt < p.n_full_tiles ? kLmBlockV : p.last_rows;
+          const int v = (quarter * 32 + lane < tile_rows) ? tile_row0(vt) + quarter * 32 + lane : p.vocab;   // past the tile: not a row
+          for (int nb = 0; nb < p.n_blocks && ok; ++nb, ++seq) {
+            const int slot = seq % p.n_bufs;
+            if (!mbar_wait(&tmem_full[slot], static_cast<uint32_t>(seq / p.n_bufs) & 1u, p.status, 6)) { ok = false; break; }
             tc_fence_after();
-            const int tile_rows = vt < p.n_full_tiles ? kLmBlockV : p.last_rows;
-            const int v = (quarter * 32 + lane < tile_rows) ? tile_row0(vt) + quarter * 32 + lane : p.vocab;   // past the tile: not a row
-            const int row_base = pass * rows_per_pass;
+            const int row_base = pass * rows_per_pass + nb * p.n_tile;
             const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                    static_cast<uint32_t>(a * acc_cols);
-            for (int c0 = 0; c0 < acc_cols; c0 += 16) {
+                                    static_cast<uint32_t>(slot * p.n_tile);
+            for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
                 if (row_base + c0 >= p.m_rows) break;    // warp-uniform
                 uint32_t r[16];
                 tmem_ld_x16(taddr0 + static_cast<uint32_t>(c0), r);
@@ -228,8 +240,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tmem_empty[a]);
-            if (++a == p.acc_stages) { a = 0; aph ^= 1u; }
+            if (lane == 0) mbar_arrive(&tmem_empty[slot]);
+          }
         }
     }
 
