@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch, per workload, from the ncu
 # captures summarised in profiles/ (a workload without a capture of the current kernel reports null)
-LM_HEAD_TRAFFIC_BYTES = {}
+LM_HEAD_TRAFFIC_BYTES = {"llama3_8b": 1051787000 + 8008448}
 FALLBACK_HBM_GBS = 6650.0
 REFERENCE_BUDGET_S = 120.0
 
@@ -272,6 +272,9 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
 
     shape = wl.CONFIGS[args.config]
+    if args.batch or args.vocab:                                         # reduced case (profiler captures)
+        shape = wl.scaled(shape, name=f"{shape.name}_b{args.batch or shape.batch}_v{args.vocab or shape.vocab}",
+                          batch=args.batch or shape.batch, vocab=args.vocab or shape.vocab)
     shape = shard_for_rank(shape, rank)                                  # every rank its own batch
     inp = wl.make_inputs(shape, device=str(dev))
     k_host, kv_host = inp.draft_len.cpu(), inp.kv_len.cpu()
@@ -457,7 +460,7 @@ def run_ours(args):
             "wall_s_timed_region": t_wall,
         }
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(wl.CONFIGS[args.config])
+            line["cpu_baseline"] = cpu_baseline(shape)
         if layers_info is not None:
             step_l = ms_per_step + layers_info["attention_ms_all_layers"] - stage_ms[1]
             layers_info["attention_share_of_step"] = layers_info["attention_ms_all_layers"] / step_l
@@ -465,7 +468,7 @@ def run_ours(args):
             line["layers"] = layers_info
         if world == 1 and args.fit_k:
             del flush
-            fit = fit_cloud_cost(args, wl.CONFIGS[args.config], dev)
+            fit = fit_cloud_cost(args, shape, dev)
             line["cloud_cost_fit"] = fit
             # the paper's objective (Eq. 2) with the fitted cloud constants: adaptive stride against fixed strides
             from paper_2601_00644_b200 import policy
@@ -489,6 +492,8 @@ def main():
     ap.add_argument("--top-p", type=float, default=1.0,
                     help="nucleus sampling of the target (the paper's stochastic regime uses 0.9); 1.0 = off")
     ap.add_argument("--top-k", type=int, default=0, help="top-k filter of the target before the nucleus; 0 = off")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (reduced cases for profiler captures)")
+    ap.add_argument("--vocab", type=int, default=0, help="override the workload's vocabulary (reduced cases for profiler captures)")
     ap.add_argument("--layers", type=int, default=1,
                     help="also time the attention stage L times back to back (one launch per layer of a real model)")
     ap.add_argument("--fit-k", action="store_true",
