@@ -17,7 +17,10 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "flexspec_oracle.c")
 _HDR = os.path.join(_HERE, "flexspec_oracle.h")
-_LIB = os.path.join(_HERE, "libflexspec_oracle.so")
+# FLEXSPEC_ORACLE_SANITIZE=1: a separate build with AddressSanitizer + UndefinedBehaviorSanitizer (the
+# process must then run with libasan preloaded; tests/test_oracle_sanitized.py does that in a child)
+_SANITIZE = os.environ.get("FLEXSPEC_ORACLE_SANITIZE", "") == "1"
+_LIB = os.path.join(_HERE, "libflexspec_oracle_san.so" if _SANITIZE else "libflexspec_oracle.so")
 
 GREEDY = 1
 SAMPLE = 0
@@ -28,8 +31,9 @@ def build(force: bool = False) -> str:
     stale = (not os.path.exists(_LIB)
              or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)))
     if force or stale:
-        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
-               "-o", _LIB, _SRC, "-lm"]
+        opt = ["-O1", "-g", "-fsanitize=address,undefined", "-fno-omit-frame-pointer"] if _SANITIZE else ["-O2"]
+        cmd = ["gcc"] + opt + ["-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+                                "-o", _LIB, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 

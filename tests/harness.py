@@ -111,15 +111,40 @@ def make_verifier(case: Case, debug=True, mode=None):
                             debug=debug)
 
 
+CANARY = -0x5A5A5A5B          # guard-band pattern around output buffers
+GUARD = 64                    # elements on either side
+
+
+def guarded(n, dtype, device="cuda"):
+    """A buffer of n elements with GUARD canary elements before and after it; returns (whole, view)."""
+    per = torch.empty(0, dtype=dtype).element_size()
+    words = ((n + 2 * GUARD) * per + 3) // 4
+    raw = torch.full((words,), CANARY, dtype=torch.int32, device=device)
+    whole = raw.view(dtype)
+    return whole, whole[GUARD:GUARD + n]
+
+
+def guards_intact(whole, n):
+    raw = whole.view(torch.int32) if whole.dtype != torch.int32 else whole
+    per = whole.element_size()
+    lo = GUARD * per // 4
+    hi = (GUARD + n) * per // 4 + (1 if ((GUARD + n) * per) % 4 else 0)
+    return bool((raw[:lo] == CANARY).all() and (raw[hi:] == CANARY).all())
+
+
 def run_gpu_verify(case: Case, ver, vocab_mask_dev=None, temperature=None):
+    """One verify call; the two output arrays sit between canary guard bands that must survive it."""
     inp = case.inp
     t = case.shape.temperature if temperature is None else temperature
-    acc, nxt = ver.verify(inp.kv_pages, inp.page_table, inp.kv_len, inp.kv_len.cpu(), inp.hidden,
-                          case.draft_tokens, case.draft_logits, inp.draft_len, inp.draft_len.cpu(),
-                          inp.seeds, temperature=t, vocab_mask=vocab_mask_dev)
+    acc_w, acc = guarded(case.batch, torch.int32)
+    nxt_w, nxt = guarded(case.batch, torch.int32)
+    ver.verify(inp.kv_pages, inp.page_table, inp.kv_len, inp.kv_len.cpu(), inp.hidden,
+               case.draft_tokens, case.draft_logits, inp.draft_len, inp.draft_len.cpu(),
+               inp.seeds, temperature=t, vocab_mask=vocab_mask_dev, accepted_len=acc, next_token=nxt)
     torch.cuda.synchronize()
     code, st = ver.status()
     assert code == 0, f"device status {code} {st}"
+    assert guards_intact(acc_w, case.batch) and guards_intact(nxt_w, case.batch), "a kernel wrote outside accepted_len / next_token"
     return acc.cpu().numpy(), nxt.cpu().numpy()
 
 

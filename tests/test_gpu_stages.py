@@ -406,3 +406,25 @@ def test_sample_stage_with_per_sequence_temperatures_matches_oracle():
     ref = oracle.accept(0, zt.astype(np.float64), zd, toks, k, seeds, 0.9)
     assert _decisions_match(k, acc.cpu().numpy(), nxt.cpu().numpy(), ref) <= 1
     ver.close()
+
+
+def test_stage_outputs_stay_inside_their_buffers():
+    """Attention output and logits written into caller buffers that sit between canary guard bands
+    (ragged batch: the last query row and the last vocabulary tile are partial): the bands survive."""
+    import tests.harness as H
+    B = _binding()
+    shape = _shape("guard", 31, batch=3, n_q_heads=8, n_kv_heads=2, head_dim=128, vocab=1000 + 37, k_min=0, k_max=6,
+                   ctx_min=5, ctx_max=300)
+    inp = wl.make_inputs(shape, device="cuda")
+    kh, kvh = inp.draft_len.cpu(), inp.kv_len.cpu()
+    ver = B.Verifier(inp.lm_head_w, 8, 2, 128, max_batch=3, k_max=6, max_kv_len=int(kvh.max()))
+    m, d, v = inp.m_rows, shape.d_model, shape.vocab
+    a_w, a = H.guarded(m * d, torch.bfloat16)
+    ver.attention(inp.kv_pages, inp.page_table, inp.kv_len, kvh, inp.hidden, inp.draft_len, kh, attn_out=a.view(m, d))
+    l_w, l = H.guarded(m * v, torch.float32)
+    ver.lm_head(a.view(m, d), logits=l.view(m, v))
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    assert H.guards_intact(a_w, m * d) and H.guards_intact(l_w, m * v)
+    assert torch.isfinite(l).all() and torch.isfinite(a.float()).all()      # and everything inside was written
+    ver.close()
