@@ -426,5 +426,5 @@ def test_stage_outputs_stay_inside_their_buffers():
     torch.cuda.synchronize()
     assert ver.status()[0] == 0
     assert H.guards_intact(a_w, m * d) and H.guards_intact(l_w, m * v)
-    assert torch.isfinite(l).all() and torch.isfinite(a.float()).all()      # and everything inside was written
+    assert int((l.view(torch.int32) == H.CANARY).sum()) == 0                # and everything inside was written
     ver.close()
