@@ -457,7 +457,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     const size_t att_slots = static_cast<size_t>(2) * h.sm_count;
     A(dev_alloc(&h.part_o, att_slots * kAttRowsPerPair * c.head_dim));
     A(dev_alloc(&h.part_ml, att_slots * 4 * kAttRowsPerPair * 2));
-    A(dev_alloc(&h.att_tickets, static_cast<size_t>(h.att_pairs_max) * 8));
+    A(dev_alloc(&h.att_tickets, static_cast<size_t>(h.att_pairs_max) * 12));
     A(dev_alloc(&h.plan.cu_q, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.cu_d, static_cast<size_t>(c.max_batch) + 1));
     A(dev_alloc(&h.plan.row_seq, static_cast<size_t>(max_m)));
@@ -479,7 +479,7 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
         if (cudaMalloc(&h.stage_dev, h.stage_bytes) != cudaSuccess) { cudaGetLastError(); rc = FLEXSPEC_ERR_OOM; }
     }
     if (rc == FLEXSPEC_OK) {
-        if (cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 8) != cudaSuccess ||
+        if (cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 12) != cudaSuccess ||
             cudaMemset(h.status, 0, sizeof(int32_t) * 4) != cudaSuccess)
             rc = FLEXSPEC_ERR_CUDA;
     }
@@ -812,7 +812,7 @@ int flexspec_status(flexspec_handle* fh, int32_t* status_host)
     if (st[0] != 0) {
         // a kernel that gave up may have left its arrival tickets half counted: start the next call clean
         if (cudaMemset(h.status, 0, sizeof(st)) != cudaSuccess ||
-            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 8) != cudaSuccess)
+            cudaMemset(h.att_tickets, 0, sizeof(int32_t) * static_cast<size_t>(h.att_pairs_max) * 12) != cudaSuccess)
             return FLEXSPEC_ERR_CUDA;
     }
     if (status_host != nullptr) memcpy(status_host, st, sizeof(st));

@@ -45,7 +45,7 @@ namespace fs {
 
 constexpr int kPageTokens = 16;
 constexpr int kAttPagesPerStage = kAttBlockTokens / kPageTokens;    // 8
-// warp order: 2 TMA producers, the S^T issuer, 4 or 8 softmax warps (HALVES = 1 or 2), the PV issuer;
+// warp order: 2 TMA producers, the S^T issuer, 4, 8 or 12 softmax warps (HALVES = 1, 2 or 3), the PV issuer;
 // named barrier 1 joins everyone who touches tensor memory: 64 + 128 * HALVES threads
 constexpr int kAttTmemCols = 512;
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO = 256;        // column offsets
@@ -58,7 +58,7 @@ struct AttBars {
     uint64_t v_full[kAttMaxStages], v_empty[kAttMaxStages];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_full[2], p_empty[2];
-    uint64_t q_full, o_full[2], group[2];       // o_full alternates with the block parity (see the PV issuer)
+    uint64_t q_full, o_full[2], group[3];       // o_full alternates with the block parity (see the PV issuer)
     uint32_t tmem_slot;
 };
 static_assert(sizeof(AttBars) <= 512, "barrier block");
@@ -76,7 +76,7 @@ struct AttCfg {
     static constexpr int kTileBytes = kSlabs * kSlabBytes;     // K (or V) of one 128-token block
     __host__ __device__ static constexpr int q_bytes(int n_pad) { return kSlabs * n_pad * 128; }
     __host__ __device__ static constexpr int p_bytes(int n_pad) { return n_pad * 256; }
-    __host__ __device__ static constexpr int col_bytes(int n_pad) { return (3 * 4 + 1) * n_pad * 4 + 64; }
+    __host__ __device__ static constexpr int col_bytes(int n_pad) { return (3 * 4 + 1) * n_pad * 4 + 128; }
     __host__ __device__ static constexpr int fixed_bytes(int n_pad, int p_bufs)
     {
         return q_bytes(n_pad) + p_bufs * p_bytes(n_pad) + 512 + col_bytes(n_pad) + 1024;
@@ -239,7 +239,7 @@ struct AttSmem {                  // pointers into dynamic shared memory
     AttBars* bars;
     float* xch;                   // [3][4][n_pad]: column maxima (by block parity) and row sums, one row per warp
     float* m_col;                 // [n_pad] running maximum of every column (query row), log2 units
-    int* flags;                   // [2][4] "a score exceeded its maximum by more than the threshold", by block parity and warp
+    int* flags;                   // [parts][2][4] "a score exceeded its maximum by more than the threshold", by block parity and warp
 };
 
 // CTA that holds block x of the batch-wide list: the last one whose range starts at or before x.
@@ -267,10 +267,10 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
     AttBars* bars = sm.bars;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
-    // HALVES == 2: two warps share every quarter (the same 32 tokens) and split the columns (query rows)
-    // chunk-wise: warp half h owns chunks h, h + 2.  Column state, exchanges and barriers of the two halves
+    // HALVES == 2 or 3: that many warps share every quarter (the same 32 tokens) and split the columns (query
+    // rows) chunk-wise: the warp of part h owns chunks h, h + HALVES.  Column state, exchanges and barriers of the two halves
     // are separate; they only meet in the hand-overs to the MMA warps.
-    const int half = HALVES == 2 ? ((warp - (kAttProducerWarps + 1)) >> 2) : 0;
+    const int half = HALVES > 1 ? ((warp - (kAttProducerWarps + 1)) >> 2) : 0;
     const int t = quarter * 32 + lane;                  // token of the block (S^T), Dh index (O^T)
     const int cta = blockIdx.x;
     const int n_pad = p.n_pad;
@@ -583,7 +583,7 @@ __device__ __forceinline__ void att_softmax(const AttnParams& p, const AttTable&
         __syncwarp();
         int last = 0;
         if (lane == 0) {
-            int32_t* tk = p.tickets + (static_cast<int64_t>(pair_global) * 4 + quarter) * 2 + half;
+            int32_t* tk = p.tickets + (static_cast<int64_t>(pair_global) * 4 + quarter) * 3 + half;
             last = (atomicAdd(tk, 1) == c_last - c_first);
             if (last) *tk = 0;                                         // ready for the next call
         }
@@ -683,8 +683,8 @@ attention_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         for (int a = 0; a < 2; ++a) {
             mbar_init(&bars->s_full[a], 1); mbar_init(&bars->s_empty[a], 4 * HALVES);   // one arrival per softmax warp
             mbar_init(&bars->p_full[a], 4 * HALVES); mbar_init(&bars->p_empty[a], 1);
-            mbar_init(&bars->group[a], 4);                                              // the four warps of one half
         }
+        for (int a = 0; a < 3; ++a) mbar_init(&bars->group[a], 4);                      // the four warps of one column part
         mbar_init(&bars->q_full, 4 * HALVES);
         mbar_init(&bars->o_full[0], 1);
         mbar_init(&bars->o_full[1], 1);
@@ -896,7 +896,7 @@ static cudaError_t att_init_dh()
 {
     cudaError_t e = att_set_smem<DH, 1, 1>();
     if (e == cudaSuccess) e = att_set_smem<DH, 2, 2>();
-    if (e == cudaSuccess) e = att_set_smem<DH, 3, 2>();
+    if (e == cudaSuccess) e = att_set_smem<DH, 3, 3>();
     if (e == cudaSuccess) e = att_set_smem<DH, 4, 2>();
     return e;
 }
@@ -915,7 +915,7 @@ static void att_launch_dh(const CUtensorMap& kv_map, const AttnParams& p, const 
     dim3 grid(n_ctas);
     if (p.n_pad <= 32) attention_kernel<DH, 1, 1><<<grid, 256, smem, stream>>>(kv_map, p, tab);
     else if (p.n_pad <= 64) attention_kernel<DH, 2, 2><<<grid, 384, smem, stream>>>(kv_map, p, tab);
-    else if (p.n_pad <= 96) attention_kernel<DH, 3, 2><<<grid, 384, smem, stream>>>(kv_map, p, tab);
+    else if (p.n_pad <= 96) attention_kernel<DH, 3, 3><<<grid, 512, smem, stream>>>(kv_map, p, tab);   // three threads per token
     else attention_kernel<DH, 4, 2><<<grid, 384, smem, stream>>>(kv_map, p, tab);
 }
 

@@ -48,7 +48,7 @@ struct AttnParams {
     float scale_log2;         // log2(e) / sqrt(head_dim)
     float* part_o;            // [2 * CTAs][Dh][128] unnormalised partial outputs (a CTA's first / last segment)
     float* part_ml;           // [2 * CTAs][4 warps][128][2]  (running max in log2 units, sum)
-    int32_t* tickets;         // [pairs][4 quarters][2 halves] self-resetting arrival counters of the split merge
+    int32_t* tickets;         // [pairs][4 quarters][3 column parts] self-resetting arrival counters of the split merge
     __nv_bfloat16* attn_out;  // [M][d_model]
     int32_t* status;
 };
