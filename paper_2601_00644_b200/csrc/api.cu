@@ -7,6 +7,8 @@
 
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "internal.h"
 
 using namespace fs;
@@ -60,6 +62,12 @@ int dev_alloc(T** p, size_t count)
     if (e != cudaSuccess) { cudaGetLastError(); return FLEXSPEC_ERR_OOM; }
     return FLEXSPEC_OK;
 }
+
+// Named range on the host timeline (header-only NVTX: a no-op unless a profiler is attached).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 struct DeviceGuard {
     int prev = -1;
@@ -531,6 +539,7 @@ int flexspec_attention(flexspec_handle* fh, const flexspec_kv* kv, const void* h
                        const int32_t* draft_len, const int32_t* draft_len_host, int32_t batch,
                        void* attn_out, void* stream)
 {
+    NvtxRange nvtx_range("flexspec_attention");
     if (fh == nullptr || hidden == nullptr || draft_len == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
     Handle& h = fh->h;
     if (!kv_args_ok(h, kv, true)) return FLEXSPEC_ERR_INVALID_ARG;
@@ -547,6 +556,7 @@ int flexspec_attention(flexspec_handle* fh, const flexspec_kv* kv, const void* h
 
 int flexspec_lm_head(flexspec_handle* fh, const void* x, int32_t m_rows, float* logits, void* stream)
 {
+    NvtxRange nvtx_range("flexspec_lm_head");
     if (fh == nullptr) return FLEXSPEC_ERR_INVALID_ARG;
     Handle& h = fh->h;
     if (m_rows < 1 || m_rows > h.max_m) return FLEXSPEC_ERR_INVALID_ARG;
@@ -561,6 +571,7 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
                     const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
                     int32_t* accepted_len, int32_t* next_token, void* stream)
 {
+    NvtxRange nvtx_range("flexspec_sample");
     if (fh == nullptr || draft_len == nullptr || accepted_len == nullptr || next_token == nullptr)
         return FLEXSPEC_ERR_INVALID_ARG;
     Handle& h = fh->h;
@@ -589,6 +600,7 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
                     const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
                     int32_t* accepted_len, int32_t* next_token, void* stream)
 {
+    NvtxRange nvtx_range("flexspec_verify");
     if (fh == nullptr || hidden == nullptr || draft_len == nullptr || accepted_len == nullptr ||
         next_token == nullptr)
         return FLEXSPEC_ERR_INVALID_ARG;
@@ -649,6 +661,7 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
                          const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
                          int32_t* accepted_len, int32_t* next_token, void* stream)
 {
+    NvtxRange nvtx_range("flexspec_verify_host");
     if (fh == nullptr || hidden == nullptr || draft_len == nullptr || accepted_len == nullptr ||
         next_token == nullptr)
         return FLEXSPEC_ERR_INVALID_ARG;

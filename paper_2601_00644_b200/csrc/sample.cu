@@ -581,12 +581,23 @@ sample_accept_kernel(const SampleParams p)
             int x = p.draft_tokens[d0 + j];
             x = min(max(x, 0), p.vocab - 1);
             if (!p.greedy) {
+                // the row's parts (at most a few per lane: kept in registers, so they are read once)
                 const float2* dp = p.stats + static_cast<int64_t>(p.m_rows + d0 + j) * p.n_chunks;
+                float2 part[4];
                 float mqf = -INFINITY;
-                for (int i = lane; i < p.n_chunks; i += 32) mqf = fmaxf(mqf, __ldcg(&dp[i].x));
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int i = lane + 32 * t;
+                    part[t] = (i < p.n_chunks) ? __ldcg(&dp[i]) : make_float2(-INFINITY, 0.f);
+                    mqf = fmaxf(mqf, part[t].x);
+                }
+                for (int i = lane + 128; i < p.n_chunks; i += 32) mqf = fmaxf(mqf, __ldcg(&dp[i].x));   // vocabularies beyond 1M / 8: none today
                 mqf = warp_max(mqf);
                 double acc = 0.0;
-                for (int i = lane; i < p.n_chunks; i += 32) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    if (part[t].x != -INFINITY) acc += static_cast<double>(part[t].y) * static_cast<double>(fast_exp2((part[t].x - mqf) * cf));
+                for (int i = lane + 128; i < p.n_chunks; i += 32) {
                     const float2 pt = __ldcg(&dp[i]);
                     if (pt.x != -INFINITY) acc += static_cast<double>(pt.y) * static_cast<double>(fast_exp2((pt.x - mqf) * cf));
                 }
