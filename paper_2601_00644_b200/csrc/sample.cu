@@ -216,20 +216,28 @@ __device__ __forceinline__ float key_to_float(uint32_t k)
 }
 
 struct FilterShared {
-    uint32_t hist[2][3][256];                           // [buffer][count, mass limb (bits 16..31), mass limb (bits 0..15)][bin]
-    unsigned long long tot[2][256];                     // cluster-wide histogram of the round
-    float red[kFilterWarps];
-    float slice_max[kAcceptCluster];
+    uint32_t hist[2][2][256];                           // [buffer][top-k: count | top-p: mass limbs (bits 16..31, bits 0..15)][bin]
+    unsigned long long tot[256];                        // cluster-wide histogram of the round (the weight that decides)
+    uint32_t red[kFilterWarps];
+    unsigned long long red64[kFilterWarps];
+    uint32_t slice_max[kAcceptCluster];
+    unsigned long long slice_mass[kAcceptCluster];
     uint32_t prefix;                                    // key bits fixed so far
-    unsigned long long above[2];                        // count / mass of the keys above the prefix's bin path
+    unsigned long long above;                           // weight of the keys above the prefix's bin path
     unsigned long long target;
     int bin;
 };
 
+// 2^((z - m) c) in fixed point (units of 2^-31, round to nearest), z given by its key
+__device__ __forceinline__ uint32_t key_mass(uint32_t key, float m, float cf)
+{
+    return __float2uint_rn(fast_exp2((key_to_float(key) - m) * cf) * kMassUnitF);   // <= 2^31
+}
+
 __global__ void __cluster_dims__(kAcceptCluster, 1, 1) __launch_bounds__(kFilterThreads)
 sample_filter_kernel(const SampleParams p)
 {
-    extern __shared__ float s_slice[];                  // this CTA's slice of the row (when it fits)
+    extern __shared__ uint32_t s_keys[];                // this CTA's slice of the row as order-preserving keys (when it fits)
     __shared__ FilterShared sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = static_cast<int>(cluster.block_rank());
@@ -246,142 +254,149 @@ sample_filter_kernel(const SampleParams p)
     const int n = v1 - v0;
     const bool staged = per <= kFilterSliceMax;
     const bool vec_ok = ((p.vocab & 3) == 0);
+    // key of entry i of the slice: 0 for entries that cannot be selected (masked, -inf), else > 0 and ordered like the logits
+    auto make_key = [&](float z, int i) -> uint32_t {
+        if (z == -INFINITY || (mask_row != nullptr && !mask_allows(mask_row, v0 + i))) return 0u;
+        return order_key(z);
+    };
     if (staged) {
+        float* s_f = reinterpret_cast<float*>(s_keys);
         if (vec_ok) {
-            for (int i = tid * 4; i < n; i += kFilterThreads * 4) cp_async_16(s_slice + i, src + v0 + i);
+            for (int i = tid * 4; i < n; i += kFilterThreads * 4) cp_async_16(s_f + i, src + v0 + i);
         } else {
-            for (int i = tid; i < n; i += kFilterThreads) cp_async_4(s_slice + i, src + v0 + i);
+            for (int i = tid; i < n; i += kFilterThreads) cp_async_4(s_f + i, src + v0 + i);
         }
         cp_async_wait_all();
         __syncthreads();
+        for (int i = tid; i < n; i += kFilterThreads) s_keys[i] = make_key(s_f[i], i);     // once, in place
+        __syncthreads();
     }
-    auto logit = [&](int i) -> float {                  // entry i of the slice; masked entries read as -inf
-        const float z = staged ? s_slice[i] : __ldg(src + v0 + i);
-        return (mask_row != nullptr && !mask_allows(mask_row, v0 + i)) ? -INFINITY : z;
-    };
+    auto key_at = [&](int i) -> uint32_t { return staged ? s_keys[i] : make_key(__ldg(src + v0 + i), i); };
 
-    // ---- row maximum: slice maxima, exchanged through the peers' shared memory
-    float m = -INFINITY;
-    for (int i = tid; i < n; i += kFilterThreads) m = fmaxf(m, logit(i));
-    m = warp_max(m);
-    if (lane == 0) sh.red[warp] = m;
+    // ---- row maximum (the largest key): slice maxima, exchanged through the peers' shared memory
+    uint32_t kmax = 0u;
+    for (int i = tid; i < n; i += kFilterThreads) kmax = max(kmax, key_at(i));
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) sh.red[warp] = kmax;
     __syncthreads();
     cluster_wait();                                     // all eight CTAs have started
     if (tid < kAcceptCluster) {
-        float mm = sh.red[0];
+        uint32_t mm = sh.red[0];
 #pragma unroll
-        for (int w = 1; w < kFilterWarps; ++w) mm = fmaxf(mm, sh.red[w]);
+        for (int w = 1; w < kFilterWarps; ++w) mm = max(mm, sh.red[w]);
         cluster.map_shared_rank(&sh.slice_max[0], tid)[rank] = mm;
     }
-    if (tid == 0) { sh.prefix = 0u; sh.above[0] = 0ull; sh.above[1] = 0ull; }
     cluster_sync();
-    m = sh.slice_max[0];
+    kmax = sh.slice_max[0];
 #pragma unroll
-    for (int c = 1; c < kAcceptCluster; ++c) m = fmaxf(m, sh.slice_max[c]);
+    for (int c = 1; c < kAcceptCluster; ++c) kmax = max(kmax, sh.slice_max[c]);
+    const float m = key_to_float(kmax);
 
     // ---- selections: top-k on counts (if on), then top-p on mass among the keys that survived
     const bool do_k = p.top_k > 0 && p.top_k < p.vocab;
     const bool do_p = p.top_p < 1.f;
-    uint32_t floor_key = 0u;                            // keys below it were cut by top-k
+    uint32_t floor_key = 1u;                            // keys below it are out: 0 = not selectable, later the top-k cut
     double kept_mass = 0.0;
-    float tau = -INFINITY;
     int round_no = 0;                                   // alternates the histogram buffers
     for (int sel = do_k ? 0 : 1; sel < (do_p ? 2 : 1); ++sel) {
         // sel 0: weight 1, target k.   sel 1: weight mass, target top_p * (mass of the keys >= floor_key)
-        if (tid == 0) { sh.prefix = 0u; sh.above[0] = 0ull; sh.above[1] = 0ull; }
+        if (tid == 0) { sh.prefix = 0u; sh.above = 0ull; }
         __syncthreads();
         for (int round = 0; round < 4; ++round, ++round_no) {
             const int shift = 24 - 8 * round;
             const int buf = round_no & 1;
-            for (int i = tid; i < 3 * 256; i += kFilterThreads) (&sh.hist[buf][0][0])[i] = 0u;
+            for (int i = tid; i < 2 * 256; i += kFilterThreads) (&sh.hist[buf][0][0])[i] = 0u;
             __syncthreads();
             const uint32_t prefix = sh.prefix;
             const uint32_t hi_mask = (round == 0) ? 0u : (0xffffffffu << (shift + 8));
-            // four entries per thread and step (their loads and exponentials overlap).  When all lanes of
-            // the warp fall into the same bin (the leading bytes of flat logits) the warp adds once, one
-            // reduction per limb; grouping the lanes by bin with a match was measured twice as slow as
-            // letting them collide.
+            const uint32_t want = prefix & hi_mask;
+            // four entries per thread and step.  A step in which no lane holds a live key (most steps after
+            // the first round) costs a load and a compare per entry.  When all lanes of the warp fall into
+            // the same bin (the leading bytes of flat logits) the warp adds once, one reduction per limb.
             for (int i0 = 0; i0 < n; i0 += kFilterThreads * 4) {
+                uint32_t key[4];
+                bool live[4];
+                bool any = false;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * kFilterThreads + tid;
+                    key[u] = (i < n) ? key_at(i) : 0u;
+                    live[u] = key[u] >= floor_key && (key[u] & hi_mask) == want;
+                    any |= live[u];
+                }
+                if (!__any_sync(0xffffffffu, any)) continue;
                 int bin[4];
                 uint32_t w[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * kFilterThreads + tid;
-                    const float z = (i < n) ? logit(i) : -INFINITY;
-                    const uint32_t key = order_key(z);
-                    const bool live = z != -INFINITY && key >= floor_key && (key & hi_mask) == (prefix & hi_mask);
-                    bin[u] = live ? static_cast<int>((key >> shift) & 255u) : -1;
-                    w[u] = live ? __float2uint_rn(fast_exp2((z - m) * cf) * kMassUnitF) : 0u;   // <= 2^31
+                    bin[u] = live[u] ? static_cast<int>((key[u] >> shift) & 255u) : -1;
+                    w[u] = !live[u] ? 0u : (sel == 0 ? 1u : key_mass(key[u], m, cf));
                 }
                 const int bin0 = __shfl_sync(0xffffffffu, bin[0], 0);
                 if (__all_sync(0xffffffffu, bin[0] == bin0 && bin[1] == bin0 && bin[2] == bin0 && bin[3] == bin0)) {
-                    const uint32_t hi = __reduce_add_sync(0xffffffffu, (w[0] >> 16) + (w[1] >> 16) + (w[2] >> 16) + (w[3] >> 16));
-                    const uint32_t lo = __reduce_add_sync(0xffffffffu, (w[0] & 0xffffu) + (w[1] & 0xffffu) + (w[2] & 0xffffu) + (w[3] & 0xffffu));
-                    if (lane == 0 && bin0 >= 0) {
-                        atomicAdd(&sh.hist[buf][0][bin0], 128u);
-                        atomicAdd(&sh.hist[buf][1][bin0], hi);
-                        atomicAdd(&sh.hist[buf][2][bin0], lo);
+                    // (all 128 entries live and in one bin; limb sums stay far below 2^32)
+                    const uint32_t a0 = __reduce_add_sync(0xffffffffu, sel == 0 ? 4u : (w[0] >> 16) + (w[1] >> 16) + (w[2] >> 16) + (w[3] >> 16));
+                    const uint32_t a1 = sel == 0 ? 0u : __reduce_add_sync(0xffffffffu, (w[0] & 0xffffu) + (w[1] & 0xffffu) + (w[2] & 0xffffu) + (w[3] & 0xffffu));
+                    if (lane == 0) {
+                        atomicAdd(&sh.hist[buf][0][bin0], a0);
+                        if (sel == 1) atomicAdd(&sh.hist[buf][1][bin0], a1);
                     }
                 } else {
 #pragma unroll
                     for (int u = 0; u < 4; ++u)
-                        if (bin[u] >= 0) {
-                            atomicAdd(&sh.hist[buf][0][bin[u]], 1u);
-                            atomicAdd(&sh.hist[buf][1][bin[u]], w[u] >> 16);
-                            atomicAdd(&sh.hist[buf][2][bin[u]], w[u] & 0xffffu);
+                        if (live[u]) {
+                            if (sel == 0) {
+                                atomicAdd(&sh.hist[buf][0][bin[u]], 1u);
+                            } else {
+                                atomicAdd(&sh.hist[buf][0][bin[u]], w[u] >> 16);
+                                atomicAdd(&sh.hist[buf][1][bin[u]], w[u] & 0xffffu);
+                            }
                         }
                 }
             }
             cluster_sync();                             // all eight histograms of this round are complete
-            // cluster-wide histogram: thread t adds bin t of the eight CTAs (both weights)
+            // cluster-wide histogram: thread t adds bin t of the eight CTAs
             {
-                unsigned long long c_sum = 0ull, m_sum = 0ull;
+                unsigned long long acc = 0ull;
 #pragma unroll
                 for (int c = 0; c < kAcceptCluster; ++c) {
                     const uint32_t* peer = cluster.map_shared_rank(&sh.hist[buf][0][0], c);
-                    c_sum += peer[tid];
-                    m_sum += (static_cast<unsigned long long>(peer[256 + tid]) << 16) + peer[512 + tid];
+                    acc += sel == 0 ? static_cast<unsigned long long>(peer[tid])
+                                    : (static_cast<unsigned long long>(peer[tid]) << 16) + peer[256 + tid];
                 }
-                sh.tot[0][tid] = c_sum;
-                sh.tot[1][tid] = m_sum;
+                sh.tot[tid] = acc;
             }
             __syncthreads();
             if (warp == 0) {
-                // walk from the top bin down: lane l owns bins 255 - 8 l ... 248 - 8 l; both weights are
-                // scanned, the one of this selection decides
-                unsigned long long mine[2] = {0ull, 0ull};
+                // walk from the top bin down: lane l owns bins 255 - 8 l ... 248 - 8 l
+                unsigned long long mine = 0ull;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    mine[0] += sh.tot[0][255 - (lane * 8 + j)];
-                    mine[1] += sh.tot[1][255 - (lane * 8 + j)];
-                }
-                unsigned long long incl[2] = {mine[0], mine[1]};      // inclusive scans over lanes (top bins first)
+                for (int j = 0; j < 8; ++j) mine += sh.tot[255 - (lane * 8 + j)];
+                unsigned long long incl = mine;          // inclusive scan over lanes (top bins first)
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    const unsigned long long t0 = __shfl_up_sync(0xffffffffu, incl[0], o);
-                    const unsigned long long t1 = __shfl_up_sync(0xffffffffu, incl[1], o);
-                    if (lane >= o) { incl[0] += t0; incl[1] += t1; }
+                    const unsigned long long t0 = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t0;
                 }
                 if (round == 0 && lane == 31) {
                     // total weight of the live keys = the base of the target
                     sh.target = (sel == 0) ? static_cast<unsigned long long>(p.top_k)
-                                           : static_cast<unsigned long long>(static_cast<double>(p.top_p) * static_cast<double>(incl[1]));
+                                           : static_cast<unsigned long long>(static_cast<double>(p.top_p) * static_cast<double>(incl));
                     if (sh.target < 1ull) sh.target = 1ull;
                 }
                 __syncwarp();
                 const unsigned long long target = sh.target;
-                unsigned long long run[2] = {sh.above[0] + incl[0] - mine[0], sh.above[1] + incl[1] - mine[1]};
-                const unsigned hit = __ballot_sync(0xffffffffu, (sel ? run[1] + mine[1] : run[0] + mine[0]) >= target);
+                unsigned long long run = sh.above + incl - mine;
+                const unsigned hit = __ballot_sync(0xffffffffu, run + mine >= target);
                 // (with exact sums the last lane always reaches the target; the guard keeps the walk defined)
                 const int l = hit != 0u ? __ffs(hit) - 1 : 31;
                 if (lane == l) {
                     int bin = 255 - lane * 8;
                     for (int j = 0; j < 7; ++j, --bin) {
-                        if ((sel ? run[1] + sh.tot[1][bin] : run[0] + sh.tot[0][bin]) >= target) break;
-                        run[0] += sh.tot[0][bin];
-                        run[1] += sh.tot[1][bin];
+                        if (run + sh.tot[bin] >= target) break;
+                        run += sh.tot[bin];
                     }
-                    sh.above[0] = run[0]; sh.above[1] = run[1];       // weights strictly above the chosen bin
+                    sh.above = run;                      // weight strictly above the chosen bin
                     sh.bin = bin;
                     sh.prefix = prefix | (static_cast<uint32_t>(bin) << shift);
                 }
@@ -389,15 +404,35 @@ sample_filter_kernel(const SampleParams p)
             __syncthreads();
         }
         // the selected key: every key >= it is kept
-        const uint32_t key_sel = sh.prefix;
-        const unsigned long long mass_int = sh.above[1] + sh.tot[1][sh.bin];
-        floor_key = key_sel;
-        tau = key_to_float(key_sel);
-        kept_mass = static_cast<double>(mass_int) / kMassUnit;
+        floor_key = sh.prefix;
+        if (sel == 1) kept_mass = static_cast<double>(sh.above + sh.tot[sh.bin]) / kMassUnit;
         __syncthreads();
     }
+    if (!do_p) {
+        // top-k alone: the mass of the kept keys is one more pass (a plain reduction, no histogram)
+        unsigned long long acc = 0ull;
+        for (int i = tid; i < n; i += kFilterThreads) {
+            const uint32_t key = key_at(i);
+            if (key >= floor_key) acc += key_mass(key, m, cf);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) sh.red64[warp] = acc;
+        __syncthreads();
+        if (tid < kAcceptCluster) {
+            unsigned long long t = 0ull;
+#pragma unroll
+            for (int w = 0; w < kFilterWarps; ++w) t += sh.red64[w];
+            cluster.map_shared_rank(&sh.slice_mass[0], tid)[rank] = t;
+        }
+        cluster_sync();
+        unsigned long long t = 0ull;
+#pragma unroll
+        for (int c = 0; c < kAcceptCluster; ++c) t += sh.slice_mass[c];
+        kept_mass = static_cast<double>(t) / kMassUnit;
+    }
     if (rank == 0 && tid == 0) {
-        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(tau);
+        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(key_to_float(floor_key));
         p.topp[static_cast<int64_t>(row) * 2 + 1] = kept_mass;
     }
     cluster_sync();                                     // no CTA leaves while a peer may still read its histograms
