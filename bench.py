@@ -44,61 +44,110 @@ def _peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks / throttle reasons sampled every 100 ms from before the warm-up until after the
-    end-to-end leg (a 20-step timed region lasts a few milliseconds: alone it would see no sample).
-    The median clock is taken over the samples drawn under load: board power at least half of the
-    run's highest sample (between phases the GPU idles and clocks down)."""
+    """SM clock and throttle reasons of one GPU, polled through NVML (read-only queries) every ~2 ms by
+    a thread, from before the warm-up until after the end-to-end leg.  mark() brackets the timed region:
+    the reported median is taken over the samples inside it (a 20-step region lasts ~5 ms and still holds
+    a few); if none fell inside, over the samples of the whole run drawn under load (board power at
+    least half of the run's highest sample).  Falls back to `nvidia-smi -lms 100` without the NVML binding."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index = index
-        self.lines = []
+        self.rows = []            # (t, sm_mhz, power_w, reasons_bitmask)
+        self.marks = []
+        self.smax = None
         self.proc = None
+        self.thread = None
+        self._stop = False
+        self.mode = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.mode = "nvml"
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.mode = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
                  "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.mode = "smi"
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except Exception:
             self.proc = None
 
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+    def mark(self):
+        self.marks.append(time.perf_counter())
 
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        rows, smax, reasons = [], [], set()
+    def _poll(self):
+        nv = self.nv
+        while not self._stop:
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                self.rows.append((time.perf_counter(), sm, pw, rs))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def _pump(self):
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+        for line in self.proc.stdout:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 7:
                 continue
             try:
-                rows.append((float(parts[0]), float(parts[2]))); smax.append(float(parts[1]))
+                sm, smax, pw = float(parts[0]), float(parts[1]), float(parts[2])
             except ValueError:
                 continue
+            self.smax = smax
+            rs = 0
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
+                    rs |= bits[name]
+            self.rows.append((time.perf_counter(), sm, pw, rs))
+
+    def stop(self):
+        if self.mode is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML binding and no nvidia-smi"], "samples": 0}
+        self._stop = True
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        rows = list(self.rows)
+        # NVML clocks-event-reasons bits: 0x4 sw power cap, 0x8 hw slowdown, 0x20 sw thermal, 0x40 hw thermal
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+        timed = [r for r in rows if len(self.marks) >= 2 and self.marks[0] <= r[0] <= self.marks[1]]
+        p_max = max((r[2] for r in rows), default=0.0)
+        loaded = [r for r in rows if r[2] >= 0.5 * p_max]
+        use = timed if timed else loaded
+        reasons = set()
+        for r in use:
+            for bit, name in names.items():
+                if r[3] & bit:
                     reasons.add(name)
-        p_max = max((p for _, p in rows), default=0.0)
-        loaded = [c for c, p in rows if p >= 0.5 * p_max]
-        return {"sm_mhz": statistics.median(loaded) if loaded else None,
-                "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(loaded), "samples_total": len(rows),
-                "power_w_max": p_max}
+        return {"sm_mhz": statistics.median([r[1] for r in use]) if use else None,
+                "sm_max_mhz": self.smax, "reasons": sorted(reasons),
+                "samples": len(use), "samples_in_timed_region": len(timed), "samples_total": len(rows),
+                "power_w_max": p_max, "source": self.mode}
 
 
 def _dist_env():
@@ -328,6 +377,8 @@ def run_ours(args):
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
+    if rank == 0:
+        sampler.mark()
     t_wall0 = time.perf_counter()
     for i in range(args.steps):
         flush_l2()
@@ -336,6 +387,8 @@ def run_ours(args):
         ends[i].record(stream)
     barrier()
     t_wall = time.perf_counter() - t_wall0
+    if rank == 0:
+        sampler.mark()
     step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
     total_ms = sum(step_ms)
     verified = int(acc.sum().item()) + batch                              # tau + 1 tokens per sequence
