@@ -139,7 +139,7 @@ __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
-// 2-D tiled load, no multicast.  c0 is the innermost coordinate (elements): c0 * elem_size
+// 2-D tiled load into this CTA only.  c0 is the innermost coordinate (elements): c0 * elem_size
 // must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar,
                                             int32_t c0, int32_t c1, uint64_t policy)
