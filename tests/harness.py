@@ -105,9 +105,10 @@ class Case:
 def make_verifier(case: Case, debug=True, mode=None):
     from paper_2601_00644_b200 import binding
     s = case.shape
+    k_max = max(int(case.k.max()), 1)
     return binding.Verifier(case.inp.lm_head_w, s.n_q_heads, s.n_kv_heads, s.head_dim,
-                            max_batch=case.batch, k_max=max(int(case.k.max()), 1),
-                            max_kv_len=int(case.kv_len.max()), mode=case.mode if mode is None else mode,
+                            max_batch=case.batch, k_max=k_max,
+                            max_kv_len=max(int(case.kv_len.max()), k_max + 1), mode=case.mode if mode is None else mode,
                             debug=debug)
 
 

@@ -91,3 +91,87 @@ def test_kv_release_matches_oracle():
     torch.cuda.synchronize()
     assert ver.status()[0] == B.ERR_INVALID_ARG
     ver.close()
+
+
+def test_serving_loop_append_verify_rollback_release():
+    """Three consecutive steps of one batch, as a serving loop would run them (Section IV-C and Algorithm 2):
+    hand pages to the sequences that need them, append the window's K/V, verify, roll kv_len back,
+    release the pages past it, draft again from the new length.  Every step's pool, attention output,
+    decisions, lengths, page table and released pages are compared with the oracle run on the same state."""
+    import tests.harness as H
+    from paper_2601_00644_b200 import binding as B
+    rng = np.random.RandomState(91)
+    Hq, Hkv, Dh, V, batch, k_max = 8, 2, 64, 2048, 5, 4
+    d = Hq * Dh
+    max_pages = 12
+    num_pages = batch * max_pages
+    gen = torch.Generator(device="cuda").manual_seed(91)
+    w = (torch.randn(V, d, generator=gen, device="cuda") * 0.05).to(torch.bfloat16)
+    pool = torch.randn(num_pages, 2, Hkv, 16, Dh, generator=gen, device="cuda").to(torch.bfloat16)
+    ver = B.Verifier(w, Hq, Hkv, Dh, max_batch=batch, k_max=k_max, max_kv_len=max_pages * 16, debug=True)
+    pt_h = np.full((batch, max_pages), -1, np.int32)             # nobody owns a page yet
+    free_h = rng.permutation(num_pages).astype(np.int32)         # the free list holds them all
+    n_free = num_pages
+    ctx = rng.randint(3, 60, batch).astype(np.int32)             # committed context per sequence
+    seeds = torch.from_numpy(rng.randint(0, 2 ** 62, batch).astype(np.int64)).cuda()
+    seeds_h = seeds.cpu().numpy().view(np.uint64)
+    released_total = 0
+    for step in range(3):
+        k = rng.randint(0, k_max + 1, batch).astype(np.int32)
+        kv_len = (ctx + k + 1).astype(np.int32)
+        # the serving loop hands pages from the free list to the sequences whose window needs them
+        for b in range(batch):
+            for i in range(-(-int(kv_len[b]) // 16)):
+                if pt_h[b, i] < 0:
+                    n_free -= 1
+                    pt_h[b, i] = free_h[n_free]
+        pt = torch.from_numpy(pt_h).cuda()
+        free = torch.from_numpy(free_h).cuda()
+        free_n = torch.tensor([n_free], dtype=torch.int32, device="cuda")
+        m, s = int(k.sum()) + batch, int(k.sum())
+        hidden = torch.randn(m, d, generator=gen, device="cuda").to(torch.bfloat16)
+        new_k = torch.randn(m, Hkv, Dh, generator=gen, device="cuda").to(torch.bfloat16)
+        new_v = torch.randn(m, Hkv, Dh, generator=gen, device="cuda").to(torch.bfloat16)
+        zd = torch.randn(max(s, 1), V, generator=gen, device="cuda")[:s] * 2
+        toks = torch.from_numpy(rng.randint(0, V, s).astype(np.int32)).cuda()
+        k_d, kv_d = torch.from_numpy(k).cuda(), torch.from_numpy(kv_len).cuda()
+        pool_before = wl.bits_u16(pool)
+        ver.kv_append(pool, pt, kv_d, torch.from_numpy(kv_len), new_k, new_v, k_d, torch.from_numpy(k))
+        acc, nxt = ver.verify(pool, pt, kv_d, torch.from_numpy(kv_len), hidden, toks, zd, k_d, torch.from_numpy(k), seeds)
+        kv_next = ver.kv_rollback(kv_d, k_d, acc)
+        ver.kv_release(pt, num_pages, kv_d, kv_next, free, free_n)
+        torch.cuda.synchronize()
+        assert ver.status()[0] == 0
+        # ---- the oracle on the same state
+        want_pool = oracle.kv_append(pool_before, pt_h, kv_len, k, wl.bits_u16(new_k), wl.bits_u16(new_v), Hkv, Dh)
+        assert np.array_equal(wl.bits_u16(pool), want_pool)
+        ref = oracle.verify(oracle.SAMPLE, wl.bits_u16(hidden), want_pool, pt_h, kv_len, k, wl.bits_u16(w),
+                            toks.cpu().numpy(), zd.cpu().numpy(), seeds_h, Hq, Hkv, Dh)
+        dbg = ver.debug(m, s)
+        err, ok = H.rel_close(dbg["attn_out"].float().cpu().numpy(), ref["attn_f64"])
+        assert ok and err < H.REL_TOL
+        iso = oracle.accept(oracle.SAMPLE, dbg["logits"].cpu().numpy().astype(np.float64), zd.cpu().numpy(), toks.cpu().numpy(),
+                            k, seeds_h)
+        acc_h, nxt_h = acc.cpu().numpy(), nxt.cpu().numpy()
+        t0 = np.concatenate([[0], np.cumsum(k)])
+        for b in range(batch):                                  # the oracle on the same logits: identical except at near-ties
+            if acc_h[b] != iso["accepted_len"][b]:
+                assert iso["acc_margin"][t0[b] + min(acc_h[b], iso["accepted_len"][b])] < H.TIE_TOL
+            elif nxt_h[b] != iso["next_token"][b]:
+                assert iso["cdf_margin"][b] < H.CDF_TIE_TOL
+        kv_next_h = kv_next.cpu().numpy()
+        assert np.array_equal(kv_next_h, oracle.kv_rollback(kv_len, k, acc_h))
+        want_pt, want_freed = oracle.kv_release(pt_h, kv_len, kv_next_h)
+        assert np.array_equal(pt.cpu().numpy(), want_pt)
+        n_after = int(free_n.item())
+        assert n_after - n_free == len(want_freed)
+        assert sorted(free.cpu().numpy()[n_free:n_after].tolist()) == sorted(want_freed.tolist())
+        released_total += len(want_freed)
+        # the next step starts from the committed context + accepted drafts + the emitted token's position
+        pt_h, free_h, n_free = want_pt, free.cpu().numpy(), n_after
+        ctx = kv_next_h.astype(np.int32)
+    # every page is either owned by exactly one sequence or on the free list
+    owned = pt_h[pt_h >= 0]
+    assert len(set(owned.tolist())) == len(owned)
+    assert set(owned.tolist()).isdisjoint(set(free_h[:n_free].tolist())) and len(owned) + n_free == num_pages
+    ver.close()

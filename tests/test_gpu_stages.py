@@ -428,3 +428,34 @@ def test_stage_outputs_stay_inside_their_buffers():
     assert H.guards_intact(a_w, m * d) and H.guards_intact(l_w, m * v)
     assert int((l.view(torch.int32) == H.CANARY).sum()) == 0                # and everything inside was written
     ver.close()
+
+
+# ------------------------------------------------------------------ attention over a sweep of seeded shapes
+
+def _random_attention_shapes():
+    """Seeded shapes that walk through every kernel instance and both cuts of the work list: head dims 64 / 128,
+    group sizes 1..16, tiles of 1..128 query rows (one, two or three threads per token, single P^T buffer),
+    contexts from empty to several blocks per CTA, batches from one sequence to more pairs than SMs."""
+    rng = np.random.RandomState(20260106)
+    shapes = []
+    for i in range(14):
+        head_dim = int(rng.choice([64, 128]))
+        n_kv = int(rng.choice([1, 2, 4, 8]))
+        group = int(rng.choice([1, 2, 4, 8, 16]))
+        k_hi = int(rng.choice([0, 1, 3, 7, 12, 20]))
+        k_hi = min(k_hi, 128 // group * 2)                 # up to two row blocks per kv head
+        ctx_hi = int(rng.choice([0, 50, 400, 1500, 4000]))
+        batch = int(rng.choice([1, 2, 5, 24]))
+        if batch * ctx_hi * n_kv * head_dim > 24 * 1500 * 8 * 64:   # keep the oracle within a second or two
+            ctx_hi = 400
+        shapes.append(dict(batch=batch, n_q_heads=n_kv * group, n_kv_heads=n_kv, head_dim=head_dim, k_min=0, k_max=k_hi,
+                           ctx_min=0, ctx_max=ctx_hi, input_std=float(rng.choice([0.02, 1.0])), idx=400 + i))
+    return shapes
+
+
+@pytest.mark.parametrize("kw", _random_attention_shapes(), ids=lambda kw: "b%dh%dx%dd%dk%dc%d" % (
+    kw["batch"], kw["n_kv_heads"], kw["n_q_heads"] // kw["n_kv_heads"], kw["head_dim"], kw["k_max"], kw["ctx_max"]))
+def test_attention_sweep_matches_oracle(kw):
+    kw = dict(kw)
+    idx = kw.pop("idx")
+    _attn_parity(_shape("att_sweep", idx, **kw))
