@@ -367,7 +367,7 @@ int run_sample(Handle& h, const float* logits, const int32_t* draft_tokens, cons
     if (launch_sample_stats(p, 0, p.greedy ? p.m_rows : p.m_rows + p.s_rows, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     if (p.filtered) {
-        if (launch_sample_filter(p, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+        if (launch_sample_filter(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
     }
     if (launch_sample_accept(p, false, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
@@ -646,11 +646,11 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);
     if (sp.filtered) {
-        if (launch_sample_filter(sp, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;      // the plan's tables are there: joined above
+        if (launch_sample_filter(sp, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;   // the plan's tables are there: joined above
         h.launches++;
     }
     mark(h, 5, s);
-    if (launch_sample_accept(sp, !sp.filtered, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_accept(sp, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 6, s);
     return FLEXSPEC_OK;

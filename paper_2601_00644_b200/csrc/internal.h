@@ -180,7 +180,7 @@ cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHe
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
 // pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
 // the stream drains; it waits on the device before touching the predecessor's results)
-cudaError_t launch_sample_filter(const SampleParams& p, cudaStream_t stream);
+cudaError_t launch_sample_filter(const SampleParams& p, bool pdl, cudaStream_t stream);
 cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream);
 
 template <typename... KArgs, typename... Args>

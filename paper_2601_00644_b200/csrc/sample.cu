@@ -184,24 +184,44 @@ __device__ __forceinline__ void cp_async_wait_all()
 // is applied first.  Both filters are thresholds on the logit: the kept set of a row is
 // {v : z_v >= tau}, tau being the k-th largest logit (top-k; ties with it are kept), respectively the
 // largest logit such that the tokens with logit >= tau hold at least top_p of the (top-k filtered)
-// mass.  tau is found exactly by a radix selection over the order-preserving 32-bit keys of the
-// logits, 8 bits per round, the weight of a key being 1 (top-k) or its probability mass (top-p).
+// mass.  tau is found exactly by a selection over an order-preserving 32-bit code of the logits:
+// round after round the interval of codes that can still hold tau is cut into up to 256 bins, every
+// live entry adds its weight (1 for top-k, its probability mass for top-p) to the bin of its code,
+// and a walk over the bins from the largest logits down finds the bin in which the running weight
+// reaches the target.  As soon as that bin holds at most kFilterCand entries they are collected and
+// ranked directly, which ends the selection.
 //
-// One cluster of eight CTAs per target row; every CTA keeps its slice of the row in shared memory
-// (one read of the logits for all rounds).  Per round each CTA builds a 256-bin histogram of its
-// slice, restricted to the keys that match the prefix found so far; after one cluster barrier every
-// CTA adds up the eight histograms (read from its peers' shared memory; histograms alternate
-// between two buffers, so one barrier per round is enough) and walks from the top bin down to the
-// bin in which the running weight reaches the target.  Masses are accumulated as fixed-point integers
-// (2^((z - max) c) rounded to units of 2^-31, added as two 16-bit limbs with the native 32-bit
-// shared-memory atomics; 64-bit shared-memory atomics were measured 15x slower): integer addition is
-// exact and order-independent, so the histograms, the totals and the comparison with the target are
-// the same whatever the order of the atomic adds, and a row's result does not depend on scheduling.
-// The rounding of one entry is at most 2^-32 and unbiased: over a 128 K row its sum stays near 1e-8 of
-// the mass.
+// The code of an entry is the bit pattern of d = m - z (m = the row maximum, known from the softmax
+// statistics of the row, so no pass over the row is spent on it): a non-negative float, whose bit
+// pattern grows with d.  Bins cut from it are equally wide on a logarithmic scale of the distance to
+// the maximum, whatever the scale of the logits, which spreads flat rows (all logits within 1e-2) and
+// peaked rows alike over dozens of bins, where the leading byte of the logit itself puts most of a
+// row into a handful of bins and its shared-memory atomics into one another's way.  Distinct logits
+// can round to the same d; should such a group ever hold more than kFilterCand entries, the selection
+// carries on over the bit pattern of z itself inside the group (second phase), so that the result is
+// exact in every case.
+//
+// One cluster of eight CTAs per target row, a contiguous slice of the vocabulary per CTA.  The first
+// round reads the slice from global memory (the one read of the logits that comes from DRAM) and
+// leaves every entry's first-round bin in shared memory, one byte per entry; the later rounds scan
+// these bytes and fetch only the logits whose byte lies in the live range (a few percent, out of
+// L2).  A round ends with one cluster barrier, after which every CTA adds up the eight histograms
+// (read from its peers' shared memory; histograms alternate between two buffers, so one barrier per
+// round is enough) and walks them; all CTAs reach the same result, so nothing is broadcast.
+// Masses are accumulated as fixed-point integers (2^((z - m) c) rounded to units of 2^-31, added as
+// two 16-bit limbs with the native 32-bit shared-memory atomics; 64-bit shared-memory atomics were
+// measured 15x slower): integer addition is exact and order-independent, so the histograms, the
+// totals and the comparison with the target are the same whatever the order of the atomic adds, and
+// a row's result does not depend on scheduling.  The rounding of one entry is at most 2^-32 and
+// unbiased: over a 128 K row its sum stays near 1e-8 of the mass.
 constexpr int kFilterThreads = 256;
 constexpr int kFilterWarps = kFilterThreads / 32;
-constexpr int kFilterSliceMax = 16384;                    // entries of a slice kept in shared memory (64 KB)
+constexpr int kFilterCodesMax = 16384;                    // entries of a slice whose first-round bin is kept in shared memory
+constexpr int kFilterList = 1024;                         // live entries of a slice listed after the first round
+constexpr int kFilterCand = 128;                          // a bin with at most this many entries is ranked directly
+constexpr int kFilterMaxRounds = 32;                      // (a selection needs at most 13: see the walk)
+constexpr int kFilterShift0 = 18;                         // first round: exponent and five mantissa bits of d, ...
+constexpr int kFilterOctaves = 8;                         // ... a window of eight octaves of d
 constexpr double kMassUnit = 2147483648.0;                // 2^31
 constexpr float kMassUnitF = 2147483648.0f;
 
@@ -215,205 +235,413 @@ __device__ __forceinline__ float key_to_float(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-struct FilterShared {
-    uint32_t hist[2][2][256];                           // [buffer][top-k: count | top-p: mass limbs (bits 16..31, bits 0..15)][bin]
-    unsigned long long tot[256];                        // cluster-wide histogram of the round (the weight that decides)
-    uint32_t red[kFilterWarps];
-    unsigned long long red64[kFilterWarps];
-    uint32_t slice_max[kAcceptCluster];
-    unsigned long long slice_mass[kAcceptCluster];
-    uint32_t prefix;                                    // key bits fixed so far
-    unsigned long long above;                           // weight of the keys above the prefix's bin path
+// what a round of the selection looks at (identical in the eight CTAs of a row)
+struct FilterRound {
+    uint32_t lo, hi;                                    // live codes: lo <= code <= hi
+    uint32_t base;                                      // bin = clamp((code >> shift) - base, 0, 255)
+    int shift;
+    int phase;                                          // 0: code = bits of (m - z);  1: code = ~key(z) among the entries with bits of (m - z) == dsel
+    uint32_t dsel;
+    int next;                                           // after the walk: 0 another round, 1 collect and rank, 2 tau is known
+    uint32_t n_sel;                                     // entries in the chosen bin (when the round counted them)
+    unsigned long long above;                           // weight of the codes below lo (the logits above the live interval)
     unsigned long long target;
-    int bin;
+    float tau;
+    unsigned long long kept;
 };
 
-// 2^((z - m) c) in fixed point (units of 2^-31, round to nearest), z given by its key
-__device__ __forceinline__ uint32_t key_mass(uint32_t key, float m, float cf)
+struct FilterShared {
+    uint32_t hist[2][3][256];                           // [buffer][mass bits 16..31 | mass bits 0..15 | entries][bin]
+    unsigned long long tot[256];                        // cluster-wide weight per bin
+    uint32_t totc[256];                                 // cluster-wide entries per bin
+    float cand_z[kFilterCand];
+    uint32_t cand_w[kFilterCand];
+    float red_hi[kFilterWarps], red_lo[kFilterWarps];
+    float slice_hi[kAcceptCluster], slice_lo[kAcceptCluster];
+    unsigned long long red64[kFilterWarps];
+    unsigned long long slice_mass[kAcceptCluster];
+    uint32_t n_cand;
+    uint32_t list_n;
+    FilterRound r;
+};
+
+// 2^(-d c) in fixed point (units of 2^-31, round to nearest), d = m - z >= 0
+__device__ __forceinline__ uint32_t mass_of(float d, float cf)
 {
-    return __float2uint_rn(fast_exp2((key_to_float(key) - m) * cf) * kMassUnitF);   // <= 2^31
+    return __float2uint_rn(fast_exp2(d * -cf) * kMassUnitF);   // <= 2^31
+}
+__device__ __forceinline__ int bin_of(uint32_t code, int shift, uint32_t base)
+{
+    const uint32_t t = code >> shift;
+    return t <= base ? 0 : static_cast<int>(min(t - base, 255u));
 }
 
-__global__ void __cluster_dims__(kAcceptCluster, 1, 1) __launch_bounds__(kFilterThreads)
+__global__ void __cluster_dims__(kAcceptCluster, 1, 1) __launch_bounds__(kFilterThreads, 6)
 sample_filter_kernel(const SampleParams p)
 {
-    extern __shared__ uint32_t s_keys[];                // this CTA's slice of the row as order-preserving keys (when it fits)
+    extern __shared__ __align__(16) uint8_t s_bin0[];   // first-round bin of every entry of this CTA's slice (when it fits), ...
     __shared__ FilterShared sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = static_cast<int>(cluster.block_rank());
     const int row = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float cf = p.row_c[row];
-    const uint32_t* mask_row = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(p.row_seq[row]) * p.mask_words : nullptr;
-    const float* src = p.logits + static_cast<int64_t>(row) * p.vocab;
     cluster_arrive();                                   // "this CTA runs" (awaited before the first peer access)
 
-    // ---- this CTA's slice: [v0, v1), a multiple of four entries long so that 16-byte copies stay aligned
+    // ---- this CTA's slice: [v0, v1), a multiple of four entries long so that 16-byte loads stay aligned
     const int per = ((p.vocab + kAcceptCluster - 1) / kAcceptCluster + 3) & ~3;
     const int v0 = min(p.vocab, rank * per), v1 = min(p.vocab, v0 + per);
     const int n = v1 - v0;
-    const bool staged = per <= kFilterSliceMax;
+    const bool coded = per <= kFilterCodesMax;
+    uint16_t* s_idx = reinterpret_cast<uint16_t*>(s_bin0 + per);                       // ... the listed entries' indices ...
+    float* s_list = reinterpret_cast<float*>(s_bin0 + per + kFilterList * sizeof(uint16_t));   // ... and their logits
     const bool vec_ok = ((p.vocab & 3) == 0);
-    // key of entry i of the slice: 0 for entries that cannot be selected (masked, -inf), else > 0 and ordered like the logits
-    auto make_key = [&](float z, int i) -> uint32_t {
-        if (z == -INFINITY || (mask_row != nullptr && !mask_allows(mask_row, v0 + i))) return 0u;
-        return order_key(z);
-    };
-    if (staged) {
-        float* s_f = reinterpret_cast<float*>(s_keys);
-        if (vec_ok) {
-            for (int i = tid * 4; i < n; i += kFilterThreads * 4) cp_async_16(s_f + i, src + v0 + i);
-        } else {
-            for (int i = tid; i < n; i += kFilterThreads) cp_async_4(s_f + i, src + v0 + i);
+    for (int i = tid; i < 3 * 256; i += kFilterThreads) (&sh.hist[0][0][0])[i] = 0u;
+    if (tid == 0) sh.n_cand = 0u;
+    pdl_wait();                                         // the logits and their statistics come from the preceding kernel
+    pdl_launch_dependents();
+    const float cf = p.row_c[row];
+    const uint32_t* mask_row = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(p.row_seq[row]) * p.mask_words : nullptr;
+    const float* src = p.logits + static_cast<int64_t>(row) * p.vocab + v0;
+
+    // ---- row maximum m and the spread of the part maxima, from the row's softmax statistics (each CTA
+    // reads an eighth of the parts; the slice results are exchanged through the peers' shared memory)
+    {
+        const float2* tp = p.tstats + static_cast<int64_t>(row) * p.n_tparts;
+        float hi = -INFINITY, lo = INFINITY;
+        for (int t = rank * kFilterThreads + tid; t < p.n_tparts; t += kAcceptCluster * kFilterThreads) {
+            const float x = __ldcg(&tp[t].x);
+            hi = fmaxf(hi, x);
+            if (x > -INFINITY) lo = fminf(lo, x);
         }
-        cp_async_wait_all();
+        hi = warp_max(hi);
+        lo = -warp_max(-lo);
+        if (lane == 0) { sh.red_hi[warp] = hi; sh.red_lo[warp] = lo; }
         __syncthreads();
-        for (int i = tid; i < n; i += kFilterThreads) s_keys[i] = make_key(s_f[i], i);     // once, in place
-        __syncthreads();
-    }
-    auto key_at = [&](int i) -> uint32_t { return staged ? s_keys[i] : make_key(__ldg(src + v0 + i), i); };
-
-    // ---- row maximum (the largest key): slice maxima, exchanged through the peers' shared memory
-    uint32_t kmax = 0u;
-    for (int i = tid; i < n; i += kFilterThreads) kmax = max(kmax, key_at(i));
-    kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) sh.red[warp] = kmax;
-    __syncthreads();
-    cluster_wait();                                     // all eight CTAs have started
-    if (tid < kAcceptCluster) {
-        uint32_t mm = sh.red[0];
+        cluster_wait();                                 // all eight CTAs have started
+        if (tid < kAcceptCluster) {
 #pragma unroll
-        for (int w = 1; w < kFilterWarps; ++w) mm = max(mm, sh.red[w]);
-        cluster.map_shared_rank(&sh.slice_max[0], tid)[rank] = mm;
+            for (int w = 0; w < kFilterWarps; ++w) { hi = fmaxf(hi, sh.red_hi[w]); lo = fminf(lo, sh.red_lo[w]); }
+            cluster.map_shared_rank(&sh.slice_hi[0], tid)[rank] = hi;
+            cluster.map_shared_rank(&sh.slice_lo[0], tid)[rank] = lo;
+        }
+        cluster_sync();
     }
-    cluster_sync();
-    kmax = sh.slice_max[0];
+    float m = sh.slice_hi[0], part_lo = sh.slice_lo[0];
 #pragma unroll
-    for (int c = 1; c < kAcceptCluster; ++c) kmax = max(kmax, sh.slice_max[c]);
-    const float m = key_to_float(kmax);
+    for (int c = 1; c < kAcceptCluster; ++c) { m = fmaxf(m, sh.slice_hi[c]); part_lo = fminf(part_lo, sh.slice_lo[c]); }
+    if (m == -INFINITY) {                               // nothing can be selected in this row
+        if (rank == 0 && tid == 0) {
+            p.topp[static_cast<int64_t>(row) * 2] = -static_cast<double>(INFINITY);
+            p.topp[static_cast<int64_t>(row) * 2 + 1] = 0.0;
+        }
+        cluster_sync();
+        return;
+    }
+    // first-round window: eight octaves of d = m - z, the top one a few octaves above the spread of the
+    // part maxima (the maxima of small parts spread almost like the row, those of large parts much
+    // less).  A window that misses only costs rounds: its end bins take what lies outside.
+    uint32_t base0;
+    {
+        const float spread = m - part_lo;
+        int e_top = 127 + 6;
+        if (spread > 0.f && spread < INFINITY)
+            e_top = static_cast<int>(__float_as_uint(spread) >> 23) + ((p.vocab / max(p.n_tparts, 1) >= 1024) ? 5 : 3);
+        e_top = min(max(e_top, kFilterOctaves), 254);
+        base0 = static_cast<uint32_t>(e_top - (kFilterOctaves - 1)) << (23 - kFilterShift0);
+    }
 
-    // ---- selections: top-k on counts (if on), then top-p on mass among the keys that survived
     const bool do_k = p.top_k > 0 && p.top_k < p.vocab;
     const bool do_p = p.top_p < 1.f;
-    uint32_t floor_key = 1u;                            // keys below it are out: 0 = not selectable, later the top-k cut
-    double kept_mass = 0.0;
+    float floor_z = -3.402823466e38f;                   // logits below it are out: first "finite", later the top-k cut
+    bool bytes_valid = false;
     int round_no = 0;                                   // alternates the histogram buffers
-    for (int sel = do_k ? 0 : 1; sel < (do_p ? 2 : 1); ++sel) {
-        // sel 0: weight 1, target k.   sel 1: weight mass, target top_p * (mass of the keys >= floor_key)
-        if (tid == 0) { sh.prefix = 0u; sh.above = 0ull; }
-        __syncthreads();
-        for (int round = 0; round < 4; ++round, ++round_no) {
-            const int shift = 24 - 8 * round;
-            const int buf = round_no & 1;
-            for (int i = tid; i < 2 * 256; i += kFilterThreads) (&sh.hist[buf][0][0])[i] = 0u;
-            __syncthreads();
-            const uint32_t prefix = sh.prefix;
-            const uint32_t hi_mask = (round == 0) ? 0u : (0xffffffffu << (shift + 8));
-            const uint32_t want = prefix & hi_mask;
-            // four entries per thread and step.  A step in which no lane holds a live key (most steps after
-            // the first round) costs a load and a compare per entry.  When all lanes of the warp fall into
-            // the same bin (the leading bytes of flat logits) the warp adds once, one reduction per limb.
-            for (int i0 = 0; i0 < n; i0 += kFilterThreads * 4) {
-                uint32_t key[4];
-                bool live[4];
-                bool any = false;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * kFilterThreads + tid;
-                    key[u] = (i < n) ? key_at(i) : 0u;
-                    live[u] = key[u] >= floor_key && (key[u] & hi_mask) == want;
-                    any |= live[u];
-                }
-                if (!__any_sync(0xffffffffu, any)) continue;
-                int bin[4];
-                uint32_t w[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    bin[u] = live[u] ? static_cast<int>((key[u] >> shift) & 255u) : -1;
-                    w[u] = !live[u] ? 0u : (sel == 0 ? 1u : key_mass(key[u], m, cf));
-                }
-                const int bin0 = __shfl_sync(0xffffffffu, bin[0], 0);
-                if (__all_sync(0xffffffffu, bin[0] == bin0 && bin[1] == bin0 && bin[2] == bin0 && bin[3] == bin0)) {
-                    // (all 128 entries live and in one bin; limb sums stay far below 2^32)
-                    const uint32_t a0 = __reduce_add_sync(0xffffffffu, sel == 0 ? 4u : (w[0] >> 16) + (w[1] >> 16) + (w[2] >> 16) + (w[3] >> 16));
-                    const uint32_t a1 = sel == 0 ? 0u : __reduce_add_sync(0xffffffffu, (w[0] & 0xffffu) + (w[1] & 0xffffu) + (w[2] & 0xffffu) + (w[3] & 0xffffu));
-                    if (lane == 0) {
-                        atomicAdd(&sh.hist[buf][0][bin0], a0);
-                        if (sel == 1) atomicAdd(&sh.hist[buf][1][bin0], a1);
-                    }
-                } else {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (live[u]) {
-                            if (sel == 0) {
-                                atomicAdd(&sh.hist[buf][0][bin[u]], 1u);
-                            } else {
-                                atomicAdd(&sh.hist[buf][0][bin[u]], w[u] >> 16);
-                                atomicAdd(&sh.hist[buf][1][bin[u]], w[u] & 0xffffu);
-                            }
-                        }
+
+    // one logit that may be live: test it, add it to the histogram or hand it over as a candidate
+    auto consider = [&](float z, int sel, const FilterRound& r, uint32_t* hist, bool collect) {
+        if (!(z >= floor_z)) return;
+        const float d = m - z;
+        const uint32_t dbits = __float_as_uint(d);
+        uint32_t code = dbits;
+        if (r.phase != 0) {
+            if (dbits != r.dsel) return;
+            code = ~order_key(z);
+        }
+        if (code - r.lo > r.hi - r.lo) return;
+        const uint32_t w = sel == 0 ? 1u : mass_of(d, cf);
+        if (collect) {
+            const uint32_t idx = atomicAdd(cluster.map_shared_rank(&sh.n_cand, 0), 1u);
+            if (idx < static_cast<uint32_t>(kFilterCand)) {
+#pragma unroll 1
+                for (int c = 0; c < kAcceptCluster; ++c) {
+                    cluster.map_shared_rank(&sh.cand_z[0], c)[idx] = z;
+                    cluster.map_shared_rank(&sh.cand_w[0], c)[idx] = w;
                 }
             }
+        } else {
+            const int bin = bin_of(code, r.shift, r.base);
+            if (sel != 0) {
+                atomicAdd(&hist[bin], w >> 16);
+                atomicAdd(&hist[256 + bin], w & 0xffffu);
+            }
+            atomicAdd(&hist[512 + bin], 1u);
+        }
+    };
+    auto fetch = [&](int i) -> float {                  // entry i of the slice, -inf when it is masked out
+        const float z = __ldg(src + i);
+        return (mask_row != nullptr && !mask_allows(mask_row, v0 + i)) ? -INFINITY : z;
+    };
+    // A pass over the slice for the round r.  The stored first-round bins tell which entries can be live; the
+    // first such pass of a selection lists them (index, then value: the fetches of a round are all in flight
+    // together instead of one after the other in a thread), and the later passes, whose live sets lie inside
+    // that one, walk the list.  A list that does not fit sends the selection back to scanning.
+    int list_state = 0;                                 // 0 none yet, 1 valid, 2 did not fit
+    auto scan = [&](int sel, const FilterRound& r, uint32_t* hist, bool collect) {
+        if (list_state == 1) {
+            const int nl = static_cast<int>(sh.list_n);
+            for (int j = tid; j < nl; j += kFilterThreads) consider(s_list[j], sel, r, hist, collect);
+            return;
+        }
+        if (!bytes_valid) {
+#pragma unroll 1
+            for (int i = tid; i < n; i += kFilterThreads) consider(fetch(i), sel, r, hist, collect);
+            return;
+        }
+        const uint32_t b_lo = static_cast<uint32_t>(bin_of(r.phase == 0 ? r.lo : r.dsel, kFilterShift0, base0));
+        const uint32_t b_span = static_cast<uint32_t>(bin_of(r.phase == 0 ? r.hi : r.dsel, kFilterShift0, base0)) - b_lo;
+        const uint32_t lo4 = b_lo * 0x01010101u, span4 = b_span * 0x01010101u;
+        // the bytes of a word that lie in the live range, four at a time (0xff where they do)
+        auto hits_of = [&](int i0) -> uint32_t {
+            const uint32_t b4 = *reinterpret_cast<const uint32_t*>(s_bin0 + i0);
+            uint32_t hits = __vcmpleu4(__vsub4(b4, lo4), span4);
+            if (i0 + 4 > n) hits &= (1u << (8 * (n - i0))) - 1u;
+            return hits;
+        };
+        if (list_state == 0) {
+            // count this thread's hits, reserve room for the warp's with one atomic, then write the indices
+            uint32_t mine = 0u;
+#pragma unroll 1
+            for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) mine += __popc(hits_of(i0) & 0x01010101u);
+            uint32_t incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t0 = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t0;
+            }
+            uint32_t at = 0u;
+            if (lane == 31) at = atomicAdd(&sh.list_n, incl);
+            at = __shfl_sync(0xffffffffu, at, 31) + incl - mine;
+            if (mine != 0u) {
+#pragma unroll 1
+                for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) {
+                    uint32_t hits = hits_of(i0);
+                    while (hits != 0u) {
+                        const int u = (__ffs(hits) - 1) >> 3;
+                        hits &= ~(0xffu << (8 * u));
+                        if (at < static_cast<uint32_t>(kFilterList)) s_idx[at] = static_cast<uint16_t>(i0 + u);
+                        ++at;
+                    }
+                }
+            }
+            __syncthreads();
+            const uint32_t total = sh.list_n;
+            if (total <= static_cast<uint32_t>(kFilterList)) {
+                list_state = 1;
+                for (int j = tid; j < static_cast<int>(total); j += kFilterThreads) {
+                    const float z = fetch(s_idx[j]);
+                    s_list[j] = z;
+                    consider(z, sel, r, hist, collect);
+                }
+                return;
+            }
+            list_state = 2;
+        }
+#pragma unroll 1
+        for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) {
+            uint32_t hits = hits_of(i0);
+            while (hits != 0u) {
+                const int u = (__ffs(hits) - 1) >> 3;
+                hits &= ~(0xffu << (8 * u));
+                consider(fetch(i0 + u), sel, r, hist, collect);
+            }
+        }
+    };
+
+    // ---- selections: top-k on counts (if on), then top-p on mass among the logits that survived
+    for (int sel = do_k ? 0 : 1; sel < (do_p ? 2 : 1); ++sel) {
+        // sel 0: weight 1, target k.   sel 1: weight mass, target top_p * (mass of the logits >= floor_z)
+        if (tid == 0) {
+            FilterRound r0;
+            r0.lo = 0u; r0.hi = min(0x7f800000u, __float_as_uint(m - floor_z));   // every d >= 0 down to the floor
+            r0.base = base0; r0.shift = kFilterShift0; r0.phase = 0; r0.dsel = 0u; r0.next = 0; r0.n_sel = 0u;
+            r0.above = 0ull; r0.target = 0ull; r0.tau = floor_z; r0.kept = 0ull;
+            sh.r = r0;
+            sh.list_n = 0u;
+        }
+        __syncthreads();
+        bool first = true;                              // first round of the selection: its total fixes the target
+        list_state = 0;
+        for (int it = 0; it < kFilterMaxRounds; ++it, ++round_no) {
+            const FilterRound r = sh.r;
+            uint32_t* hist = &sh.hist[round_no & 1][0][0];
+            bool counted = true;                        // the round records how many entries each bin holds
+            if (!bytes_valid && first) {
+                // the first pass of the kernel: every entry of the slice, straight from global memory; leaves the
+                // bins in shared memory.  For top-p the entry count is left out (two atomics per entry, not three).
+                counted = sel == 0;
+#pragma unroll 2
+                for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) {
+                    float z[4];
+                    if (vec_ok) {
+                        const float4 x = __ldg(reinterpret_cast<const float4*>(src + i0));
+                        z[0] = x.x; z[1] = x.y; z[2] = x.z; z[3] = x.w;
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) z[u] = (i0 + u < n) ? __ldg(src + i0 + u) : -INFINITY;
+                    }
+                    if (mask_row != nullptr) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (i0 + u < n && !mask_allows(mask_row, v0 + i0 + u)) z[u] = -INFINITY;
+                    }
+                    uint32_t b4 = 0u;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float d = m - z[u];
+                        const uint32_t dbits = __float_as_uint(d);
+                        const bool live = z[u] >= floor_z && dbits <= 0x7f800000u;
+                        const int bin = live ? bin_of(dbits, kFilterShift0, base0) : 255;
+                        b4 |= static_cast<uint32_t>(bin) << (8 * u);
+                        if (live) {
+                            if (sel == 0) {
+                                atomicAdd(&hist[512 + bin], 1u);
+                            } else {
+                                const uint32_t w = mass_of(d, cf);
+                                atomicAdd(&hist[bin], w >> 16);
+                                atomicAdd(&hist[256 + bin], w & 0xffffu);
+                            }
+                        }
+                    }
+                    if (coded) *reinterpret_cast<uint32_t*>(s_bin0 + i0) = b4;
+                }
+                bytes_valid = coded;
+            } else {
+                scan(sel, r, hist, false);
+            }
             cluster_sync();                             // all eight histograms of this round are complete
-            // cluster-wide histogram: thread t adds bin t of the eight CTAs
+            // cluster-wide histogram: thread t adds bin t of the eight CTAs; the other buffer is cleared for the
+            // next round (its last readers arrived at the barrier above after they were done with it)
             {
                 unsigned long long acc = 0ull;
+                uint32_t cnt = 0u;
 #pragma unroll
                 for (int c = 0; c < kAcceptCluster; ++c) {
-                    const uint32_t* peer = cluster.map_shared_rank(&sh.hist[buf][0][0], c);
-                    acc += sel == 0 ? static_cast<unsigned long long>(peer[tid])
-                                    : (static_cast<unsigned long long>(peer[tid]) << 16) + peer[256 + tid];
+                    const uint32_t* peer = cluster.map_shared_rank(hist, c);
+                    if (sel != 0) acc += (static_cast<unsigned long long>(peer[tid]) << 16) + peer[256 + tid];
+                    if (counted) cnt += peer[512 + tid];
                 }
-                sh.tot[tid] = acc;
+                sh.tot[tid] = sel == 0 ? static_cast<unsigned long long>(cnt) : acc;
+                sh.totc[tid] = cnt;
+                uint32_t* other = &sh.hist[(round_no & 1) ^ 1][0][0];
+                other[tid] = 0u; other[256 + tid] = 0u; other[512 + tid] = 0u;
             }
             __syncthreads();
             if (warp == 0) {
-                // walk from the top bin down: lane l owns bins 255 - 8 l ... 248 - 8 l
+                // walk from the largest logits (bin 0) down: lane l owns bins 8 l ... 8 l + 7
                 unsigned long long mine = 0ull;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) mine += sh.tot[255 - (lane * 8 + j)];
-                unsigned long long incl = mine;          // inclusive scan over lanes (top bins first)
+                for (int j = 0; j < 8; ++j) mine += sh.tot[lane * 8 + j];
+                unsigned long long incl = mine;          // inclusive scan over lanes
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const unsigned long long t0 = __shfl_up_sync(0xffffffffu, incl, o);
                     if (lane >= o) incl += t0;
                 }
-                if (round == 0 && lane == 31) {
-                    // total weight of the live keys = the base of the target
-                    sh.target = (sel == 0) ? static_cast<unsigned long long>(p.top_k)
-                                           : static_cast<unsigned long long>(static_cast<double>(p.top_p) * static_cast<double>(incl));
-                    if (sh.target < 1ull) sh.target = 1ull;
+                unsigned long long target = r.target;
+                if (first) {
+                    // total weight of the live entries = the base of the target
+                    const unsigned long long total = __shfl_sync(0xffffffffu, incl, 31);
+                    target = (sel == 0) ? static_cast<unsigned long long>(p.top_k)
+                                        : static_cast<unsigned long long>(static_cast<double>(p.top_p) * static_cast<double>(total));
+                    if (target < 1ull) target = 1ull;
                 }
-                __syncwarp();
-                const unsigned long long target = sh.target;
-                unsigned long long run = sh.above + incl - mine;
+                unsigned long long run = r.above + incl - mine;
                 const unsigned hit = __ballot_sync(0xffffffffu, run + mine >= target);
                 // (with exact sums the last lane always reaches the target; the guard keeps the walk defined)
                 const int l = hit != 0u ? __ffs(hit) - 1 : 31;
                 if (lane == l) {
-                    int bin = 255 - lane * 8;
-                    for (int j = 0; j < 7; ++j, --bin) {
+                    int bin = lane * 8;
+                    for (int j = 0; j < 7; ++j, ++bin) {
                         if (run + sh.tot[bin] >= target) break;
                         run += sh.tot[bin];
                     }
-                    sh.above = run;                      // weight strictly above the chosen bin
-                    sh.bin = bin;
-                    sh.prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+                    // the codes of the chosen bin; the end bins of a window also hold what lies outside it
+                    const unsigned long long v = static_cast<unsigned long long>(r.base) + static_cast<unsigned long long>(bin);
+                    uint32_t lo = r.lo, hi = r.hi;
+                    if (bin > 0) lo = static_cast<uint32_t>(max(static_cast<unsigned long long>(lo), v << r.shift));
+                    if (bin < 255) hi = static_cast<uint32_t>(min(static_cast<unsigned long long>(hi), ((v + 1ull) << r.shift) - 1ull));
+                    FilterRound q = r;
+                    q.target = target; q.above = run; q.lo = lo; q.hi = hi;
+                    q.n_sel = counted ? sh.totc[bin] : 0xffffffffu;
+                    if (q.n_sel <= static_cast<uint32_t>(kFilterCand)) {
+                        q.next = 1;                     // few enough: collect them and rank them directly
+                    } else if (lo == hi) {
+                        if (r.phase == 0) {
+                            // one value of d, many entries: go on over the bits of z itself inside this group
+                            q.phase = 1; q.dsel = lo; q.lo = 0u; q.hi = 0xffffffffu; q.shift = 24; q.base = 0u;
+                        } else {
+                            q.next = 2;                 // one logit value: it is tau, and all its entries are kept
+                            q.tau = key_to_float(~lo);
+                            q.kept = run + sh.tot[bin];
+                        }
+                    } else {
+                        // cut the interval into (at most 257, the last two sharing a bin) equal parts
+                        const int width = 32 - __clz(hi - lo);
+                        q.shift = max(0, width - 8);
+                        q.base = lo >> q.shift;
+                    }
+                    sh.r = q;
                 }
             }
             __syncthreads();
+            first = false;
+            if (sh.r.next != 0) { ++round_no; break; }
         }
-        // the selected key: every key >= it is kept
-        floor_key = sh.prefix;
-        if (sel == 1) kept_mass = static_cast<double>(sh.above + sh.tot[sh.bin]) / kMassUnit;
+        const FilterRound r = sh.r;
+        if (r.next == 1) {
+            // every CTA hands its entries of the chosen bin to all eight CTAs; each ranks them on its own
+            scan(sel, r, nullptr, true);
+            cluster_sync();
+            const int nc = static_cast<int>(min(r.n_sel, static_cast<uint32_t>(kFilterCand)));
+            if (tid < nc) {
+                const float zt = sh.cand_z[tid];
+                unsigned long long gt = 0ull, ge = 0ull;   // weight of the candidates above zt / not below zt
+#pragma unroll 4
+                for (int j = 0; j < nc; ++j) {
+                    const float zj = sh.cand_z[j];
+                    const unsigned long long wj = sh.cand_w[j];
+                    gt += zj > zt ? wj : 0ull;
+                    ge += zj >= zt ? wj : 0ull;
+                }
+                if (r.above + gt < r.target && r.above + ge >= r.target) { sh.r.tau = zt; sh.r.kept = r.above + ge; }
+            }
+            __syncthreads();
+            if (tid == 0) sh.n_cand = 0u;               // (rank 0's counter; the next hand-over is two barriers away)
+        } else if (r.next == 0 && rank == 0 && tid == 0) {
+            report_error(p.status, kErrTimeout, row, 7);   // cannot happen: every round shrinks the interval
+        }
+        floor_z = sh.r.tau;                             // every logit >= it is kept
         __syncthreads();
     }
+    double kept_mass = static_cast<double>(sh.r.kept) / kMassUnit;
     if (!do_p) {
-        // top-k alone: the mass of the kept keys is one more pass (a plain reduction, no histogram)
+        // top-k alone: the mass of the kept logits is one more pass (a plain reduction, no histogram)
         unsigned long long acc = 0ull;
+        const uint32_t b_hi = static_cast<uint32_t>(bin_of(__float_as_uint(m - floor_z), kFilterShift0, base0));
         for (int i = tid; i < n; i += kFilterThreads) {
-            const uint32_t key = key_at(i);
-            if (key >= floor_key) acc += key_mass(key, m, cf);
+            if (bytes_valid && s_bin0[i] > b_hi) continue;
+            const float z = __ldg(src + i);
+            if (mask_row != nullptr && !mask_allows(mask_row, v0 + i)) continue;
+            if (z >= floor_z) acc += mass_of(m - z, cf);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
@@ -432,18 +660,17 @@ sample_filter_kernel(const SampleParams p)
         kept_mass = static_cast<double>(t) / kMassUnit;
     }
     if (rank == 0 && tid == 0) {
-        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(key_to_float(floor_key));
+        p.topp[static_cast<int64_t>(row) * 2] = static_cast<double>(floor_z);
         p.topp[static_cast<int64_t>(row) * 2 + 1] = kept_mass;
     }
-    cluster_sync();                                     // no CTA leaves while a peer may still read its histograms
+    cluster_sync();                                     // no CTA leaves while a peer may still read its shared memory
 }
 
-cudaError_t launch_sample_filter(const SampleParams& p, cudaStream_t stream)
+cudaError_t launch_sample_filter(const SampleParams& p, bool pdl, cudaStream_t stream)
 {
     const int per = ((p.vocab + kAcceptCluster - 1) / kAcceptCluster + 3) & ~3;
-    const size_t smem = per <= kFilterSliceMax ? static_cast<size_t>(per) * sizeof(float) : 0;
-    sample_filter_kernel<<<dim3(kAcceptCluster, p.m_rows), kFilterThreads, smem, stream>>>(p);
-    return cudaGetLastError();
+    const size_t smem = per <= kFilterCodesMax ? static_cast<size_t>(per) + kFilterList * (sizeof(uint16_t) + sizeof(float)) : 0;
+    return launch_kernel_ex(sample_filter_kernel, dim3(kAcceptCluster, p.m_rows), dim3(kFilterThreads), smem, stream, pdl, p);
 }
 
 // ------------------------------------------------------------------------------------ acceptance
@@ -903,12 +1130,8 @@ constexpr size_t kAcceptSmemMax = static_cast<size_t>(kAcceptWarps) * 4 * kSubCh
 
 cudaError_t sample_init()
 {
-    cudaError_t e = cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(kAcceptSmemMax));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(sample_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kFilterSliceMax * sizeof(float)));
-    return e;
+    return cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(kAcceptSmemMax));
 }
 
 cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream)
