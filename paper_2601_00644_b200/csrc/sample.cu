@@ -184,44 +184,49 @@ __device__ __forceinline__ void cp_async_wait_all()
 // is applied first.  Both filters are thresholds on the logit: the kept set of a row is
 // {v : z_v >= tau}, tau being the k-th largest logit (top-k; ties with it are kept), respectively the
 // largest logit such that the tokens with logit >= tau hold at least top_p of the (top-k filtered)
-// mass.  tau is found exactly by a selection over an order-preserving 32-bit code of the logits:
-// round after round the interval of codes that can still hold tau is cut into up to 256 bins, every
+// mass.  tau is found exactly by a selection over an order-preserving integer code of the logits:
+// round after round the interval of codes that can still hold tau is cut into up to 128 bins, every
 // live entry adds its weight (1 for top-k, its probability mass for top-p) to the bin of its code,
 // and a walk over the bins from the largest logits down finds the bin in which the running weight
 // reaches the target.  As soon as that bin holds at most kFilterCand entries they are collected and
-// ranked directly, which ends the selection.
+// ranked directly by their logits, which ends the selection.
 //
-// The code of an entry is the bit pattern of d = m - z (m = the row maximum, known from the softmax
-// statistics of the row, so no pass over the row is spent on it): a non-negative float, whose bit
-// pattern grows with d.  Bins cut from it are equally wide on a logarithmic scale of the distance to
-// the maximum, whatever the scale of the logits, which spreads flat rows (all logits within 1e-2) and
-// peaked rows alike over dozens of bins, where the leading byte of the logit itself puts most of a
-// row into a handful of bins and its shared-memory atomics into one another's way.  Distinct logits
-// can round to the same d; should such a group ever hold more than kFilterCand entries, the selection
-// carries on over the bit pattern of z itself inside the group (second phase), so that the result is
-// exact in every case.
+// The code of an entry is a 23-bit fixed-point image of d = m - z over [0, d_max]: the mantissa of
+// 1 + d / d_max (one fused multiply-add; values past d_max share the last code).  m is the row
+// maximum and d_max a multiple of the spread of the part maxima, both taken from the softmax
+// statistics of the row, so no pass over the row is spent on them.  The code grows with d but is not
+// one-to-one; that is harmless: entries that share a code are told apart when they are ranked by
+// their logits, and should a single code ever hold more than kFilterCand entries, the selection
+// carries on over the bit pattern of z itself inside that group (second phase).  The result is exact
+// whatever d_max was; a poor d_max only costs rounds.
 //
-// One cluster of eight CTAs per target row, a contiguous slice of the vocabulary per CTA.  The first
-// round reads the slice from global memory (the one read of the logits that comes from DRAM) and
-// leaves every entry's first-round bin in shared memory, one byte per entry; the later rounds scan
-// these bytes and fetch only the logits whose byte lies in the live range (a few percent, out of
-// L2).  A round ends with one cluster barrier, after which every CTA adds up the eight histograms
-// (read from its peers' shared memory; histograms alternate between two buffers, so one barrier per
-// round is enough) and walks them; all CTAs reach the same result, so nothing is broadcast.
-// Masses are accumulated as fixed-point integers (2^((z - m) c) rounded to units of 2^-31, added as
-// two 16-bit limbs with the native 32-bit shared-memory atomics; 64-bit shared-memory atomics were
+// One cluster of four CTAs per target row, a contiguous slice of the vocabulary per CTA.  The first
+// round reads the slice from global memory (the one read of the logits that comes from DRAM), leaves
+// every entry's first-round bin in shared memory (one byte per entry) and accumulates into a
+// histogram with one column per lane (bank = lane: an atomic instruction of a warp is one wavefront,
+// where 32 lanes falling into a few dozen bins of a plain histogram were measured at 3.8 wavefronts
+// per instruction and bound the whole kernel); the columns are added up before the hand-over.  The
+// later rounds scan the stored bytes, list the entries whose byte lies in the live range (a few
+// percent), fetch those logits out of L2 all at once and from then on work on the list.  A round
+// ends with one cluster barrier, after which every CTA adds up the four histograms (read from its
+// peers' shared memory; histograms alternate between two buffers, so one barrier per round is
+// enough) and walks them; all CTAs reach the same result, so nothing is broadcast.
+// Masses are accumulated as fixed-point integers (2^(-d c) rounded to units of 2^-31, added as two
+// 16-bit limbs with the native 32-bit shared-memory atomics; 64-bit shared-memory atomics were
 // measured 15x slower): integer addition is exact and order-independent, so the histograms, the
 // totals and the comparison with the target are the same whatever the order of the atomic adds, and
 // a row's result does not depend on scheduling.  The rounding of one entry is at most 2^-32 and
 // unbiased: over a 128 K row its sum stays near 1e-8 of the mass.
-constexpr int kFilterThreads = 256;
+constexpr int kFilterCluster = 4;
+constexpr int kFilterThreads = 512;
 constexpr int kFilterWarps = kFilterThreads / 32;
-constexpr int kFilterCodesMax = 16384;                    // entries of a slice whose first-round bin is kept in shared memory
-constexpr int kFilterList = 1024;                         // live entries of a slice listed after the first round
+constexpr int kFilterBins = 128;
+constexpr int kFilterCodeBits = 23;
+constexpr int kFilterShift0 = kFilterCodeBits - 7;        // first round: the leading seven bits of the code
+constexpr int kFilterCodesMax = 32768;                    // entries of a slice whose first-round bin is kept in shared memory
+constexpr int kFilterList = 2048;                         // live entries of a slice listed after the first round
 constexpr int kFilterCand = 128;                          // a bin with at most this many entries is ranked directly
-constexpr int kFilterMaxRounds = 32;                      // (a selection needs at most 13: see the walk)
-constexpr int kFilterShift0 = 18;                         // first round: exponent and five mantissa bits of d, ...
-constexpr int kFilterOctaves = 8;                         // ... a window of eight octaves of d
+constexpr int kFilterMaxRounds = 32;                      // (a selection needs far fewer: every round shrinks the interval)
 constexpr double kMassUnit = 2147483648.0;                // 2^31
 constexpr float kMassUnitF = 2147483648.0f;
 
@@ -235,12 +240,12 @@ __device__ __forceinline__ float key_to_float(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// what a round of the selection looks at (identical in the eight CTAs of a row)
+// what a round of the selection looks at (identical in the four CTAs of a row)
 struct FilterRound {
     uint32_t lo, hi;                                    // live codes: lo <= code <= hi
-    uint32_t base;                                      // bin = clamp((code >> shift) - base, 0, 255)
+    uint32_t base;                                      // bin = clamp((code >> shift) - base, 0, kFilterBins - 1)
     int shift;
-    int phase;                                          // 0: code = bits of (m - z);  1: code = ~key(z) among the entries with bits of (m - z) == dsel
+    int phase;                                          // 0: code of d;  1: code = ~key(z) among the entries whose code of d is dsel
     uint32_t dsel;
     int next;                                           // after the walk: 0 another round, 1 collect and rank, 2 tau is known
     uint32_t n_sel;                                     // entries in the chosen bin (when the round counted them)
@@ -251,15 +256,14 @@ struct FilterRound {
 };
 
 struct FilterShared {
-    uint32_t hist[2][3][256];                           // [buffer][mass bits 16..31 | mass bits 0..15 | entries][bin]
-    unsigned long long tot[256];                        // cluster-wide weight per bin
-    uint32_t totc[256];                                 // cluster-wide entries per bin
+    uint32_t hist[2][3][kFilterBins];                   // [buffer][mass bits 16..31 | mass bits 0..15 | entries][bin]
+    unsigned long long tot[kFilterBins];                // cluster-wide weight per bin
+    uint32_t totc[kFilterBins];                         // cluster-wide entries per bin
     float cand_z[kFilterCand];
     uint32_t cand_w[kFilterCand];
     float red_hi[kFilterWarps], red_lo[kFilterWarps];
-    float slice_hi[kAcceptCluster], slice_lo[kAcceptCluster];
     unsigned long long red64[kFilterWarps];
-    unsigned long long slice_mass[kAcceptCluster];
+    unsigned long long slice_mass[kFilterCluster];
     uint32_t n_cand;
     uint32_t list_n;
     FilterRound r;
@@ -270,16 +274,24 @@ __device__ __forceinline__ uint32_t mass_of(float d, float cf)
 {
     return __float2uint_rn(fast_exp2(d * -cf) * kMassUnitF);   // <= 2^31
 }
+// 23-bit code of d >= 0: the mantissa of min(1 + d * inv_dmax, 2 - 2^-23)
+__device__ __forceinline__ uint32_t code_of(float d, float inv_dmax)
+{
+    return __float_as_uint(fminf(fmaf(d, inv_dmax, 1.f), 1.99999988f)) - 0x3f800000u;
+}
 __device__ __forceinline__ int bin_of(uint32_t code, int shift, uint32_t base)
 {
     const uint32_t t = code >> shift;
-    return t <= base ? 0 : static_cast<int>(min(t - base, 255u));
+    return t <= base ? 0 : static_cast<int>(min(t - base, static_cast<uint32_t>(kFilterBins - 1)));
 }
 
-__global__ void __cluster_dims__(kAcceptCluster, 1, 1) __launch_bounds__(kFilterThreads, 6)
+__global__ void __cluster_dims__(kFilterCluster, 1, 1) __launch_bounds__(kFilterThreads, 3)
 sample_filter_kernel(const SampleParams p)
 {
-    extern __shared__ __align__(16) uint8_t s_bin0[];   // first-round bin of every entry of this CTA's slice (when it fits), ...
+    // first-round bin of every entry of this CTA's slice (when it fits), then the first round's histogram with one
+    // column per lane: [limb][bin][lane].  Once its columns are added up the histogram is dead and its room holds
+    // the list of live entries (indices, then logits).
+    extern __shared__ __align__(16) uint8_t s_bin0[];
     __shared__ FilterShared sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = static_cast<int>(cluster.block_rank());
@@ -288,14 +300,16 @@ sample_filter_kernel(const SampleParams p)
     cluster_arrive();                                   // "this CTA runs" (awaited before the first peer access)
 
     // ---- this CTA's slice: [v0, v1), a multiple of four entries long so that 16-byte loads stay aligned
-    const int per = ((p.vocab + kAcceptCluster - 1) / kAcceptCluster + 3) & ~3;
+    const int per = ((p.vocab + kFilterCluster - 1) / kFilterCluster + 3) & ~3;
     const int v0 = min(p.vocab, rank * per), v1 = min(p.vocab, v0 + per);
     const int n = v1 - v0;
     const bool coded = per <= kFilterCodesMax;
-    uint16_t* s_idx = reinterpret_cast<uint16_t*>(s_bin0 + per);                       // ... the listed entries' indices ...
-    float* s_list = reinterpret_cast<float*>(s_bin0 + per + kFilterList * sizeof(uint16_t));   // ... and their logits
     const bool vec_ok = ((p.vocab & 3) == 0);
-    for (int i = tid; i < 3 * 256; i += kFilterThreads) (&sh.hist[0][0][0])[i] = 0u;
+    uint32_t* s_big = reinterpret_cast<uint32_t*>(s_bin0 + (coded ? per : 0));
+    uint16_t* s_idx = reinterpret_cast<uint16_t*>(s_big);
+    float* s_list = reinterpret_cast<float*>(s_big + kFilterList * sizeof(uint16_t) / sizeof(uint32_t));
+    for (int i = tid; i < 3 * kFilterBins; i += kFilterThreads) (&sh.hist[0][0][0])[i] = 0u;
+    for (int i = tid; i < 2 * kFilterBins * 32; i += kFilterThreads) s_big[i] = 0u;
     if (tid == 0) sh.n_cand = 0u;
     pdl_wait();                                         // the logits and their statistics come from the preceding kernel
     pdl_launch_dependents();
@@ -303,12 +317,14 @@ sample_filter_kernel(const SampleParams p)
     const uint32_t* mask_row = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(p.row_seq[row]) * p.mask_words : nullptr;
     const float* src = p.logits + static_cast<int64_t>(row) * p.vocab + v0;
 
-    // ---- row maximum m and the spread of the part maxima, from the row's softmax statistics (each CTA
-    // reads an eighth of the parts; the slice results are exchanged through the peers' shared memory)
+    // ---- row maximum m and the spread of the part maxima, from the row's softmax statistics (every CTA reads all
+    // the parts, a few loads per thread all in flight at once: cheaper than an exchange between the CTAs)
+    float m, part_lo;
     {
         const float2* tp = p.tstats + static_cast<int64_t>(row) * p.n_tparts;
         float hi = -INFINITY, lo = INFINITY;
-        for (int t = rank * kFilterThreads + tid; t < p.n_tparts; t += kAcceptCluster * kFilterThreads) {
+#pragma unroll 4
+        for (int t = tid; t < p.n_tparts; t += kFilterThreads) {
             const float x = __ldcg(&tp[t].x);
             hi = fmaxf(hi, x);
             if (x > -INFINITY) lo = fminf(lo, x);
@@ -317,18 +333,11 @@ sample_filter_kernel(const SampleParams p)
         lo = -warp_max(-lo);
         if (lane == 0) { sh.red_hi[warp] = hi; sh.red_lo[warp] = lo; }
         __syncthreads();
-        cluster_wait();                                 // all eight CTAs have started
-        if (tid < kAcceptCluster) {
+        m = sh.red_hi[0]; part_lo = sh.red_lo[0];
 #pragma unroll
-            for (int w = 0; w < kFilterWarps; ++w) { hi = fmaxf(hi, sh.red_hi[w]); lo = fminf(lo, sh.red_lo[w]); }
-            cluster.map_shared_rank(&sh.slice_hi[0], tid)[rank] = hi;
-            cluster.map_shared_rank(&sh.slice_lo[0], tid)[rank] = lo;
-        }
-        cluster_sync();
+        for (int w = 1; w < kFilterWarps; ++w) { m = fmaxf(m, sh.red_hi[w]); part_lo = fminf(part_lo, sh.red_lo[w]); }
+        cluster_wait();                                 // all four CTAs have started
     }
-    float m = sh.slice_hi[0], part_lo = sh.slice_lo[0];
-#pragma unroll
-    for (int c = 1; c < kAcceptCluster; ++c) { m = fmaxf(m, sh.slice_hi[c]); part_lo = fminf(part_lo, sh.slice_lo[c]); }
     if (m == -INFINITY) {                               // nothing can be selected in this row
         if (rank == 0 && tid == 0) {
             p.topp[static_cast<int64_t>(row) * 2] = -static_cast<double>(INFINITY);
@@ -337,17 +346,15 @@ sample_filter_kernel(const SampleParams p)
         cluster_sync();
         return;
     }
-    // first-round window: eight octaves of d = m - z, the top one a few octaves above the spread of the
-    // part maxima (the maxima of small parts spread almost like the row, those of large parts much
-    // less).  A window that misses only costs rounds: its end bins take what lies outside.
-    uint32_t base0;
+    // d_max: a multiple of the spread of the part maxima (the maxima of 32-entry parts spread almost like the
+    // row's bulk, those of large parts much less), and no more than where the mass vanishes (2^-40 of the
+    // largest).  A d_max that misses only costs rounds: the last code takes what lies beyond it.
+    float inv_dmax;
     {
         const float spread = m - part_lo;
-        int e_top = 127 + 6;
-        if (spread > 0.f && spread < INFINITY)
-            e_top = static_cast<int>(__float_as_uint(spread) >> 23) + ((p.vocab / max(p.n_tparts, 1) >= 1024) ? 5 : 3);
-        e_top = min(max(e_top, kFilterOctaves), 254);
-        base0 = static_cast<uint32_t>(e_top - (kFilterOctaves - 1)) << (23 - kFilterShift0);
+        float dmax = 40.f / cf;
+        if (spread > 0.f && spread < INFINITY) dmax = fminf(dmax, spread * ((p.vocab / max(p.n_tparts, 1) >= 1024) ? 8.f : 2.25f));
+        inv_dmax = 1.f / dmax;
     }
 
     const bool do_k = p.top_k > 0 && p.top_k < p.vocab;
@@ -360,10 +367,11 @@ sample_filter_kernel(const SampleParams p)
     auto consider = [&](float z, int sel, const FilterRound& r, uint32_t* hist, bool collect) {
         if (!(z >= floor_z)) return;
         const float d = m - z;
-        const uint32_t dbits = __float_as_uint(d);
-        uint32_t code = dbits;
+        if (!(d >= 0.f)) return;
+        const uint32_t dcode = code_of(d, inv_dmax);
+        uint32_t code = dcode;
         if (r.phase != 0) {
-            if (dbits != r.dsel) return;
+            if (dcode != r.dsel) return;
             code = ~order_key(z);
         }
         if (code - r.lo > r.hi - r.lo) return;
@@ -372,7 +380,7 @@ sample_filter_kernel(const SampleParams p)
             const uint32_t idx = atomicAdd(cluster.map_shared_rank(&sh.n_cand, 0), 1u);
             if (idx < static_cast<uint32_t>(kFilterCand)) {
 #pragma unroll 1
-                for (int c = 0; c < kAcceptCluster; ++c) {
+                for (int c = 0; c < kFilterCluster; ++c) {
                     cluster.map_shared_rank(&sh.cand_z[0], c)[idx] = z;
                     cluster.map_shared_rank(&sh.cand_w[0], c)[idx] = w;
                 }
@@ -381,9 +389,9 @@ sample_filter_kernel(const SampleParams p)
             const int bin = bin_of(code, r.shift, r.base);
             if (sel != 0) {
                 atomicAdd(&hist[bin], w >> 16);
-                atomicAdd(&hist[256 + bin], w & 0xffffu);
+                atomicAdd(&hist[kFilterBins + bin], w & 0xffffu);
             }
-            atomicAdd(&hist[512 + bin], 1u);
+            atomicAdd(&hist[2 * kFilterBins + bin], 1u);
         }
     };
     auto fetch = [&](int i) -> float {                  // entry i of the slice, -inf when it is masked out
@@ -406,21 +414,33 @@ sample_filter_kernel(const SampleParams p)
             for (int i = tid; i < n; i += kFilterThreads) consider(fetch(i), sel, r, hist, collect);
             return;
         }
-        const uint32_t b_lo = static_cast<uint32_t>(bin_of(r.phase == 0 ? r.lo : r.dsel, kFilterShift0, base0));
-        const uint32_t b_span = static_cast<uint32_t>(bin_of(r.phase == 0 ? r.hi : r.dsel, kFilterShift0, base0)) - b_lo;
+        // live range of the stored bytes: the first-round bins of the interval's ends (of the group's code in phase 1)
+        const uint32_t b_lo = (r.phase == 0 ? r.lo : r.dsel) >> kFilterShift0;
+        const uint32_t b_span = ((r.phase == 0 ? r.hi : r.dsel) >> kFilterShift0) - b_lo;
         const uint32_t lo4 = b_lo * 0x01010101u, span4 = b_span * 0x01010101u;
-        // the bytes of a word that lie in the live range, four at a time (0xff where they do)
+        // the bytes of a word that lie in the live range, as four flag bits
         auto hits_of = [&](int i0) -> uint32_t {
             const uint32_t b4 = *reinterpret_cast<const uint32_t*>(s_bin0 + i0);
-            uint32_t hits = __vcmpleu4(__vsub4(b4, lo4), span4);
-            if (i0 + 4 > n) hits &= (1u << (8 * (n - i0))) - 1u;
-            return hits;
+            uint32_t flags;                             // bit 7 of every byte that hits
+            if (b_span == 0u) {
+                const uint32_t x = b4 ^ lo4;            // zero bytes hit
+                flags = ~(((x & 0x7f7f7f7fu) + 0x7f7f7f7fu) | x) & 0x80808080u;
+            } else {
+                flags = __vcmpleu4(__vsub4(b4, lo4), span4) & 0x80808080u;
+            }
+            uint32_t nib = ((flags >> 7) * 0x00204081u >> 21) & 15u;
+            if (!vec_ok && i0 + 4 > n) nib &= (1u << (n - i0)) - 1u;   // (a slice is a multiple of four entries otherwise)
+            return nib;
         };
         if (list_state == 0) {
-            // count this thread's hits, reserve room for the warp's with one atomic, then write the indices
-            uint32_t mine = 0u;
+            // one look at this thread's (at most 16) words: the hits as a 64-bit mask; room for the warp's hits is
+            // reserved with one atomic, then the indices are written
+            unsigned long long mask = 0ull;
+            int word = 0;
 #pragma unroll 1
-            for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) mine += __popc(hits_of(i0) & 0x01010101u);
+            for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4, ++word)
+                mask |= static_cast<unsigned long long>(hits_of(i0)) << (4 * word);
+            const uint32_t mine = static_cast<uint32_t>(__popcll(mask));
             uint32_t incl = mine;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -430,17 +450,12 @@ sample_filter_kernel(const SampleParams p)
             uint32_t at = 0u;
             if (lane == 31) at = atomicAdd(&sh.list_n, incl);
             at = __shfl_sync(0xffffffffu, at, 31) + incl - mine;
-            if (mine != 0u) {
-#pragma unroll 1
-                for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) {
-                    uint32_t hits = hits_of(i0);
-                    while (hits != 0u) {
-                        const int u = (__ffs(hits) - 1) >> 3;
-                        hits &= ~(0xffu << (8 * u));
-                        if (at < static_cast<uint32_t>(kFilterList)) s_idx[at] = static_cast<uint16_t>(i0 + u);
-                        ++at;
-                    }
-                }
+            while (mask != 0ull) {
+                const int pos = __ffsll(static_cast<long long>(mask)) - 1;
+                mask &= mask - 1ull;
+                if (at < static_cast<uint32_t>(kFilterList))
+                    s_idx[at] = static_cast<uint16_t>(tid * 4 + (pos >> 2) * (kFilterThreads * 4) + (pos & 3));
+                ++at;
             }
             __syncthreads();
             const uint32_t total = sh.list_n;
@@ -457,10 +472,10 @@ sample_filter_kernel(const SampleParams p)
         }
 #pragma unroll 1
         for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) {
-            uint32_t hits = hits_of(i0);
-            while (hits != 0u) {
-                const int u = (__ffs(hits) - 1) >> 3;
-                hits &= ~(0xffu << (8 * u));
+            uint32_t nib = hits_of(i0);
+            while (nib != 0u) {
+                const int u = __ffs(nib) - 1;
+                nib &= nib - 1u;
                 consider(fetch(i0 + u), sel, r, hist, collect);
             }
         }
@@ -471,8 +486,8 @@ sample_filter_kernel(const SampleParams p)
         // sel 0: weight 1, target k.   sel 1: weight mass, target top_p * (mass of the logits >= floor_z)
         if (tid == 0) {
             FilterRound r0;
-            r0.lo = 0u; r0.hi = min(0x7f800000u, __float_as_uint(m - floor_z));   // every d >= 0 down to the floor
-            r0.base = base0; r0.shift = kFilterShift0; r0.phase = 0; r0.dsel = 0u; r0.next = 0; r0.n_sel = 0u;
+            r0.lo = 0u; r0.hi = code_of(m - floor_z, inv_dmax);   // every code down to the floor's
+            r0.base = 0u; r0.shift = kFilterShift0; r0.phase = 0; r0.dsel = 0u; r0.next = 0; r0.n_sel = 0u;
             r0.above = 0ull; r0.target = 0ull; r0.tau = floor_z; r0.kept = 0ull;
             sh.r = r0;
             sh.list_n = 0u;
@@ -485,71 +500,112 @@ sample_filter_kernel(const SampleParams p)
             uint32_t* hist = &sh.hist[round_no & 1][0][0];
             bool counted = true;                        // the round records how many entries each bin holds
             if (!bytes_valid && first) {
-                // the first pass of the kernel: every entry of the slice, straight from global memory; leaves the
-                // bins in shared memory.  For top-p the entry count is left out (two atomics per entry, not three).
+                // The first pass of the kernel: every entry of the slice, straight from global memory; leaves the
+                // bins in shared memory.  Lane l adds into column l of the histogram, so the 32 atomics of a warp
+                // instruction go to 32 banks.  For top-p the entry count is left out (two atomics per entry).
                 counted = sel == 0;
-#pragma unroll 2
-                for (int i0 = tid * 4; i0 < n; i0 += kFilterThreads * 4) {
-                    float z[4];
-                    if (vec_ok) {
-                        const float4 x = __ldg(reinterpret_cast<const float4*>(src + i0));
-                        z[0] = x.x; z[1] = x.y; z[2] = x.z; z[3] = x.w;
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) z[u] = (i0 + u < n) ? __ldg(src + i0 + u) : -INFINITY;
-                    }
+                if (round_no != 0) {                    // (cleared in the prologue for the kernel's first round)
+                    for (int i = tid; i < 2 * kFilterBins * 32; i += kFilterThreads) s_big[i] = 0u;
+                    __syncthreads();
+                }
+                uint32_t* col = s_big + lane;
+                // (top-p as the first selection has no floor yet, and an entry that cannot be selected is -inf: its
+                // distance clamps into the last bin and its mass is 0, so it needs no test of its own)
+                const bool plain = sel != 0 && !do_k;
+                auto entries4 = [&](const float* zin, int i0) {
+                    float z[4] = {zin[0], zin[1], zin[2], zin[3]};
                     if (mask_row != nullptr) {
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
                             if (i0 + u < n && !mask_allows(mask_row, v0 + i0 + u)) z[u] = -INFINITY;
                     }
-                    uint32_t b4 = 0u;
+                    uint32_t tb[4];                     // bits of min(1 + d / d_max, 2 - 2^-23): byte 2 = 0x80 | bin
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const float d = m - z[u];
-                        const uint32_t dbits = __float_as_uint(d);
-                        const bool live = z[u] >= floor_z && dbits <= 0x7f800000u;
-                        const int bin = live ? bin_of(dbits, kFilterShift0, base0) : 255;
-                        b4 |= static_cast<uint32_t>(bin) << (8 * u);
-                        if (live) {
-                            if (sel == 0) {
-                                atomicAdd(&hist[512 + bin], 1u);
-                            } else {
-                                const uint32_t w = mass_of(d, cf);
-                                atomicAdd(&hist[bin], w >> 16);
-                                atomicAdd(&hist[256 + bin], w & 0xffffu);
+                        tb[u] = __float_as_uint(fminf(fmaf(d, inv_dmax, 1.f), 1.99999988f));
+                        if (plain) {
+                            const uint32_t w = mass_of(d, cf);
+                            uint32_t* at = col + ((tb[u] >> 11) & 0xfe0u);         // bin * 32 words
+                            atomicAdd(at, w >> 16);
+                            atomicAdd(at + kFilterBins * 32, w & 0xffffu);
+                        } else {
+                            const bool live = z[u] >= floor_z && d >= 0.f;
+                            if (!live) tb[u] = 0x3fff0000u;                         // the last bin
+                            const uint32_t bin = (tb[u] >> 16) & 0x7fu;
+                            if (live) {
+                                if (sel == 0) {
+                                    atomicAdd(col + bin * 32u, 1u);
+                                } else {
+                                    const uint32_t w = mass_of(d, cf);
+                                    atomicAdd(col + bin * 32u, w >> 16);
+                                    atomicAdd(col + (kFilterBins + bin) * 32u, w & 0xffffu);
+                                }
                             }
                         }
                     }
-                    if (coded) *reinterpret_cast<uint32_t*>(s_bin0 + i0) = b4;
+                    if (coded)
+                        *reinterpret_cast<uint32_t*>(s_bin0 + i0) =
+                            __byte_perm(__byte_perm(tb[0], tb[1], 0x0062), __byte_perm(tb[2], tb[3], 0x0062), 0x5410) ^ 0x80808080u;
+                };
+                // four loads of a thread are in flight before the first of them is used
+                constexpr int kStep = kFilterThreads * 4;
+#pragma unroll 1
+                for (int base = tid * 4; base < n; base += 4 * kStep) {
+                    float z[4][4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int i0 = base + q * kStep;
+                        if (vec_ok && i0 < n) {
+                            const float4 x = __ldg(reinterpret_cast<const float4*>(src + i0));
+                            z[q][0] = x.x; z[q][1] = x.y; z[q][2] = x.z; z[q][3] = x.w;
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) z[q][u] = (i0 + u < n) ? __ldg(src + i0 + u) : -INFINITY;
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (base + q * kStep < n) entries4(z[q], base + q * kStep);
+                }
+                __syncthreads();
+                // add up the columns: thread (limb, bin) reads its 32 columns, rotated so that a warp's reads fall
+                // into 32 banks
+                if (tid < 2 * kFilterBins) {
+                    uint32_t sum = 0u;
+#pragma unroll 8
+                    for (int k = 0; k < 32; ++k) sum += s_big[tid * 32 + ((k + tid) & 31)];
+                    if (sel != 0) hist[tid] = sum;
+                    else if (tid < kFilterBins) hist[2 * kFilterBins + tid] = sum;
                 }
                 bytes_valid = coded;
             } else {
                 scan(sel, r, hist, false);
             }
-            cluster_sync();                             // all eight histograms of this round are complete
-            // cluster-wide histogram: thread t adds bin t of the eight CTAs; the other buffer is cleared for the
+            cluster_sync();                             // all four histograms of this round are complete
+            // cluster-wide histogram: thread t adds bin t of the four CTAs; the other buffer is cleared for the
             // next round (its last readers arrived at the barrier above after they were done with it)
-            {
+            if (tid < kFilterBins) {
                 unsigned long long acc = 0ull;
                 uint32_t cnt = 0u;
 #pragma unroll
-                for (int c = 0; c < kAcceptCluster; ++c) {
+                for (int c = 0; c < kFilterCluster; ++c) {
                     const uint32_t* peer = cluster.map_shared_rank(hist, c);
-                    if (sel != 0) acc += (static_cast<unsigned long long>(peer[tid]) << 16) + peer[256 + tid];
-                    if (counted) cnt += peer[512 + tid];
+                    if (sel != 0) acc += (static_cast<unsigned long long>(peer[tid]) << 16) + peer[kFilterBins + tid];
+                    if (counted) cnt += peer[2 * kFilterBins + tid];
                 }
                 sh.tot[tid] = sel == 0 ? static_cast<unsigned long long>(cnt) : acc;
                 sh.totc[tid] = cnt;
                 uint32_t* other = &sh.hist[(round_no & 1) ^ 1][0][0];
-                other[tid] = 0u; other[256 + tid] = 0u; other[512 + tid] = 0u;
+                other[tid] = 0u; other[kFilterBins + tid] = 0u; other[2 * kFilterBins + tid] = 0u;
             }
             __syncthreads();
             if (warp == 0) {
-                // walk from the largest logits (bin 0) down: lane l owns bins 8 l ... 8 l + 7
+                // walk from the largest logits (bin 0) down: lane l owns bins 4 l ... 4 l + 3
+                constexpr int kPerLane = kFilterBins / 32;
                 unsigned long long mine = 0ull;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) mine += sh.tot[lane * 8 + j];
+                for (int j = 0; j < kPerLane; ++j) mine += sh.tot[lane * kPerLane + j];
                 unsigned long long incl = mine;          // inclusive scan over lanes
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -569,8 +625,8 @@ sample_filter_kernel(const SampleParams p)
                 // (with exact sums the last lane always reaches the target; the guard keeps the walk defined)
                 const int l = hit != 0u ? __ffs(hit) - 1 : 31;
                 if (lane == l) {
-                    int bin = lane * 8;
-                    for (int j = 0; j < 7; ++j, ++bin) {
+                    int bin = lane * kPerLane;
+                    for (int j = 0; j < kPerLane - 1; ++j, ++bin) {
                         if (run + sh.tot[bin] >= target) break;
                         run += sh.tot[bin];
                     }
@@ -578,7 +634,7 @@ sample_filter_kernel(const SampleParams p)
                     const unsigned long long v = static_cast<unsigned long long>(r.base) + static_cast<unsigned long long>(bin);
                     uint32_t lo = r.lo, hi = r.hi;
                     if (bin > 0) lo = static_cast<uint32_t>(max(static_cast<unsigned long long>(lo), v << r.shift));
-                    if (bin < 255) hi = static_cast<uint32_t>(min(static_cast<unsigned long long>(hi), ((v + 1ull) << r.shift) - 1ull));
+                    if (bin < kFilterBins - 1) hi = static_cast<uint32_t>(min(static_cast<unsigned long long>(hi), ((v + 1ull) << r.shift) - 1ull));
                     FilterRound q = r;
                     q.target = target; q.above = run; q.lo = lo; q.hi = hi;
                     q.n_sel = counted ? sh.totc[bin] : 0xffffffffu;
@@ -586,17 +642,17 @@ sample_filter_kernel(const SampleParams p)
                         q.next = 1;                     // few enough: collect them and rank them directly
                     } else if (lo == hi) {
                         if (r.phase == 0) {
-                            // one value of d, many entries: go on over the bits of z itself inside this group
-                            q.phase = 1; q.dsel = lo; q.lo = 0u; q.hi = 0xffffffffu; q.shift = 24; q.base = 0u;
+                            // one code of d, many entries: go on over the bits of z itself inside this group
+                            q.phase = 1; q.dsel = lo; q.lo = 0u; q.hi = 0xffffffffu; q.shift = 25; q.base = 0u;
                         } else {
                             q.next = 2;                 // one logit value: it is tau, and all its entries are kept
                             q.tau = key_to_float(~lo);
                             q.kept = run + sh.tot[bin];
                         }
                     } else {
-                        // cut the interval into (at most 257, the last two sharing a bin) equal parts
+                        // cut the interval into (at most 129, the last two sharing a bin) equal parts
                         const int width = 32 - __clz(hi - lo);
-                        q.shift = max(0, width - 8);
+                        q.shift = max(0, width - 7);
                         q.base = lo >> q.shift;
                     }
                     sh.r = q;
@@ -608,7 +664,7 @@ sample_filter_kernel(const SampleParams p)
         }
         const FilterRound r = sh.r;
         if (r.next == 1) {
-            // every CTA hands its entries of the chosen bin to all eight CTAs; each ranks them on its own
+            // every CTA hands its entries of the chosen bin to all four CTAs; each ranks them on its own
             scan(sel, r, nullptr, true);
             cluster_sync();
             const int nc = static_cast<int>(min(r.n_sel, static_cast<uint32_t>(kFilterCand)));
@@ -636,18 +692,17 @@ sample_filter_kernel(const SampleParams p)
     if (!do_p) {
         // top-k alone: the mass of the kept logits is one more pass (a plain reduction, no histogram)
         unsigned long long acc = 0ull;
-        const uint32_t b_hi = static_cast<uint32_t>(bin_of(__float_as_uint(m - floor_z), kFilterShift0, base0));
+        const uint32_t b_hi = code_of(m - floor_z, inv_dmax) >> kFilterShift0;
         for (int i = tid; i < n; i += kFilterThreads) {
             if (bytes_valid && s_bin0[i] > b_hi) continue;
-            const float z = __ldg(src + i);
-            if (mask_row != nullptr && !mask_allows(mask_row, v0 + i)) continue;
+            const float z = fetch(i);
             if (z >= floor_z) acc += mass_of(m - z, cf);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (lane == 0) sh.red64[warp] = acc;
         __syncthreads();
-        if (tid < kAcceptCluster) {
+        if (tid < kFilterCluster) {
             unsigned long long t = 0ull;
 #pragma unroll
             for (int w = 0; w < kFilterWarps; ++w) t += sh.red64[w];
@@ -656,7 +711,7 @@ sample_filter_kernel(const SampleParams p)
         cluster_sync();
         unsigned long long t = 0ull;
 #pragma unroll
-        for (int c = 0; c < kAcceptCluster; ++c) t += sh.slice_mass[c];
+        for (int c = 0; c < kFilterCluster; ++c) t += sh.slice_mass[c];
         kept_mass = static_cast<double>(t) / kMassUnit;
     }
     if (rank == 0 && tid == 0) {
@@ -666,11 +721,16 @@ sample_filter_kernel(const SampleParams p)
     cluster_sync();                                     // no CTA leaves while a peer may still read its shared memory
 }
 
+static size_t filter_smem_bytes(int vocab)
+{
+    const int per = ((vocab + kFilterCluster - 1) / kFilterCluster + 3) & ~3;
+    return (per <= kFilterCodesMax ? static_cast<size_t>(per) : 0) + static_cast<size_t>(2 * kFilterBins * 32) * sizeof(uint32_t);
+}
+
 cudaError_t launch_sample_filter(const SampleParams& p, bool pdl, cudaStream_t stream)
 {
-    const int per = ((p.vocab + kAcceptCluster - 1) / kAcceptCluster + 3) & ~3;
-    const size_t smem = per <= kFilterCodesMax ? static_cast<size_t>(per) + kFilterList * (sizeof(uint16_t) + sizeof(float)) : 0;
-    return launch_kernel_ex(sample_filter_kernel, dim3(kAcceptCluster, p.m_rows), dim3(kFilterThreads), smem, stream, pdl, p);
+    return launch_kernel_ex(sample_filter_kernel, dim3(kFilterCluster, p.m_rows), dim3(kFilterThreads), filter_smem_bytes(p.vocab),
+                            stream, pdl, p);
 }
 
 // ------------------------------------------------------------------------------------ acceptance
@@ -1130,8 +1190,12 @@ constexpr size_t kAcceptSmemMax = static_cast<size_t>(kAcceptWarps) * 4 * kSubCh
 
 cudaError_t sample_init()
 {
-    return cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                static_cast<int>(kAcceptSmemMax));
+    cudaError_t e = cudaFuncSetAttribute(sample_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kAcceptSmemMax));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(sample_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(filter_smem_bytes(kFilterCluster * kFilterCodesMax)));
+    return e;
 }
 
 cudaError_t launch_sample_accept(const SampleParams& p, bool pdl, cudaStream_t stream)
