@@ -92,6 +92,7 @@ void free_workspace(Handle& h)
         if (h.ev[i]) cudaEventDestroy(h.ev[i]);
     if (h.ev_fork) cudaEventDestroy(h.ev_fork);
     if (h.ev_join) cudaEventDestroy(h.ev_join);
+    if (h.ev_plan) cudaEventDestroy(h.ev_plan);
     if (h.side) cudaStreamDestroy(h.side);
     free(h.att_seq);
     h.att_seq = nullptr;
@@ -496,7 +497,8 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     if (rc == FLEXSPEC_OK &&
         (cudaStreamCreateWithFlags(&h.side, cudaStreamNonBlocking) != cudaSuccess ||
          cudaEventCreateWithFlags(&h.ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-         cudaEventCreateWithFlags(&h.ev_join, cudaEventDisableTiming) != cudaSuccess))
+         cudaEventCreateWithFlags(&h.ev_join, cudaEventDisableTiming) != cudaSuccess ||
+         cudaEventCreateWithFlags(&h.ev_plan, cudaEventDisableTiming) != cudaSuccess))
         rc = FLEXSPEC_ERR_CUDA;
     if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map, lm_head_w, static_cast<uint64_t>(c.vocab),
                                             static_cast<uint64_t>(d_model), 128);
@@ -594,13 +596,16 @@ int flexspec_sample(flexspec_handle* fh, const float* logits, const int32_t* dra
                       temperature, vocab_mask, accepted_len, next_token, s);
 }
 
-int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
-                    const int32_t* draft_tokens, const float* draft_logits,
-                    const int32_t* draft_len, const int32_t* draft_len_host,
-                    const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
-                    int32_t* accepted_len, int32_t* next_token, void* stream)
+// The step on device buffers.  dlog_in_flight: the draft logits are still being copied from the host on the
+// second stream (queued there by the caller before anything else).  Then the plan runs on the main stream,
+// the statistics of the draft logits wait for it behind the copy, and the main stream joins the second one
+// only before the decision, so that attention and the LM head run beside the copy.
+static int verify_impl(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
+                       const int32_t* draft_tokens, const float* draft_logits, bool dlog_in_flight,
+                       const int32_t* draft_len, const int32_t* draft_len_host,
+                       const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
+                       int32_t* accepted_len, int32_t* next_token, void* stream)
 {
-    NvtxRange nvtx_range("flexspec_verify");
     if (fh == nullptr || hidden == nullptr || draft_len == nullptr || accepted_len == nullptr ||
         next_token == nullptr)
         return FLEXSPEC_ERR_INVALID_ARG;
@@ -622,10 +627,18 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     mark(h, 0, s);
     // ---- second stream: row offsets of the ragged batch and the statistics of the draft logits need
     // nothing from the target model, so they run beside attention and the LM head
-    if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess)
-        return FLEXSPEC_ERR_CUDA;
-    rc = run_plan(h, draft_len, draft_tokens, batch, g, sp, h.side);
-    if (rc != FLEXSPEC_OK) return rc;
+    const bool host_copy = dlog_in_flight && draft_logits != nullptr && g.s_rows > 0;
+    if (host_copy) {
+        rc = run_plan(h, draft_len, draft_tokens, batch, g, sp, s);
+        if (rc != FLEXSPEC_OK) return rc;
+        if (cudaEventRecord(h.ev_plan, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_plan, 0) != cudaSuccess)
+            return FLEXSPEC_ERR_CUDA;
+    } else {
+        if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess)
+            return FLEXSPEC_ERR_CUDA;
+        rc = run_plan(h, draft_len, draft_tokens, batch, g, sp, h.side);
+        if (rc != FLEXSPEC_OK) return rc;
+    }
     if (!sp.greedy && sp.s_rows > 0) {
         if (launch_sample_stats(sp, sp.m_rows, sp.s_rows, h.side) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
         h.launches++;
@@ -637,9 +650,10 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 2, s);
     mark(h, 3, s);
-    // the second stream's work is long done by now; joining here keeps LM head -> decision -> draw
-    // back to back on this stream, so that the last two can be launched programmatically
-    if (cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    // With device inputs the second stream's work is long done by now; joining here keeps LM head -> decision
+    // -> draw back to back on this stream, so that the last two can be launched programmatically.  With the
+    // draft logits still on their way from the host the join waits until just before the decision.
+    if (!host_copy && cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     sp.tstats = h.tstats;                                                     // the LM head leaves the target rows' parts
     sp.n_tparts = 4 * (g.m_rows <= 512 ? h.lm_full_tiles + h.lm_last_tiles : (h.cfg.vocab + 127) / 128);
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
@@ -649,11 +663,23 @@ int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidd
         if (launch_sample_filter(sp, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;   // the plan's tables are there: joined above
         h.launches++;
     }
+    if (host_copy && cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     mark(h, 5, s);
-    if (launch_sample_accept(sp, true, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
+    if (launch_sample_accept(sp, !host_copy, s) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     h.launches++;
     mark(h, 6, s);
     return FLEXSPEC_OK;
+}
+
+int flexspec_verify(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
+                    const int32_t* draft_tokens, const float* draft_logits,
+                    const int32_t* draft_len, const int32_t* draft_len_host,
+                    const uint64_t* seeds, int32_t batch, float temperature, const uint32_t* vocab_mask,
+                    int32_t* accepted_len, int32_t* next_token, void* stream)
+{
+    NvtxRange nvtx_range("flexspec_verify");
+    return verify_impl(fh, kv, hidden, draft_tokens, draft_logits, false, draft_len, draft_len_host, seeds, batch,
+                       temperature, vocab_mask, accepted_len, next_token, stream);
 }
 
 int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void* hidden,
@@ -692,9 +718,10 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     auto H2D = [&](void* dst, const void* src, size_t bytes) {
         if (bytes > 0 && src != nullptr) ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
     };
-    // The draft logits are by far the largest input and nothing on the main stream needs them before the
-    // decision: they are copied on the second stream, beside attention and the LM head (the statistics
-    // kernel that reads them runs on that stream, behind the copy).
+    // The small inputs go first: host-to-device copies are served in the order they were issued, whatever their
+    // stream, and attention needs these.  The draft logits, by far the largest input, follow on the second
+    // stream (idle: the previous call ended with a synchronisation); nothing on the main stream needs them
+    // before the decision, so attention and the LM head run beside their copy.
     H2D(d_hidden, hidden, static_cast<size_t>(g.m_rows) * h.d_model * 2);
     H2D(d_tok, draft_tokens, static_cast<size_t>(g.s_rows) * 4);
     H2D(d_len, draft_len, static_cast<size_t>(batch) * 4);
@@ -702,20 +729,18 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
     H2D(d_seed, seeds, static_cast<size_t>(batch) * 8);
     H2D(d_mask, vocab_mask, mask_bytes);
     if (!ok) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
-    if (draft_logits != nullptr && g.s_rows > 0) {
-        if (cudaEventRecord(h.ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h.side, h.ev_fork, 0) != cudaSuccess ||
-            cudaMemcpyAsync(d_dlog, draft_logits, static_cast<size_t>(g.s_rows) * h.cfg.vocab * 4, cudaMemcpyHostToDevice,
-                            h.side) != cudaSuccess) {
-            cudaGetLastError();
-            return FLEXSPEC_ERR_CUDA;
-        }
+    const bool big = draft_logits != nullptr && g.s_rows > 0;
+    if (big && cudaMemcpyAsync(d_dlog, draft_logits, static_cast<size_t>(g.s_rows) * h.cfg.vocab * 4, cudaMemcpyHostToDevice,
+                               h.side) != cudaSuccess) {
+        cudaGetLastError();
+        return FLEXSPEC_ERR_CUDA;
     }
 
     flexspec_kv kv_dev = *kv;
     kv_dev.kv_len = d_kvl;
-    rc = flexspec_verify(fh, &kv_dev, d_hidden, d_tok, draft_logits ? d_dlog : nullptr, d_len, draft_len,
-                         seeds ? d_seed : nullptr, batch, temperature, vocab_mask ? d_mask : nullptr, h.out_dev,
-                         h.out_dev + batch, s);
+    rc = verify_impl(fh, &kv_dev, d_hidden, d_tok, draft_logits ? d_dlog : nullptr, big, d_len, draft_len,
+                     seeds ? d_seed : nullptr, batch, temperature, vocab_mask ? d_mask : nullptr, h.out_dev,
+                     h.out_dev + batch, s);
     if (rc != FLEXSPEC_OK) return rc;
     ok = cudaMemcpyAsync(accepted_len, h.out_dev, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(next_token, h.out_dev + batch, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;

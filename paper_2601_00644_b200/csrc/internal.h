@@ -160,7 +160,7 @@ struct Handle {
     void* stage_dev; size_t stage_bytes;
     int32_t* out_dev;
     // second stream: the plan and the draft-logit statistics run beside attention and the LM head
-    cudaStream_t side; cudaEvent_t ev_fork, ev_join;
+    cudaStream_t side; cudaEvent_t ev_fork, ev_join, ev_plan;
     // profiling
     int32_t profiling, launches;
     cudaEvent_t ev[kNumStageEvents];
