@@ -104,6 +104,8 @@ typedef struct {            /* DEVICE pointers into the handle's workspace, vali
     const double*  q_tok;      /* fp64 [S]  q_j(x_j)                                              */
     const float*   u_acc;      /* fp32 [S]  u_j                                                   */
     const int32_t* status;     /* int32 [4] device status word: [0] first error code, [1] detail  */
+    const double*  topp;       /* fp64 [M][2] per target row, written when top-k / top-p is on: the lowest kept
+                                  logit and the kept mass in units of the row's largest term          */
 } flexspec_debug;
 
 /* Create a handle for one target model's verification step (the frozen head and the KV-session

@@ -45,7 +45,7 @@ class KV(C.Structure):
 
 class Debug(C.Structure):
     _fields_ = [("attn_out", C.c_void_p), ("logits", C.c_void_p), ("p_tok", C.c_void_p),
-                ("q_tok", C.c_void_p), ("u_acc", C.c_void_p), ("status", C.c_void_p)]
+                ("q_tok", C.c_void_p), ("u_acc", C.c_void_p), ("status", C.c_void_p), ("topp", C.c_void_p)]
 
 
 def _load() -> C.CDLL:
@@ -313,6 +313,7 @@ class Verifier:
             "p_tok": self._view(d.p_tok, (s_rows,), torch.float64),
             "q_tok": self._view(d.q_tok, (s_rows,), torch.float64),
             "u": self._view(d.u_acc, (s_rows,), torch.float32),
+            "topp": self._view(d.topp, (m_rows, 2), torch.float64),
         }
 
     def set_top_p(self, top_p: float):

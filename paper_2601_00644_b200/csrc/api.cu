@@ -836,6 +836,7 @@ int flexspec_get_debug(flexspec_handle* fh, flexspec_debug* out)
     out->q_tok = h.dbg_q;
     out->u_acc = h.dbg_u;
     out->status = h.status;
+    out->topp = h.topp;
     return FLEXSPEC_OK;
 }
 

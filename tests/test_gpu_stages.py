@@ -459,3 +459,75 @@ def test_attention_sweep_matches_oracle(kw):
     kw = dict(kw)
     idx = kw.pop("idx")
     _attn_parity(_shape("att_sweep", idx, **kw))
+
+
+# ------------------------------------------------------------------ the filter's thresholds themselves
+
+def _filter_rows(vocab, seed):
+    """Rows that stress every path of the selection: ties by the thousand, one dominant token, duplicates
+    around the cut, a spread of 1e-4, -inf entries, a heavy tail, plain normal rows."""
+    rng = np.random.RandomState(seed)
+    rows = [
+        np.zeros(vocab),                                                     # all equal: one code, one logit value
+        (rng.rand(vocab) < 0.5).astype(np.float64),                          # two values
+        np.where(np.arange(vocab) == vocab // 3, 30.0, rng.standard_normal(vocab)),   # one dominant token
+        np.round(rng.standard_normal(vocab) * 2.0 * 4.0) / 4.0,              # multiples of 0.25: many exact duplicates
+        rng.standard_normal(vocab),
+        rng.standard_normal(vocab) * 1e-4,                                   # flatter than any window guess
+        np.where(rng.rand(vocab) < 0.2, -np.inf, rng.standard_normal(vocab)),
+        rng.exponential(5.0, vocab),                                         # heavy upper tail
+        rng.standard_normal(vocab) * 3.0 + 100.0,                            # large offset: coarse float grid
+        -rng.exponential(0.01, vocab),                                       # most entries a hair below the maximum
+    ]
+    return np.stack(rows).astype(np.float32)
+
+
+@pytest.mark.parametrize("top_p,top_k,temperature", [(0.9, 0, 1.0), (0.5, 0, 0.7), (0.999, 0, 1.0), (1.0, 1, 1.0),
+                                                      (1.0, 7, 1.0), (0.9, 50, 1.3), (1.0, 900, 1.0), (0.3, 3, 1.0)])
+@pytest.mark.parametrize("vocab", [1000, 1003, 32000, 140003])
+def test_filter_thresholds_match_their_definition(top_p, top_k, temperature, vocab):
+    """The lowest kept logit and the kept mass that the filter kernel leaves per row, against the definition
+    (sorted prefix in fp64 through the oracle's top-k / nucleus routines) on the same fp32 logits."""
+    B = _binding()
+    zt = _filter_rows(vocab, 13 * vocab + top_k)
+    rows = zt.shape[0]
+    k = np.zeros(rows, np.int32)
+    w = torch.zeros(vocab, 64, dtype=torch.bfloat16, device="cuda")
+    ver = B.Verifier(w, 1, 1, 64, max_batch=rows, k_max=1, max_kv_len=64, mode=0, debug=True)
+    ver.set_sampling(top_p=top_p, top_k=top_k)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).cuda()
+    seeds = np.arange(1, rows + 1, dtype=np.int64)
+    acc, nxt = ver.sample(dev(zt, torch.float32), dev(np.zeros(0, np.int32), torch.int32),
+                          dev(np.zeros((0, vocab), np.float32), torch.float32), dev(k, torch.int32),
+                          torch.from_numpy(k), dev(seeds, torch.int64), temperature=temperature)
+    torch.cuda.synchronize()
+    assert ver.status()[0] == 0
+    got = ver.debug(rows, 0)["topp"].cpu().numpy()
+    nxt = nxt.cpu().numpy()
+    checked = 0
+    for r in range(rows):
+        z = zt[r].astype(np.float64)
+        e = np.exp((z - z.max()) / temperature)
+        p = e / e.sum()
+        if 0 < top_k < vocab:
+            p = oracle.topk(p, top_k)
+        pk = p.copy()                                                        # the distribution the nucleus is cut from
+        margin = np.inf
+        if top_p < 1.0:
+            p, margin = oracle.nucleus(p, top_p)
+        kept = p > 0
+        assert kept[nxt[r]], (r, "emitted token outside the kept set")
+        kept_g = (z >= got[r, 0]) & np.isfinite(z)
+        if margin < 1e-6:
+            # the cut itself is a near-tie: the kernel's set must still be a minimal prefix within that slack
+            assert kept_g[pk > 0].any() and not kept_g[pk == 0].any(), r
+            assert pk[kept_g].sum() >= top_p - 2e-6 and pk[z > got[r, 0]].sum() < top_p + 2e-6, (r, pk[kept_g].sum())
+            continue
+        # the threshold is unique up to the gap below the lowest kept logit: compare the sets it defines
+        assert np.array_equal(kept_g, kept), (r, got[r, 0], z[kept].min(), int(kept.sum()), int(kept_g.sum()))
+        if kept.sum() < np.isfinite(z).sum():
+            assert got[r, 0] == z[kept].min(), (r, got[r, 0], z[kept].min())  # and it is the lowest kept logit itself
+        assert abs(got[r, 1] - e[kept].sum()) <= 2e-6 * e[kept].sum(), (r, got[r, 1], e[kept].sum())
+        checked += 1
+    assert checked >= 2
+    ver.close()
