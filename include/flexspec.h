@@ -110,10 +110,13 @@ typedef struct {            /* DEVICE pointers into the handle's workspace, vali
 
 /* Create a handle for one target model's verification step (the frozen head and the KV-session
  * layout of Sections IV-A and IV-C): validates the shape, allocates the workspace on cfg->device
- * (logits [max_batch*(k_max+1)][vocab] fp32, attention partials, small tables)
- * and builds the TMA descriptor of the LM-head weights.
+ * (logits [max_batch*(k_max+1)][vocab] fp32, the re-tiled copy of the LM-head weights, attention
+ * partials, small tables) and builds the TMA descriptors of that copy.
  *   lm_head_w : DEVICE bf16 [vocab][d_model] (row v is the output embedding of
- *               token v), 16-byte aligned, borrowed until flexspec_destroy.
+ *               token v), 16-byte aligned.  It is read during this call only: the handle keeps
+ *               its own copy (vocab * d_model * 2 bytes, rounded up to whole tiles) in the order
+ *               the LM head streams it, one contiguous block per pipeline stage; the caller may
+ *               free or overwrite its buffer afterwards (later changes are not seen).
  * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA, NO_DEVICE. */
 int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_handle** out);
 

@@ -85,7 +85,7 @@ void free_workspace(Handle& h)
 {
     cudaFree(h.attn_out); cudaFree(h.logits); cudaFree(h.part_o); cudaFree(h.part_ml); cudaFree(h.att_tickets);
     cudaFree(h.plan.cu_q); cudaFree(h.plan.cu_d); cudaFree(h.plan.row_seq); cudaFree(h.plan.k_eff); cudaFree(h.plan.row_c);
-    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.topp);
+    cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.topp); cudaFree(h.w_tiled);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
     for (int i = 0; i < kNumStageEvents; ++i)
@@ -310,8 +310,7 @@ int run_lm_head(Handle& h, const void* x, int32_t m_rows, float* logits, const S
     else { p.n_tile = 256; p.n_blocks = 2; }
     const int rows_per_pass = p.n_tile * p.n_blocks;
     p.n_pass = (m_rows + rows_per_pass - 1) / rows_per_pass;
-    if (p.n_pass == 1) { p.n_full_tiles = h.lm_full_tiles; p.last_rows = h.lm_last_rows; p.n_vtiles = h.lm_full_tiles + h.lm_last_tiles; }
-    else { p.n_vtiles = (c.vocab + 127) / 128; p.n_full_tiles = p.n_vtiles; p.last_rows = 128; }
+    p.n_full_tiles = h.lm_full_tiles; p.last_rows = h.lm_last_rows; p.n_vtiles = h.lm_full_tiles + h.lm_last_tiles;
     p.num_stages = lm_head_pick_stages(p.n_tile, p.n_blocks);
     p.n_bufs = 512 / p.n_tile < 4 ? 512 / p.n_tile : 4;       // what fits into the 512 TMEM columns, four at most
     p.tstats = nullptr; p.n_tparts = 0; p.inv_temp_log2 = 1.f; p.greedy = 0;
@@ -435,7 +434,6 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     h.max_m = static_cast<int32_t>(max_m);
     h.max_s = c.max_batch * c.k_max;
     h.sm_count = prop.multiProcessorCount;
-    h.w = static_cast<const __nv_bfloat16*>(lm_head_w);
     h.top_p = 1.f;
     h.att_seq = static_cast<SeqBlocks*>(malloc(sizeof(SeqBlocks) * static_cast<size_t>(c.max_batch)));
     if (h.att_seq == nullptr) { delete fh; return FLEXSPEC_ERR_OOM; }
@@ -500,10 +498,16 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
          cudaEventCreateWithFlags(&h.ev_join, cudaEventDisableTiming) != cudaSuccess ||
          cudaEventCreateWithFlags(&h.ev_plan, cudaEventDisableTiming) != cudaSuccess))
         rc = FLEXSPEC_ERR_CUDA;
-    if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map, lm_head_w, static_cast<uint64_t>(c.vocab),
-                                            static_cast<uint64_t>(d_model), 128);
-    if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map_last, lm_head_w, static_cast<uint64_t>(c.vocab),
-                                            static_cast<uint64_t>(d_model), static_cast<uint32_t>(h.lm_last_rows));
+    // W is copied once into the order the LM head streams it (a stage of its pipeline = one contiguous block);
+    // the caller's buffer is not needed afterwards
+    const uint64_t w_rows = static_cast<uint64_t>(h.lm_full_tiles) * 128 + static_cast<uint64_t>(h.lm_last_tiles) * h.lm_last_rows;
+    A(dev_alloc(&h.w_tiled, static_cast<size_t>(w_rows) * d_model));
+    if (rc == FLEXSPEC_OK &&
+        (launch_retile_w(lm_head_w, h.w_tiled, c.vocab, d_model, h.lm_full_tiles, h.lm_last_tiles, h.lm_last_rows, nullptr) != cudaSuccess ||
+         cudaStreamSynchronize(nullptr) != cudaSuccess))
+        rc = FLEXSPEC_ERR_CUDA;
+    if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map, h.w_tiled, w_rows * (d_model / 64), 64, 128);
+    if (rc == FLEXSPEC_OK) rc = make_map_2d(&h.w_map_last, h.w_tiled, w_rows * (d_model / 64), 64, static_cast<uint32_t>(h.lm_last_rows));
     if (rc == FLEXSPEC_OK && (attention_init(c.head_dim) != cudaSuccess || lm_head_init() != cudaSuccess || sample_init() != cudaSuccess))
         rc = FLEXSPEC_ERR_CUDA;
     if (rc != FLEXSPEC_OK) {
@@ -655,7 +659,7 @@ static int verify_impl(flexspec_handle* fh, const flexspec_kv* kv, const void* h
     // draft logits still on their way from the host the join waits until just before the decision.
     if (!host_copy && cudaStreamWaitEvent(s, h.ev_join, 0) != cudaSuccess) return FLEXSPEC_ERR_CUDA;
     sp.tstats = h.tstats;                                                     // the LM head leaves the target rows' parts
-    sp.n_tparts = 4 * (g.m_rows <= 512 ? h.lm_full_tiles + h.lm_last_tiles : (h.cfg.vocab + 127) / 128);
+    sp.n_tparts = 4 * (h.lm_full_tiles + h.lm_last_tiles);
     rc = run_lm_head(h, h.attn_out, g.m_rows, h.logits, &sp, s);
     if (rc != FLEXSPEC_OK) return rc;
     mark(h, 4, s);

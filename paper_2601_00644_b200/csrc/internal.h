@@ -144,8 +144,8 @@ struct Handle {
     SeqBlocks* att_seq;       // HOST [max_batch]
     int32_t d_model, max_m, max_s;
     int32_t sm_count;
-    const __nv_bfloat16* w;
-    CUtensorMap w_map;
+    __nv_bfloat16* w_tiled;   // the handle's copy of W in streaming order: [tile][k block][tile rows][64]
+    CUtensorMap w_map;        // over w_tiled viewed as rows of 64 elements, box of 128 rows (one k block of a full tile)
     CUtensorMap w_map_last;   // same tensor, box of lm_last_rows rows (tiles of the last wave)
     int32_t lm_full_tiles, lm_last_rows, lm_last_tiles;
     // workspace
@@ -177,6 +177,8 @@ cudaError_t launch_plan(const int32_t* draft_len, const int32_t* draft_tokens, i
 cudaError_t launch_attention(const Handle& h, const CUtensorMap& kv_map, const AttnParams& p, const AttTable& table,
                              int32_t n_ctas, cudaStream_t stream);
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream);
+cudaError_t launch_retile_w(const void* w, void* out, int vocab, int d_model, int n_full, int n_last, int last_rows,
+                            cudaStream_t stream);
 cudaError_t launch_sample_stats(const SampleParams& p, int32_t row_begin, int32_t row_count, cudaStream_t stream);
 // pdl: launch with programmatic stream serialization (the kernel may start while its predecessor in
 // the stream drains; it waits on the device before touching the predecessor's results)

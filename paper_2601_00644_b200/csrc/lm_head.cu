@@ -105,13 +105,17 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int vt = tile / p.n_pass, pass = tile % p.n_pass;
+                // the tile's k blocks lie one after the other in the re-tiled copy of W, w_rows rows of 64 elements each
+                const int w_rows = vt < p.n_full_tiles ? kLmBlockV : p.last_rows;
+                const int w_row0 = vt < p.n_full_tiles ? vt * num_kb * kLmBlockV
+                                                       : (p.n_full_tiles * kLmBlockV + (vt - p.n_full_tiles) * p.last_rows) * num_kb;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, p.status, 2)) { ok = false; break; }
                     uint8_t* st = smem + s * stage_bytes;
                     const bool full_tile = vt < p.n_full_tiles;
                     mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(full_tile ? stage_bytes
                                                                                           : p.last_rows * 128 + b_bytes));
-                    tma_load_2d(st, full_tile ? &w_map : &w_map_last, &full_bar[s], kb * kLmBlockK, tile_row0(vt), pol_w);
+                    tma_load_2d(st, full_tile ? &w_map : &w_map_last, &full_bar[s], 0, w_row0 + kb * w_rows, pol_w);
                     for (int nb = 0; nb < p.n_blocks; ++nb)
                         tma_load_2d(st + kLmATileBytes + nb * p.n_tile * 128, &x_map, &full_bar[s], kb * kLmBlockK,
                                     pass * rows_per_pass + nb * p.n_tile, pol_x);
@@ -256,6 +260,45 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 cudaError_t lm_head_init()
 {
     return cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmemLimit);
+}
+
+// W in the order the kernel streams it: for every vocabulary tile (n_full tiles of 128 rows, then n_last tiles of
+// last_rows rows) its d / 64 k blocks one after the other, each a [tile rows][64] bf16 block (16 KB for a full
+// tile), so that a stage of the pipeline is one contiguous piece of memory instead of 128 pieces of 128 bytes a
+// whole row of W apart.  Rows past the vocabulary are zero.  One thread moves 16 bytes.
+__global__ void retile_w_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ out, int vocab, int d_model,
+                                int n_full, int n_last, int last_rows)
+{
+    const int num_kb = d_model / kLmBlockK;
+    const int64_t rows_total = static_cast<int64_t>(n_full) * kLmBlockV + static_cast<int64_t>(n_last) * last_rows;
+    const int64_t n_chunks = rows_total * num_kb * 8;                 // 16-byte chunks of the copy
+    const int64_t full_rows = static_cast<int64_t>(n_full) * num_kb * kLmBlockV;
+    for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; q < n_chunks; q += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t R = q >> 3;                                     // row of 64 elements in the copy
+        const int c = static_cast<int>(q & 7);
+        int64_t src_row;
+        int kb;
+        if (R < full_rows) {
+            const int64_t t = R / kLmBlockV;
+            src_row = (t / num_kb) * kLmBlockV + R % kLmBlockV;
+            kb = static_cast<int>(t % num_kb);
+        } else {
+            const int64_t t = (R - full_rows) / last_rows;
+            src_row = static_cast<int64_t>(n_full) * kLmBlockV + (t / num_kb) * last_rows + (R - full_rows) % last_rows;
+            kb = static_cast<int>(t % num_kb);
+        }
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (src_row < vocab) v = *reinterpret_cast<const uint4*>(w + src_row * d_model + kb * kLmBlockK + c * 8);
+        *reinterpret_cast<uint4*>(out + q * 8) = v;
+    }
+}
+
+cudaError_t launch_retile_w(const void* w, void* out, int vocab, int d_model, int n_full, int n_last, int last_rows,
+                            cudaStream_t stream)
+{
+    retile_w_kernel<<<2048, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(w), static_cast<__nv_bfloat16*>(out), vocab, d_model,
+                                              n_full, n_last, last_rows);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_lm_head(const Handle& h, const CUtensorMap& x_map, const LmHeadParams& p, cudaStream_t stream)

@@ -27,6 +27,8 @@ def _rand_bf16(gen, shape, std):
     (100, 256, 777),         # vocab not a multiple of 4, rows not a multiple of 16
     (300, 512, 1300),        # two accumulator blocks (single TMEM buffer)
     (600, 256, 1000),        # two passes over W
+    (40, 192, 20011),        # more tiles than SMs: full waves, then a wave of short tiles (re-tiled copy of W, both boxes)
+    (530, 128, 19500),       # the same with two passes
 ])
 def test_lm_head_matches_oracle(m, d, v):
     B = _binding()
