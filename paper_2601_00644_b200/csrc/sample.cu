@@ -509,9 +509,11 @@ sample_filter_kernel(const SampleParams p)
                     __syncthreads();
                 }
                 uint32_t* col = s_big + lane;
-                // (top-p as the first selection has no floor yet, and an entry that cannot be selected is -inf: its
-                // distance clamps into the last bin and its mass is 0, so it needs no test of its own)
-                const bool plain = sel != 0 && !do_k;
+                // (the first selection of the kernel has no floor yet, and an entry that cannot be selected is -inf: its
+                // distance clamps into the last bin, where its mass is 0 and a count too many only matters to a
+                // top-k that reaches down there -- the next round counts that bin's live entries exactly, and a k
+                // beyond them keeps every logit, as it should)
+                const bool plain = round_no == 0;
                 auto entries4 = [&](const float* zin, int i0) {
                     float z[4] = {zin[0], zin[1], zin[2], zin[3]};
                     if (mask_row != nullptr) {
@@ -525,10 +527,14 @@ sample_filter_kernel(const SampleParams p)
                         const float d = m - z[u];
                         tb[u] = __float_as_uint(fminf(fmaf(d, inv_dmax, 1.f), 1.99999988f));
                         if (plain) {
-                            const uint32_t w = mass_of(d, cf);
                             uint32_t* at = col + ((tb[u] >> 11) & 0xfe0u);         // bin * 32 words
-                            atomicAdd(at, w >> 16);
-                            atomicAdd(at + kFilterBins * 32, w & 0xffffu);
+                            if (sel == 0) {
+                                atomicAdd(at, 1u);
+                            } else {
+                                const uint32_t w = mass_of(d, cf);
+                                atomicAdd(at, w >> 16);
+                                atomicAdd(at + kFilterBins * 32, w & 0xffffu);
+                            }
                         } else {
                             const bool live = z[u] >= floor_z && d >= 0.f;
                             if (!live) tb[u] = 0x3fff0000u;                         // the last bin
