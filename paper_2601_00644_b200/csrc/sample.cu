@@ -1095,20 +1095,47 @@ sample_accept_kernel(const SampleParams p)
             const float* zd_s = zt_s + kSubChunk;
             const int v0 = sub_base(sidx) + lane * kGroup;
             float mr = 0.f, mp = 0.f;
+            if (row.plain && sub_base(sidx) + kSubChunk <= p.vocab) {
+                // no mask, no nucleus, no ragged end: nothing depends on the entry's index, so the 16 exponentials
+                // of a lane (32 with the draft's) are independent instructions the scheduler can overlap; the
+                // sums are then taken in the entries' order, exactly as in the general loop below
+                float ze[kGroup], zq[kGroup];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int pos = lane * kGroup + ((j ^ ((lane >> 1) & 3)) << 2);
-                const float4 a = *reinterpret_cast<const float4*>(zt_s + pos);
-                float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (row.residual) d = *reinterpret_cast<const float4*>(zd_s + pos);
-                const float za[4] = {a.x, a.y, a.z, a.w}, zq[4] = {d.x, d.y, d.z, d.w};
+                for (int j = 0; j < 4; ++j) {
+                    const int pos = lane * kGroup + ((j ^ ((lane >> 1) & 3)) << 2);
+                    const float4 a = *reinterpret_cast<const float4*>(zt_s + pos);
+                    ze[4 * j + 0] = a.x; ze[4 * j + 1] = a.y; ze[4 * j + 2] = a.z; ze[4 * j + 3] = a.w;
+                    if (row.residual) {
+                        const float4 d = *reinterpret_cast<const float4*>(zd_s + pos);
+                        zq[4 * j + 0] = d.x; zq[4 * j + 1] = d.y; zq[4 * j + 2] = d.z; zq[4 * j + 3] = d.w;
+                    }
+                }
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int v = v0 + 4 * j + e;
-                    if (v < p.vocab) {
-                        const float ep = row.e_p(za[e], v);
-                        mp += ep;
-                        if (row.residual) mr += fmaxf(fmaf(-row.rho, row.e_q(zq[e]), ep), 0.f);
+                for (int i = 0; i < kGroup; ++i) ze[i] = fast_exp2((ze[i] - row.mp) * row.c);
+                if (row.residual) {
+#pragma unroll
+                    for (int i = 0; i < kGroup; ++i) zq[i] = fmaxf(fmaf(-row.rho, fast_exp2((zq[i] - row.mq) * row.c), ze[i]), 0.f);
+#pragma unroll
+                    for (int i = 0; i < kGroup; ++i) mr += zq[i];
+                }
+#pragma unroll
+                for (int i = 0; i < kGroup; ++i) mp += ze[i];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int pos = lane * kGroup + ((j ^ ((lane >> 1) & 3)) << 2);
+                    const float4 a = *reinterpret_cast<const float4*>(zt_s + pos);
+                    float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (row.residual) d = *reinterpret_cast<const float4*>(zd_s + pos);
+                    const float za[4] = {a.x, a.y, a.z, a.w}, zq[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int v = v0 + 4 * j + e;
+                        if (v < p.vocab) {
+                            const float ep = row.e_p(za[e], v);
+                            mp += ep;
+                            if (row.residual) mr += fmaxf(fmaf(-row.rho, row.e_q(zq[e]), ep), 0.f);
+                        }
                     }
                 }
             }
