@@ -779,6 +779,7 @@ constexpr int kAcceptRowsPerCta = (kMaxK + 1 + kAcceptCluster - 1) / kAcceptClus
 struct RowResult {
     double s_p, s_q, tau;             // sum of 2^((z - max) * c) of the target / draft row; lowest kept logit of the nucleus
     float m_p, m_q;                   // maxima (logit units)
+    float rho;                        // s_p / s_q of a row that has a draft row (the residual's scale), else 0
     int32_t rej;                      // 1: this row's draft token is rejected
     int32_t argmax;                   // GREEDY: lowest index holding the row's maximum
 };
@@ -981,7 +982,7 @@ sample_accept_kernel(const SampleParams p)
                     if (red_f[w] > m || (red_f[w] == m && red_i[w] < best)) { m = red_f[w]; best = red_i[w]; }
                 s_tmp.argmax = best;
                 s_tmp.rej = (test_row && x != best) ? 1 : 0;
-                s_tmp.m_p = m; s_tmp.m_q = 0.f; s_tmp.s_p = 1.0; s_tmp.s_q = 1.0; s_tmp.tau = -INFINITY;
+                s_tmp.m_p = m; s_tmp.m_q = 0.f; s_tmp.s_p = 1.0; s_tmp.s_q = 1.0; s_tmp.tau = -INFINITY; s_tmp.rho = 0.f;
             }
         } else {
             float m = -INFINITY, sf = 0.f;
@@ -1022,6 +1023,7 @@ sample_accept_kernel(const SampleParams p)
                 }
                 s_tmp.m_p = m; s_tmp.s_p = sm; s_tmp.tau = tau;
                 s_tmp.m_q = static_cast<float>(s_mq[i]); s_tmp.s_q = s_sq[i];
+                s_tmp.rho = test_row ? static_cast<float>(sm / s_sq[i]) : 0.f;
                 s_tmp.rej = rej; s_tmp.argmax = 0;
             }
         }
@@ -1061,7 +1063,7 @@ sample_accept_kernel(const SampleParams p)
     row.mask = (p.vocab_mask != nullptr) ? p.vocab_mask + static_cast<int64_t>(b) * p.mask_words : nullptr;
     row.mp = s_row[n].m_p;
     row.mq = row.residual ? s_row[n].m_q : 0.f;
-    row.rho = row.residual ? static_cast<float>(s_row[n].s_p / s_row[n].s_q) : 0.f;
+    row.rho = row.residual ? s_row[n].rho : 0.f;
     row.tau = static_cast<float>(s_row[n].tau);
     row.plain = (row.mask == nullptr && row.tau == -INFINITY);
     row.c = cf;
