@@ -88,6 +88,7 @@ void free_workspace(Handle& h)
     cudaFree(h.stats); cudaFree(h.tstats); cudaFree(h.topp); cudaFree(h.w_tiled);
     cudaFree(h.dbg_p); cudaFree(h.dbg_q); cudaFree(h.dbg_u); cudaFree(h.status);
     cudaFree(h.stage_dev); cudaFree(h.out_dev);
+    if (h.out_host) cudaFreeHost(h.out_host);
     for (int i = 0; i < kNumStageEvents; ++i)
         if (h.ev[i]) cudaEventDestroy(h.ev[i]);
     if (h.ev_fork) cudaEventDestroy(h.ev_fork);
@@ -478,6 +479,11 @@ int flexspec_create(const flexspec_config* cfg, const void* lm_head_w, flexspec_
     A(dev_alloc(&h.dbg_u, static_cast<size_t>(h.max_s)));
     A(dev_alloc(&h.status, 4));
     A(dev_alloc(&h.out_dev, static_cast<size_t>(2) * c.max_batch));
+    if (rc == FLEXSPEC_OK && cudaMallocHost(reinterpret_cast<void**>(&h.out_host), static_cast<size_t>(2) * c.max_batch * sizeof(int32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        h.out_host = nullptr;
+        rc = FLEXSPEC_ERR_OOM;
+    }
     if (rc == FLEXSPEC_OK) {
         // staging for flexspec_verify_host: hidden | draft logits | tokens | lengths (2) | seeds
         h.stage_bytes = static_cast<size_t>(max_m) * d_model * 2 + static_cast<size_t>(h.max_s) * c.vocab * 4 +
@@ -746,10 +752,13 @@ int flexspec_verify_host(flexspec_handle* fh, const flexspec_kv* kv, const void*
                      seeds ? d_seed : nullptr, batch, temperature, vocab_mask ? d_mask : nullptr, h.out_dev,
                      h.out_dev + batch, s);
     if (rc != FLEXSPEC_OK) return rc;
-    ok = cudaMemcpyAsync(accepted_len, h.out_dev, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(next_token, h.out_dev + batch, static_cast<size_t>(batch) * 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    // both result arrays lie side by side on the device: one copy into the handle's pinned buffer, then two
+    // 4 * batch byte copies on the host
+    ok = cudaMemcpyAsync(h.out_host, h.out_dev, static_cast<size_t>(batch) * 8, cudaMemcpyDeviceToHost, s) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return FLEXSPEC_ERR_CUDA; }
+    memcpy(accepted_len, h.out_host, static_cast<size_t>(batch) * 4);
+    memcpy(next_token, h.out_host + batch, static_cast<size_t>(batch) * 4);
     return FLEXSPEC_OK;
 }
 

@@ -159,6 +159,7 @@ struct Handle {
     // host staging for flexspec_verify_host
     void* stage_dev; size_t stage_bytes;
     int32_t* out_dev;
+    int32_t* out_host;        // pinned: both result arrays of the host-buffer entry point come back in one copy
     // second stream: the plan and the draft-logit statistics run beside attention and the LM head
     cudaStream_t side; cudaEvent_t ev_fork, ev_join, ev_plan;
     // profiling
