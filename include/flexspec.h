@@ -27,8 +27,8 @@
  *     host before any launch.
  *   - "DEVICE" pointers are CUDA global-memory addresses on the handle's
  *     device, "HOST" pointers ordinary host memory.  The caller owns every
- *     input and output buffer; the handle owns only its workspace and borrows
- *     the LM-head weight pointer for its lifetime.
+ *     input and output buffer; the handle owns its workspace, which includes
+ *     its own re-tiled copy of the LM-head weights (made by flexspec_create).
  *   - Calls that take a stream are asynchronous on it; outputs are valid once
  *     the stream has been synchronised.  A handle is not thread-safe and must
  *     be used on one stream at a time.

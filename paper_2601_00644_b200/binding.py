@@ -153,7 +153,6 @@ class Verifier:
                  max_batch: int, k_max: int, max_kv_len: int, mode: int = MODE_SAMPLE,
                  debug: bool = False, page_size: int = 16):
         _dev(lm_head_w, torch.bfloat16, "lm_head_w")
-        self.w = lm_head_w                      # keep alive: the handle borrows the pointer
         self.vocab = int(lm_head_w.shape[0])
         self.d_model = int(lm_head_w.shape[1])
         self.cfg = Config(n_q_heads, n_kv_heads, head_dim, self.vocab, page_size, max_batch, k_max,
