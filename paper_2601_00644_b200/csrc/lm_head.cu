@@ -149,12 +149,25 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
                     const uint32_t b_addr = a_addr + kLmATileBytes;
-                    for (int nb = 0; nb < p.n_blocks; ++nb) {
+                    if (p.n_blocks == 1) {
 #pragma unroll
                         for (int k = 0; k < kLmBlockK / kLmUmmaK; ++k) {
                             const uint64_t da = umma_desc_k_sw128(a_addr + k * kLmUmmaK * 2);
-                            const uint64_t db = umma_desc_k_sw128(b_addr + nb * p.n_tile * 128 + k * kLmUmmaK * 2);
-                            umma_bf16(nb ? acc1 : acc0, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                            const uint64_t db = umma_desc_k_sw128(b_addr + k * kLmUmmaK * 2);
+                            umma_bf16(acc0, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        }
+                    } else {
+                        // two blocks of token columns share the W tile: the two MMAs of a 16-wide slice follow one
+                        // another, the first keeps its A operand in the collector and the second takes it from
+                        // there, so the slice of W is read from shared memory once, not twice
+#pragma unroll
+                        for (int k = 0; k < kLmBlockK / kLmUmmaK; ++k) {
+                            const uint64_t da = umma_desc_k_sw128(a_addr + k * kLmUmmaK * 2);
+                            const uint64_t db0 = umma_desc_k_sw128(b_addr + k * kLmUmmaK * 2);
+                            const uint64_t db1 = umma_desc_k_sw128(b_addr + p.n_tile * 128 + k * kLmUmmaK * 2);
+                            const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
+                            umma_bf16_a_fill(acc0, da, db0, idesc, accum);
+                            umma_bf16_a_lastuse(acc1, da, db1, idesc, accum);
                         }
                     }
                     umma_commit(&empty_bar[s]);          // stage is free once these MMAs have read it
