@@ -8,7 +8,7 @@
 // vocabulary rows, a warp's store of one token column is 32 consecutive floats of a logits row.
 //
 // Persistent CTAs (one per SM) walk over the vocabulary tiles.  Warp 0 is the TMA producer, warp 1
-// issues tcgen05.mma from one thread and owns the TMEM allocation, warps 2..5 drain the
+// issues tcgen05.mma from one thread and owns the TMEM allocation, warps 2..9 drain the
 // accumulators.  Shared-memory stages and the (double-buffered, when it fits) accumulators are
 // handed over through mbarriers; every wait is bounded.
 //
@@ -24,7 +24,8 @@ namespace fs {
 constexpr int kLmBlockV = 128;          // vocabulary rows per tile (MMA M)
 constexpr int kLmBlockK = 64;           // bf16 elements per 128-byte swizzle row
 constexpr int kLmUmmaK = 16;
-constexpr int kLmThreads = 192;
+constexpr int kLmThreads = 320;         // TMA warp, MMA warp, eight epilogue warps
+constexpr int kLmEpilogueWarps = 8;
 constexpr int kLmMaxStages = 12;
 constexpr int kLmATileBytes = kLmBlockV * kLmBlockK * 2;     // 16 KB
 constexpr int kLmTmemCols = 512;
@@ -65,7 +66,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int a = 0; a < p.n_bufs; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 4); }
+        for (int a = 0; a < p.n_bufs; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], kLmEpilogueWarps); }
         fence_barrier_init();
         tma_prefetch_desc(&w_map);
         tma_prefetch_desc(&w_map_last);
@@ -181,8 +182,11 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (4 warps)
+        // ------------------------------------------------------------------ epilogue (8 warps)
+        // two warps per quarter of the TMEM lanes (a warp reaches the lanes 32 * (warp % 4) ...): one takes the
+        // even groups of 16 token columns, the other the odd ones
         const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31
+        const int half = (warp - 2) >> 2;
         int seq = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -196,7 +200,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             const int row_base = pass * rows_per_pass + nb * p.n_tile;
             const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                     static_cast<uint32_t>(slot * p.n_tile);
-            for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+            for (int c0 = half * 16; c0 < p.n_tile; c0 += 32) {
                 if (row_base + c0 >= p.m_rows) break;    // warp-uniform
                 uint32_t r[16];
                 tmem_ld_x16(taddr0 + static_cast<uint32_t>(c0), r);
@@ -241,17 +245,31 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                         for (int i = 0; i < 16; ++i)
                             sc[i] = fast_exp2((zv[i] - ((mx[i] == -INFINITY) ? 0.f : mx[i])) *
                                               (p.row_c != nullptr ? __shfl_sync(0xffffffffu, c_lane, i) : p.inv_temp_log2));
+                        // 16 sums over the 32 lanes by halving exchanges (8 + 4 + 2 + 1 + 1 shuffles instead of 80):
+                        // a lane keeps the half of the columns its lane bit selects and adds its partner's share,
+                        // so that lanes 2 c and 2 c + 1 end up with the sum of column c
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1)
+                        for (int o = 16, w = 8; o > 1; o >>= 1, w >>= 1) {
+                            const bool up = (lane & o) != 0;
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) sc[i] += __shfl_xor_sync(0xffffffffu, sc[i], o);
+                            for (int i = 0; i < 8; ++i) {
+                                if (i < w) {
+                                    const float give = up ? sc[i] : sc[i + w];
+                                    const float keep = up ? sc[i + w] : sc[i];
+                                    sc[i] = keep + __shfl_xor_sync(0xffffffffu, give, o);
+                                }
+                            }
+                        }
+                        sc[0] += __shfl_xor_sync(0xffffffffu, sc[0], 1);
                     }
-                    float part_m = -INFINITY, part_s = 0.f;
+                    // lane l now holds column l >> 1 (GREEDY: every lane holds all 16 arg-max indices)
+                    const int col = lane >> 1;
+                    float part_m = -INFINITY, part_s = p.greedy ? 0.f : sc[0];
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        if (lane == i) { part_m = mx[i]; part_s = sc[i]; }
-                    if (lane < 16 && row_base + c0 + lane < p.m_rows)
-                        p.tstats[static_cast<int64_t>(row_base + c0 + lane) * p.n_tparts + vt * 4 + quarter] =
+                        if (col == i) { part_m = mx[i]; if (p.greedy) part_s = sc[i]; }
+                    if ((lane & 1) == 0 && row_base + c0 + col < p.m_rows)
+                        p.tstats[static_cast<int64_t>(row_base + c0 + col) * p.n_tparts + vt * 4 + quarter] =
                             make_float2(part_m, part_s);
                 }
             }
