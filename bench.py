@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one lm_head_kernel launch, per workload, from the ncu
 # captures summarised in profiles/ (a workload without a capture of the current kernel reports null)
-LM_HEAD_TRAFFIC_BYTES = {"llama3_8b": 1051993000 + 8599552}
+LM_HEAD_TRAFFIC_BYTES = {"llama3_8b": 1052039000 + 9035520}
 FALLBACK_HBM_GBS = 6650.0
 REFERENCE_BUDGET_S = 120.0
 
