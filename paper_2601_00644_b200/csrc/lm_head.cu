@@ -8,7 +8,7 @@
 // vocabulary rows, a warp's store of one token column is 32 consecutive floats of a logits row.
 //
 // Persistent CTAs (one per SM) walk over the vocabulary tiles.  Warp 0 is the TMA producer, warp 1
-// issues tcgen05.mma from one thread and owns the TMEM allocation, warps 2..9 drain the
+// issues tcgen05.mma from one thread and owns the TMEM allocation, warps 2..17 drain the
 // accumulators.  Shared-memory stages and the (double-buffered, when it fits) accumulators are
 // handed over through mbarriers; every wait is bounded.
 //
@@ -24,8 +24,8 @@ namespace fs {
 constexpr int kLmBlockV = 128;          // vocabulary rows per tile (MMA M)
 constexpr int kLmBlockK = 64;           // bf16 elements per 128-byte swizzle row
 constexpr int kLmUmmaK = 16;
-constexpr int kLmThreads = 320;         // TMA warp, MMA warp, eight epilogue warps
-constexpr int kLmEpilogueWarps = 8;
+constexpr int kLmEpilogueWarps = 16;
+constexpr int kLmThreads = (2 + kLmEpilogueWarps) * 32;   // TMA warp, MMA warp, epilogue warps
 constexpr int kLmMaxStages = 12;
 constexpr int kLmATileBytes = kLmBlockV * kLmBlockK * 2;     // 16 KB
 constexpr int kLmTmemCols = 512;
@@ -182,9 +182,9 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (8 warps)
-        // two warps per quarter of the TMEM lanes (a warp reaches the lanes 32 * (warp % 4) ...): one takes the
-        // even groups of 16 token columns, the other the odd ones
+        // ------------------------------------------------------------------ epilogue (16 warps)
+        // four warps per quarter of the TMEM lanes (a warp reaches the lanes 32 * (warp % 4) ...), each taking
+        // every fourth group of 16 token columns
         const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31
         const int half = (warp - 2) >> 2;
         int seq = 0;
@@ -200,7 +200,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             const int row_base = pass * rows_per_pass + nb * p.n_tile;
             const uint32_t taddr0 = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                     static_cast<uint32_t>(slot * p.n_tile);
-            for (int c0 = half * 16; c0 < p.n_tile; c0 += 32) {
+            for (int c0 = half * 16; c0 < p.n_tile; c0 += (kLmEpilogueWarps / 4) * 16) {
                 if (row_base + c0 >= p.m_rows) break;    // warp-uniform
                 uint32_t r[16];
                 tmem_ld_x16(taddr0 + static_cast<uint32_t>(c0), r);
