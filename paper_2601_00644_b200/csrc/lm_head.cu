@@ -104,24 +104,28 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             int last_s = -1;
             uint32_t last_ph = 0;
             bool ok = true;
+            uint8_t* st = smem;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int vt = tile / p.n_pass, pass = tile % p.n_pass;
                 // the tile's k blocks lie one after the other in the re-tiled copy of W, w_rows rows of 64 elements each
                 const int w_rows = vt < p.n_full_tiles ? kLmBlockV : p.last_rows;
                 const int w_row0 = vt < p.n_full_tiles ? vt * num_kb * kLmBlockV
                                                        : (p.n_full_tiles * kLmBlockV + (vt - p.n_full_tiles) * p.last_rows) * num_kb;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const bool full_tile = vt < p.n_full_tiles;
+                const CUtensorMap* wm = full_tile ? &w_map : &w_map_last;
+                const uint32_t tx = static_cast<uint32_t>(full_tile ? stage_bytes : p.last_rows * 128 + b_bytes);
+                const int x_row0 = pass * rows_per_pass;
+                int w_row = w_row0;
+                for (int kb = 0; kb < num_kb; ++kb, w_row += w_rows) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, p.status, 2)) { ok = false; break; }
-                    uint8_t* st = smem + s * stage_bytes;
-                    const bool full_tile = vt < p.n_full_tiles;
-                    mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(full_tile ? stage_bytes
-                                                                                          : p.last_rows * 128 + b_bytes));
-                    tma_load_2d(st, full_tile ? &w_map : &w_map_last, &full_bar[s], 0, w_row0 + kb * w_rows, pol_w);
-                    for (int nb = 0; nb < p.n_blocks; ++nb)
-                        tma_load_2d(st + kLmATileBytes + nb * p.n_tile * 128, &x_map, &full_bar[s], kb * kLmBlockK,
-                                    pass * rows_per_pass + nb * p.n_tile, pol_x);
+                    mbar_arrive_expect_tx(&full_bar[s], tx);
+                    tma_load_2d(st, wm, &full_bar[s], 0, w_row, pol_w);
+                    tma_load_2d(st + kLmATileBytes, &x_map, &full_bar[s], kb * kLmBlockK, x_row0, pol_x);
+                    if (p.n_blocks > 1)
+                        tma_load_2d(st + kLmATileBytes + p.n_tile * 128, &x_map, &full_bar[s], kb * kLmBlockK, x_row0 + p.n_tile, pol_x);
                     last_s = s; last_ph = ph;
-                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                    st += stage_bytes;
+                    if (++s == p.num_stages) { s = 0; ph ^= 1u; st = smem; }
                 }
             }
             // do not leave while a copy of ours may still be landing in shared memory
@@ -135,6 +139,7 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
             uint32_t ph = 0;
             int seq = 0;                                 // accumulator buffers handed out so far
             bool ok = true;
+            uint32_t a_addr = smem_u32(smem);
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 // the tile's accumulator buffers: their previous contents must have been drained (use u of a
                 // buffer waits for the epilogue of use u - 1; a fresh barrier lets use 0 through)
@@ -148,7 +153,6 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, p.status, 5)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
                     const uint32_t b_addr = a_addr + kLmATileBytes;
                     if (p.n_blocks == 1) {
 #pragma unroll
@@ -172,7 +176,8 @@ lm_head_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
                         }
                     }
                     umma_commit(&empty_bar[s]);          // stage is free once these MMAs have read it
-                    if (++s == p.num_stages) { s = 0; ph ^= 1u; }
+                    a_addr += static_cast<uint32_t>(stage_bytes);
+                    if (++s == p.num_stages) { s = 0; ph ^= 1u; a_addr = smem_u32(smem); }
                 }
                 if (ok) {                                // accumulators complete
                     umma_commit(&tmem_full[slot0]);
